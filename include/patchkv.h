@@ -1,0 +1,247 @@
+/*
+ * patchkv.h -- C ABI of the PatchKV suffix-restore library for NVIDIA B200 (sm_100a).
+ *
+ * After a middle edit of an LLM context, C_new = P + M_new + S keeps a token-identical suffix S
+ * whose KV cache was offloaded (Section II-A, Eq. 1).  This library runs the two data-parallel
+ * steps of resuming that suffix:
+ *
+ *   1. patchkv_select_repair -- fix the block partition (R, F) of the suffix before any
+ *      reconstruction: per-block attention mass from stored attention (Section IV-C, Eq. 10), the
+ *      edit-local dirty window (Section IV-B, Eq. 9), the top-k non-local blocks outside it (Eq. 11),
+ *      and R = BlockRound(D u H), F = B(S) \ R (Eq. 12).
+ *   2. patchkv_restore / patchkv_restore_from_host -- rebuild every block of F in one fused pass:
+ *      dequantise it by its frozen per-block precision tag (Section IV-D, Eq. 14 gives the tags),
+ *      correct the RoPE phase of K by the position delta, K_corr = R(rho) R(omega)^-1 K_old
+ *      (Section II-B, Eq. 3; values are never rotated, Section IV-C), and write the rows straight
+ *      into the request's destination KV pages (Section IV-D, last paragraph).  Blocks of R are
+ *      never read and never written: they belong to the recompute path.
+ *
+ * Conventions
+ *   - Every function returns a patchkv_status (0 = ok, < 0 = error); nothing throws or prints.
+ *   - "DEVICE" pointers are CUDA device memory of the context's device; "HOST" pointers are host
+ *     memory; "PINNED" is page-locked host memory (cudaHostAlloc / cudaHostRegister).
+ *   - The caller owns every buffer it passes and keeps it alive and unmodified until the work
+ *     enqueued on `stream` has completed.  The library owns only the context's workspace.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls are
+ *     asynchronous with respect to the host unless stated otherwise; completion is stream order,
+ *     which is how "decode starts only after both groups have been placed" (Section IV-C) is kept.
+ *   - Device-side faults are never raised.  A work item whose directory entry, record extent or
+ *     destination pages are out of range is skipped whole, the first such error is latched in the
+ *     context's status word, and the rest of the call proceeds; see patchkv_query_status.
+ *   - Every struct starts with struct_size = sizeof(that struct) as compiled by the caller.
+ *
+ * Checkpoint byte layout ("PKV1"; the paper prescribes none beyond same-representation runs)
+ *   - per layer one payload buffer, 16-byte aligned; tags u8 [L][NB] and blk_off u64 [L][NB] give the
+ *     tag and the byte offset (multiple of 16) of each block's record inside its layer payload;
+ *   - one block record = [K codes][K scales][V codes][V scales]; codes are [token][head][channel]
+ *     row-major; bf16 codes 2 bytes; int8 codes 1 byte two's complement; int4 codes pack channel c
+ *     (even) in bits 0-3 and channel c+1 in bits 4-7 of one byte, two's-complement nibbles; scales
+ *     are fp16 [token][head][channel / group], symmetric (no zero point); a bf16 section has no
+ *     scales; a partial last block is zero-padded to block_tokens tokens.
+ *   - value = code * scale formed in fp32 (exact), rounded once to bf16 (nearest even); a bf16 code
+ *     is copied bit for bit (V always; K when delta == 0).
+ *   - K rotation: theta_i = rope_base^(-2i/rotary_dim) (or inv_freq[i]); c_i, s_i = cos, sin of
+ *     (double)delta * theta_i evaluated in double on the host and rounded once to fp32; each rotary
+ *     pair (a, b) -> (a*c_i - b*s_i, a*s_i + b*c_i) with every fp32 operation rounded on its own (no
+ *     FMA contraction), then one rounding to bf16.  delta == 0 skips the rotation.
+ *   - destination: suffix token u = j*block_tokens + t + dst_shift goes to slot u % page_tokens of
+ *     page block_table[u / page_tokens]; element offset = layer*stride_layer + page*stride_page +
+ *     slot*stride_token + head*stride_head + channel from k_base / v_base.
+ */
+#ifndef PATCHKV_H_
+#define PATCHKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(_WIN32)
+#define PATCHKV_API __declspec(dllexport)
+#else
+#define PATCHKV_API __attribute__((visibility("default")))
+#endif
+
+typedef struct patchkv_ctx patchkv_ctx; /* opaque: streams, events, staging ring, workspace, status word */
+
+typedef enum {
+    PATCHKV_OK = 0,
+    PATCHKV_E_INVALID = -1,     /* bad argument (null pointer, inconsistent geometry, misalignment, pageable payload) */
+    PATCHKV_E_CUDA = -2,        /* a CUDA runtime call failed; text in patchkv_last_error */
+    PATCHKV_E_BOUNDS = -3,      /* device side: an item was out of range and was skipped */
+    PATCHKV_E_NOMEM = -4,       /* workspace or staging allocation failed */
+    PATCHKV_E_TIMEOUT = -5,     /* reserved: a bounded device-side wait gave up */
+    PATCHKV_E_UNSUPPORTED = -6, /* valid but outside the compiled kernels' geometry limits */
+    PATCHKV_E_BADINPUT = -7     /* device side: stored attention held a negative, infinite or NaN entry */
+} patchkv_status;
+
+/* Per-block precision tags (the frozen policy pi_b of Section IV-D: FP16 | K8/V8 | K8/V4). */
+enum {
+    PATCHKV_TAG_BF16 = 0, /* K bf16, V bf16 (the full-precision tier; this build stores bf16) */
+    PATCHKV_TAG_INT8 = 1, /* K int8, V int8 */
+    PATCHKV_TAG_INT4 = 2, /* K int8, V int4 -- keys stay at 8 bits, only values enter the 4-bit tier */
+    PATCHKV_TAG_K4V4 = 3  /* K int4, V int4 -- the uniform-INT4 ablation of Section V-C */
+};
+enum { PATCHKV_ROPE_HALF = 0 /* pairs (i, i + rotary_dim/2) */, PATCHKV_ROPE_INTERLEAVED = 1 /* pairs (2i, 2i+1) */ };
+enum { PATCHKV_LAYERS_INDEPENDENT = 0 /* one (R_l, F_l) per layer */, PATCHKV_LAYERS_SHARED = 1 /* rank on the mass summed over layers */ };
+enum { PATCHKV_SCORE_ATTN_F16 = 0 /* stored attention */, PATCHKV_SCORE_BLOCK_MASS = 1 /* stored per-block mass */ };
+
+enum {
+    PATCHKV_MAX_SESSIONS = 8,      /* sessions per restore call */
+    PATCHKV_MAX_ROTARY_DIM = 256,  /* rotary_dim <= 256 */
+    PATCHKV_MAX_BLOCK_VECTORS = 2048 /* block_tokens * n_kv_heads <= 2048 */
+};
+
+typedef struct {
+    uint32_t struct_size;
+    int32_t device;            /* CUDA device ordinal */
+    int32_t staging_slots;     /* restore_from_host: depth of the device staging ring (0 = 4) */
+    int32_t reserved;
+    uint64_t merge_gap_bytes;  /* restore_from_host: two reused records closer than this are fetched by one copy
+                                  (the bytes between them are transferred and ignored); UINT64_MAX = default 64 KiB */
+} patchkv_config;
+
+/* Model / cache geometry shared by all sessions of a call. */
+typedef struct {
+    uint32_t struct_size;
+    int32_t n_layers;       /* L */
+    int32_t n_kv_heads;     /* H */
+    int32_t head_dim;       /* D, multiple of 8 */
+    int32_t rotary_dim;     /* Dr <= D; multiple of 16 (HALF) or 8 (INTERLEAVED); channels >= Dr are not rotated */
+    int32_t rope_style;     /* PATCHKV_ROPE_* */
+    int32_t block_tokens;   /* B: tokens per checkpoint block */
+    int32_t page_tokens;    /* P: tokens per destination page */
+    int32_t group;          /* G: channels per fp16 scale, multiple of 8, divides D */
+    double rope_base;
+    const float* inv_freq;  /* HOST, optional [Dr/2]; overrides rope_base (frequency-scaled RoPE variants) */
+} patchkv_geom;
+
+/* Destination paged KV pool: two bf16 tensors addressed by element strides. */
+typedef struct {
+    uint32_t struct_size;
+    int32_t n_pages;
+    void* k_base;           /* DEVICE bf16, 16-byte aligned */
+    void* v_base;           /* DEVICE bf16, 16-byte aligned */
+    int64_t stride_layer;   /* elements; every stride a multiple of 8; the channel stride is 1 */
+    int64_t stride_page;
+    int64_t stride_token;
+    int64_t stride_head;
+} patchkv_pool;
+
+/* One resumed session whose checkpoint is resident in device memory.  NB = ceil(n_suffix_tokens / B). */
+typedef struct {
+    uint32_t struct_size;
+    int32_t n_suffix_tokens;            /* |S| */
+    int32_t delta;                      /* rho_i - omega_i = |M_new| - |M_old|, the same for every suffix token */
+    int32_t dst_shift;                  /* 0 .. P-1: slot of the first suffix token in logical page 0 of block_table */
+    int32_t n_table;                    /* entries of block_table */
+    int32_t reserved;
+    const int32_t* block_table;         /* DEVICE i32 [n_table]: logical page -> physical page */
+    const uint8_t* tags;                /* DEVICE u8  [L][NB] */
+    const uint64_t* blk_off;            /* DEVICE u64 [L][NB] */
+    const void* const* layer_payload;   /* DEVICE array of L DEVICE pointers (each 16-byte aligned) */
+    const uint64_t* layer_bytes;        /* DEVICE u64 [L]: size of each layer payload */
+    const int32_t* reuse_idx;           /* DEVICE i32 [L][NB]: F_l ascending in the first reuse_cnt[l] entries */
+    const int32_t* reuse_cnt;           /* DEVICE i32 [L] */
+} patchkv_session;
+
+/* The same session with its checkpoint in pinned host memory; every pointer here is a HOST pointer
+ * except block_table's target pool.  The planner reads tags, blk_off and the reuse lists on the host. */
+typedef struct {
+    uint32_t struct_size;
+    int32_t n_suffix_tokens;
+    int32_t delta;
+    int32_t dst_shift;
+    int32_t n_table;
+    int32_t reserved;
+    const int32_t* block_table;         /* HOST i32 [n_table] */
+    const uint8_t* tags;                /* HOST u8  [L][NB] */
+    const uint64_t* blk_off;            /* HOST u64 [L][NB] */
+    const void* const* layer_payload;   /* HOST array of L PINNED pointers (each 16-byte aligned) */
+    const uint64_t* layer_bytes;        /* HOST u64 [L] */
+    const int32_t* reuse_idx;           /* HOST i32 [L][NB] */
+    const int32_t* reuse_cnt;           /* HOST i32 [L] */
+} patchkv_session_host;
+
+typedef struct {
+    uint32_t struct_size;
+    int32_t kind;                /* PATCHKV_SCORE_* */
+    int32_t n_layers;            /* L */
+    int32_t n_q_heads;           /* Hq (ATTN_F16 only) */
+    int32_t n_queries;           /* Q: stored decode query positions (ATTN_F16 only) */
+    int32_t n_suffix_tokens;     /* n = |S| */
+    int32_t block_tokens;        /* B */
+    int32_t dirty_tokens;        /* d-hat of Eq. 9; clamped to [0, n] */
+    int32_t top_k;               /* blocks taken outside the dirty window, per layer (or once, LAYERS_SHARED) */
+    int32_t layer_mode;          /* PATCHKV_LAYERS_* */
+    const void* attn;            /* DEVICE fp16 [L][Hq][Q][n], token stride 1 (ATTN_F16) */
+    int64_t attn_stride_layer;   /* elements */
+    int64_t attn_stride_head;
+    int64_t attn_stride_query;
+    const uint64_t* mass;        /* DEVICE u64 [L][NB], units of 2^-24 (BLOCK_MASS) */
+    uint64_t* mass_out;          /* DEVICE u64 [L][NB], optional: receives the exact block masses (ATTN_F16);
+                                    when NULL the context's workspace holds them */
+    uint8_t* repair_mask;        /* DEVICE u8  [L][NB]: 1 = block is in R_l */
+    int32_t* repair_idx;         /* DEVICE i32 [L][NB]: R_l ascending, then -1 */
+    int32_t* repair_cnt;         /* DEVICE i32 [L] */
+    int32_t* reuse_idx;          /* DEVICE i32 [L][NB]: F_l ascending, then -1 */
+    int32_t* reuse_cnt;          /* DEVICE i32 [L] */
+} patchkv_select_args;
+
+typedef struct {
+    uint32_t struct_size;
+    uint32_t n_copies;           /* host->device copies issued */
+    uint64_t bytes_copied;       /* bytes that crossed the link */
+    uint64_t bytes_useful;       /* bytes of reused records among them */
+    uint64_t n_block_layers;     /* reused (layer, block) records */
+} patchkv_restore_stats;
+
+/* Create / destroy a context bound to one device.  Creation allocates two streams, a few events and the
+ * 4-byte status word; workspaces grow on first use (a growing call synchronises the device once). */
+PATCHKV_API int patchkv_create(patchkv_ctx** out, const patchkv_config* cfg);
+PATCHKV_API int patchkv_destroy(patchkv_ctx* ctx);
+
+/* Copies the text of the last host-side error of this context into buf (NUL-terminated, truncated to n). */
+PATCHKV_API int patchkv_last_error(patchkv_ctx* ctx, char* buf, size_t n);
+
+/* Section IV-C Eqs. 10-12 with the dirty window of Section IV-B Eq. 9, at block granularity.
+ *   mass[l][j] = exact sum over heads, stored query positions and the tokens of block j of attn (each
+ *                finite fp16 >= 0 is an integer number of 2^-24 units, so the sum is order-independent);
+ *                a negative non-zero, infinite or NaN entry counts as zero and latches PATCHKV_E_BADINPUT.
+ *   dirty      = blocks [0, ceil(min(max(dirty_tokens, 0), n) / B)).
+ *   H_l        = the min(top_k, #candidates) non-dirty blocks of largest mass; ties go to the lower index.
+ *   R_l = dirty u H_l and F_l = the rest, both ascending; unused list entries are set to -1.
+ * Asynchronous on `stream`; all outputs are caller-allocated DEVICE arrays. */
+PATCHKV_API int patchkv_select_repair(patchkv_ctx* ctx, const patchkv_select_args* args, void* stream);
+
+/* Section IV-D fused restore (dequantise, Eq. 3 RoPE correction of K, page placement) of the reuse sets of
+ * up to PATCHKV_MAX_SESSIONS sessions whose payloads are in device memory.  One kernel launch, asynchronous
+ * on `stream`, no host synchronisation, no allocation. */
+PATCHKV_API int patchkv_restore(patchkv_ctx* ctx, const patchkv_geom* geom, const patchkv_pool* pool,
+                                const patchkv_session* sessions, int n_sessions, void* stream);
+
+/* The same restore with the payloads in PINNED host memory (the CPU-resident checkpoint of Section II-C /
+ * Section V-A): only the records of F are fetched, by asynchronous copies on an internal copy stream into a
+ * ring of device staging slots (one layer of one session per slot), each decoded by the restore kernel on
+ * an internal decode stream as soon as it has landed, so that transfer and decode overlap.  The internal
+ * streams start after the work already on `stream` and `stream` waits for them before anything enqueued
+ * later, so pages are complete for whatever follows on `stream`.  The call returns once everything is
+ * enqueued; host arrays are consumed before it returns, the pinned payload must stay valid until the
+ * stream work completes.  `stats` is optional. */
+PATCHKV_API int patchkv_restore_from_host(patchkv_ctx* ctx, const patchkv_geom* geom, const patchkv_pool* pool,
+                                          const patchkv_session_host* sessions, int n_sessions, void* stream,
+                                          patchkv_restore_stats* stats);
+
+/* Synchronises the context's device work and returns in *device_status the first device-side error latched
+ * since the last query (PATCHKV_OK, PATCHKV_E_BOUNDS or PATCHKV_E_BADINPUT), then clears it. */
+PATCHKV_API int patchkv_query_status(patchkv_ctx* ctx, int* device_status);
+
+/* Bytes of one block record for a tag under a geometry; 0 for an unknown tag. */
+PATCHKV_API uint64_t patchkv_record_bytes(int tag, int block_tokens, int n_kv_heads, int head_dim, int group);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PATCHKV_H_ */

@@ -1,0 +1,129 @@
+// Internal declarations shared by the translation units of libpatchkv (not part of the C ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <mutex>
+#include <string>
+#include <vector>
+
+#include "patchkv.h"
+
+namespace patchkv {
+
+enum { FMT_BF16 = 0, FMT_INT8 = 1, FMT_INT4 = 2 };
+
+__host__ __device__ inline int k_format(int tag) {
+    return tag == PATCHKV_TAG_BF16 ? FMT_BF16 : (tag == PATCHKV_TAG_K4V4 ? FMT_INT4 : FMT_INT8);
+}
+__host__ __device__ inline int v_format(int tag) {
+    return tag == PATCHKV_TAG_BF16 ? FMT_BF16 : (tag == PATCHKV_TAG_INT8 ? FMT_INT8 : FMT_INT4);
+}
+// Code bytes and scale bytes of one K or V section holding `elems` elements.
+__host__ __device__ inline uint64_t code_bytes(int fmt, uint64_t elems) {
+    return fmt == FMT_BF16 ? 2 * elems : (fmt == FMT_INT8 ? elems : elems / 2);
+}
+__host__ __device__ inline uint64_t scale_bytes(int fmt, uint64_t elems, int group) {
+    return fmt == FMT_BF16 ? 0 : 2 * (elems / (uint64_t)group);
+}
+__host__ __device__ inline uint64_t record_bytes(int tag, uint64_t elems, int group) {
+    if (tag < 0 || tag > PATCHKV_TAG_K4V4) return 0;
+    const int kf = k_format(tag), vf = v_format(tag);
+    return code_bytes(kf, elems) + scale_bytes(kf, elems, group) + code_bytes(vf, elems) + scale_bytes(vf, elems, group);
+}
+
+// One session as the restore kernel sees it (all pointers device memory).
+struct SessionDev {
+    const int32_t* block_table;
+    const uint8_t* tags;
+    const unsigned long long* blk_off;
+    const void* const* layer_payload;
+    const unsigned long long* layer_bytes;
+    const int32_t* reuse_idx;
+    const int32_t* reuse_cnt;
+    int32_t n, nb, delta, dst_shift, n_table;
+    int32_t item_begin;     // first work item of this session in the launch's item numbering
+};
+
+struct RestoreParams {
+    // geometry
+    int32_t L, H, D, Dr, rope_style, B, P, G;
+    // pool
+    uint16_t* k_base;
+    uint16_t* v_base;
+    long long stride_layer, stride_page, stride_token, stride_head;
+    int32_t n_pages;
+    // work: items are (session, layer in [layer_begin, layer_end), position r in the reuse list)
+    int32_t n_sessions, layer_begin, layer_end, total_items;
+    int32_t* status;        // device status word
+    SessionDev s[PATCHKV_MAX_SESSIONS];
+    // cos / sin of delta * theta_i per session, fp32, built on the host in double
+    float cs[PATCHKV_MAX_SESSIONS][2][PATCHKV_MAX_ROTARY_DIM / 2];
+};
+
+struct Staging {
+    void* base = nullptr;
+    size_t bytes = 0;
+    cudaEvent_t copied = nullptr;   // recorded on the copy stream when the slot's copies are enqueued
+    cudaEvent_t freed = nullptr;    // recorded on the decode stream after the kernel that read the slot
+};
+
+}  // namespace patchkv
+
+struct patchkv_ctx {
+    int device = 0;
+    int sm_count = 0;
+    int staging_slots = 4;
+    uint64_t merge_gap = 64 * 1024;
+    cudaStream_t copy_stream = nullptr, decode_stream = nullptr;
+    cudaEvent_t ev_begin = nullptr, ev_done = nullptr;
+    int32_t* d_status = nullptr;
+    // select workspace (block masses when the caller gives no mass_out; summed mass for LAYERS_SHARED)
+    unsigned long long* d_mass_ws = nullptr;
+    size_t mass_ws_elems = 0;
+    // restore_from_host: staging ring, metadata arenas
+    std::vector<patchkv::Staging> slots;
+    uint8_t* d_meta = nullptr;
+    uint8_t* h_meta = nullptr;      // pinned mirror
+    size_t meta_bytes = 0;
+    bool host_call_pending = false;
+    std::string last_error;
+    std::mutex mu;
+};
+
+namespace patchkv {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+inline int fail(patchkv_ctx* ctx, int code, const std::string& msg) {
+    if (ctx) ctx->last_error = msg;
+    return code;
+}
+
+#define PKV_CUDA(ctx, expr)                                                                       \
+    do {                                                                                          \
+        cudaError_t e_ = (expr);                                                                  \
+        if (e_ != cudaSuccess)                                                                    \
+            return ::patchkv::fail((ctx), e_ == cudaErrorMemoryAllocation ? PATCHKV_E_NOMEM : PATCHKV_E_CUDA, \
+                                   std::string(#expr) + ": " + cudaGetErrorString(e_));           \
+    } while (0)
+
+// Validates geometry + pool and fills the geometry / pool part of RestoreParams.
+int fill_geometry(patchkv_ctx* ctx, const patchkv_geom* g, const patchkv_pool* pool, RestoreParams* p);
+// cos / sin table of one session (double on the host, rounded once to fp32).
+void build_rope_table(const patchkv_geom* g, int delta, float* cos_out, float* sin_out);
+// Launches the restore kernel for layers [layer_begin, layer_end) of the sessions already filled in p.
+int launch_restore(patchkv_ctx* ctx, RestoreParams* p, cudaStream_t stream);
+
+}  // namespace patchkv

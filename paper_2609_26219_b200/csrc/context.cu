@@ -1,0 +1,80 @@
+// Context life cycle, error text and the device status word.
+#include "common.cuh"
+
+using namespace patchkv;
+
+extern "C" int patchkv_create(patchkv_ctx** out, const patchkv_config* cfg) {
+    if (!out || !cfg || cfg->struct_size != sizeof(patchkv_config)) return PATCHKV_E_INVALID;
+    *out = nullptr;
+    int n_dev = 0;
+    if (cudaGetDeviceCount(&n_dev) != cudaSuccess || cfg->device < 0 || cfg->device >= n_dev) return PATCHKV_E_CUDA;
+    DeviceGuard guard(cfg->device);
+    if (!guard.ok) return PATCHKV_E_CUDA;
+    patchkv_ctx* ctx = new patchkv_ctx();
+    ctx->device = cfg->device;
+    ctx->staging_slots = cfg->staging_slots > 0 ? cfg->staging_slots : 4;
+    if (ctx->staging_slots > 64) ctx->staging_slots = 64;
+    ctx->merge_gap = cfg->merge_gap_bytes == UINT64_MAX ? 64 * 1024 : cfg->merge_gap_bytes;
+    bool ok = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, cfg->device) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&ctx->decode_stream, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&ctx->ev_begin, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&ctx->ev_done, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaMalloc(&ctx->d_status, sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMemset(ctx->d_status, 0, sizeof(int32_t)) == cudaSuccess;
+    if (!ok) {
+        patchkv_destroy(ctx);
+        return PATCHKV_E_CUDA;
+    }
+    *out = ctx;
+    return PATCHKV_OK;
+}
+
+extern "C" int patchkv_destroy(patchkv_ctx* ctx) {
+    if (!ctx) return PATCHKV_OK;
+    {
+        DeviceGuard guard(ctx->device);
+        cudaDeviceSynchronize();
+        for (auto& s : ctx->slots) {
+            if (s.base) cudaFree(s.base);
+            if (s.copied) cudaEventDestroy(s.copied);
+            if (s.freed) cudaEventDestroy(s.freed);
+        }
+        if (ctx->d_meta) cudaFree(ctx->d_meta);
+        if (ctx->h_meta) cudaFreeHost(ctx->h_meta);
+        if (ctx->d_mass_ws) cudaFree(ctx->d_mass_ws);
+        if (ctx->d_status) cudaFree(ctx->d_status);
+        if (ctx->ev_begin) cudaEventDestroy(ctx->ev_begin);
+        if (ctx->ev_done) cudaEventDestroy(ctx->ev_done);
+        if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+        if (ctx->decode_stream) cudaStreamDestroy(ctx->decode_stream);
+    }
+    delete ctx;
+    return PATCHKV_OK;
+}
+
+extern "C" int patchkv_last_error(patchkv_ctx* ctx, char* buf, size_t n) {
+    if (!ctx || !buf || n == 0) return PATCHKV_E_INVALID;
+    std::lock_guard<std::mutex> lock(ctx->mu);
+    strncpy(buf, ctx->last_error.c_str(), n - 1);
+    buf[n - 1] = '\0';
+    return PATCHKV_OK;
+}
+
+extern "C" int patchkv_query_status(patchkv_ctx* ctx, int* device_status) {
+    if (!ctx || !device_status) return PATCHKV_E_INVALID;
+    std::lock_guard<std::mutex> lock(ctx->mu);
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, PATCHKV_E_CUDA, "cudaSetDevice failed");
+    PKV_CUDA(ctx, cudaDeviceSynchronize());
+    int32_t v = 0;
+    PKV_CUDA(ctx, cudaMemcpy(&v, ctx->d_status, sizeof(v), cudaMemcpyDeviceToHost));
+    PKV_CUDA(ctx, cudaMemset(ctx->d_status, 0, sizeof(v)));
+    *device_status = v;
+    return PATCHKV_OK;
+}
+
+extern "C" uint64_t patchkv_record_bytes(int tag, int block_tokens, int n_kv_heads, int head_dim, int group) {
+    if (block_tokens <= 0 || n_kv_heads <= 0 || head_dim <= 0 || group <= 0) return 0;
+    return record_bytes(tag, (uint64_t)block_tokens * n_kv_heads * head_dim, group);
+}

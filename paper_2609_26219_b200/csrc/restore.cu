@@ -1,0 +1,369 @@
+// Fused restore of reused suffix blocks: dequantise by precision tag, RoPE phase correction of K (Eq. 3),
+// placement into destination KV pages through the block table (Section IV-D).  HBM-bound streaming codec:
+// no tensor cores, coalesced 128/64/32-bit code loads, 128-bit bf16 stores, persistent grid over block records.
+#include <cuda_fp16.h>
+#include <math.h>
+
+#include "common.cuh"
+
+namespace patchkv {
+
+constexpr int kThreads = 256;
+constexpr int kCtasPerSm = 6;
+
+// ---------------------------------------------------------------- conversions
+// Four biased bytes -> four exact floats: byte b placed in the low mantissa byte of 2^23, minus (2^23 + bias).
+__device__ __forceinline__ void s8x4_to_f32(uint32_t w, float* o) {
+    const uint32_t x = w ^ 0x80808080u;      // two's complement -> offset binary
+    o[0] = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7650)) - 8388736.0f;
+    o[1] = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7651)) - 8388736.0f;
+    o[2] = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7652)) - 8388736.0f;
+    o[3] = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7653)) - 8388736.0f;
+}
+// Eight nibbles (channel 2k in the low nibble of byte k) -> eight exact floats in channel order.
+__device__ __forceinline__ void s4x8_to_f32(uint32_t w, float* o) {
+    const uint32_t x = w ^ 0x88888888u;
+    const uint32_t lo = x & 0x0F0F0F0Fu, hi = (x >> 4) & 0x0F0F0F0Fu;
+    o[0] = __uint_as_float(__byte_perm(lo, 0x4B000000u, 0x7650)) - 8388616.0f;
+    o[1] = __uint_as_float(__byte_perm(hi, 0x4B000000u, 0x7650)) - 8388616.0f;
+    o[2] = __uint_as_float(__byte_perm(lo, 0x4B000000u, 0x7651)) - 8388616.0f;
+    o[3] = __uint_as_float(__byte_perm(hi, 0x4B000000u, 0x7651)) - 8388616.0f;
+    o[4] = __uint_as_float(__byte_perm(lo, 0x4B000000u, 0x7652)) - 8388616.0f;
+    o[5] = __uint_as_float(__byte_perm(hi, 0x4B000000u, 0x7652)) - 8388616.0f;
+    o[6] = __uint_as_float(__byte_perm(lo, 0x4B000000u, 0x7653)) - 8388616.0f;
+    o[7] = __uint_as_float(__byte_perm(hi, 0x4B000000u, 0x7653)) - 8388616.0f;
+}
+__device__ __forceinline__ float fp16_bits_to_f32(uint16_t h) { return __half2float(__ushort_as_half(h)); }
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));   // first source -> upper half
+    return r;
+}
+__device__ __forceinline__ uint4 pack8(const float* v) {
+    return make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
+}
+
+// Eight consecutive channels of one (token, head) vector, as stored.
+struct Chunk {
+    uint4 w;        // bf16: 16 bytes; int8: x,y; int4: x
+    uint16_t s;     // fp16 scale bits (quantised formats)
+};
+
+template <int FMT>
+__device__ __forceinline__ Chunk load_chunk(const uint8_t* codes, const uint8_t* scales, uint32_t vec, int D,
+                                            int groups_per_vec, int c0, int g0) {
+    Chunk c;
+    c.w = make_uint4(0, 0, 0, 0);
+    c.s = 0;
+    const size_t e = (size_t)vec * D + c0;
+    if (FMT == FMT_BF16) {
+        c.w = __ldg(reinterpret_cast<const uint4*>(codes + 2 * e));
+    } else if (FMT == FMT_INT8) {
+        const uint2 t = __ldg(reinterpret_cast<const uint2*>(codes + e));
+        c.w.x = t.x; c.w.y = t.y;
+        c.s = __ldg(reinterpret_cast<const uint16_t*>(scales) + (size_t)vec * groups_per_vec + g0);
+    } else {
+        c.w.x = __ldg(reinterpret_cast<const uint32_t*>(codes + (e >> 1)));
+        c.s = __ldg(reinterpret_cast<const uint16_t*>(scales) + (size_t)vec * groups_per_vec + g0);
+    }
+    return c;
+}
+
+template <int FMT>
+__device__ __forceinline__ void chunk_to_f32(const Chunk& c, float* v) {
+    if (FMT == FMT_BF16) {
+        v[0] = __uint_as_float(c.w.x << 16); v[1] = __uint_as_float(c.w.x & 0xFFFF0000u);
+        v[2] = __uint_as_float(c.w.y << 16); v[3] = __uint_as_float(c.w.y & 0xFFFF0000u);
+        v[4] = __uint_as_float(c.w.z << 16); v[5] = __uint_as_float(c.w.z & 0xFFFF0000u);
+        v[6] = __uint_as_float(c.w.w << 16); v[7] = __uint_as_float(c.w.w & 0xFFFF0000u);
+    } else {
+        if (FMT == FMT_INT8) { s8x4_to_f32(c.w.x, v); s8x4_to_f32(c.w.y, v + 4); }
+        else s4x8_to_f32(c.w.x, v);
+        const float s = fp16_bits_to_f32(c.s);
+#pragma unroll
+        for (int i = 0; i < 8; i++) v[i] = __fmul_rn(v[i], s);   // exact: < 2^8 times an 11-bit significand
+    }
+}
+
+// (a, b) -> (a c - b s, a s + b c), every operation rounded on its own.
+__device__ __forceinline__ void rotate_pair(float& a, float& b, float c, float s) {
+    const float ac = __fmul_rn(a, c), bs = __fmul_rn(b, s), as = __fmul_rn(a, s), bc = __fmul_rn(b, c);
+    a = __fsub_rn(ac, bs);
+    b = __fadd_rn(as, bc);
+}
+
+// Which two 8-channel chunks of a head vector a thread owns, and how they rotate.
+struct ThreadMap {
+    int ty, TY;         // vector lane of this thread, vector lanes per CTA
+    int cA, cB;         // first channel of chunk A / chunk B (cB < 0: absent)
+    int gA, gB;         // scale group of each chunk
+    bool rotA, rotB;    // chunk holds rotary channels (HALF: A and B are partners and rotate together)
+    int tab;            // HALF: table index of the first pair; INTERLEAVED: unused
+};
+
+template <int KF, int VF, bool INTER>
+__device__ __forceinline__ void restore_vectors(const RestoreParams& p, const uint8_t* rec, int nvec,
+                                                const long long* vec_off, const ThreadMap& tm,
+                                                const float* tc, const float* ts, bool rotate) {
+    const uint64_t elems = (uint64_t)p.B * p.H * p.D;
+    const uint8_t* kc = rec;
+    const uint8_t* ks = kc + code_bytes(KF, elems);
+    const uint8_t* vc = ks + scale_bytes(KF, elems, p.G);
+    const uint8_t* vs = vc + code_bytes(VF, elems);
+    const int gpv = p.D / p.G;
+    const bool hasB = tm.cB >= 0;
+    const bool rotA = rotate && tm.rotA, rotB = rotate && tm.rotB;
+
+#pragma unroll 2
+    for (int vec = tm.ty; vec < nvec; vec += tm.TY) {
+        const long long off = vec_off[vec];
+        Chunk ka = load_chunk<KF>(kc, ks, vec, p.D, gpv, tm.cA, tm.gA);
+        Chunk kb = ka, va, vb;
+        if (hasB) kb = load_chunk<KF>(kc, ks, vec, p.D, gpv, tm.cB, tm.gB);
+        va = load_chunk<VF>(vc, vs, vec, p.D, gpv, tm.cA, tm.gA);
+        vb = va;
+        if (hasB) vb = load_chunk<VF>(vc, vs, vec, p.D, gpv, tm.cB, tm.gB);
+
+        // ---- K: dequantise, rotate, round once
+        uint16_t* kd = p.k_base + off;
+        {
+            float a[8], b[8];
+            chunk_to_f32<KF>(ka, a);
+            chunk_to_f32<KF>(kb, b);
+            if (!INTER) {
+                if (rotA) {
+#pragma unroll
+                    for (int i = 0; i < 8; i++) rotate_pair(a[i], b[i], tc[i], ts[i]);
+                }
+            } else {
+                if (rotA) {
+#pragma unroll
+                    for (int i = 0; i < 4; i++) rotate_pair(a[2 * i], a[2 * i + 1], tc[i], ts[i]);
+                }
+                if (rotB) {
+#pragma unroll
+                    for (int i = 0; i < 4; i++) rotate_pair(b[2 * i], b[2 * i + 1], tc[4 + i], ts[4 + i]);
+                }
+            }
+            // a bf16 code that is not rotated is copied bit for bit
+            const uint4 oa = (KF == FMT_BF16 && !rotA) ? ka.w : pack8(a);
+            *reinterpret_cast<uint4*>(kd + tm.cA) = oa;
+            if (hasB) {
+                const uint4 ob = (KF == FMT_BF16 && !rotB) ? kb.w : pack8(b);
+                *reinterpret_cast<uint4*>(kd + tm.cB) = ob;
+            }
+        }
+        // ---- V: dequantise and round once; never rotated
+        uint16_t* vd = p.v_base + off;
+        {
+            float a[8];
+            uint4 oa = va.w;
+            if (VF != FMT_BF16) { chunk_to_f32<VF>(va, a); oa = pack8(a); }
+            *reinterpret_cast<uint4*>(vd + tm.cA) = oa;
+            if (hasB) {
+                uint4 ob = vb.w;
+                if (VF != FMT_BF16) { chunk_to_f32<VF>(vb, a); ob = pack8(a); }
+                *reinterpret_cast<uint4*>(vd + tm.cB) = ob;
+            }
+        }
+    }
+}
+
+template <bool INTER>
+__global__ void __launch_bounds__(kThreads)
+restore_kernel(const __grid_constant__ RestoreParams p) {
+    __shared__ long long vec_off[PATCHKV_MAX_BLOCK_VECTORS];
+
+    // ---- per-thread channel map (fixed for the whole launch)
+    ThreadMap tm;
+    const int TX = (p.D + 15) >> 4;
+    tm.TY = kThreads / TX;
+    const int tx = threadIdx.x % TX;
+    tm.ty = threadIdx.x / TX;
+    const bool lane_active = tm.ty < tm.TY;
+    if (!INTER) {
+        const int n_rot = p.Dr >> 4;
+        if (tx < n_rot) { tm.cA = 8 * tx; tm.cB = (p.Dr >> 1) + 8 * tx; tm.rotA = tm.rotB = true; tm.tab = 8 * tx; }
+        else { tm.cA = p.Dr + 16 * (tx - n_rot); tm.cB = tm.cA + 8; tm.rotA = tm.rotB = false; tm.tab = 0; }
+    } else {
+        tm.cA = 16 * tx; tm.cB = tm.cA + 8;
+        tm.rotA = tm.cA < p.Dr; tm.rotB = tm.cB < p.Dr; tm.tab = 0;
+    }
+    if (tm.cB >= p.D) { tm.cB = -1; tm.rotB = INTER ? false : tm.rotB; }
+    tm.gA = tm.cA / p.G;
+    tm.gB = tm.cB >= 0 ? tm.cB / p.G : 0;
+
+    float tc[8], ts[8];
+    int cur_session = -1;
+
+    for (int item = blockIdx.x; item < p.total_items; item += gridDim.x) {
+        int si = 0;
+#pragma unroll 1
+        for (int k = 1; k < p.n_sessions; k++) if (item >= p.s[k].item_begin) si = k;
+        const SessionDev& S = p.s[si];
+        const int local = item - S.item_begin;
+        const int l = p.layer_begin + local / S.nb;
+        const int r = local - (l - p.layer_begin) * S.nb;
+        if (r >= __ldg(S.reuse_cnt + l)) continue;                     // uniform over the CTA
+
+        if (si != cur_session) {                                        // this thread's cos / sin entries
+            cur_session = si;
+#pragma unroll
+            for (int i = 0; i < 8; i++) {
+                int idx;
+                if (!INTER) idx = tm.tab + i;
+                else idx = (i < 4) ? (tm.cA >> 1) + i : ((tm.cB >= 0 ? tm.cB : 0) >> 1) + (i - 4);
+                idx = min(idx, PATCHKV_MAX_ROTARY_DIM / 2 - 1);
+                tc[i] = p.cs[si][0][idx];
+                ts[i] = p.cs[si][1][idx];
+            }
+        }
+
+        // ---- directory entry of the block; every thread reads the same words (broadcast)
+        const int j = __ldg(S.reuse_idx + (size_t)l * S.nb + r);
+        bool bad = j < 0 || j >= S.nb;
+        int tag = 0;
+        unsigned long long off = 0, rec = 0, lbytes = 0;
+        const uint8_t* base = nullptr;
+        if (!bad) {
+            tag = __ldg(S.tags + (size_t)l * S.nb + j);
+            off = __ldg(S.blk_off + (size_t)l * S.nb + j);
+            lbytes = __ldg(S.layer_bytes + l);
+            base = reinterpret_cast<const uint8_t*>(
+                static_cast<uintptr_t>(__ldg(reinterpret_cast<const unsigned long long*>(S.layer_payload) + l)));
+            rec = record_bytes(tag, (uint64_t)p.B * p.H * p.D, p.G);
+            bad = rec == 0 || off > lbytes || rec > lbytes - off || base == nullptr ||
+                  ((reinterpret_cast<uintptr_t>(base) + off) & 15u) != 0;
+        }
+        const int valid = bad ? 0 : min(p.B, S.n - j * p.B);
+        const int nvec = valid * p.H;
+
+        __syncthreads();                                                // previous item's vec_off no longer in use
+        // ---- destination offset of every (token, head) vector; all pages validated before any write
+        for (int i = threadIdx.x; i < nvec; i += kThreads) {
+            const int t = i / p.H, h = i - t * p.H;
+            const long long u = (long long)j * p.B + t + S.dst_shift;
+            const long long lp = u / p.P;
+            int page = -1;
+            if (lp < S.n_table) page = __ldg(S.block_table + lp);
+            if (page < 0 || page >= p.n_pages) bad = true;
+            vec_off[i] = (long long)l * p.stride_layer + (long long)page * p.stride_page +
+                         (u - lp * p.P) * p.stride_token + (long long)h * p.stride_head;
+        }
+        if (__syncthreads_or(bad)) {                                    // skip the block whole, latch the error
+            if (threadIdx.x == 0) atomicCAS(p.status, 0, (int)PATCHKV_E_BOUNDS);
+            continue;
+        }
+        if (!lane_active) continue;
+
+        const uint8_t* recp = base + off;
+        const bool rotate = S.delta != 0;
+        switch (tag) {
+            case PATCHKV_TAG_BF16: restore_vectors<FMT_BF16, FMT_BF16, INTER>(p, recp, nvec, vec_off, tm, tc, ts, rotate); break;
+            case PATCHKV_TAG_INT8: restore_vectors<FMT_INT8, FMT_INT8, INTER>(p, recp, nvec, vec_off, tm, tc, ts, rotate); break;
+            case PATCHKV_TAG_INT4: restore_vectors<FMT_INT8, FMT_INT4, INTER>(p, recp, nvec, vec_off, tm, tc, ts, rotate); break;
+            default:               restore_vectors<FMT_INT4, FMT_INT4, INTER>(p, recp, nvec, vec_off, tm, tc, ts, rotate); break;
+        }
+    }
+}
+
+// ---------------------------------------------------------------- host side
+void build_rope_table(const patchkv_geom* g, int delta, float* cos_out, float* sin_out) {
+    const int half = g->rotary_dim / 2;
+    for (int i = 0; i < half; i++) {
+        const double theta = g->inv_freq ? (double)g->inv_freq[i]
+                                         : pow(g->rope_base, -2.0 * (double)i / (double)g->rotary_dim);
+        const double phi = (double)delta * theta;
+        cos_out[i] = (float)cos(phi);
+        sin_out[i] = (float)sin(phi);
+    }
+}
+
+int fill_geometry(patchkv_ctx* ctx, const patchkv_geom* g, const patchkv_pool* pool, RestoreParams* p) {
+    if (!g || !pool || g->struct_size != sizeof(patchkv_geom) || pool->struct_size != sizeof(patchkv_pool))
+        return fail(ctx, PATCHKV_E_INVALID, "geometry / pool: null or struct_size mismatch");
+    if (g->n_layers <= 0 || g->n_kv_heads <= 0 || g->head_dim <= 0 || g->block_tokens <= 0 || g->page_tokens <= 0 ||
+        g->group <= 0 || g->rotary_dim < 0 || g->rotary_dim > g->head_dim || (g->head_dim & 1) || (g->rotary_dim & 1) ||
+        g->head_dim % g->group != 0)
+        return fail(ctx, PATCHKV_E_INVALID, "geometry: need L,H,D,B,P,G > 0, D and Dr even, Dr <= D, G | D");
+    if (g->rope_style != PATCHKV_ROPE_HALF && g->rope_style != PATCHKV_ROPE_INTERLEAVED)
+        return fail(ctx, PATCHKV_E_INVALID, "geometry: unknown rope_style");
+    if (!g->inv_freq && g->rotary_dim > 0 && !(g->rope_base > 0.0))
+        return fail(ctx, PATCHKV_E_INVALID, "geometry: rope_base must be positive");
+    const int rot_mult = g->rope_style == PATCHKV_ROPE_HALF ? 16 : 8;
+    const long long vecs = (long long)g->block_tokens * g->n_kv_heads;
+    if (g->head_dim % 8 || g->group % 8 || g->rotary_dim % rot_mult || g->rotary_dim > PATCHKV_MAX_ROTARY_DIM ||
+        vecs > PATCHKV_MAX_BLOCK_VECTORS || g->head_dim > 16 * kThreads ||
+        (vecs * g->head_dim) % 32 != 0 || (vecs * (g->head_dim / g->group)) % 8 != 0)
+        return fail(ctx, PATCHKV_E_UNSUPPORTED,
+                    "geometry outside kernel limits: D % 8, G % 8, Dr % 16 (half) or % 8 (interleaved), Dr <= 256, "
+                    "B*H <= 2048, record sections multiples of 16 bytes");
+    if (!pool->k_base || !pool->v_base || pool->n_pages <= 0)
+        return fail(ctx, PATCHKV_E_INVALID, "pool: null base or n_pages <= 0");
+    if ((reinterpret_cast<uintptr_t>(pool->k_base) | reinterpret_cast<uintptr_t>(pool->v_base)) & 15u)
+        return fail(ctx, PATCHKV_E_INVALID, "pool: bases must be 16-byte aligned");
+    if (pool->stride_layer < 0 || pool->stride_page < 0 || pool->stride_token < 0 || pool->stride_head < 0 ||
+        ((pool->stride_layer | pool->stride_page | pool->stride_token | pool->stride_head) & 7))
+        return fail(ctx, PATCHKV_E_INVALID, "pool: strides must be non-negative multiples of 8 elements");
+    p->L = g->n_layers; p->H = g->n_kv_heads; p->D = g->head_dim; p->Dr = g->rotary_dim; p->rope_style = g->rope_style;
+    p->B = g->block_tokens; p->P = g->page_tokens; p->G = g->group;
+    p->k_base = static_cast<uint16_t*>(pool->k_base);
+    p->v_base = static_cast<uint16_t*>(pool->v_base);
+    p->stride_layer = pool->stride_layer; p->stride_page = pool->stride_page;
+    p->stride_token = pool->stride_token; p->stride_head = pool->stride_head;
+    p->n_pages = pool->n_pages;
+    p->status = ctx->d_status;
+    return PATCHKV_OK;
+}
+
+int launch_restore(patchkv_ctx* ctx, RestoreParams* p, cudaStream_t stream) {
+    if (p->total_items <= 0) return PATCHKV_OK;
+    int grid = ctx->sm_count * kCtasPerSm;
+    if (grid > p->total_items) grid = p->total_items;
+    if (p->rope_style == PATCHKV_ROPE_INTERLEAVED) restore_kernel<true><<<grid, kThreads, 0, stream>>>(*p);
+    else restore_kernel<false><<<grid, kThreads, 0, stream>>>(*p);
+    PKV_CUDA(ctx, cudaGetLastError());
+    return PATCHKV_OK;
+}
+
+}  // namespace patchkv
+
+using namespace patchkv;
+
+extern "C" int patchkv_restore(patchkv_ctx* ctx, const patchkv_geom* geom, const patchkv_pool* pool,
+                               const patchkv_session* sessions, int n_sessions, void* stream) {
+    if (!ctx) return PATCHKV_E_INVALID;
+    std::lock_guard<std::mutex> lock(ctx->mu);
+    if (n_sessions < 0 || n_sessions > PATCHKV_MAX_SESSIONS || (n_sessions > 0 && !sessions))
+        return fail(ctx, PATCHKV_E_INVALID, "restore: n_sessions must be 0..PATCHKV_MAX_SESSIONS");
+    static thread_local RestoreParams p;
+    int rc = fill_geometry(ctx, geom, pool, &p);
+    if (rc != PATCHKV_OK) return rc;
+    p.n_sessions = n_sessions; p.layer_begin = 0; p.layer_end = geom->n_layers;
+    long long items = 0;
+    for (int i = 0; i < n_sessions; i++) {
+        const patchkv_session& s = sessions[i];
+        if (s.struct_size != sizeof(patchkv_session)) return fail(ctx, PATCHKV_E_INVALID, "session: struct_size mismatch");
+        if (s.n_suffix_tokens < 0 || s.dst_shift < 0 || s.dst_shift >= geom->page_tokens || s.n_table < 0)
+            return fail(ctx, PATCHKV_E_INVALID, "session: n_suffix_tokens >= 0, 0 <= dst_shift < P, n_table >= 0");
+        const int nb = (s.n_suffix_tokens + geom->block_tokens - 1) / geom->block_tokens;
+        if (nb > 0 && (!s.block_table || !s.tags || !s.blk_off || !s.layer_payload || !s.layer_bytes || !s.reuse_idx || !s.reuse_cnt))
+            return fail(ctx, PATCHKV_E_INVALID, "session: null pointer");
+        SessionDev& d = p.s[i];
+        d.block_table = s.block_table; d.tags = s.tags;
+        d.blk_off = reinterpret_cast<const unsigned long long*>(s.blk_off);
+        d.layer_payload = s.layer_payload;
+        d.layer_bytes = reinterpret_cast<const unsigned long long*>(s.layer_bytes);
+        d.reuse_idx = s.reuse_idx; d.reuse_cnt = s.reuse_cnt;
+        d.n = s.n_suffix_tokens; d.nb = nb; d.delta = s.delta; d.dst_shift = s.dst_shift; d.n_table = s.n_table;
+        d.item_begin = (int32_t)items;
+        items += (long long)nb * geom->n_layers;
+        if (items > 0x7fffffffLL) return fail(ctx, PATCHKV_E_UNSUPPORTED, "restore: more than 2^31 work items");
+        build_rope_table(geom, s.delta, p.cs[i][0], p.cs[i][1]);
+    }
+    p.total_items = (int32_t)items;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, PATCHKV_E_CUDA, "cudaSetDevice failed");
+    return launch_restore(ctx, &p, static_cast<cudaStream_t>(stream));
+}

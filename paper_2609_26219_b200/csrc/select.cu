@@ -1,0 +1,347 @@
+// Repair-set selection (Section IV-B Eq. 9, Section IV-C Eqs. 10-12) at block granularity:
+//   1. exact per-block attention mass from stored fp16 attention (integer units of 2^-24, so any reduction
+//      order gives the same bits): 128-bit streaming loads, per-thread integer accumulation over rows,
+//      warp-shuffle segmented reduction over the octets of a block, one 64-bit atomic per block per CTA;
+//   2. per layer one CTA: radix select of the k-th largest candidate mass (8 passes of 8 bits over u64 keys),
+//      ties resolved towards the lower block index by a prefix count, then union with the dirty window and
+//      prefix-sum compaction into ascending repair / reuse lists.
+#include <cuda_fp16.h>
+
+#include "common.cuh"
+
+namespace patchkv {
+
+// ---------------------------------------------------------------- block mass
+// Units of 2^-24 of a finite fp16 in [0, 2): exact through fp32 (value * 2^24 <= 2^25 is an integer).
+__device__ __forceinline__ uint32_t units2_fast(uint32_t w) {
+    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w));
+    return __float2uint_rz(f.x * 16777216.0f) + __float2uint_rz(f.y * 16777216.0f);
+}
+// Any fp16 bit pattern: negative non-zero / inf / NaN count as zero and raise *bad.
+__device__ __forceinline__ unsigned long long units_any(uint32_t h, bool* bad) {
+    h &= 0xFFFFu;
+    if ((h & 0x7FFFu) == 0) return 0;
+    const uint32_t e = (h >> 10) & 31u, m = h & 1023u;
+    if ((h & 0x8000u) || e == 31u) { *bad = true; return 0; }
+    return e == 0 ? (unsigned long long)m : (unsigned long long)(1024u + m) << (e - 1);
+}
+
+struct MassParams {
+    const uint16_t* attn;
+    long long stride_layer, stride_head, stride_query;
+    int Hq, Q, n, B, NB;
+    int rows_per_cta;
+    unsigned long long* mass;   // [L][NB], zeroed before the launch
+    int32_t* status;
+};
+
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+// One thread owns one octet (8 consecutive key positions, all in one block because B % 8 == 0) and walks the
+// rows (head, query) assigned to its CTA.  grid = (octet tiles, row groups, layers).
+__global__ void __launch_bounds__(256)
+block_mass_octet_kernel(const MassParams p) {
+    const int oct = blockIdx.x * blockDim.x + threadIdx.x;
+    const int col = oct * 8;
+    const int l = blockIdx.z;
+    const int R = p.Hq * p.Q;
+    const int r0 = blockIdx.y * p.rows_per_cta;
+    const int r1 = min(R, r0 + p.rows_per_cta);
+    const bool in_range = col < p.n;
+    const int n_valid = in_range ? min(8, p.n - col) : 0;
+
+    unsigned long long acc = 0;
+    uint32_t acc32 = 0;
+    bool bad = false;
+    if (in_range) {
+        const uint16_t* base = p.attn + (long long)l * p.stride_layer + col;
+        int h = r0 / p.Q, q = r0 - h * p.Q;
+        const uint16_t* row = base + (long long)h * p.stride_head + (long long)q * p.stride_query;
+        int since_flush = 0;
+#pragma unroll 4
+        for (int r = r0; r < r1; r++) {
+            uint4 w;
+            if (n_valid == 8) w = ld_stream(reinterpret_cast<const uint4*>(row));
+            else {                                   // ragged last octet of a row: element loads, zero fill
+                uint16_t e[8];
+#pragma unroll
+                for (int i = 0; i < 8; i++) e[i] = i < n_valid ? __ldg(row + i) : (uint16_t)0;
+                w = make_uint4(e[0] | (uint32_t)e[1] << 16, e[2] | (uint32_t)e[3] << 16,
+                               e[4] | (uint32_t)e[5] << 16, e[6] | (uint32_t)e[7] << 16);
+            }
+            if (((w.x | w.y | w.z | w.w) & 0xC000C000u) == 0) {          // every entry in [0, 2)
+                acc32 += units2_fast(w.x) + units2_fast(w.y) + units2_fast(w.z) + units2_fast(w.w);
+                if (++since_flush == 8) { acc += acc32; acc32 = 0; since_flush = 0; }   // 8 * 8 * 2^25 = 2^31
+            } else {
+                const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                for (int i = 0; i < 4; i++) acc += units_any(ww[i], &bad) + units_any(ww[i] >> 16, &bad);
+            }
+            if (++q == p.Q) { q = 0; h++; row = base + (long long)h * p.stride_head; }
+            else row += p.stride_query;
+        }
+        acc += acc32;
+    }
+    if (bad) atomicCAS(p.status, 0, (int)PATCHKV_E_BADINPUT);
+
+    // segmented reduction over the octets of one block (segments are aligned groups of B/8 lanes)
+    const int opb = p.B >> 3;
+    const unsigned lane = threadIdx.x & 31u;
+    if (opb <= 32 && (opb & (opb - 1)) == 0) {
+        for (int d = 1; d < opb; d <<= 1) {
+            const unsigned long long o = __shfl_down_sync(0xFFFFFFFFu, acc, d);
+            if ((lane & (2 * d - 1)) == 0) acc += o;     // only segment-aligned lanes keep a full sum
+        }
+        if (in_range && (lane & (opb - 1)) == 0 && acc) atomicAdd(p.mass + (long long)l * p.NB + col / p.B, acc);
+    } else if (in_range && acc) {
+        atomicAdd(p.mass + (long long)l * p.NB + col / p.B, acc);
+    }
+}
+
+// Any B, any strides, any alignment: one thread per key position.
+__global__ void __launch_bounds__(256)
+block_mass_generic_kernel(const MassParams p) {
+    const int col = blockIdx.x * blockDim.x + threadIdx.x;
+    const int l = blockIdx.z;
+    const int R = p.Hq * p.Q;
+    const int r0 = blockIdx.y * p.rows_per_cta;
+    const int r1 = min(R, r0 + p.rows_per_cta);
+    if (col >= p.n) return;
+    unsigned long long acc = 0;
+    bool bad = false;
+    for (int r = r0; r < r1; r++) {
+        const int h = r / p.Q, q = r - h * p.Q;
+        const uint16_t x = __ldg(p.attn + (long long)l * p.stride_layer + (long long)h * p.stride_head +
+                                 (long long)q * p.stride_query + col);
+        acc += units_any(x, &bad);
+    }
+    if (bad) atomicCAS(p.status, 0, (int)PATCHKV_E_BADINPUT);
+    if (acc) atomicAdd(p.mass + (long long)l * p.NB + col / p.B, acc);
+}
+
+__global__ void sum_layers_kernel(const unsigned long long* mass, int L, int NB, unsigned long long* out) {
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= NB) return;
+    unsigned long long s = 0;
+    for (int l = 0; l < L; l++) s += mass[(long long)l * NB + j];
+    out[j] = s;
+}
+
+// ---------------------------------------------------------------- top-k + union + lists
+struct TopkParams {
+    const unsigned long long* mass;     // [L][NB], or [NB] when shared
+    int shared;                         // 1: every layer ranks on mass[0..NB)
+    int NB, n_dirty, top_k;
+    uint8_t* mask;
+    int32_t* repair_idx; int32_t* repair_cnt;
+    int32_t* reuse_idx;  int32_t* reuse_cnt;
+};
+
+constexpr int kSelThreads = 1024;
+
+// Exclusive prefix sum of v over the CTA; *total receives the CTA sum.  `warp_sums` is 33 ints of shared memory.
+__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int* total) {
+    const unsigned lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    int inc = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int o = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+        if (lane >= (unsigned)d) inc += o;
+    }
+    __syncthreads();                                 // warp_sums free to overwrite
+    if (lane == 31) warp_sums[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        int w = lane < (kSelThreads >> 5) ? warp_sums[lane] : 0;
+        int winc = w;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int o = __shfl_up_sync(0xFFFFFFFFu, winc, d);
+            if (lane >= (unsigned)d) winc += o;
+        }
+        warp_sums[lane] = winc - w;                  // exclusive offset of each warp
+        if (lane == 31) warp_sums[32] = winc;
+    }
+    __syncthreads();
+    *total = warp_sums[32];
+    return warp_sums[warp] + inc - v;
+}
+
+__global__ void __launch_bounds__(kSelThreads)
+select_kernel(const TopkParams p) {
+    __shared__ unsigned int hist[256];
+    __shared__ int warp_sums[33];
+    __shared__ unsigned long long s_prefix;
+    __shared__ int s_krem;
+
+    const int l = blockIdx.x;
+    const unsigned long long* key = p.mass + (p.shared ? 0 : (long long)l * p.NB);
+    const int NB = p.NB, n_dirty = min(p.n_dirty, NB);
+    const int ncand = NB - n_dirty;
+    const int k = min(p.top_k, ncand);
+    const bool take_all = k == ncand, take_none = k == 0;
+
+    unsigned long long T = 0;
+    int krem = 0;
+    if (!take_all && !take_none) {
+        // radix select: after the pass over byte b, `prefix` holds the top (8 - b) bytes of the k-th largest key
+        if (threadIdx.x == 0) { s_prefix = 0; s_krem = k; }
+        for (int b = 7; b >= 0; b--) {
+            if (threadIdx.x < 256) hist[threadIdx.x] = 0;
+            __syncthreads();
+            const unsigned long long prefix = s_prefix;
+            for (int j = n_dirty + threadIdx.x; j < NB; j += kSelThreads) {
+                const unsigned long long x = key[j];
+                const bool match = b == 7 || ((x ^ prefix) >> (8 * (b + 1))) == 0;
+                if (match) atomicAdd(&hist[(unsigned)(x >> (8 * b)) & 255u], 1u);
+            }
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                int need = s_krem, cum = 0, d = 255;
+                for (; d > 0; d--) {
+                    const int c = (int)hist[d];
+                    if (cum + c >= need) break;
+                    cum += c;
+                }
+                s_prefix = prefix | ((unsigned long long)d << (8 * b));
+                s_krem = need - cum;             // how many keys with this digit (and prefix) are still to take
+            }
+            __syncthreads();
+        }
+        T = s_prefix;
+        krem = s_krem;                           // keys equal to T to take, lowest block index first
+    }
+
+    // ---- emit mask and ascending lists
+    int run_r = 0, run_eq = 0;
+    uint8_t* mask = p.mask + (long long)l * NB;
+    int32_t* ridx = p.repair_idx + (long long)l * NB;
+    int32_t* fidx = p.reuse_idx + (long long)l * NB;
+    for (int j0 = 0; j0 < NB; j0 += kSelThreads) {
+        const int j = j0 + threadIdx.x;
+        const bool in = j < NB;
+        const bool dirty = in && j < n_dirty;
+        const unsigned long long x = (in && !dirty) ? key[j] : 0;
+        const bool cand = in && !dirty;
+        bool sel = dirty;
+        if (take_all) sel = in;
+        else if (!take_none) {
+            const int eq = cand && x == T;
+            int tot_eq;
+            const int rank = block_exclusive_scan(eq, warp_sums, &tot_eq) + run_eq;
+            run_eq += tot_eq;
+            sel = dirty || (cand && x > T) || (eq && rank < krem);
+        }
+        int tot_r;
+        const int pos = block_exclusive_scan(sel ? 1 : 0, warp_sums, &tot_r) + run_r;
+        run_r += tot_r;
+        if (in) {
+            mask[j] = sel ? 1 : 0;
+            if (sel) ridx[pos] = j;
+            else fidx[j - pos] = j;
+        }
+    }
+    const int n_r = run_r, n_f = NB - run_r;
+    for (int i = n_r + threadIdx.x; i < NB; i += kSelThreads) ridx[i] = -1;
+    for (int i = n_f + threadIdx.x; i < NB; i += kSelThreads) fidx[i] = -1;
+    if (threadIdx.x == 0) { p.repair_cnt[l] = n_r; p.reuse_cnt[l] = n_f; }
+}
+
+static int ensure_mass_ws(patchkv_ctx* ctx, size_t elems) {
+    if (elems <= ctx->mass_ws_elems) return PATCHKV_OK;
+    PKV_CUDA(ctx, cudaDeviceSynchronize());
+    if (ctx->d_mass_ws) { cudaFree(ctx->d_mass_ws); ctx->d_mass_ws = nullptr; ctx->mass_ws_elems = 0; }
+    PKV_CUDA(ctx, cudaMalloc(&ctx->d_mass_ws, elems * sizeof(unsigned long long)));
+    ctx->mass_ws_elems = elems;
+    return PATCHKV_OK;
+}
+
+}  // namespace patchkv
+
+using namespace patchkv;
+
+extern "C" int patchkv_select_repair(patchkv_ctx* ctx, const patchkv_select_args* a, void* stream_) {
+    if (!ctx) return PATCHKV_E_INVALID;
+    std::lock_guard<std::mutex> lock(ctx->mu);
+    if (!a || a->struct_size != sizeof(patchkv_select_args)) return fail(ctx, PATCHKV_E_INVALID, "select: null args or struct_size mismatch");
+    if (a->n_layers <= 0 || a->n_suffix_tokens < 0 || a->block_tokens <= 0 || a->top_k < 0)
+        return fail(ctx, PATCHKV_E_INVALID, "select: need L > 0, n >= 0, B > 0, top_k >= 0");
+    if (a->layer_mode != PATCHKV_LAYERS_INDEPENDENT && a->layer_mode != PATCHKV_LAYERS_SHARED)
+        return fail(ctx, PATCHKV_E_INVALID, "select: unknown layer_mode");
+    if (a->kind != PATCHKV_SCORE_ATTN_F16 && a->kind != PATCHKV_SCORE_BLOCK_MASS)
+        return fail(ctx, PATCHKV_E_INVALID, "select: unknown kind");
+    if (!a->repair_mask || !a->repair_idx || !a->repair_cnt || !a->reuse_idx || !a->reuse_cnt)
+        return fail(ctx, PATCHKV_E_INVALID, "select: null output");
+    const int L = a->n_layers, n = a->n_suffix_tokens, B = a->block_tokens;
+    const int NB = (int)(((long long)n + B - 1) / B);
+    long long nd = a->dirty_tokens < 0 ? 0 : a->dirty_tokens;
+    if (nd > n) nd = n;
+    const int n_dirty = (int)((nd + B - 1) / B);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, PATCHKV_E_CUDA, "cudaSetDevice failed");
+
+    const bool shared = a->layer_mode == PATCHKV_LAYERS_SHARED && L > 1;
+    const bool from_attn = a->kind == PATCHKV_SCORE_ATTN_F16;
+    size_t ws_need = (from_attn && !a->mass_out ? (size_t)L * NB : 0) + (shared ? (size_t)NB : 0);
+    if (ws_need) { int rc = ensure_mass_ws(ctx, ws_need); if (rc != PATCHKV_OK) return rc; }
+    unsigned long long* ws = ctx->d_mass_ws;
+
+    const unsigned long long* mass = reinterpret_cast<const unsigned long long*>(a->mass);
+    if (from_attn) {
+        if (a->n_q_heads < 0 || a->n_queries < 0 || (NB > 0 && a->n_q_heads > 0 && a->n_queries > 0 && !a->attn))
+            return fail(ctx, PATCHKV_E_INVALID, "select: attention shape / pointer");
+        unsigned long long* m = a->mass_out ? reinterpret_cast<unsigned long long*>(a->mass_out) : ws;
+        if (!a->mass_out) ws += (size_t)L * NB;
+        const long long rows = (long long)a->n_q_heads * a->n_queries;
+        if (NB > 0) PKV_CUDA(ctx, cudaMemsetAsync(m, 0, (size_t)L * NB * sizeof(unsigned long long), stream));
+        if (NB > 0 && rows > 0) {
+            if (rows > 0x7fffffffLL) return fail(ctx, PATCHKV_E_UNSUPPORTED, "select: Hq * Q too large");
+            MassParams mp;
+            mp.attn = static_cast<const uint16_t*>(a->attn);
+            mp.stride_layer = a->attn_stride_layer; mp.stride_head = a->attn_stride_head; mp.stride_query = a->attn_stride_query;
+            mp.Hq = a->n_q_heads; mp.Q = a->n_queries; mp.n = n; mp.B = B; mp.NB = NB;
+            mp.mass = m; mp.status = ctx->d_status;
+            const bool octet = (B % 8 == 0) && ((reinterpret_cast<uintptr_t>(a->attn) & 15u) == 0) &&
+                               ((a->attn_stride_layer | a->attn_stride_head | a->attn_stride_query) & 7) == 0;
+            const int cols = octet ? (n + 7) / 8 : n;
+            const int tiles = (cols + 255) / 256;
+            // enough CTAs for ~8 waves of 8 CTAs per SM, at least 16 rows each so that atomics stay rare
+            long long want = (long long)ctx->sm_count * 64;
+            long long groups = want / ((long long)tiles * L);
+            if (groups < 1) groups = 1;
+            long long rpc = (rows + groups - 1) / groups;
+            if (rpc < 16) rpc = 16;
+            if (rpc > rows) rpc = rows;
+            groups = (rows + rpc - 1) / rpc;
+            if (groups > 65535 || L > 65535) return fail(ctx, PATCHKV_E_UNSUPPORTED, "select: grid too large");
+            mp.rows_per_cta = (int)rpc;
+            dim3 grid(tiles, (unsigned)groups, L);
+            if (octet) block_mass_octet_kernel<<<grid, 256, 0, stream>>>(mp);
+            else block_mass_generic_kernel<<<grid, 256, 0, stream>>>(mp);
+            PKV_CUDA(ctx, cudaGetLastError());
+        }
+        mass = m;
+    } else if (NB > 0 && !mass) {
+        return fail(ctx, PATCHKV_E_INVALID, "select: null mass");
+    }
+
+    TopkParams tp;
+    tp.mass = mass; tp.shared = 0;
+    if (shared && NB > 0) {
+        sum_layers_kernel<<<(NB + 255) / 256, 256, 0, stream>>>(mass, L, NB, ws);
+        PKV_CUDA(ctx, cudaGetLastError());
+        tp.mass = ws; tp.shared = 1;
+    }
+    tp.NB = NB; tp.n_dirty = n_dirty; tp.top_k = a->top_k;
+    tp.mask = a->repair_mask; tp.repair_idx = a->repair_idx; tp.repair_cnt = a->repair_cnt;
+    tp.reuse_idx = a->reuse_idx; tp.reuse_cnt = a->reuse_cnt;
+    select_kernel<<<L, kSelThreads, 0, stream>>>(tp);
+    PKV_CUDA(ctx, cudaGetLastError());
+    return PATCHKV_OK;
+}

@@ -1,0 +1,267 @@
+"""GPU parity of patchkv_restore / patchkv_restore_from_host against the oracle on the same seeded inputs:
+V, placement and untouched pages bit-exact; rotated K within 2 bf16 ulp (and expected bit-exact)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import patchkv_inputs as pin
+from gpu_common import DEV, check_pools, gpu_pool, new_context, run_select_and_restore, staged
+from helpers import np_u16, oracle_restore, oracle_select
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = new_context()
+    yield c
+    c.close()
+
+
+def test_tiny(ctx):
+    run_select_and_restore(ctx, pin.config_tiny())
+
+
+TINY_VARIANTS = {
+    "delta0": dict(delta=0),
+    "delta_neg": dict(delta=-137),
+    "shift5": dict(dst_shift=5, n_pages=300),
+    "P32": dict(geom=pin.Geometry(2, 4, 64, 64, pin.ROPE_HALF, 1e4, 16, 32, 32)),
+    "P8_shift3": dict(geom=pin.Geometry(2, 4, 64, 64, pin.ROPE_HALF, 1e4, 16, 8, 32), dst_shift=3),
+    "interleaved": dict(geom=pin.Geometry(2, 4, 64, 64, pin.ROPE_INTERLEAVED, 1e4, 16, 16, 32)),
+    "partial_rotary_half": dict(geom=pin.Geometry(2, 4, 64, 32, pin.ROPE_HALF, 1e4, 16, 16, 32)),
+    "partial_rotary_interleaved": dict(geom=pin.Geometry(2, 4, 64, 40, pin.ROPE_INTERLEAVED, 1e4, 16, 16, 32)),
+    "ragged_n1000": dict(n=1000),
+    "G64": dict(geom=pin.Geometry(2, 4, 64, 64, pin.ROPE_HALF, 1e4, 16, 16, 64)),
+    "G8": dict(geom=pin.Geometry(2, 4, 64, 64, pin.ROPE_HALF, 1e4, 16, 16, 8)),
+    "k4v4": dict(tag_probs=(0.25, 0.25, 0.25, 0.25)),
+    "one_head_D128": dict(geom=pin.Geometry(3, 1, 128, 128, pin.ROPE_HALF, 5e5, 16, 16, 32)),
+    "D72_odd_chunks": dict(geom=pin.Geometry(2, 2, 72, 48, pin.ROPE_HALF, 1e4, 16, 16, 24)),
+    "D256": dict(geom=pin.Geometry(1, 2, 256, 256, pin.ROPE_HALF, 1e4, 16, 16, 128)),
+    "B32_P16": dict(geom=pin.Geometry(2, 4, 64, 64, pin.ROPE_HALF, 1e4, 32, 16, 32)),
+    "all_dirty": dict(dirty_tokens=10 ** 6),
+    "nothing_dirty_k0": dict(dirty_tokens=0, top_k=0),
+    "shared_layers": dict(layer_mode=pin.LAYERS_SHARED, top_k=4),
+}
+
+
+@pytest.mark.parametrize("name", sorted(TINY_VARIANTS))
+def test_tiny_variants(ctx, name):
+    kw = dict(TINY_VARIANTS[name])
+    kw.setdefault("n_pages", 256)
+    run_select_and_restore(ctx, pin.config_tiny(**kw))
+
+
+def test_inv_freq_override(ctx):
+    inv = (1e4 ** (-2.0 * np.arange(32) / 64) / 8.0).astype(np.float32)      # a frequency-scaled variant
+    run_select_and_restore(ctx, pin.config_tiny(), inv_freq=inv)
+
+
+def test_empty_suffix_and_no_sessions(ctx):
+    ck = pin.config_tiny()
+    st = staged(ck)
+    k, v, pool = gpu_pool(ck)
+    assert ctx.restore(st.geom(), pool, []) == 0
+    ctx.select_repair(st.select_args())
+    assert ctx.restore(st.geom(), pool, [st.session(n_suffix_tokens=0)]) == 0
+    torch.cuda.synchronize()
+    assert bool((k == k[0, 0, 0, 0, 0]).all()) and bool((v == v[0, 0, 0, 0, 0]).all())
+
+
+@pytest.mark.parametrize("what", ["page", "negative_page", "tag", "offset", "reuse_index", "table_short", "misaligned"])
+def test_out_of_range_items_are_skipped_and_latched(ctx, what):
+    ck = pin.config_tiny(tag_probs=(0.3, 0.4, 0.3, 0.0))
+    st = staged(ck)
+    _, sel = oracle_select(ck)
+    ctx.select_repair(st.select_args())
+    torch.cuda.synchronize()
+    F0 = [int(x) for x in sel["reuse_idx"][0, :sel["reuse_cnt"][0]]]
+    bad_block = F0[3]
+    over_o, over_g = {}, {}
+    table = ck.block_table.clone()
+    tags = ck.tags.clone()
+    off = ck.blk_off.clone()
+    if what == "page":
+        table[bad_block] = ck.n_pages
+    elif what == "negative_page":
+        table[bad_block] = -1
+    elif what == "tag":
+        tags[:, bad_block] = 9
+    elif what == "offset":
+        off[:, bad_block] = max(ck.layer_bytes) - 16
+    elif what == "misaligned":
+        off[:, bad_block] += 8
+    elif what == "reuse_index":
+        ridx = sel["reuse_idx"].copy()
+        ridx[:, 3] = ck.n_blocks
+        st.reuse_idx.copy_(torch.from_numpy(ridx))
+        over_o["reuse_idx"] = ridx
+    elif what == "table_short":
+        bad_block = ck.n_blocks - 1
+        table = table[:-1]
+    over_o.update(block_table=table.numpy(), tags=tags.numpy(), blk_off=off.numpy())
+    k, v, pool = gpu_pool(ck)
+    sess = st.session(block_table=table.to(DEV), tags=tags.to(DEV), blk_off=off.to(DEV))
+    assert ctx.restore(st.geom(), pool, [sess]) == 0
+    torch.cuda.synchronize()
+    assert ctx.query_status() == -3
+    if what == "misaligned":
+        # the oracle has no alignment rule; compare against a run without that block
+        ridx = sel["reuse_idx"].copy()
+        cnt = sel["reuse_cnt"].copy()
+        for l in range(2):
+            row = [x for x in ridx[l, :cnt[l]] if x != bad_block]
+            ridx[l, :len(row)] = row
+            cnt[l] = len(row)
+        rc, k_ref, v_ref, _ = oracle_restore(ck, ridx, cnt)
+    else:
+        ridx = over_o.pop("reuse_idx", sel["reuse_idx"])
+        rc, k_ref, v_ref, _ = oracle_restore(ck, ridx, sel["reuse_cnt"], **over_o)
+        assert rc == oracle.E_BOUNDS
+    check_pools(k, v, k_ref, v_ref, ck.geom)
+
+
+def test_invalid_arguments_are_rejected_on_the_host(ctx):
+    from paper_2609_26219_b200 import binding as pk
+    ck = pin.config_tiny()
+    st = staged(ck)
+    ctx.select_repair(st.select_args())
+    k, v, pool = gpu_pool(ck)
+    g = st.geom()
+    assert ctx.restore(g, pool, [st.session(dst_shift=16)], check=False) == pk.E_INVALID
+    assert "dst_shift" in ctx.last_error()
+    bad = st.geom(); bad.head_dim = 63
+    assert ctx.restore(bad, pool, [st.session()], check=False) == pk.E_INVALID
+    bad = st.geom(); bad.group = 4
+    assert ctx.restore(bad, pool, [st.session()], check=False) == pk.E_UNSUPPORTED
+    bad = st.geom(); bad.rotary_dim = 24
+    assert ctx.restore(bad, pool, [st.session()], check=False) == pk.E_UNSUPPORTED
+    badp = pk.make_pool(k, v, ck.n_pages, (7, 8, 8, 8))
+    assert ctx.restore(g, badp, [st.session()], check=False) == pk.E_INVALID
+    assert ctx.restore(g, pool, [st.session()] * 9, check=False) == pk.E_INVALID
+    a = st.select_args(); a.top_k = -1
+    assert ctx.select_repair(a, check=False) == pk.E_INVALID
+    # a pageable payload is not accepted by the host-resident entry point
+    hs = st.host_session()
+    pageable = torch.zeros(ck.payload.numel(), dtype=torch.uint8)
+    ptrs = torch.tensor([pageable.data_ptr() // 256 * 256 + 256 + o for o in ck.layer_off], dtype=torch.int64)
+    hs2 = st.host_session(layer_payload=ptrs)
+    rc, _ = ctx.restore_from_host(g, pool, [hs2], check=False)
+    assert rc == pk.E_INVALID
+    torch.cuda.synchronize()
+    assert bool((k == k[0, 0, 0, 0, 0]).all())
+
+
+def test_two_sessions_in_one_call_share_a_pool(ctx):
+    a = pin.config_tiny(n_pages=256)
+    b = pin.config_tiny(seed=77, delta=-999, n=700, dirty_tokens=40, top_k=5, n_pages=256)
+    pin.shared_free_list(5, 256, [a, b])
+    sa, sb = staged(a), staged(b)
+    ctx.select_repair(sa.select_args())
+    ctx.select_repair(sb.select_args())
+    k, v, pool = gpu_pool(a)
+    ctx.restore(sa.geom(), pool, [sa.session(), sb.session()])
+    torch.cuda.synchronize()
+    assert ctx.query_status() == 0
+    _, sela = oracle_select(a)
+    _, selb = oracle_select(b)
+    rc, k_ref, v_ref, _ = oracle_restore(a, sela["reuse_idx"], sela["reuse_cnt"])
+    rc, k_ref, v_ref, _ = oracle_restore(b, selb["reuse_idx"], selb["reuse_cnt"], pools=(k_ref, v_ref))
+    check_pools(k, v, k_ref, v_ref, a.geom)
+
+
+def test_noncontiguous_pool_strides(ctx):
+    """Pool laid out [page][L][slot][H][D+pad]: every stride differs from the benchmark layout."""
+    from paper_2609_26219_b200 import binding as pk
+    ck = pin.config_tiny()
+    g = ck.geom
+    st = staged(ck)
+    ctx.select_repair(st.select_args())
+    Dp = g.head_dim + 8
+    shape = (ck.n_pages, g.n_layers, g.page_tokens, g.n_kv_heads, Dp)
+    fill = pin.SENTINEL - 0x10000
+    k = torch.full(shape, fill, dtype=torch.int16, device=DEV)
+    v = torch.full(shape, fill, dtype=torch.int16, device=DEV)
+    s_head, s_tok = Dp, g.n_kv_heads * Dp
+    s_layer = g.page_tokens * s_tok
+    s_page = g.n_layers * s_layer
+    pool = pk.make_pool(k, v, ck.n_pages, (s_layer, s_page, s_tok, s_head))
+    ctx.restore(st.geom(), pool, [st.session()])
+    torch.cuda.synchronize()
+    _, sel = oracle_select(ck)
+    rc, k_ref, v_ref, _ = oracle_restore(ck, sel["reuse_idx"], sel["reuse_cnt"])
+    kk = k.permute(1, 0, 2, 3, 4)
+    check_pools(kk[..., :g.head_dim].contiguous(), v.permute(1, 0, 2, 3, 4)[..., :g.head_dim].contiguous(), k_ref, v_ref, g)
+    assert bool((k[..., g.head_dim:] == fill).all()) and bool((v[..., g.head_dim:] == fill).all())
+
+
+def test_tiny_from_pinned_host(ctx):
+    run_select_and_restore(ctx, pin.config_tiny(), host=True)
+
+
+@pytest.mark.parametrize("name", ["delta0", "shift5", "ragged_n1000", "k4v4", "all_dirty", "interleaved"])
+def test_tiny_variants_from_pinned_host(ctx, name):
+    kw = dict(TINY_VARIANTS[name])
+    kw.setdefault("n_pages", 256)
+    run_select_and_restore(ctx, pin.config_tiny(**kw), host=True)
+
+
+def test_host_restore_small_ring_and_no_merging():
+    c = new_context(staging_slots=1, merge_gap_bytes=0)
+    try:
+        st, sel, pools, _ = run_select_and_restore(c, pin.config_tiny(), host=True)
+        # twice in a row on the same context: the ring and the metadata arena are reused
+        run_select_and_restore(c, pin.config_tiny(seed=9), host=True)
+    finally:
+        c.close()
+
+
+def test_host_restore_stats_and_two_sessions(ctx):
+    a = pin.config_tiny(n_pages=256)
+    b = pin.config_tiny(seed=78, delta=-5, n=900, n_pages=256)
+    pin.shared_free_list(6, 256, [a, b])
+    sa, sb = staged(a, payload_on_host=True), staged(b, payload_on_host=True)
+    ctx.select_repair(sa.select_args())
+    ctx.select_repair(sb.select_args())
+    k, v, pool = gpu_pool(a)
+    rc, stats = ctx.restore_from_host(sa.geom(), pool, [sa.host_session(), sb.host_session()])
+    torch.cuda.synchronize()
+    assert ctx.query_status() == 0
+    _, sela = oracle_select(a)
+    _, selb = oracle_select(b)
+    rc, k_ref, v_ref, _ = oracle_restore(a, sela["reuse_idx"], sela["reuse_cnt"])
+    rc, k_ref, v_ref, _ = oracle_restore(b, selb["reuse_idx"], selb["reuse_cnt"], pools=(k_ref, v_ref))
+    check_pools(k, v, k_ref, v_ref, a.geom)
+    useful = 0
+    for ck, sel in ((a, sela), (b, selb)):
+        for l in range(2):
+            for j in sel["reuse_idx"][l, :sel["reuse_cnt"][l]]:
+                useful += pin.record_bytes(int(ck.tags[l, j]), ck.geom)
+    assert stats.bytes_useful == useful
+    assert stats.bytes_copied >= useful and stats.n_copies >= 4
+    assert stats.n_block_layers == int(sela["reuse_cnt"].sum() + selb["reuse_cnt"].sum())
+
+
+def test_llama8b_shape_full_size_sampled_layers(ctx):
+    """The benchmark configuration (32 layers, 16384-token suffix, device-resident payload): every layer is
+    restored on the GPU; sampled layers are compared in full, the rest by their untouched-page invariant."""
+    for delta in (-2048, 0, 2048, None):
+        ck = pin.config_llama8b(device=DEV, delta=delta)
+        st, sel, (k, v), frac = run_select_and_restore(ctx, ck, layers=[0, 17, 31], oracle_threads=0)
+        table = ck.block_table.cpu().numpy()
+        fill = pin.SENTINEL - 0x10000
+        for l in (5, 23):
+            R = sel["repair_idx"][l, :sel["repair_cnt"][l]]
+            untouched = np.setdiff1d(np.arange(ck.n_pages), table[np.setdiff1d(np.arange(1024), R)])
+            idx = torch.from_numpy(untouched).to(DEV)
+            assert bool((k[l, idx] == fill).all()) and bool((v[l, idx] == fill).all())
+            Fp = torch.from_numpy(table[sel["reuse_idx"][l, :sel["reuse_cnt"][l]]].astype(np.int64)).to(DEV)
+            assert not bool((v[l, Fp] == fill).all(dim=(1, 2, 3)).any())
+        del st, k, v
+        torch.cuda.empty_cache()
+
+
+def test_7b_shape_from_pinned_host_sampled_layers(ctx):
+    ck = pin.config_7b_host(device=DEV, pin_payload=True)
+    run_select_and_restore(ctx, ck, layers=[0, 11, 27], host=True)

@@ -1,0 +1,145 @@
+"""GPU parity of patchkv_select_repair against the oracle: bit-exact masses, masks, lists and counts."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import patchkv_inputs as pin
+from gpu_common import DEV, check_select, new_context, staged
+from helpers import oracle_select
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = new_context()
+    yield c
+    c.close()
+
+
+def _run(ctx, ck, **over):
+    st = staged(ck)
+    mass, sel = oracle_select(ck)
+    ctx.select_repair(st.select_args(**over))
+    check_select(st, sel, mass if ck.attn is not None else None)
+    assert ctx.query_status() == 0
+    return st, sel
+
+
+def test_tiny_from_attention(ctx):
+    st, sel = _run(ctx, pin.config_tiny())
+    assert list(sel["reuse_cnt"]) == [56, 56]
+
+
+@pytest.mark.parametrize("n,B,d_hat,k", [(1000, 16, 90, 2), (1024, 32, 64, 3), (1024, 8, 0, 5), (1019, 24, 100, 4),
+                                         (1024, 16, -5, 0), (1024, 16, 5000, 3), (1024, 16, 90, 1000), (7, 16, 0, 1),
+                                         (1024, 20, 33, 6)])
+def test_attention_shapes_and_edge_parameters(ctx, n, B, d_hat, k):
+    ck = pin.config_tiny(n=n, dirty_tokens=d_hat, top_k=k, n_pages=512)
+    # the selection block size is independent of the payload geometry: only select is exercised here
+    ck.geom = pin.Geometry(2, 4, 64, 64, pin.ROPE_HALF, 1e4, B, 16, 32)
+    st = staged(ck)
+    rc, mass = oracle.block_mass(ck.attn.numpy(), B)
+    sel = oracle.select(mass, n, B, d_hat, k)
+    ctx.select_repair(st.select_args())
+    check_select(st, sel, mass)
+
+
+def test_layers_shared(ctx):
+    _run(ctx, pin.config_tiny(layer_mode=pin.LAYERS_SHARED, top_k=5))
+
+
+def test_strided_and_unaligned_attention_uses_the_general_kernel(ctx):
+    ck = pin.config_tiny()
+    st = staged(ck)
+    big = torch.zeros((2, 8, 16, 1024 + 3), dtype=torch.float16, device=DEV)
+    big[..., 3:] = st.attn
+    view = big[..., 3:]                  # rows start 6 bytes past a 16-byte boundary
+    mass, sel = oracle_select(ck)
+    ctx.select_repair(st.select_args(attn=view))
+    check_select(st, sel, mass)
+    wide = torch.zeros((2, 16, 16, 1024), dtype=torch.float16, device=DEV)
+    wide[:, ::2] = st.attn
+    ctx.select_repair(st.select_args(attn=wide[:, ::2]))      # strided heads, still 16-byte aligned rows
+    check_select(st, sel, mass)
+
+
+def test_values_outside_the_unit_interval_and_bad_entries(ctx):
+    rng = np.random.default_rng(3)
+    bits = rng.integers(0, 0x7C00, size=(2, 3, 5, 512)).astype(np.uint16)     # whole finite fp16 range
+    attn = torch.from_numpy(bits.view(np.float16).copy())
+    g = pin.Geometry(2, 4, 64, 64, pin.ROPE_HALF, 1e4, 16, 16, 32)
+    ck = pin.config_tiny(n=512, geom=g)
+    ck.attn = attn
+    _run(ctx, ck)
+    bad = bits.copy()
+    bad[0, 0, 0, 3] = 0xBC00
+    bad[1, 1, 1, 40] = 0x7C00
+    bad[1, 2, 4, 41] = 0x7E00
+    bad[0, 0, 0, 4] = 0x8000
+    ck.attn = torch.from_numpy(bad.view(np.float16).copy())
+    st = staged(ck)
+    rc, mass = oracle.block_mass(bad, 16)
+    assert rc == oracle.E_BADINPUT
+    sel = oracle.select(mass, 512, 16, ck.dirty_tokens, ck.top_k)
+    ctx.select_repair(st.select_args())
+    check_select(st, sel, mass)
+    assert ctx.query_status() == -7
+    assert ctx.query_status() == 0          # the latch clears on read
+
+
+def test_ties_constant_mass_and_one_unit_difference(ctx):
+    ck = pin.config_llama8b(n_layers=2)
+    ck.mass = torch.full_like(ck.mass, 12345)
+    ck.mass[1, 700] += 1
+    st, sel = _run(ctx, ck)
+    assert 700 in sel["repair_idx"][1, :sel["repair_cnt"][1]]
+
+
+def test_zipf_masses_8b_shape_and_workspace_path(ctx):
+    ck = pin.config_llama8b(n_layers=4)
+    st, sel = _run(ctx, ck)
+    assert list(sel["repair_cnt"]) == [154] * 4 and list(sel["reuse_cnt"]) == [870] * 4
+    ck2 = pin.config_tiny()
+    _run(ctx, ck2, use_mass_out=False)      # masses kept in the context's workspace
+
+
+def test_many_blocks_many_ties(ctx):
+    g = pin.Geometry(3, 8, 128, 128, pin.ROPE_HALF, 5e5, 16, 16, 32)
+    rng = np.random.default_rng(4)
+    NB = 5000
+    mass = torch.from_numpy(rng.integers(0, 40, size=(3, NB)).astype(np.int64))
+    sel = oracle.select(mass.numpy().astype(np.uint64), NB * 16, 16, 333, 777)
+    ctxm = ctx
+    from paper_2609_26219_b200 import binding as pk
+    out = dict(repair_mask=torch.zeros((3, NB), dtype=torch.uint8, device=DEV),
+               repair_idx=torch.zeros((3, NB), dtype=torch.int32, device=DEV),
+               repair_cnt=torch.zeros(3, dtype=torch.int32, device=DEV),
+               reuse_idx=torch.zeros((3, NB), dtype=torch.int32, device=DEV),
+               reuse_cnt=torch.zeros(3, dtype=torch.int32, device=DEV))
+    md = mass.to(DEV)
+    a = pk.select_args(kind=pk.SCORE_BLOCK_MASS, n_layers=3, n_suffix_tokens=NB * 16, block_tokens=16,
+                       dirty_tokens=333, top_k=777, layer_mode=0, mass=md, **out)
+    ctxm.select_repair(a)
+    torch.cuda.synchronize()
+    assert np.array_equal(out["repair_idx"].cpu().numpy(), sel["repair_idx"])
+    assert np.array_equal(out["reuse_idx"].cpu().numpy(), sel["reuse_idx"])
+    assert np.array_equal(out["repair_mask"].cpu().numpy(), sel["mask"])
+
+
+def test_selection_at_scale_full_size_sampled_layers(ctx):
+    """Stored attention [32][32][64][16384] fp16 (2 GiB): masses and lists compared on sampled layers."""
+    ck = pin.config_select_scale(device=DEV, n_layers=32)   # payload of 32 layers is built too (1.4 GB)
+    st = staged(ck)
+    ctx.select_repair(st.select_args())
+    torch.cuda.synchronize()
+    assert ctx.query_status() == 0
+    for l in (0, 13, 31):
+        rc, mass = oracle.block_mass(ck.attn[l:l + 1].cpu().numpy(), 16)
+        assert rc == oracle.OK
+        assert np.array_equal(st.mass_out[l].cpu().numpy().astype(np.uint64), mass[0])
+        sel = oracle.select(mass, ck.n_suffix_tokens, 16, ck.dirty_tokens, ck.top_k)
+        assert np.array_equal(st.repair_idx[l].cpu().numpy(), sel["repair_idx"][0])
+        assert np.array_equal(st.reuse_idx[l].cpu().numpy(), sel["reuse_idx"][0])
+        assert int(st.reuse_cnt[l]) == 952 and int(st.repair_cnt[l]) == 72

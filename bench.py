@@ -1,0 +1,393 @@
+#!/usr/bin/env python
+"""Benchmark of the PatchKV suffix-restore hot path on B200.
+
+One step = one pass of the whole hot path over one batch of synthetic input: patchkv_select_repair (dirty
+window, top-k of stored block masses, union, lists) followed by patchkv_restore (dequantise by tag, RoPE
+phase correction of K, page placement) of every reused block, on the Llama-3-8B-shaped workload (32 layers,
+8 KV heads, head_dim 128, 16384-token suffix, 16-token blocks, tags 30/50/20 bf16/int8/int4, repair set
+15 %, device-resident payload, 1280-page pool).  Prints ONE JSON line (rank 0).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+value      restored KV GB/s (bf16-equivalent: bytes of bf16 K+V written to the pool / time), inputs in HBM.
+e2e        the same metric through the host-resident entry point: block masses copied from pinned host
+           memory, selection lists read back, patchkv_restore_from_host streaming the pinned payload.
+roofline   the restore kernel against the measured HBM copy bandwidth.
+cpu_baseline / --impl reference   the CPU checker in oracle/ timed on the machine's host cores (a reported
+           baseline only; it is a deliberately plain program).
+With N > 1 (torchrun) every rank restores its own copy of the workload on its own GPU: the path has no
+exchange step, so this is weak scaling without any data-path collective.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+import patchkv_inputs as pin
+
+METRIC = "restored_kv_gbps_bf16_equiv"
+UNIT = "GB/s"
+WORKLOAD = "llama3-8b-shaped: L=32 H=8 D=128 base=5e5 n=16384 B=P=16 G=32 tags 30/50/20 repair 15% device-resident"
+FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one restore_kernel launch on this workload, from the ncu
+# capture summarised in profiles/ (None until a capture exists)
+RESTORE_KERNEL_DRAM_TRAFFIC_BYTES = None
+
+
+# ------------------------------------------------------------------------------------------ helpers
+def algorithmic_bytes(ck: pin.SuffixCheckpoint, reuse_idx: np.ndarray, reuse_cnt: np.ndarray):
+    """(payload bytes read, bf16 bytes written, reused block-layers) of one restore of `ck`."""
+    g = ck.geom
+    tags = ck.tags.cpu().numpy()
+    rec = np.array([pin.record_bytes(t, g) for t in range(4)], dtype=np.int64)
+    read = 0
+    items = 0
+    for l in range(g.n_layers):
+        F = reuse_idx[l, :reuse_cnt[l]]
+        read += int(rec[tags[l, F]].sum())
+        items += len(F)
+    # every reused block writes B tokens of K and V in bf16 (the suffix here is a whole number of blocks)
+    written = items * 2 * g.block_tokens * g.n_kv_heads * g.head_dim * 2
+    return read, written, items
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.gpu_index), "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        rows = [l for (t, l) in self.lines if t0 - 0.05 <= t <= t1 + 0.25] or [l for (_, l) in self.lines]
+        for line in rows:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def measured_hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+def oracle_sample(ck: pin.SuffixCheckpoint, layers, repeats: int = 1):
+    """Time the CPU checker (select + restore) on `layers` of the workload.  Returns (seconds per pass,
+    bf16-equivalent bytes per pass, threads)."""
+    import oracle
+    g = ck.geom
+    L = len(layers)
+    mass = ck.mass.cpu().numpy().astype(np.uint64)[layers]
+    pay = ck.payload.cpu().numpy()
+    payloads = [pay[ck.layer_off[l]:ck.layer_off[l] + ck.layer_bytes[l]] for l in layers]
+    sub = pin.Geometry(L, g.n_kv_heads, g.head_dim, g.rotary_dim, g.rope_style, g.rope_base, g.block_tokens,
+                       g.page_tokens, g.group)
+    shape = (L, ck.n_pages, g.page_tokens, g.n_kv_heads, g.head_dim)
+    k = np.full(shape, pin.SENTINEL, dtype=np.uint16)
+    v = np.full(shape, pin.SENTINEL, dtype=np.uint16)
+    tags = ck.tags.cpu().numpy()[layers]
+    off = ck.blk_off.cpu().numpy()[layers]
+    table = ck.block_table.cpu().numpy()
+    threads = oracle.max_threads()
+    best, written = None, 0
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        sel = oracle.select(mass, ck.n_suffix_tokens, g.block_tokens, ck.dirty_tokens, ck.top_k, ck.layer_mode)
+        rc, _ = oracle.restore(L=L, H=g.n_kv_heads, D=g.head_dim, Dr=g.rotary_dim, rope_style=g.rope_style,
+                               rope_base=g.rope_base, B=g.block_tokens, P=g.page_tokens, G=g.group, k_pool=k,
+                               v_pool=v, strides=pin.pool_strides(sub, ck.n_pages), n_pages=ck.n_pages,
+                               n=ck.n_suffix_tokens, delta=ck.delta, dst_shift=ck.dst_shift, block_table=table,
+                               tags=tags, blk_off=off, layer_payload=payloads, reuse_idx=sel["reuse_idx"],
+                               reuse_cnt=sel["reuse_cnt"], n_threads=threads)
+        dt = time.perf_counter() - t0
+        assert rc == 0
+        best = dt if best is None else min(best, dt)
+        written = int(sel["reuse_cnt"].sum()) * 2 * g.block_tokens * g.n_kv_heads * g.head_dim * 2
+    return best, written, threads
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def max_over_ranks(x: float, world: int, device) -> float:
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def barrier(world: int):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+# ------------------------------------------------------------------------------------------ reference arm
+def run_reference(args):
+    """The CPU checker as the reference arm: each step is a bounded sample (2 layers of the 32) of the same
+    workload, select + restore, on all host cores.  Rank 0 only."""
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    sample_layers = [0, 1]
+    ck = pin.config_llama8b(device="cpu", n_layers=len(sample_layers))
+    times = []
+    written = 0
+    for i in range(args.warmup + args.steps):
+        dt, written, threads = oracle_sample(ck, list(range(len(sample_layers))))
+        if i >= args.warmup:
+            times.append(dt)
+    total = sum(times)
+    value = written * len(times) / total / 1e9
+    sample = f"{len(sample_layers)} of 32 layers per step (select + restore of 870 reused blocks per layer)"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------ our arm
+def pinned_copy_ceiling(device, nbytes=1 << 30, reps=10):
+    src = torch.empty(nbytes, dtype=torch.uint8).pin_memory()
+    dst = torch.empty(nbytes, dtype=torch.uint8, device=device)
+    best = None
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        dst.copy_(src, non_blocking=True)
+        e1.record()
+        e1.synchronize()
+        ms = e0.elapsed_time(e1)
+        best = ms if best is None else min(best, ms)
+    del src, dst
+    return nbytes / (best * 1e-3) / 1e9
+
+
+def run_ours(args):
+    rank, local_rank, world = dist_env()
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device(f"cuda:{local_rank}")
+
+    from paper_2609_26219_b200 import binding as pk
+    from paper_2609_26219_b200 import build as pkbuild
+    from paper_2609_26219_b200.harness import StagedCheckpoint, device_pool
+    if rank == 0:
+        pkbuild.build()
+    barrier(world)
+    ctx = pk.Context(device=local_rank)
+
+    # ---- inputs, resident in HBM before the timed region
+    ck = pin.config_llama8b(device=dev)
+    st = StagedCheckpoint(ck, dev)
+    k, v, pool = device_pool(ck, dev)
+    geom = st.geom()
+    sel_args = st.select_args()
+    sess = st.session()
+    stream = torch.cuda.current_stream()
+
+    def step(ev=None):
+        ctx.select_repair(sel_args, stream)
+        if ev:
+            ev[0].record(stream)
+        ctx.restore(geom, pool, [sess], stream)
+        if ev:
+            ev[1].record(stream)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    assert ctx.query_status() == 0
+    reuse_idx, reuse_cnt = st.reuse_idx.cpu().numpy(), st.reuse_cnt.cpu().numpy()
+    read_b, written_b, items = algorithmic_bytes(ck, reuse_idx, reuse_cnt)
+
+    # ---- timed region: K steps, CUDA events on the launching stream, clocks sampled alongside
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    e_begin, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier(world)
+    torch.cuda.synchronize()
+    t0 = time.time()
+    e_begin.record(stream)
+    for i in range(args.steps):
+        step(evs[i])
+    e_end.record(stream)
+    torch.cuda.synchronize()
+    barrier(world)
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1)
+    total_ms = max_over_ranks(e_begin.elapsed_time(e_end), world, dev)
+    restore_ms = [a.elapsed_time(b) for a, b in evs]
+    restore_avg_ms = sum(restore_ms) / len(restore_ms)
+    ms_per_step = total_ms / args.steps
+    select_us = 1e3 * (total_ms / args.steps - restore_avg_ms) if world == 1 else None
+    value = world * written_b / (ms_per_step * 1e-3) / 1e9
+    assert ctx.query_status() == 0
+
+    peak, peak_kind = measured_hbm_peak()
+    achieved = (read_b + written_b) / (restore_avg_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "restore_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_kind": f"of {peak_kind} copy bandwidth (burst)",
+                "frac_of_nominal_8tbs": achieved / 8000.0, "traffic": RESTORE_KERNEL_DRAM_TRAFFIC_BYTES,
+                "algorithmic_bytes_per_launch": read_b + written_b, "kernel_ms": restore_avg_ms}
+
+    # ---- end to end: host buffers, copies inside the timed region
+    e2e = None
+    host_link = None
+    if not args.no_e2e:
+        ceiling = pinned_copy_ceiling(dev)
+        hst = StagedCheckpoint(ck, dev, payload_on_host=True)
+        mass_host = ck.mass.cpu().pin_memory()
+        idx_host = torch.empty_like(hst.reuse_idx, device="cpu").pin_memory()
+        cnt_host = torch.empty_like(hst.reuse_cnt, device="cpu").pin_memory()
+        hsel = hst.select_args()
+        hs = hst.host_session(reuse_idx=idx_host, reuse_cnt=cnt_host)
+        dir_bytes = ck.tags.numel() + ck.blk_off.numel() * 8 + idx_host.numel() * 4 + cnt_host.numel() * 4 + \
+            ck.block_table.numel() * 4 + 16 * ck.geom.n_layers
+        e2e_steps = max(3, min(args.steps, 10))
+        times, copied = [], 0
+        for i in range(3 + e2e_steps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            barrier(world)
+            a.record(stream)
+            hst.mass.copy_(mass_host, non_blocking=True)                 # stored block masses: host -> device
+            ctx.select_repair(hsel, stream)
+            idx_host.copy_(hst.reuse_idx, non_blocking=True)             # selection result: device -> host
+            cnt_host.copy_(hst.reuse_cnt, non_blocking=True)
+            stream.synchronize()                                          # the host planner needs the lists
+            rc, stats = ctx.restore_from_host(geom, pool, [hs], stream)
+            b.record(stream)
+            status = ctx.query_status()                                   # reads the device status word back
+            assert status == 0
+            if i >= 3:
+                times.append(max_over_ranks(a.elapsed_time(b), world, dev))
+                copied = stats.bytes_copied
+        e_ms = sum(times) / len(times)
+        e2e = {"value": world * written_b / (e_ms * 1e-3) / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": int(copied + mass_host.numel() * 8 + dir_bytes),
+               "d2h_bytes_per_step": int(idx_host.numel() * 4 + cnt_host.numel() * 4 + 4),
+               "ms_per_step": e_ms, "steps": len(times),
+               "path": "pinned masses H2D, select_repair, lists D2H, restore_from_host (pinned payload), status D2H"}
+        host_link = {"ceiling_gbps": ceiling, "ceiling": "1 GiB pinned cudaMemcpyAsync H2D, best of 10, same run",
+                     "payload_gbps": read_b / (e_ms * 1e-3) / 1e9, "frac": read_b / (e_ms * 1e-3) / 1e9 / ceiling,
+                     "bytes_copied": int(copied), "bytes_useful": int(read_b), "copies": int(stats.n_copies)}
+
+    # ---- CPU baseline: the checker, as it stands, on a bounded sample of the same workload (rank 0, N = 1)
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        import oracle
+        oracle.build()
+        sample_layers = list(range(0, 32, 4))
+        dt, wb, threads = oracle_sample(ck, sample_layers, repeats=2)
+        cpu_baseline = {"value": wb / dt / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
+                        "sample": f"{len(sample_layers)} of 32 layers (select + restore), best of 2, {dt:.2f} s"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "delta": ck.delta, "l2": "working set 3.0 GB per step >> 126 MB L2, no flush",
+                       "parallelism": f"independent replicas x{world}" if world > 1 else "1 gpu"},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": 2 * args.steps,
+            "roofline": roofline, "cpu_baseline": cpu_baseline,
+            "select_us": select_us, "restore_ms": restore_avg_ms,
+            "block_layers_per_s": world * items / (ms_per_step * 1e-3),
+            "real_gbps": world * (read_b + written_b) / (ms_per_step * 1e-3) / 1e9,
+            "host_link": host_link,
+        }
+        print(json.dumps(line), flush=True)
+    ctx.close()
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

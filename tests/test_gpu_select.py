@@ -22,7 +22,7 @@ def _run(ctx, ck, **over):
     st = staged(ck)
     mass, sel = oracle_select(ck)
     ctx.select_repair(st.select_args(**over))
-    check_select(st, sel, mass if ck.attn is not None else None)
+    check_select(st, sel, mass if (ck.attn is not None and over.get("use_mass_out", True)) else None)
     assert ctx.query_status() == 0
     return st, sel
 

@@ -246,7 +246,7 @@ def run_ours(args):
     ctx = pk.Context(device=local_rank)
 
     # ---- inputs, resident in HBM before the timed region
-    ck = pin.config_llama8b(device=dev)
+    ck = pin.config_llama8b(device=dev, n_layers=args.layers)
     st = StagedCheckpoint(ck, dev)
     k, v, pool = device_pool(ck, dev)
     geom = st.geom()
@@ -348,7 +348,7 @@ def run_ours(args):
     if rank == 0 and world == 1 and not args.no_cpu:
         import oracle
         oracle.build()
-        sample_layers = list(range(0, 32, 4))
+        sample_layers = list(range(0, ck.geom.n_layers, 4))
         dt, wb, threads = oracle_sample(ck, sample_layers, repeats=2)
         cpu_baseline = {"value": wb / dt / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
                         "sample": f"{len(sample_layers)} of 32 layers (select + restore), best of 2, {dt:.2f} s"}
@@ -358,7 +358,8 @@ def run_ours(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "delta": ck.delta, "l2": "working set 3.0 GB per step >> 126 MB L2, no flush",
+            "config": {"workload": WORKLOAD if args.layers == 32 else WORKLOAD + f" [PROFILING SLICE: {args.layers} layers]",
+                       "delta": ck.delta, "l2": "working set 3.0 GB per step >> 126 MB L2, no flush",
                        "parallelism": f"independent replicas x{world}" if world > 1 else "1 gpu"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": 2 * args.steps,
             "roofline": roofline, "cpu_baseline": cpu_baseline,
@@ -382,6 +383,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--layers", type=int, default=32,
+                    help="profiling only: fewer layers of the same workload (the bench line is quoted on 32)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

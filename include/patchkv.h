@@ -72,7 +72,7 @@ typedef enum {
     PATCHKV_E_CUDA = -2,        /* a CUDA runtime call failed; text in patchkv_last_error */
     PATCHKV_E_BOUNDS = -3,      /* device side: an item was out of range and was skipped */
     PATCHKV_E_NOMEM = -4,       /* workspace or staging allocation failed */
-    PATCHKV_E_TIMEOUT = -5,     /* reserved: a bounded device-side wait gave up */
+    PATCHKV_E_TIMEOUT = -5,     /* device side: a bounded wait inside a kernel gave up; the launch ended early */
     PATCHKV_E_UNSUPPORTED = -6, /* valid but outside the compiled kernels' geometry limits */
     PATCHKV_E_BADINPUT = -7     /* device side: stored attention held a negative, infinite or NaN entry */
 } patchkv_status;
@@ -89,6 +89,10 @@ enum { PATCHKV_LAYERS_INDEPENDENT = 0 /* one (R_l, F_l) per layer */, PATCHKV_LA
 enum { PATCHKV_SCORE_ATTN_F16 = 0 /* stored attention */, PATCHKV_SCORE_BLOCK_MASS = 1 /* stored per-block mass */ };
 
 enum {
+    PATCHKV_FLAG_DIRECT_LOADS = 1  /* restore with the plain-load kernel even where the bulk-copy pipeline applies */
+};
+
+enum {
     PATCHKV_MAX_SESSIONS = 8,      /* sessions per restore call */
     PATCHKV_MAX_ROTARY_DIM = 256,  /* rotary_dim <= 256 */
     PATCHKV_MAX_BLOCK_VECTORS = 2048 /* block_tokens * n_kv_heads <= 2048 */
@@ -98,7 +102,7 @@ typedef struct {
     uint32_t struct_size;
     int32_t device;            /* CUDA device ordinal */
     int32_t staging_slots;     /* restore_from_host: depth of the device staging ring (0 = 4) */
-    int32_t reserved;
+    int32_t flags;             /* PATCHKV_FLAG_* */
     uint64_t merge_gap_bytes;  /* restore_from_host: two reused records closer than this are fetched by one copy
                                   (the bytes between them are transferred and ignored); UINT64_MAX = default 64 KiB */
 } patchkv_config;
@@ -235,7 +239,7 @@ PATCHKV_API int patchkv_restore_from_host(patchkv_ctx* ctx, const patchkv_geom* 
                                           patchkv_restore_stats* stats);
 
 /* Synchronises the context's device work and returns in *device_status the first device-side error latched
- * since the last query (PATCHKV_OK, PATCHKV_E_BOUNDS or PATCHKV_E_BADINPUT), then clears it. */
+ * since the last query (PATCHKV_OK, PATCHKV_E_BOUNDS, PATCHKV_E_BADINPUT or PATCHKV_E_TIMEOUT), then clears it. */
 PATCHKV_API int patchkv_query_status(patchkv_ctx* ctx, int* device_status);
 
 /* Bytes of one block record for a tag under a geometry; 0 for an unknown tag. */

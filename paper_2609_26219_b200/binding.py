@@ -21,11 +21,12 @@ ROPE_HALF, ROPE_INTERLEAVED = 0, 1
 LAYERS_INDEPENDENT, LAYERS_SHARED = 0, 1
 SCORE_ATTN_F16, SCORE_BLOCK_MASS = 0, 1
 MAX_SESSIONS = 8
+FLAG_DIRECT_LOADS = 1
 
 
 class Config(C.Structure):
     _fields_ = [("struct_size", C.c_uint32), ("device", C.c_int32), ("staging_slots", C.c_int32),
-                ("reserved", C.c_int32), ("merge_gap_bytes", C.c_uint64)]
+                ("flags", C.c_int32), ("merge_gap_bytes", C.c_uint64)]
 
 
 class Geom(C.Structure):
@@ -132,9 +133,10 @@ def make_session(*, n_suffix_tokens, delta, dst_shift, block_table, tags, blk_of
 class Context:
     """Owns one patchkv_ctx.  Methods are the C entry points with the `patchkv_` prefix dropped."""
 
-    def __init__(self, device: int = 0, staging_slots: int = 0, merge_gap_bytes: Optional[int] = None):
+    def __init__(self, device: int = 0, staging_slots: int = 0, merge_gap_bytes: Optional[int] = None,
+                 flags: int = 0):
         self._h = C.c_void_p()
-        cfg = Config(C.sizeof(Config), device, staging_slots, 0,
+        cfg = Config(C.sizeof(Config), device, staging_slots, flags,
                      0xFFFFFFFFFFFFFFFF if merge_gap_bytes is None else merge_gap_bytes)
         rc = lib().patchkv_create(C.byref(self._h), C.byref(cfg))
         if rc != OK:

@@ -59,6 +59,8 @@ struct RestoreParams {
     // work: items are (session, layer in [layer_begin, layer_end), position r in the reuse list)
     int32_t n_sessions, layer_begin, layer_end, total_items;
     int32_t* status;        // device status word
+    // bulk-copy pipeline: tokens per staged unit, bytes of one stage's code / scale / offset areas, ring depth
+    int32_t unit_tokens, stage_code_bytes, stage_scale_bytes, stage_bytes, n_stages;
     SessionDev s[PATCHKV_MAX_SESSIONS];
     // cos / sin of delta * theta_i per session, fp32, built on the host in double
     float cs[PATCHKV_MAX_SESSIONS][2][PATCHKV_MAX_ROTARY_DIM / 2];
@@ -77,6 +79,8 @@ struct patchkv_ctx {
     int device = 0;
     int sm_count = 0;
     int staging_slots = 4;
+    int flags = 0;
+    int max_smem_optin = 0;
     uint64_t merge_gap = 64 * 1024;
     cudaStream_t copy_stream = nullptr, decode_stream = nullptr;
     cudaEvent_t ev_begin = nullptr, ev_done = nullptr;

@@ -14,8 +14,10 @@ extern "C" int patchkv_create(patchkv_ctx** out, const patchkv_config* cfg) {
     ctx->device = cfg->device;
     ctx->staging_slots = cfg->staging_slots > 0 ? cfg->staging_slots : 4;
     if (ctx->staging_slots > 64) ctx->staging_slots = 64;
+    ctx->flags = cfg->flags;
     ctx->merge_gap = cfg->merge_gap_bytes == UINT64_MAX ? 64 * 1024 : cfg->merge_gap_bytes;
     bool ok = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, cfg->device) == cudaSuccess;
+    ok = ok && cudaDeviceGetAttribute(&ctx->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, cfg->device) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&ctx->decode_stream, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&ctx->ev_begin, cudaEventDisableTiming) == cudaSuccess;

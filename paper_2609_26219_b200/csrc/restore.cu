@@ -268,6 +268,323 @@ restore_kernel(const __grid_constant__ RestoreParams p) {
     }
 }
 
+// ---------------------------------------------------------------- bulk-copy pipeline
+// One producer warp walks the work list, resolves the directory and the destination pages of each block a few
+// stages ahead, and stages the block's K and V sections (in units of a few tokens) into a shared-memory ring
+// with bulk asynchronous copies that complete on an mbarrier.  Eight consumer warps dequantise / rotate from
+// shared memory and write the bf16 rows to the pool with 128-bit stores.  Directory latency and HBM read
+// latency are hidden by the ring instead of by occupancy.  Every wait is bounded.
+constexpr int kPipeConsumers = 256;
+constexpr int kPipeThreads = kPipeConsumers + 32;
+constexpr int kMaxStages = 8;
+constexpr uint32_t kWaitLimit = 1u << 22;
+
+struct StageMeta { int32_t nvec, fmt, flags, session; };   // nvec < 0: no more work; flags bit0 = K section, bit1 = rotate
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false when the limit ran out (the abort flag is then raised) or another role aborted.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    for (uint32_t i = 0; i < kWaitLimit; i++) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (i > 32) __nanosleep(40);
+    }
+    *abort_flag = 1;
+    return false;
+}
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t a) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint2 lds64(uint32_t a) {
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t a) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint16_t lds16(uint32_t a) {
+    uint16_t v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(a));
+    return v;
+}
+
+template <int FMT>
+__device__ __forceinline__ Chunk lds_chunk(uint32_t codes, uint32_t scales, int vec, int D, int gpv, int c0, int g0) {
+    Chunk c;
+    c.w = make_uint4(0, 0, 0, 0);
+    c.s = 0;
+    const uint32_t e = (uint32_t)vec * D + c0;
+    if (FMT == FMT_BF16) {
+        c.w = lds128(codes + 2 * e);
+    } else if (FMT == FMT_INT8) {
+        const uint2 t = lds64(codes + e);
+        c.w.x = t.x; c.w.y = t.y;
+        c.s = lds16(scales + 2 * ((uint32_t)vec * gpv + g0));
+    } else {
+        c.w.x = lds32(codes + (e >> 1));
+        c.s = lds16(scales + 2 * ((uint32_t)vec * gpv + g0));
+    }
+    return c;
+}
+
+template <int FMT, bool INTER>
+__device__ __forceinline__ void consume_unit(const RestoreParams& p, uint32_t codes, uint32_t scales,
+                                             const long long* vec_off, int nvec, uint16_t* dst_base,
+                                             const ThreadMap& tm, int gpv, const float* tc, const float* ts, bool rotate) {
+    const bool hasB = tm.cB >= 0;
+    const bool rotA = rotate && tm.rotA, rotB = rotate && tm.rotB;
+#pragma unroll 2
+    for (int vec = tm.ty; vec < nvec; vec += tm.TY) {
+        const Chunk ca = lds_chunk<FMT>(codes, scales, vec, p.D, gpv, tm.cA, tm.gA);
+        Chunk cb = ca;
+        if (hasB) cb = lds_chunk<FMT>(codes, scales, vec, p.D, gpv, tm.cB, tm.gB);
+        uint16_t* d = dst_base + vec_off[vec];
+        uint4 oa = ca.w, ob = cb.w;
+        if (FMT != FMT_BF16 || rotA || rotB) {
+            float a[8], b[8];
+            chunk_to_f32<FMT>(ca, a);
+            chunk_to_f32<FMT>(cb, b);
+            if (!INTER) {
+                if (rotA) {
+#pragma unroll
+                    for (int i = 0; i < 8; i++) rotate_pair(a[i], b[i], tc[i], ts[i]);
+                }
+            } else {
+                if (rotA) {
+#pragma unroll
+                    for (int i = 0; i < 4; i++) rotate_pair(a[2 * i], a[2 * i + 1], tc[i], ts[i]);
+                }
+                if (rotB) {
+#pragma unroll
+                    for (int i = 0; i < 4; i++) rotate_pair(b[2 * i], b[2 * i + 1], tc[4 + i], ts[4 + i]);
+                }
+            }
+            if (FMT != FMT_BF16 || rotA) oa = pack8(a);      // a bf16 code that is not rotated is copied bit for bit
+            if (FMT != FMT_BF16 || rotB) ob = pack8(b);
+        }
+        *reinterpret_cast<uint4*>(d + tm.cA) = oa;
+        if (hasB) *reinterpret_cast<uint4*>(d + tm.cB) = ob;
+    }
+}
+
+template <bool INTER>
+__global__ void __launch_bounds__(kPipeThreads, 2)
+restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
+    extern __shared__ __align__(128) uint8_t ring[];
+    __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages];
+    __shared__ int abort_flag;
+
+    const int S = p.n_stages;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; s++) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], kPipeConsumers / 32); }
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const int off_scales = p.stage_code_bytes;
+    const int off_vec = off_scales + p.stage_scale_bytes;
+    const int off_meta = off_vec + 8 * p.unit_tokens * p.H;
+    volatile int* abortp = &abort_flag;
+
+    if (threadIdx.x < 32) {
+        // ================================================================ producer warp
+        const int lane = threadIdx.x;
+        const uint64_t elems = (uint64_t)p.B * p.H * p.D;
+        const uint32_t hd = (uint32_t)p.H * p.D;
+        uint32_t q = 0;
+        bool alive = true;
+        for (int item = blockIdx.x; alive && item < p.total_items; item += gridDim.x) {
+            int si = 0;
+#pragma unroll 1
+            for (int k = 1; k < p.n_sessions; k++) if (item >= p.s[k].item_begin) si = k;
+            const SessionDev& Sd = p.s[si];
+            const int local = item - Sd.item_begin;
+            const int l = p.layer_begin + local / Sd.nb;
+            const int r = local - (l - p.layer_begin) * Sd.nb;
+            if (r >= __ldg(Sd.reuse_cnt + l)) continue;
+            const int j = __ldg(Sd.reuse_idx + (size_t)l * Sd.nb + r);
+            bool bad = j < 0 || j >= Sd.nb;
+            int tag = 0, valid = 0;
+            const uint8_t* rec = nullptr;
+            if (!bad) {
+                tag = __ldg(Sd.tags + (size_t)l * Sd.nb + j);
+                const unsigned long long off = __ldg(Sd.blk_off + (size_t)l * Sd.nb + j);
+                const unsigned long long lbytes = __ldg(Sd.layer_bytes + l);
+                const uint8_t* base = reinterpret_cast<const uint8_t*>(
+                    static_cast<uintptr_t>(__ldg(reinterpret_cast<const unsigned long long*>(Sd.layer_payload) + l)));
+                const unsigned long long rb = record_bytes(tag, elems, p.G);
+                bad = rb == 0 || off > lbytes || rb > lbytes - off || base == nullptr ||
+                      ((reinterpret_cast<uintptr_t>(base) + off) & 15u) != 0;
+                rec = base + off;
+                valid = min(p.B, Sd.n - j * p.B);
+            }
+            if (!bad) {                                  // all destination pages are validated before any write
+                for (int t = lane; t < valid; t += 32) {
+                    const long long u = (long long)j * p.B + t + Sd.dst_shift;
+                    const long long lp = u / p.P;
+                    const int page = lp < Sd.n_table ? __ldg(Sd.block_table + lp) : -1;
+                    if (page < 0 || page >= p.n_pages) bad = true;
+                }
+            }
+            if (__any_sync(0xFFFFFFFFu, bad)) {
+                if (lane == 0) atomicCAS(p.status, 0, (int)PATCHKV_E_BOUNDS);
+                continue;
+            }
+            const int kf = k_format(tag), vf = v_format(tag);
+            const uint8_t* sec_codes[2];
+            const uint8_t* sec_scales[2];
+            sec_codes[0] = rec;
+            sec_scales[0] = sec_codes[0] + code_bytes(kf, elems);
+            sec_codes[1] = sec_scales[0] + scale_bytes(kf, elems, p.G);
+            sec_scales[1] = sec_codes[1] + code_bytes(vf, elems);
+#pragma unroll 1
+            for (int sec = 0; sec < 2 && alive; sec++) {
+                const int fmt = sec ? vf : kf;
+                const uint32_t ctok = (uint32_t)code_bytes(fmt, hd), stok = (uint32_t)scale_bytes(fmt, hd, p.G);
+#pragma unroll 1
+                for (int t0 = 0; t0 < valid; t0 += p.unit_tokens) {
+                    const int nt = min(p.unit_tokens, valid - t0);
+                    const int stage = q % S;
+                    // the verdict is made warp-uniform: the lanes meet again at __syncwarp below
+                    if (!__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], ((q / S) & 1) ^ 1, abortp))) { alive = false; break; }
+                    uint8_t* sp = ring + (size_t)stage * p.stage_bytes;
+                    long long* voff = reinterpret_cast<long long*>(sp + off_vec);
+                    for (int i = lane; i < nt * p.H; i += 32) {
+                        const int tt = i / p.H, h = i - tt * p.H;
+                        const long long u = (long long)j * p.B + t0 + tt + Sd.dst_shift;
+                        const long long lp = u / p.P;
+                        const int page = __ldg(Sd.block_table + lp);
+                        voff[i] = (long long)l * p.stride_layer + (long long)page * p.stride_page +
+                                  (u - lp * p.P) * p.stride_token + (long long)h * p.stride_head;
+                    }
+                    if (lane == 0) {
+                        StageMeta m;
+                        m.nvec = nt * p.H; m.fmt = fmt; m.session = si;
+                        m.flags = (sec == 0 ? 1 : 0) | ((sec == 0 && Sd.delta != 0) ? 2 : 0);
+                        *reinterpret_cast<StageMeta*>(sp + off_meta) = m;
+                    }
+                    __syncwarp();
+                    if (lane == 0) {
+                        const uint32_t cb = nt * ctok, sb = nt * stok;
+                        mbar_arrive_expect_tx(&full_bar[stage], cb + sb);
+                        bulk_g2s(sp, sec_codes[sec] + (size_t)t0 * ctok, cb, &full_bar[stage]);
+                        if (sb) bulk_g2s(sp + off_scales, sec_scales[sec] + (size_t)t0 * stok, sb, &full_bar[stage]);
+                    }
+                    q++;
+                }
+            }
+        }
+        if (alive) {                                     // tell the consumers that the work list is exhausted
+            const int stage = q % S;
+            if (__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], ((q / S) & 1) ^ 1, abortp))) {
+                if (lane == 0) {
+                    StageMeta m; m.nvec = -1; m.fmt = 0; m.flags = 0; m.session = 0;
+                    *reinterpret_cast<StageMeta*>(ring + (size_t)stage * p.stage_bytes + off_meta) = m;
+                    mbar_arrive(&full_bar[stage]);
+                }
+            } else alive = false;
+        }
+        if (!alive) {
+            // a wait gave up: before leaving, let the copies already issued land (bounded), so that no bulk copy
+            // is still writing this CTA's shared memory after it exits
+            const uint32_t issued = q < (uint32_t)S ? q : (uint32_t)S;
+            for (uint32_t k = 0; k < issued; k++) {
+                const uint32_t qq = q - 1 - k;
+                for (uint32_t i = 0; i < kWaitLimit; i++) {
+                    if (mbar_try_wait(&full_bar[qq % S], (qq / S) & 1)) break;
+                    __nanosleep(100);
+                }
+            }
+            if (lane == 0) atomicCAS(p.status, 0, (int)PATCHKV_E_TIMEOUT);
+        }
+    } else {
+        // ================================================================ consumer warps
+        const int c = threadIdx.x - 32;
+        ThreadMap tm;
+        const int TX = (p.D + 15) >> 4;
+        tm.TY = kPipeConsumers / TX;
+        const int tx = c % TX;
+        tm.ty = c / TX;
+        const bool lane_active = tm.ty < tm.TY;
+        if (!INTER) {
+            const int n_rot = p.Dr >> 4;
+            if (tx < n_rot) { tm.cA = 8 * tx; tm.cB = (p.Dr >> 1) + 8 * tx; tm.rotA = tm.rotB = true; tm.tab = 8 * tx; }
+            else { tm.cA = p.Dr + 16 * (tx - n_rot); tm.cB = tm.cA + 8; tm.rotA = tm.rotB = false; tm.tab = 0; }
+        } else {
+            tm.cA = 16 * tx; tm.cB = tm.cA + 8;
+            tm.rotA = tm.cA < p.Dr; tm.rotB = tm.cB < p.Dr; tm.tab = 0;
+        }
+        if (tm.cB >= p.D) { tm.cB = -1; if (INTER) tm.rotB = false; }
+        tm.gA = tm.cA / p.G;
+        tm.gB = tm.cB >= 0 ? tm.cB / p.G : 0;
+        const int gpv = p.D / p.G;
+        float tc[8], ts[8];
+        int cur_session = -1;
+        uint32_t q = 0;
+        while (true) {
+            const int stage = q % S;
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait(&full_bar[stage], (q / S) & 1, abortp))) break;
+            uint8_t* sp = ring + (size_t)stage * p.stage_bytes;
+            const StageMeta m = *reinterpret_cast<const StageMeta*>(sp + off_meta);
+            if (m.nvec < 0) break;
+            if (m.session != cur_session) {
+                cur_session = m.session;
+#pragma unroll
+                for (int i = 0; i < 8; i++) {
+                    int idx;
+                    if (!INTER) idx = tm.tab + i;
+                    else idx = (i < 4) ? (tm.cA >> 1) + i : ((tm.cB >= 0 ? tm.cB : 0) >> 1) + (i - 4);
+                    idx = min(idx, PATCHKV_MAX_ROTARY_DIM / 2 - 1);
+                    tc[i] = p.cs[cur_session][0][idx];
+                    ts[i] = p.cs[cur_session][1][idx];
+                }
+            }
+            if (lane_active) {
+                const uint32_t codes = smem_u32(sp), scales = codes + off_scales;
+                const long long* voff = reinterpret_cast<const long long*>(sp + off_vec);
+                uint16_t* dst = (m.flags & 1) ? p.k_base : p.v_base;
+                const bool rotate = (m.flags & 2) != 0;
+                switch (m.fmt) {
+                    case FMT_BF16: consume_unit<FMT_BF16, INTER>(p, codes, scales, voff, m.nvec, dst, tm, gpv, tc, ts, rotate); break;
+                    case FMT_INT8: consume_unit<FMT_INT8, INTER>(p, codes, scales, voff, m.nvec, dst, tm, gpv, tc, ts, rotate); break;
+                    default:       consume_unit<FMT_INT4, INTER>(p, codes, scales, voff, m.nvec, dst, tm, gpv, tc, ts, rotate); break;
+                }
+            }
+            __syncwarp();
+            if ((c & 31) == 0) mbar_arrive(&empty_bar[stage]);
+            q++;
+        }
+        if (c == 0 && *abortp) atomicCAS(p.status, 0, (int)PATCHKV_E_TIMEOUT);
+    }
+}
+
 // ---------------------------------------------------------------- host side
 void build_rope_table(const patchkv_geom* g, int delta, float* cos_out, float* sin_out) {
     const int half = g->rotary_dim / 2;
@@ -317,11 +634,47 @@ int fill_geometry(patchkv_ctx* ctx, const patchkv_geom* g, const patchkv_pool* p
     return PATCHKV_OK;
 }
 
+// Sizes the shared-memory ring for a geometry.  Returns false when the bulk-copy pipeline does not apply:
+// per-token code / scale runs that are not multiples of 16 bytes, or a token row too large for one stage.
+static bool plan_pipeline(const patchkv_ctx* ctx, RestoreParams* p) {
+    if (ctx->flags & PATCHKV_FLAG_DIRECT_LOADS) return false;
+    const long long hd = (long long)p->H * p->D;
+    if (hd % 32 != 0 || (hd / p->G) % 8 != 0) return false;
+    long long ut = 16384 / hd;                       // at most 32 KiB of bf16 codes per stage
+    if (ut > p->B) ut = p->B;
+    if (ut > 256 / p->H) ut = 256 / p->H;            // at most 256 (token, head) vectors per stage
+    if (ut < 1) return false;
+    p->unit_tokens = (int32_t)ut;
+    p->stage_code_bytes = (int32_t)(ut * hd * 2);
+    p->stage_scale_bytes = (int32_t)(ut * (hd / p->G) * 2);
+    const long long raw = (long long)p->stage_code_bytes + p->stage_scale_bytes + 8 * ut * p->H + 16;
+    p->stage_bytes = (int32_t)((raw + 127) / 128 * 128);
+    long long budget = ((long long)ctx->max_smem_optin - 2048) / 2;   // two CTAs per SM
+    if (budget > 112 * 1024) budget = 112 * 1024;
+    long long stages = budget / p->stage_bytes;
+    if (stages > kMaxStages) stages = kMaxStages;
+    if (stages < 2) return false;
+    p->n_stages = (int32_t)stages;
+    return true;
+}
+
 int launch_restore(patchkv_ctx* ctx, RestoreParams* p, cudaStream_t stream) {
     if (p->total_items <= 0) return PATCHKV_OK;
+    const bool inter = p->rope_style == PATCHKV_ROPE_INTERLEAVED;
+    if (plan_pipeline(ctx, p)) {
+        const int smem = p->n_stages * p->stage_bytes;
+        if (inter) PKV_CUDA(ctx, cudaFuncSetAttribute(restore_pipe_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        else PKV_CUDA(ctx, cudaFuncSetAttribute(restore_pipe_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        int grid = ctx->sm_count * 2;
+        if (grid > p->total_items) grid = p->total_items;
+        if (inter) restore_pipe_kernel<true><<<grid, kPipeThreads, smem, stream>>>(*p);
+        else restore_pipe_kernel<false><<<grid, kPipeThreads, smem, stream>>>(*p);
+        PKV_CUDA(ctx, cudaGetLastError());
+        return PATCHKV_OK;
+    }
     int grid = ctx->sm_count * kCtasPerSm;
     if (grid > p->total_items) grid = p->total_items;
-    if (p->rope_style == PATCHKV_ROPE_INTERLEAVED) restore_kernel<true><<<grid, kThreads, 0, stream>>>(*p);
+    if (inter) restore_kernel<true><<<grid, kThreads, 0, stream>>>(*p);
     else restore_kernel<false><<<grid, kThreads, 0, stream>>>(*p);
     PKV_CUDA(ctx, cudaGetLastError());
     return PATCHKV_OK;

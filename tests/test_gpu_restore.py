@@ -12,9 +12,11 @@ from helpers import np_u16, oracle_restore, oracle_select
 pytestmark = pytest.mark.gpu
 
 
-@pytest.fixture(scope="module")
-def ctx():
-    c = new_context()
+@pytest.fixture(scope="module", params=[0, 1], ids=["bulk_copy_pipeline", "direct_loads"])
+def ctx(request):
+    """Both restore kernels run every case: the shared-memory pipeline (where the geometry allows it) and the
+    plain-load kernel (PATCHKV_FLAG_DIRECT_LOADS)."""
+    c = new_context(flags=request.param)
     yield c
     c.close()
 

@@ -280,6 +280,12 @@ constexpr int kMaxStages = 8;
 constexpr uint32_t kWaitLimit = 1u << 22;
 
 struct StageMeta { int32_t nvec, fmt, flags, session; };   // nvec < 0: no more work; flags bit0 = K section, bit1 = rotate
+constexpr int kMaxItemPages = 8;                            // destination pages one block may touch in this kernel
+struct ItemDesc {                                           // one resolved, validated block (valid == 0: nothing to do)
+    const uint8_t* rec;
+    int32_t valid, tag, l, si, slot0;
+    int32_t pages[kMaxItemPages];
+};
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
@@ -356,7 +362,7 @@ __device__ __forceinline__ Chunk lds_chunk(uint32_t codes, uint32_t scales, int 
 
 template <int FMT, bool INTER>
 __device__ __forceinline__ void consume_unit(const RestoreParams& p, uint32_t codes, uint32_t scales,
-                                             const long long* vec_off, int nvec, uint16_t* dst_base,
+                                             uint32_t vec_off, int nvec, uint16_t* dst_base,
                                              const ThreadMap& tm, int gpv, const float* tc, const float* ts, bool rotate) {
     const bool hasB = tm.cB >= 0;
     const bool rotA = rotate && tm.rotA, rotB = rotate && tm.rotB;
@@ -365,7 +371,8 @@ __device__ __forceinline__ void consume_unit(const RestoreParams& p, uint32_t co
         const Chunk ca = lds_chunk<FMT>(codes, scales, vec, p.D, gpv, tm.cA, tm.gA);
         Chunk cb = ca;
         if (hasB) cb = lds_chunk<FMT>(codes, scales, vec, p.D, gpv, tm.cB, tm.gB);
-        uint16_t* d = dst_base + vec_off[vec];
+        const uint2 vo = lds64(vec_off + 8u * (uint32_t)vec);
+        uint16_t* d = dst_base + (long long)(((unsigned long long)vo.y << 32) | vo.x);
         uint4 oa = ca.w, ob = cb.w;
         if (FMT != FMT_BF16 || rotA || rotB) {
             float a[8], b[8];
@@ -400,6 +407,7 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
     extern __shared__ __align__(128) uint8_t ring[];
     __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages];
     __shared__ int abort_flag;
+    __shared__ ItemDesc descs[32];
 
     const int S = p.n_stages;
     if (threadIdx.x == 0) {
@@ -410,96 +418,116 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
     __syncthreads();
     const int off_scales = p.stage_code_bytes;
     const int off_vec = off_scales + p.stage_scale_bytes;
-    const int off_meta = off_vec + 8 * p.unit_tokens * p.H;
+    const int off_meta = (off_vec + 8 * p.unit_tokens * p.H + 15) & ~15;
     volatile int* abortp = &abort_flag;
 
     if (threadIdx.x < 32) {
         // ================================================================ producer warp
+        // Each lane resolves one upcoming block on its own (directory entry, record extent, destination pages),
+        // so the dependent global loads of 32 blocks overlap; the results are parked in shared memory and the
+        // warp then feeds the ring from them without touching global memory again.
         const int lane = threadIdx.x;
         const uint64_t elems = (uint64_t)p.B * p.H * p.D;
         const uint32_t hd = (uint32_t)p.H * p.D;
         uint32_t q = 0;
         bool alive = true;
-        for (int item = blockIdx.x; alive && item < p.total_items; item += gridDim.x) {
-            int si = 0;
 #pragma unroll 1
-            for (int k = 1; k < p.n_sessions; k++) if (item >= p.s[k].item_begin) si = k;
-            const SessionDev& Sd = p.s[si];
-            const int local = item - Sd.item_begin;
-            const int l = p.layer_begin + local / Sd.nb;
-            const int r = local - (l - p.layer_begin) * Sd.nb;
-            if (r >= __ldg(Sd.reuse_cnt + l)) continue;
-            const int j = __ldg(Sd.reuse_idx + (size_t)l * Sd.nb + r);
-            bool bad = j < 0 || j >= Sd.nb;
-            int tag = 0, valid = 0;
-            const uint8_t* rec = nullptr;
-            if (!bad) {
-                tag = __ldg(Sd.tags + (size_t)l * Sd.nb + j);
-                const unsigned long long off = __ldg(Sd.blk_off + (size_t)l * Sd.nb + j);
-                const unsigned long long lbytes = __ldg(Sd.layer_bytes + l);
-                const uint8_t* base = reinterpret_cast<const uint8_t*>(
-                    static_cast<uintptr_t>(__ldg(reinterpret_cast<const unsigned long long*>(Sd.layer_payload) + l)));
-                const unsigned long long rb = record_bytes(tag, elems, p.G);
-                bad = rb == 0 || off > lbytes || rb > lbytes - off || base == nullptr ||
-                      ((reinterpret_cast<uintptr_t>(base) + off) & 15u) != 0;
-                rec = base + off;
-                valid = min(p.B, Sd.n - j * p.B);
+        for (long long first = blockIdx.x; alive && first < p.total_items; first += 32ll * gridDim.x) {
+            {
+                ItemDesc d;
+                d.valid = 0;
+                const long long item = first + (long long)lane * gridDim.x;
+                if (item < p.total_items) {
+                    int si = 0;
+#pragma unroll 1
+                    for (int k = 1; k < p.n_sessions; k++) if (item >= p.s[k].item_begin) si = k;
+                    const SessionDev& Sd = p.s[si];
+                    const int local = (int)item - Sd.item_begin;
+                    const int l = p.layer_begin + local / Sd.nb;
+                    const int r = local - (l - p.layer_begin) * Sd.nb;
+                    if (r < __ldg(Sd.reuse_cnt + l)) {
+                        const int j = __ldg(Sd.reuse_idx + (size_t)l * Sd.nb + r);
+                        bool bad = j < 0 || j >= Sd.nb;
+                        if (!bad) {
+                            const int tag = __ldg(Sd.tags + (size_t)l * Sd.nb + j);
+                            const unsigned long long off = __ldg(Sd.blk_off + (size_t)l * Sd.nb + j);
+                            const unsigned long long lbytes = __ldg(Sd.layer_bytes + l);
+                            const uint8_t* base = reinterpret_cast<const uint8_t*>(static_cast<uintptr_t>(
+                                __ldg(reinterpret_cast<const unsigned long long*>(Sd.layer_payload) + l)));
+                            const unsigned long long rb = record_bytes(tag, elems, p.G);
+                            bad = rb == 0 || off > lbytes || rb > lbytes - off || base == nullptr ||
+                                  ((reinterpret_cast<uintptr_t>(base) + off) & 15u) != 0;
+                            const int valid = min(p.B, Sd.n - j * p.B);
+                            const long long u0 = (long long)j * p.B + Sd.dst_shift;
+                            const long long lp0 = u0 / p.P, lp1 = (u0 + valid - 1) / p.P;
+                            if (!bad) {                  // every destination page is validated before any write
+                                for (long long lp = lp0; lp <= lp1; lp++) {
+                                    const int page = lp < Sd.n_table ? __ldg(Sd.block_table + lp) : -1;
+                                    if (page < 0 || page >= p.n_pages) bad = true;
+                                    d.pages[lp - lp0] = page;
+                                }
+                            }
+                            d.rec = base + off;
+                            d.valid = valid; d.tag = tag; d.l = l; d.si = si;
+                            d.slot0 = (int)(u0 - lp0 * p.P);
+                        }
+                        if (bad) { d.valid = 0; atomicCAS(p.status, 0, (int)PATCHKV_E_BOUNDS); }
+                    }
+                }
+                descs[lane] = d;
             }
-            if (!bad) {                                  // all destination pages are validated before any write
-                for (int t = lane; t < valid; t += 32) {
-                    const long long u = (long long)j * p.B + t + Sd.dst_shift;
-                    const long long lp = u / p.P;
-                    const int page = lp < Sd.n_table ? __ldg(Sd.block_table + lp) : -1;
-                    if (page < 0 || page >= p.n_pages) bad = true;
+            __syncwarp();
+#pragma unroll 1
+            for (int di = 0; di < 32 && alive; di++) {
+                const ItemDesc& d = descs[di];
+                const int valid = d.valid;
+                if (valid == 0) continue;
+                const int tag = d.tag, l = d.l, si = d.si;
+                const int kf = k_format(tag), vf = v_format(tag);
+                const uint8_t* sec_codes[2];
+                const uint8_t* sec_scales[2];
+                sec_codes[0] = d.rec;
+                sec_scales[0] = sec_codes[0] + code_bytes(kf, elems);
+                sec_codes[1] = sec_scales[0] + scale_bytes(kf, elems, p.G);
+                sec_scales[1] = sec_codes[1] + code_bytes(vf, elems);
+                const bool shifted = p.s[si].delta != 0;
+#pragma unroll 1
+                for (int sec = 0; sec < 2 && alive; sec++) {
+                    const int fmt = sec ? vf : kf;
+                    const uint32_t ctok = (uint32_t)code_bytes(fmt, hd), stok = (uint32_t)scale_bytes(fmt, hd, p.G);
+#pragma unroll 1
+                    for (int t0 = 0; t0 < valid; t0 += p.unit_tokens) {
+                        const int nt = min(p.unit_tokens, valid - t0);
+                        const int stage = q % S;
+                        // the verdict is made warp-uniform: the lanes meet again at __syncwarp below
+                        if (!__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], ((q / S) & 1) ^ 1, abortp))) { alive = false; break; }
+                        uint8_t* sp = ring + (size_t)stage * p.stage_bytes;
+                        long long* voff = reinterpret_cast<long long*>(sp + off_vec);
+                        for (int i = lane; i < nt * p.H; i += 32) {
+                            const int tt = i / p.H, h = i - tt * p.H;
+                            const int us = d.slot0 + t0 + tt;               // slot counted from the first page
+                            const int pi = us / p.P;
+                            voff[i] = (long long)l * p.stride_layer + (long long)d.pages[pi] * p.stride_page +
+                                      (long long)(us - pi * p.P) * p.stride_token + (long long)h * p.stride_head;
+                        }
+                        if (lane == 0) {
+                            StageMeta m;
+                            m.nvec = nt * p.H; m.fmt = fmt; m.session = si;
+                            m.flags = (sec == 0 ? 1 : 0) | ((sec == 0 && shifted) ? 2 : 0);
+                            *reinterpret_cast<StageMeta*>(sp + off_meta) = m;
+                        }
+                        __syncwarp();
+                        if (lane == 0) {
+                            const uint32_t cb = nt * ctok, sb = nt * stok;
+                            mbar_arrive_expect_tx(&full_bar[stage], cb + sb);
+                            bulk_g2s(sp, sec_codes[sec] + (size_t)t0 * ctok, cb, &full_bar[stage]);
+                            if (sb) bulk_g2s(sp + off_scales, sec_scales[sec] + (size_t)t0 * stok, sb, &full_bar[stage]);
+                        }
+                        q++;
+                    }
                 }
             }
-            if (__any_sync(0xFFFFFFFFu, bad)) {
-                if (lane == 0) atomicCAS(p.status, 0, (int)PATCHKV_E_BOUNDS);
-                continue;
-            }
-            const int kf = k_format(tag), vf = v_format(tag);
-            const uint8_t* sec_codes[2];
-            const uint8_t* sec_scales[2];
-            sec_codes[0] = rec;
-            sec_scales[0] = sec_codes[0] + code_bytes(kf, elems);
-            sec_codes[1] = sec_scales[0] + scale_bytes(kf, elems, p.G);
-            sec_scales[1] = sec_codes[1] + code_bytes(vf, elems);
-#pragma unroll 1
-            for (int sec = 0; sec < 2 && alive; sec++) {
-                const int fmt = sec ? vf : kf;
-                const uint32_t ctok = (uint32_t)code_bytes(fmt, hd), stok = (uint32_t)scale_bytes(fmt, hd, p.G);
-#pragma unroll 1
-                for (int t0 = 0; t0 < valid; t0 += p.unit_tokens) {
-                    const int nt = min(p.unit_tokens, valid - t0);
-                    const int stage = q % S;
-                    // the verdict is made warp-uniform: the lanes meet again at __syncwarp below
-                    if (!__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], ((q / S) & 1) ^ 1, abortp))) { alive = false; break; }
-                    uint8_t* sp = ring + (size_t)stage * p.stage_bytes;
-                    long long* voff = reinterpret_cast<long long*>(sp + off_vec);
-                    for (int i = lane; i < nt * p.H; i += 32) {
-                        const int tt = i / p.H, h = i - tt * p.H;
-                        const long long u = (long long)j * p.B + t0 + tt + Sd.dst_shift;
-                        const long long lp = u / p.P;
-                        const int page = __ldg(Sd.block_table + lp);
-                        voff[i] = (long long)l * p.stride_layer + (long long)page * p.stride_page +
-                                  (u - lp * p.P) * p.stride_token + (long long)h * p.stride_head;
-                    }
-                    if (lane == 0) {
-                        StageMeta m;
-                        m.nvec = nt * p.H; m.fmt = fmt; m.session = si;
-                        m.flags = (sec == 0 ? 1 : 0) | ((sec == 0 && Sd.delta != 0) ? 2 : 0);
-                        *reinterpret_cast<StageMeta*>(sp + off_meta) = m;
-                    }
-                    __syncwarp();
-                    if (lane == 0) {
-                        const uint32_t cb = nt * ctok, sb = nt * stok;
-                        mbar_arrive_expect_tx(&full_bar[stage], cb + sb);
-                        bulk_g2s(sp, sec_codes[sec] + (size_t)t0 * ctok, cb, &full_bar[stage]);
-                        if (sb) bulk_g2s(sp + off_scales, sec_scales[sec] + (size_t)t0 * stok, sb, &full_bar[stage]);
-                    }
-                    q++;
-                }
-            }
+            __syncwarp();                                 // descs are rewritten by the next round
         }
         if (alive) {                                     // tell the consumers that the work list is exhausted
             const int stage = q % S;
@@ -552,7 +580,9 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
             const int stage = q % S;
             if (!__all_sync(0xFFFFFFFFu, mbar_wait(&full_bar[stage], (q / S) & 1, abortp))) break;
             uint8_t* sp = ring + (size_t)stage * p.stage_bytes;
-            const StageMeta m = *reinterpret_cast<const StageMeta*>(sp + off_meta);
+            const uint4 mw = lds128(smem_u32(sp) + off_meta);
+            StageMeta m;
+            m.nvec = (int)mw.x; m.fmt = (int)mw.y; m.flags = (int)mw.z; m.session = (int)mw.w;
             if (m.nvec < 0) break;
             if (m.session != cur_session) {
                 cur_session = m.session;
@@ -568,7 +598,7 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
             }
             if (lane_active) {
                 const uint32_t codes = smem_u32(sp), scales = codes + off_scales;
-                const long long* voff = reinterpret_cast<const long long*>(sp + off_vec);
+                const uint32_t voff = codes + off_vec;
                 uint16_t* dst = (m.flags & 1) ? p.k_base : p.v_base;
                 const bool rotate = (m.flags & 2) != 0;
                 switch (m.fmt) {
@@ -644,10 +674,11 @@ static bool plan_pipeline(const patchkv_ctx* ctx, RestoreParams* p) {
     if (ut > p->B) ut = p->B;
     if (ut > 256 / p->H) ut = 256 / p->H;            // at most 256 (token, head) vectors per stage
     if (ut < 1) return false;
+    if ((p->B + p->P - 2) / p->P + 1 > kMaxItemPages) return false;   // pages one block can straddle
     p->unit_tokens = (int32_t)ut;
     p->stage_code_bytes = (int32_t)(ut * hd * 2);
     p->stage_scale_bytes = (int32_t)(ut * (hd / p->G) * 2);
-    const long long raw = (long long)p->stage_code_bytes + p->stage_scale_bytes + 8 * ut * p->H + 16;
+    const long long raw = (long long)p->stage_code_bytes + p->stage_scale_bytes + 8 * ut * p->H + 32;
     p->stage_bytes = (int32_t)((raw + 127) / 128 * 128);
     long long budget = ((long long)ctx->max_smem_optin - 2048) / 2;   // two CTAs per SM
     if (budget > 112 * 1024) budget = 112 * 1024;

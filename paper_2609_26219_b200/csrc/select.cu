@@ -172,12 +172,15 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int* 
     return warp_sums[warp] + inc - v;
 }
 
+constexpr int kKeysPerThread = 8;      // candidate masses cached in registers: covers NB - n_dirty <= 8192
+
 __global__ void __launch_bounds__(kSelThreads)
 select_kernel(const TopkParams p) {
     __shared__ unsigned int hist[256];
     __shared__ int warp_sums[33];
     __shared__ unsigned long long s_prefix;
     __shared__ int s_krem;
+    __shared__ unsigned int s_or[2];
 
     const int l = blockIdx.x;
     const unsigned long long* key = p.mass + (p.shared ? 0 : (long long)l * p.NB);
@@ -185,31 +188,83 @@ select_kernel(const TopkParams p) {
     const int ncand = NB - n_dirty;
     const int k = min(p.top_k, ncand);
     const bool take_all = k == ncand, take_none = k == 0;
+    const int iters = (ncand + kSelThreads - 1) / kSelThreads;
+    const unsigned lane = threadIdx.x & 31u;
+
+    // candidate c = threadIdx.x + i * kSelThreads is block n_dirty + c; the first kKeysPerThread rounds live in registers
+    unsigned long long kreg[kKeysPerThread];
+#pragma unroll
+    for (int i = 0; i < kKeysPerThread; i++) {
+        const int c = threadIdx.x + i * kSelThreads;
+        kreg[i] = c < ncand ? key[n_dirty + c] : 0ull;
+    }
 
     unsigned long long T = 0;
     int krem = 0;
     if (!take_all && !take_none) {
-        // radix select: after the pass over byte b, `prefix` holds the top (8 - b) bytes of the k-th largest key
-        if (threadIdx.x == 0) { s_prefix = 0; s_krem = k; }
-        for (int b = 7; b >= 0; b--) {
+        // highest byte that is non-zero in any candidate: the passes above it would all pick digit 0
+        unsigned long long orv = 0;
+#pragma unroll
+        for (int i = 0; i < kKeysPerThread; i++) orv |= kreg[i];
+        for (int i = kKeysPerThread; i < iters; i++) {
+            const int c = threadIdx.x + i * kSelThreads;
+            if (c < ncand) orv |= key[n_dirty + c];
+        }
+        if (threadIdx.x == 0) { s_or[0] = 0; s_or[1] = 0; s_prefix = 0; s_krem = k; }
+        __syncthreads();
+        const unsigned lo = __reduce_or_sync(0xFFFFFFFFu, (unsigned)orv);
+        const unsigned hi = __reduce_or_sync(0xFFFFFFFFu, (unsigned)(orv >> 32));
+        if (lane == 0) { if (lo) atomicOr(&s_or[0], lo); if (hi) atomicOr(&s_or[1], hi); }
+        __syncthreads();
+        const unsigned long long all_or = ((unsigned long long)s_or[1] << 32) | s_or[0];
+        const int top_byte = all_or ? (63 - __clzll((long long)all_or)) >> 3 : -1;
+
+        // radix select, 8 bits per pass from the top: after the pass over byte b, `prefix` holds the bytes >= b of
+        // the k-th largest key and `krem` how many keys with that prefix are still to be taken
+        for (int b = top_byte; b >= 0; b--) {
             if (threadIdx.x < 256) hist[threadIdx.x] = 0;
             __syncthreads();
             const unsigned long long prefix = s_prefix;
-            for (int j = n_dirty + threadIdx.x; j < NB; j += kSelThreads) {
-                const unsigned long long x = key[j];
-                const bool match = b == 7 || ((x ^ prefix) >> (8 * (b + 1))) == 0;
-                if (match) atomicAdd(&hist[(unsigned)(x >> (8 * b)) & 255u], 1u);
+            const int need = s_krem;
+#pragma unroll
+            for (int i = 0; i < kKeysPerThread; i++) {
+                const int c = threadIdx.x + i * kSelThreads;
+                const unsigned long long x = kreg[i];
+                if (c < ncand && (b == 7 || ((x ^ prefix) >> (8 * (b + 1))) == 0))
+                    atomicAdd(&hist[(unsigned)(x >> (8 * b)) & 255u], 1u);
+            }
+            for (int i = kKeysPerThread; i < iters; i++) {
+                const int c = threadIdx.x + i * kSelThreads;
+                if (c < ncand) {
+                    const unsigned long long x = key[n_dirty + c];
+                    if (b == 7 || ((x ^ prefix) >> (8 * (b + 1))) == 0)
+                        atomicAdd(&hist[(unsigned)(x >> (8 * b)) & 255u], 1u);
+                }
             }
             __syncthreads();
-            if (threadIdx.x == 0) {
-                int need = s_krem, cum = 0, d = 255;
-                for (; d > 0; d--) {
-                    const int c = (int)hist[d];
-                    if (cum + c >= need) break;
-                    cum += c;
+            if (threadIdx.x < 32) {
+                // lane owns the 8 digits 255-8*lane ... 248-8*lane; a warp scan finds the digit where the running
+                // count from the top first reaches `need`
+                int cnt[8], sum = 0;
+#pragma unroll
+                for (int t = 0; t < 8; t++) { cnt[t] = (int)hist[255 - 8 * (int)lane - t]; sum += cnt[t]; }
+                int inc = sum;
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    const int o = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+                    if (lane >= (unsigned)d) inc += o;
                 }
-                s_prefix = prefix | ((unsigned long long)d << (8 * b));
-                s_krem = need - cum;             // how many keys with this digit (and prefix) are still to take
+                int cum = inc - sum;
+                if (cum < need && need <= inc) {
+#pragma unroll
+                    for (int t = 0; t < 8; t++) {
+                        if (cum < need && need <= cum + cnt[t]) {
+                            s_prefix = prefix | ((unsigned long long)(255 - 8 * (int)lane - t) << (8 * b));
+                            s_krem = need - cum;
+                        }
+                        cum += cnt[t];
+                    }
+                }
             }
             __syncthreads();
         }
@@ -217,36 +272,40 @@ select_kernel(const TopkParams p) {
         krem = s_krem;                           // keys equal to T to take, lowest block index first
     }
 
-    // ---- emit mask and ascending lists
-    int run_r = 0, run_eq = 0;
+    // ---- emit mask and ascending lists: the dirty window first, then the candidates in index order
     uint8_t* mask = p.mask + (long long)l * NB;
     int32_t* ridx = p.repair_idx + (long long)l * NB;
     int32_t* fidx = p.reuse_idx + (long long)l * NB;
-    for (int j0 = 0; j0 < NB; j0 += kSelThreads) {
-        const int j = j0 + threadIdx.x;
-        const bool in = j < NB;
-        const bool dirty = in && j < n_dirty;
-        const unsigned long long x = (in && !dirty) ? key[j] : 0;
-        const bool cand = in && !dirty;
-        bool sel = dirty;
+    for (int j = threadIdx.x; j < n_dirty; j += kSelThreads) { mask[j] = 1; ridx[j] = j; }
+    int run_sel = 0, run_eq = 0;
+    for (int i = 0; i < iters; i++) {
+        const int c = threadIdx.x + i * kSelThreads;
+        const bool in = c < ncand;
+        unsigned long long x = 0;
+        if (i < kKeysPerThread) {
+#pragma unroll
+            for (int t = 0; t < kKeysPerThread; t++) if (t == i) x = kreg[t];
+        } else if (in) x = key[n_dirty + c];
+        bool sel = false;
         if (take_all) sel = in;
         else if (!take_none) {
-            const int eq = cand && x == T;
+            const int eq = in && x == T;
             int tot_eq;
             const int rank = block_exclusive_scan(eq, warp_sums, &tot_eq) + run_eq;
             run_eq += tot_eq;
-            sel = dirty || (cand && x > T) || (eq && rank < krem);
+            sel = in && (x > T || (eq && rank < krem));
         }
-        int tot_r;
-        const int pos = block_exclusive_scan(sel ? 1 : 0, warp_sums, &tot_r) + run_r;
-        run_r += tot_r;
+        int tot_sel;
+        const int before = block_exclusive_scan(sel ? 1 : 0, warp_sums, &tot_sel) + run_sel;
+        run_sel += tot_sel;
         if (in) {
+            const int j = n_dirty + c;
             mask[j] = sel ? 1 : 0;
-            if (sel) ridx[pos] = j;
-            else fidx[j - pos] = j;
+            if (sel) ridx[n_dirty + before] = j;
+            else fidx[c - before] = j;
         }
     }
-    const int n_r = run_r, n_f = NB - run_r;
+    const int n_r = n_dirty + run_sel, n_f = NB - n_r;
     for (int i = n_r + threadIdx.x; i < NB; i += kSelThreads) ridx[i] = -1;
     for (int i = n_f + threadIdx.x; i < NB; i += kSelThreads) fidx[i] = -1;
     if (threadIdx.x == 0) { p.repair_cnt[l] = n_r; p.reuse_cnt[l] = n_f; }

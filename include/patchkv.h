@@ -74,7 +74,8 @@ typedef enum {
     PATCHKV_E_NOMEM = -4,       /* workspace or staging allocation failed */
     PATCHKV_E_TIMEOUT = -5,     /* device side: a bounded wait inside a kernel gave up; the launch ended early */
     PATCHKV_E_UNSUPPORTED = -6, /* valid but outside the compiled kernels' geometry limits */
-    PATCHKV_E_BADINPUT = -7     /* device side: stored attention held a negative, infinite or NaN entry */
+    PATCHKV_E_BADINPUT = -7,    /* device side: stored attention held a negative, infinite or NaN entry */
+    PATCHKV_E_TOO_LARGE = -8    /* patchkv_select_repair_static: the problem needs more than its fixed scratch */
 } patchkv_status;
 
 /* Per-block precision tags (the frozen policy pi_b of Section IV-D: FP16 | K8/V8 | K8/V4). */
@@ -95,7 +96,8 @@ enum {
 enum {
     PATCHKV_MAX_SESSIONS = 8,      /* sessions per restore call */
     PATCHKV_MAX_ROTARY_DIM = 256,  /* rotary_dim <= 256 */
-    PATCHKV_MAX_BLOCK_VECTORS = 2048 /* block_tokens * n_kv_heads <= 2048 */
+    PATCHKV_MAX_BLOCK_VECTORS = 2048, /* block_tokens * n_kv_heads <= 2048 */
+    PATCHKV_STATIC_MAX_MASS_ELEMS = 262144 /* u64 entries (2 MiB) of patchkv_select_repair_static's fixed scratch */
 };
 
 typedef struct {
@@ -219,6 +221,31 @@ PATCHKV_API int patchkv_last_error(patchkv_ctx* ctx, char* buf, size_t n);
  *   R_l = dirty u H_l and F_l = the rest, both ascending; unused list entries are set to -1.
  * Asynchronous on `stream`; all outputs are caller-allocated DEVICE arrays. */
 PATCHKV_API int patchkv_select_repair(patchkv_ctx* ctx, const patchkv_select_args* args, void* stream);
+
+/* The selection of patchkv_select_repair for callers that must not allocate device memory.  (The paper has no
+ * counterpart: this is a packaging variant of the same kernels, not another step of the method.)
+ *
+ * Who needs it: a serving engine that reserves nearly all of HBM for its KV pool at start-up, after which a
+ * cudaMalloc may simply fail; and a resume path that runs next to decode streams and cannot afford the
+ * device-wide stall that creating a context, or growing its workspace, brings.  This entry point takes no
+ * context and calls no cudaMalloc / cudaFree / allocating routine, now or later.  Its scratch -- the exact block
+ * masses (L*NB u64 when kind is ATTN_F16) and the layer-summed masses (NB u64 when layer_mode is
+ * LAYERS_SHARED) -- is a fixed array of PATCHKV_STATIC_MAX_MASS_ELEMS u64 inside the library image; each GPU
+ * that loads the library holds those 2 MiB until the process exits.
+ *
+ *   - Runs on the CURRENT device; every pointer in `args` is memory of that device.  Inputs and outputs are
+ *     the caller's, exactly as for patchkv_select_repair (mass_out, if given, receives a copy of the masses).
+ *   - A problem whose scratch need, (ATTN_F16 ? L*NB : 0) + (LAYERS_SHARED ? NB : 0), exceeds
+ *     PATCHKV_STATIC_MAX_MASS_ELEMS is refused with PATCHKV_E_TOO_LARGE and nothing is launched.
+ *   - The first call on each device looks up the device address of the array (a host-side query, no
+ *     allocation); make that first call outside any stream capture.
+ *   - All calls on a device share the one array, which keeps the previous call's contents; the part that must
+ *     start at zero is cleared on `stream` at each call.  Two calls whose work overlaps on the GPU (different
+ *     streams, or a second call before the first has finished on another stream) race on it: serialise them.
+ *   - `device_status` (DEVICE int32, optional, caller-zeroed) receives PATCHKV_E_BADINPUT if the stored
+ *     attention held a negative, infinite or NaN entry; with NULL that latch is dropped.
+ * Asynchronous on `stream`; results are bit-identical to patchkv_select_repair. */
+PATCHKV_API int patchkv_select_repair_static(const patchkv_select_args* args, void* stream, int32_t* device_status);
 
 /* Section IV-D fused restore (dequantise, Eq. 3 RoPE correction of K, page placement) of the reuse sets of
  * up to PATCHKV_MAX_SESSIONS sessions whose payloads are in device memory.  One kernel launch, asynchronous

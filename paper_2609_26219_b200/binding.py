@@ -16,6 +16,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libpatchkv.so")
 
 OK, E_INVALID, E_CUDA, E_BOUNDS, E_NOMEM, E_TIMEOUT, E_UNSUPPORTED, E_BADINPUT = 0, -1, -2, -3, -4, -5, -6, -7
+E_TOO_LARGE = -8
+STATIC_MAX_MASS_ELEMS = 262144
 TAG_BF16, TAG_INT8, TAG_INT4, TAG_K4V4 = 0, 1, 2, 3
 ROPE_HALF, ROPE_INTERLEAVED = 0, 1
 LAYERS_INDEPENDENT, LAYERS_SHARED = 0, 1
@@ -81,6 +83,8 @@ def lib():
         l.patchkv_destroy.argtypes = [C.c_void_p]
         l.patchkv_last_error.argtypes = [C.c_void_p, C.c_char_p, C.c_size_t]
         l.patchkv_select_repair.argtypes = [C.c_void_p, C.POINTER(SelectArgs), C.c_void_p]
+        l.patchkv_select_repair_static.argtypes = [C.POINTER(SelectArgs), C.c_void_p, C.c_void_p]
+        l.patchkv_select_repair_static.restype = C.c_int
         l.patchkv_restore.argtypes = [C.c_void_p, C.POINTER(Geom), C.POINTER(Pool), C.c_void_p, C.c_int, C.c_void_p]
         l.patchkv_restore_from_host.argtypes = [C.c_void_p, C.POINTER(Geom), C.POINTER(Pool), C.c_void_p, C.c_int,
                                                 C.c_void_p, C.POINTER(RestoreStats)]
@@ -181,6 +185,15 @@ class Context:
         if rc != OK:
             raise PatchKVError(rc, self.last_error())
         return v.value
+
+
+def select_repair_static(args: SelectArgs, stream=None, device_status: Optional[torch.Tensor] = None) -> int:
+    """patchkv_select_repair_static: the selection for callers that cannot allocate device memory (an engine
+    that has handed all of HBM to its KV pool, or a resume path that must not stall the device).  No context,
+    no allocation; scratch is a fixed 2 MiB array inside the library, shared by all calls on the device, so
+    calls must not overlap on the GPU.  Runs on the current device; returns the status code (E_TOO_LARGE when
+    the problem does not fit the fixed scratch).  `device_status`: optional zeroed int32 device tensor."""
+    return int(lib().patchkv_select_repair_static(C.byref(args), _stream_handle(stream), _ptr(device_status)))
 
 
 def record_bytes(tag: int, block_tokens: int, n_kv_heads: int, head_dim: int, group: int) -> int:

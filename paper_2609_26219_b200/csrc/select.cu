@@ -404,3 +404,118 @@ extern "C" int patchkv_select_repair(patchkv_ctx* ctx, const patchkv_select_args
     PKV_CUDA(ctx, cudaGetLastError());
     return PATCHKV_OK;
 }
+
+// ---------------------------------------------------------------- selection without any allocation
+// Scratch of patchkv_select_repair_static: block masses, the layer-summed masses of LAYERS_SHARED, and one
+// status word behind them.  It lives in the library image, so every GPU that loads the library holds these
+// ~2 MiB until the process exits, and every call on a device shares them.
+namespace patchkv {
+
+constexpr size_t kStaticMassElems = PATCHKV_STATIC_MAX_MASS_ELEMS;
+static __device__ __align__(256) unsigned long long g_static_scratch[kStaticMassElems + 32];
+
+constexpr int kMaxStaticDevices = 64;
+static unsigned long long* g_static_ptr[kMaxStaticDevices];   // device address of g_static_scratch, per device
+static std::mutex g_static_mu;
+
+// In host code `g_static_scratch` only names the symbol; the address a kernel can use has to be asked for,
+// once per device, while that device is current.
+static int static_scratch(unsigned long long** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxStaticDevices) return PATCHKV_E_CUDA;
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_ptr[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) {
+            cudaGetLastError();
+            return PATCHKV_E_CUDA;
+        }
+        g_static_ptr[dev] = static_cast<unsigned long long*>(ptr);
+    }
+    *out = g_static_ptr[dev];
+    return PATCHKV_OK;
+}
+
+}  // namespace patchkv
+
+extern "C" int patchkv_select_repair_static(const patchkv_select_args* a, void* stream_, int32_t* device_status) {
+    if (!a || a->struct_size != sizeof(patchkv_select_args)) return PATCHKV_E_INVALID;
+    if (a->n_layers <= 0 || a->n_suffix_tokens < 0 || a->block_tokens <= 0 || a->top_k < 0) return PATCHKV_E_INVALID;
+    if (a->layer_mode != PATCHKV_LAYERS_INDEPENDENT && a->layer_mode != PATCHKV_LAYERS_SHARED) return PATCHKV_E_INVALID;
+    if (a->kind != PATCHKV_SCORE_ATTN_F16 && a->kind != PATCHKV_SCORE_BLOCK_MASS) return PATCHKV_E_INVALID;
+    if (!a->repair_mask || !a->repair_idx || !a->repair_cnt || !a->reuse_idx || !a->reuse_cnt) return PATCHKV_E_INVALID;
+    const int L = a->n_layers, n = a->n_suffix_tokens, B = a->block_tokens;
+    const int NB = (int)(((long long)n + B - 1) / B);
+    long long nd = a->dirty_tokens < 0 ? 0 : a->dirty_tokens;
+    if (nd > n) nd = n;
+    const int n_dirty = (int)((nd + B - 1) / B);
+    const bool shared = a->layer_mode == PATCHKV_LAYERS_SHARED && L > 1;
+    const bool from_attn = a->kind == PATCHKV_SCORE_ATTN_F16;
+    // the fixed scratch must hold the block masses (when they are computed here) and the layer-summed masses
+    const unsigned long long need = (from_attn ? (unsigned long long)L * NB : 0ull) + (shared ? (unsigned long long)NB : 0ull);
+    if (need > kStaticMassElems) return PATCHKV_E_TOO_LARGE;
+    if (L > 65535) return PATCHKV_E_TOO_LARGE;
+
+    unsigned long long* scratch = nullptr;
+    int rc = static_scratch(&scratch);
+    if (rc != PATCHKV_OK) return rc;
+    int32_t* status = device_status ? device_status : reinterpret_cast<int32_t*>(scratch + kStaticMassElems);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+
+    const unsigned long long* mass = reinterpret_cast<const unsigned long long*>(a->mass);
+    unsigned long long* ws = scratch;
+    if (from_attn) {
+        if (a->n_q_heads < 0 || a->n_queries < 0 || (NB > 0 && a->n_q_heads > 0 && a->n_queries > 0 && !a->attn))
+            return PATCHKV_E_INVALID;
+        unsigned long long* m = ws;
+        ws += (size_t)L * NB;
+        const long long rows = (long long)a->n_q_heads * a->n_queries;
+        if (rows > 0x7fffffffLL) return PATCHKV_E_TOO_LARGE;
+        // the array keeps whatever the previous call left: the sums must start from zero
+        if (NB > 0 && cudaMemsetAsync(m, 0, (size_t)L * NB * sizeof(unsigned long long), stream) != cudaSuccess)
+            return PATCHKV_E_CUDA;
+        if (NB > 0 && rows > 0) {
+            MassParams mp;
+            mp.attn = static_cast<const uint16_t*>(a->attn);
+            mp.stride_layer = a->attn_stride_layer; mp.stride_head = a->attn_stride_head; mp.stride_query = a->attn_stride_query;
+            mp.Hq = a->n_q_heads; mp.Q = a->n_queries; mp.n = n; mp.B = B; mp.NB = NB;
+            mp.mass = m; mp.status = status;
+            const bool octet = (B % 8 == 0) && ((reinterpret_cast<uintptr_t>(a->attn) & 15u) == 0) &&
+                               ((a->attn_stride_layer | a->attn_stride_head | a->attn_stride_query) & 7) == 0;
+            const int cols = octet ? (n + 7) / 8 : n;
+            const int tiles = (cols + 255) / 256;
+            long long groups = 8192 / ((long long)tiles * L);       // about 8192 CTAs, at least 16 rows each
+            if (groups < 1) groups = 1;
+            long long rpc = (rows + groups - 1) / groups;
+            if (rpc < 16) rpc = 16;
+            if (rpc > rows) rpc = rows;
+            groups = (rows + rpc - 1) / rpc;
+            if (groups > 65535) return PATCHKV_E_TOO_LARGE;
+            mp.rows_per_cta = (int)rpc;
+            dim3 grid(tiles, (unsigned)groups, L);
+            if (octet) block_mass_octet_kernel<<<grid, 256, 0, stream>>>(mp);
+            else block_mass_generic_kernel<<<grid, 256, 0, stream>>>(mp);
+            if (cudaGetLastError() != cudaSuccess) return PATCHKV_E_CUDA;
+        }
+        if (a->mass_out && NB > 0 &&
+            cudaMemcpyAsync(a->mass_out, m, (size_t)L * NB * sizeof(unsigned long long), cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
+            return PATCHKV_E_CUDA;
+        mass = m;
+    } else if (NB > 0 && !mass) {
+        return PATCHKV_E_INVALID;
+    }
+
+    TopkParams tp;
+    tp.mass = mass; tp.shared = 0;
+    if (shared && NB > 0) {
+        sum_layers_kernel<<<(NB + 255) / 256, 256, 0, stream>>>(mass, L, NB, ws);
+        if (cudaGetLastError() != cudaSuccess) return PATCHKV_E_CUDA;
+        tp.mass = ws; tp.shared = 1;
+    }
+    tp.NB = NB; tp.n_dirty = n_dirty; tp.top_k = a->top_k;
+    tp.mask = a->repair_mask; tp.repair_idx = a->repair_idx; tp.repair_cnt = a->repair_cnt;
+    tp.reuse_idx = a->reuse_idx; tp.reuse_cnt = a->reuse_cnt;
+    select_kernel<<<L, kSelThreads, 0, stream>>>(tp);
+    if (cudaGetLastError() != cudaSuccess) return PATCHKV_E_CUDA;
+    return PATCHKV_OK;
+}

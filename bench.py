@@ -343,6 +343,42 @@ def run_ours(args):
                      "payload_gbps": read_b / (e_ms * 1e-3) / 1e9, "frac": read_b / (e_ms * 1e-3) / 1e9 / ceiling,
                      "bytes_copied": int(copied), "bytes_useful": int(read_b), "copies": int(stats.n_copies)}
 
+    # ---- selection at scale: stored attention [32][32][64][16384] fp16 (2 GiB) -> masses -> lists
+    select_scale = None
+    if not args.no_scale_select:
+        del st, k, v
+        torch.cuda.empty_cache()
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(1004)
+        SL = args.scale_layers
+        attn = pin.zipf_attention(gen, SL, 32, 64, 16384, dev)
+        NBs = 1024
+        out = dict(repair_mask=torch.empty((SL, NBs), dtype=torch.uint8, device=dev),
+                   repair_idx=torch.empty((SL, NBs), dtype=torch.int32, device=dev),
+                   repair_cnt=torch.empty(SL, dtype=torch.int32, device=dev),
+                   reuse_idx=torch.empty((SL, NBs), dtype=torch.int32, device=dev),
+                   reuse_cnt=torch.empty(SL, dtype=torch.int32, device=dev))
+        mass_out = torch.empty((SL, NBs), dtype=torch.int64, device=dev)
+        sa = pk.select_args(kind=pk.SCORE_ATTN_F16, n_layers=SL, n_suffix_tokens=16384, block_tokens=16,
+                            dirty_tokens=640, top_k=32, layer_mode=pk.LAYERS_INDEPENDENT, attn=attn,
+                            mass_out=mass_out, **out)
+        ts = []
+        for i in range(13):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            ctx.select_repair(sa, stream)
+            b.record(stream)
+            b.synchronize()
+            if i >= 3:
+                ts.append(a.elapsed_time(b))
+        assert ctx.query_status() == 0 and int(out["reuse_cnt"][0]) == 952
+        t_ms = statistics.median(ts)
+        nbytes = attn.numel() * 2
+        select_scale = {"workload": f"stored attention fp16 [{SL}][32][64][16384] ({SL * 64} MiB), 40-block dirty window, top-32 per layer",
+                        "select_us": 1e3 * t_ms, "attn_gbps": nbytes / (t_ms * 1e-3) / 1e9,
+                        "frac_of_hbm_peak": nbytes / (t_ms * 1e-3) / 1e9 / peak, "launches": 3}
+        del attn
+
     # ---- CPU baseline: the checker, as it stands, on a bounded sample of the same workload (rank 0, N = 1)
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu:
@@ -366,7 +402,7 @@ def run_ours(args):
             "select_us": select_us, "restore_ms": restore_avg_ms,
             "block_layers_per_s": world * items / (ms_per_step * 1e-3),
             "real_gbps": world * (read_b + written_b) / (ms_per_step * 1e-3) / 1e9,
-            "host_link": host_link,
+            "host_link": host_link, "select_at_scale": select_scale,
         }
         print(json.dumps(line), flush=True)
     ctx.close()
@@ -383,6 +419,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-scale-select", action="store_true")
+    ap.add_argument("--scale-layers", type=int, default=32, help="layers of the selection-at-scale leg (profiling: fewer)")
     ap.add_argument("--layers", type=int, default=32,
                     help="profiling only: fewer layers of the same workload (the bench line is quoted on 32)")
     args = ap.parse_args()

@@ -12,7 +12,7 @@
  *   2. patchkv_restore / patchkv_restore_from_host -- rebuild every block of F in one fused pass:
  *      dequantise it by its frozen per-block precision tag (Section IV-D, Eq. 14 gives the tags),
  *      correct the RoPE phase of K by the position delta, K_corr = R(rho) R(omega)^-1 K_old
- *      (Section II-B, Eq. 3; values are never rotated, Section IV-C), and write the rows straight
+ *      (Section II-B, Eq. 3; V gets no rotation, Section IV-C), and write the rows straight
  *      into the request's destination KV pages (Section IV-D, last paragraph).  Blocks of R are
  *      never read and never written: they belong to the recompute path.
  *
@@ -24,7 +24,7 @@
  *     enqueued on `stream` has completed.  The library owns only the context's workspace.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls are
  *     asynchronous with respect to the host unless stated otherwise; completion is stream order,
- *     which is how "decode starts only after both groups have been placed" (Section IV-C) is kept.
+ *     which is how the rule that decoding waits for every restored page (Section IV-C) is kept.
  *   - Device-side faults are never raised.  A work item whose directory entry, record extent or
  *     destination pages are out of range is skipped whole, the first such error is latched in the
  *     context's status word, and the rest of the call proceeds; see patchkv_query_status.
@@ -82,7 +82,7 @@ typedef enum {
 enum {
     PATCHKV_TAG_BF16 = 0, /* K bf16, V bf16 (the full-precision tier; this build stores bf16) */
     PATCHKV_TAG_INT8 = 1, /* K int8, V int8 */
-    PATCHKV_TAG_INT4 = 2, /* K int8, V int4 -- keys stay at 8 bits, only values enter the 4-bit tier */
+    PATCHKV_TAG_INT4 = 2, /* K int8, V int4 -- the low-bit tier of Section IV-D quantises V to 4 bits and leaves K at 8 */
     PATCHKV_TAG_K4V4 = 3  /* K int4, V int4 -- the uniform-INT4 ablation of Section V-C */
 };
 enum { PATCHKV_ROPE_HALF = 0 /* pairs (i, i + rotary_dim/2) */, PATCHKV_ROPE_INTERLEAVED = 1 /* pairs (2i, 2i+1) */ };

@@ -342,7 +342,7 @@ static int restore_item(const pkvo_restore_args* a, const float* ct, const float
         for (int h = 0; h < H; h++) {
             uint16_t* kd = a->k_pool + base + (int64_t)h * a->stride_head;
             uint16_t* vd = a->v_pool + base + (int64_t)h * a->stride_head;
-            /* V: dequantise and round once; a bf16 code is copied bit for bit; values are never rotated */
+            /* V: dequantise and round once; a bf16 code is copied bit for bit; V gets no rotation (Section IV-C) */
             for (int c = 0; c < D; c++) {
                 uint16_t rb; float v = dequant_elem(vc, vs, vf, H, D, G, t, h, c, &rb);
                 vd[c] = vf == PKVO_FMT_BF16 ? rb : pkvo_f32_to_bf16(v);

@@ -42,9 +42,10 @@ METRIC = "restored_kv_gbps_bf16_equiv"
 UNIT = "GB/s"
 WORKLOAD = "llama3-8b-shaped: L=32 H=8 D=128 base=5e5 n=16384 B=P=16 G=32 tags 30/50/20 repair 15% device-resident"
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one restore_kernel launch on this workload, from the ncu
-# capture summarised in profiles/ (None until a capture exists)
-RESTORE_KERNEL_DRAM_TRAFFIC_BYTES = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one restore launch on this workload, from the ncu capture of a
+# 4-layer slice summarised in profiles/restore_pipe_kernel_llama8b_slice.md: reads scale with the layers
+# (8 x 150.6 MB); writes are the algorithmic 1824 MB minus the ~54 MB still dirty in L2 when the kernel ends
+RESTORE_KERNEL_DRAM_TRAFFIC_BYTES = 2_975_000_000
 
 
 # ------------------------------------------------------------------------------------------ helpers
@@ -78,7 +79,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-i", str(self.gpu_index), "-lms", "100"],
+                                          "-i", str(self.gpu_index), "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -296,7 +297,7 @@ def run_ours(args):
 
     peak, peak_kind = measured_hbm_peak()
     achieved = (read_b + written_b) / (restore_avg_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "restore_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+    roofline = {"bound": "hbm", "kernel": "restore_pipe_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": f"of {peak_kind} copy bandwidth (burst)",
                 "frac_of_nominal_8tbs": achieved / 8000.0, "traffic": RESTORE_KERNEL_DRAM_TRAFFIC_BYTES,
                 "algorithmic_bytes_per_launch": read_b + written_b, "kernel_ms": restore_avg_ms}
@@ -414,7 +415,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=400)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")

@@ -42,8 +42,44 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
     return v;
 }
 
+// Exact running sum of one thread's octet over rows, in units of 2^-24.
+struct OctetSum {
+    unsigned long long acc = 0;
+    uint32_t acc32 = 0;
+    float facc = 0.0f;
+    int n32 = 0, nf = 0;
+    bool bad = false;
+
+    __device__ __forceinline__ void add(const uint4& w) {
+        const uint32_t any = w.x | w.y | w.z | w.w;
+        if ((any & 0xE000E000u) == 0) {
+            // every entry in [0, 2^-7): multiples of 2^-24 below 2^-7, so the eight add up exactly in fp32 (< 2^-4)
+            // and fifteen such rows still fit 24 bits (< 1): one float->int conversion per 15 rows
+            const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&w.x));
+            const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&w.y));
+            const float2 c = __half22float2(*reinterpret_cast<const __half2*>(&w.z));
+            const float2 d = __half22float2(*reinterpret_cast<const __half2*>(&w.w));
+            facc += ((a.x + a.y) + (b.x + b.y)) + ((c.x + c.y) + (d.x + d.y));
+            if (++nf == 15) { acc += __float2uint_rz(facc * 16777216.0f); facc = 0.0f; nf = 0; }
+        } else if ((any & 0xC000C000u) == 0) {                       // every entry in [0, 2)
+            acc32 += units2_fast(w.x) + units2_fast(w.y) + units2_fast(w.z) + units2_fast(w.w);
+            if (++n32 == 8) { acc += acc32; acc32 = 0; n32 = 0; }    // 8 * 8 * 2^25 = 2^31
+        } else {
+            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+            for (int i = 0; i < 4; i++) acc += units_any(ww[i], &bad) + units_any(ww[i] >> 16, &bad);
+        }
+    }
+    __device__ __forceinline__ unsigned long long total() const {
+        return acc + acc32 + __float2uint_rz(facc * 16777216.0f);
+    }
+};
+
+constexpr int kMassBatch = 8;      // rows whose loads are issued before any of them is consumed
+
 // One thread owns one octet (8 consecutive key positions, all in one block because B % 8 == 0) and walks the
-// rows (head, query) assigned to its CTA.  grid = (octet tiles, row groups, layers).
+// rows (head, query) assigned to its CTA, eight 128-bit loads in flight at a time.
+// grid = (octet tiles, row groups, layers).
 __global__ void __launch_bounds__(256)
 block_mass_octet_kernel(const MassParams p) {
     const int oct = blockIdx.x * blockDim.x + threadIdx.x;
@@ -55,39 +91,39 @@ block_mass_octet_kernel(const MassParams p) {
     const bool in_range = col < p.n;
     const int n_valid = in_range ? min(8, p.n - col) : 0;
 
-    unsigned long long acc = 0;
-    uint32_t acc32 = 0;
-    bool bad = false;
+    OctetSum sum;
     if (in_range) {
         const uint16_t* base = p.attn + (long long)l * p.stride_layer + col;
         int h = r0 / p.Q, q = r0 - h * p.Q;
-        const uint16_t* row = base + (long long)h * p.stride_head + (long long)q * p.stride_query;
-        int since_flush = 0;
-#pragma unroll 4
-        for (int r = r0; r < r1; r++) {
-            uint4 w;
-            if (n_valid == 8) w = ld_stream(reinterpret_cast<const uint4*>(row));
-            else {                                   // ragged last octet of a row: element loads, zero fill
+        if (n_valid == 8) {
+            for (int r = r0; r < r1; r += kMassBatch) {
+                uint4 w[kMassBatch];
+#pragma unroll
+                for (int i = 0; i < kMassBatch; i++) {
+                    w[i] = make_uint4(0, 0, 0, 0);              // a zero row adds nothing
+                    if (r + i < r1) {
+                        w[i] = __ldcs(reinterpret_cast<const uint4*>(base + (long long)h * p.stride_head +
+                                                                     (long long)q * p.stride_query));
+                        if (++q == p.Q) { q = 0; h++; }
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < kMassBatch; i++) sum.add(w[i]);
+            }
+        } else {                                                // ragged last octet of a row: element loads
+            for (int r = r0; r < r1; r++) {
+                const uint16_t* row = base + (long long)h * p.stride_head + (long long)q * p.stride_query;
                 uint16_t e[8];
 #pragma unroll
                 for (int i = 0; i < 8; i++) e[i] = i < n_valid ? __ldg(row + i) : (uint16_t)0;
-                w = make_uint4(e[0] | (uint32_t)e[1] << 16, e[2] | (uint32_t)e[3] << 16,
-                               e[4] | (uint32_t)e[5] << 16, e[6] | (uint32_t)e[7] << 16);
+                sum.add(make_uint4(e[0] | (uint32_t)e[1] << 16, e[2] | (uint32_t)e[3] << 16,
+                                   e[4] | (uint32_t)e[5] << 16, e[6] | (uint32_t)e[7] << 16));
+                if (++q == p.Q) { q = 0; h++; }
             }
-            if (((w.x | w.y | w.z | w.w) & 0xC000C000u) == 0) {          // every entry in [0, 2)
-                acc32 += units2_fast(w.x) + units2_fast(w.y) + units2_fast(w.z) + units2_fast(w.w);
-                if (++since_flush == 8) { acc += acc32; acc32 = 0; since_flush = 0; }   // 8 * 8 * 2^25 = 2^31
-            } else {
-                const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-                for (int i = 0; i < 4; i++) acc += units_any(ww[i], &bad) + units_any(ww[i] >> 16, &bad);
-            }
-            if (++q == p.Q) { q = 0; h++; row = base + (long long)h * p.stride_head; }
-            else row += p.stride_query;
         }
-        acc += acc32;
     }
-    if (bad) atomicCAS(p.status, 0, (int)PATCHKV_E_BADINPUT);
+    if (sum.bad) atomicCAS(p.status, 0, (int)PATCHKV_E_BADINPUT);
+    unsigned long long acc = sum.total();
 
     // segmented reduction over the octets of one block (segments are aligned groups of B/8 lanes)
     const int opb = p.B >> 3;

@@ -176,6 +176,11 @@ def max_over_ranks(x: float, world: int, device) -> float:
     return float(t.item())
 
 
+def aggregate_value(bytes_per_rank: float, ms: float, world: int) -> float:
+    """Whole-job GB/s when every rank moved bytes_per_rank in ms (the max over ranks)."""
+    return world * bytes_per_rank / (ms * 1e-3) / 1e9
+
+
 def barrier(world: int):
     if world > 1:
         import torch.distributed as dist
@@ -292,7 +297,7 @@ def run_ours(args):
     restore_avg_ms = sum(restore_ms) / len(restore_ms)
     ms_per_step = total_ms / args.steps
     select_us = 1e3 * (total_ms / args.steps - restore_avg_ms) if world == 1 else None
-    value = world * written_b / (ms_per_step * 1e-3) / 1e9
+    value = aggregate_value(written_b, ms_per_step, world)
     assert ctx.query_status() == 0
 
     peak, peak_kind = measured_hbm_peak()
@@ -347,7 +352,6 @@ def run_ours(args):
     # ---- selection at scale: stored attention [32][32][64][16384] fp16 (2 GiB) -> masses -> lists
     select_scale = None
     if not args.no_scale_select:
-        del st, k, v
         torch.cuda.empty_cache()
         gen = torch.Generator(device=dev)
         gen.manual_seed(1004)
@@ -380,6 +384,61 @@ def run_ours(args):
                         "frac_of_hbm_peak": nbytes / (t_ms * 1e-3) / 1e9 / peak, "launches": 3}
         del attn
 
+    # ---- the two host-resident workloads: 7B-shaped / 4 KV heads (one session), 70B-shaped stress (8 sessions)
+    host_cfg3 = stress = None
+    if not args.no_host_configs:
+        ceiling = pinned_copy_ceiling(dev)
+
+        def host_leg(cks, label, reps=5):
+            sts = [StagedCheckpoint(c, dev, payload_on_host=True) for c in cks]
+            for s_ in sts:
+                ctx.select_repair(s_.select_args(), stream)
+            torch.cuda.synchronize()
+            hk, hv, hpool = device_pool(cks[0], dev)
+            hgeom = sts[0].geom()
+            hss = [s_.host_session() for s_ in sts]
+            useful = written = items_h = 0
+            for c, s_ in zip(cks, sts):
+                r_, w_, i_ = algorithmic_bytes(c, s_.reuse_idx.cpu().numpy(), s_.reuse_cnt.cpu().numpy())
+                useful, written, items_h = useful + r_, written + w_, items_h + i_
+            ts_, stats_ = [], None
+            for i in range(2 + reps):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                a.record(stream)
+                rc_, stats_ = ctx.restore_from_host(hgeom, hpool, hss, stream)
+                b.record(stream)
+                b.synchronize()
+                if i >= 2:
+                    ts_.append(a.elapsed_time(b))
+            assert ctx.query_status() == 0 and stats_.bytes_useful == useful
+            t_ms = statistics.median(ts_)
+            out_ = {"workload": label, "ms": t_ms, "restored_kv_gbps_bf16_equiv": written / (t_ms * 1e-3) / 1e9,
+                    "payload_gbps": useful / (t_ms * 1e-3) / 1e9, "link_ceiling_gbps": ceiling,
+                    "frac_of_link": useful / (t_ms * 1e-3) / 1e9 / ceiling, "bytes_useful": int(useful),
+                    "bytes_copied": int(stats_.bytes_copied), "copies": int(stats_.n_copies),
+                    "block_layers": int(items_h), "block_layers_per_s": items_h / (t_ms * 1e-3)}
+            del sts, hk, hv, hss
+            torch.cuda.empty_cache()
+            return out_
+
+        try:
+            del st, k, v
+        except NameError:
+            pass
+        torch.cuda.empty_cache()
+        c3 = pin.config_7b_host(device=dev, pin_payload=True)
+        host_cfg3 = host_leg([c3], "7b-shaped: L=28 H=4 D=128 base=1e6 n=32768 delta=-3000, pinned host payload, "
+                                   "4096-page pool (2x), shuffled free list")
+        del c3
+        SLy = args.stress_layers
+        sess = [pin.config_stress_session(i, device=dev, n_layers=SLy, pin_payload=True) for i in range(8)]
+        pin.shared_free_list(1005, 8 * 4096, sess)
+        stress = host_leg(sess, f"70b-shaped stress: 8 sessions x 64k-token suffix, H=8 D=128, int4 share 10-60 %, "
+                                f"one shared pool of 32768 pages, pinned host payload; {SLy} of 80 layers resident "
+                                f"per wave (fit rule: the 80-layer pool is 172 GB)", reps=3)
+        del sess
+
     # ---- CPU baseline: the checker, as it stands, on a bounded sample of the same workload (rank 0, N = 1)
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu:
@@ -403,7 +462,7 @@ def run_ours(args):
             "select_us": select_us, "restore_ms": restore_avg_ms,
             "block_layers_per_s": world * items / (ms_per_step * 1e-3),
             "real_gbps": world * (read_b + written_b) / (ms_per_step * 1e-3) / 1e9,
-            "host_link": host_link, "select_at_scale": select_scale,
+            "host_link": host_link, "select_at_scale": select_scale, "host_7b": host_cfg3, "stress": stress,
         }
         print(json.dumps(line), flush=True)
     ctx.close()
@@ -421,6 +480,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-scale-select", action="store_true")
+    ap.add_argument("--no-host-configs", action="store_true")
+    ap.add_argument("--stress-layers", type=int, default=10)
     ap.add_argument("--scale-layers", type=int, default=32, help="layers of the selection-at-scale leg (profiling: fewer)")
     ap.add_argument("--layers", type=int, default=32,
                     help="profiling only: fewer layers of the same workload (the bench line is quoted on 32)")

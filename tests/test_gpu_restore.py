@@ -267,3 +267,49 @@ def test_llama8b_shape_full_size_sampled_layers(ctx):
 def test_7b_shape_from_pinned_host_sampled_layers(ctx):
     ck = pin.config_7b_host(device=DEV, pin_payload=True)
     run_select_and_restore(ctx, ck, layers=[0, 11, 27], host=True)
+
+
+def _stress_sessions(n_layers, n, n_sessions=8):
+    nb = -(-n // 16)
+    sess = [pin.config_stress_session(i, device=DEV, n_layers=n_layers, n=n, n_pages=nb, pin_payload=True,
+                                      dirty_tokens=min(5760, n // 8), top_k=min(254, nb // 16))
+            for i in range(n_sessions)]
+    pin.shared_free_list(1005, n_sessions * nb, sess)
+    return sess
+
+
+def _run_stress(ctx, sess, check_sessions, check_layers):
+    sts = [staged(c, payload_on_host=True) for c in sess]
+    for s in sts:
+        ctx.select_repair(s.select_args())
+    torch.cuda.synchronize()
+    k, v, pool = gpu_pool(sess[0])
+    rc, stats = ctx.restore_from_host(sts[0].geom(), pool, [s.host_session() for s in sts])
+    torch.cuda.synchronize()
+    assert ctx.query_status() == 0
+    sels = [oracle_select(c)[1] for c in sess]
+    for s, sel in zip(sts, sels):
+        assert np.array_equal(s.reuse_idx.cpu().numpy(), sel["reuse_idx"])
+    # the oracle restores every session into one shared pool (sampled layers), like the library did
+    k_ref = v_ref = None
+    for c, sel in zip(sess, sels):
+        pools = None if k_ref is None else (k_ref, v_ref)
+        rc, k_ref, v_ref, _ = oracle_restore(c, sel["reuse_idx"], sel["reuse_cnt"], layers=check_layers, pools=pools)
+        assert rc == oracle.OK
+    check_pools(k[check_layers], v[check_layers], k_ref, v_ref, sess[0].geom)
+    assert stats.n_block_layers == sum(int(sel["reuse_cnt"].sum()) for sel in sels)
+    return stats
+
+
+def test_stress_shape_eight_sessions_reduced_suffix(ctx):
+    """70B-shaped geometry, 8 concurrent sessions with their own delta and tag mix, interleaved pages of one
+    shared pool, payloads in pinned host memory; 4096-token suffixes, 3 layers, compared in full."""
+    sess = _stress_sessions(n_layers=3, n=4096)
+    assert len({c.delta for c in sess}) == 8
+    _run_stress(ctx, sess, range(8), [0, 1, 2])
+
+
+def test_stress_shape_full_suffix_one_layer(ctx):
+    """The same at the full 64k-token suffix per session (4096 blocks each, 32768 shared pages), one layer."""
+    sess = _stress_sessions(n_layers=1, n=65536)
+    _run_stress(ctx, sess, range(8), [0])

@@ -59,6 +59,7 @@ struct RestoreParams {
     // work: items are (session, layer in [layer_begin, layer_end), position r in the reuse list)
     int32_t n_sessions, layer_begin, layer_end, total_items;
     int32_t* status;        // device status word
+    int32_t* sched;         // work counter of this launch (zeroed on the stream right before it)
     // bulk-copy pipeline: tokens per staged unit, bytes of one stage's code / scale / offset areas, ring depth
     int32_t unit_tokens, stage_code_bytes, stage_scale_bytes, stage_bytes, n_stages;
     SessionDev s[PATCHKV_MAX_SESSIONS];
@@ -85,6 +86,8 @@ struct patchkv_ctx {
     cudaStream_t copy_stream = nullptr, decode_stream = nullptr;
     cudaEvent_t ev_begin = nullptr, ev_done = nullptr;
     int32_t* d_status = nullptr;
+    int32_t* d_sched = nullptr;     // ring of work counters, one per restore launch in flight
+    unsigned sched_seq = 0;
     // select workspace (block masses when the caller gives no mass_out; summed mass for LAYERS_SHARED)
     unsigned long long* d_mass_ws = nullptr;
     size_t mass_ws_elems = 0;
@@ -99,6 +102,8 @@ struct patchkv_ctx {
 };
 
 namespace patchkv {
+
+constexpr int kSchedSlots = 256;
 
 struct DeviceGuard {
     int prev = -1;

@@ -24,6 +24,7 @@ extern "C" int patchkv_create(patchkv_ctx** out, const patchkv_config* cfg) {
     ok = ok && cudaEventCreateWithFlags(&ctx->ev_done, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->d_status, sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMemset(ctx->d_status, 0, sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc(&ctx->d_sched, kSchedSlots * sizeof(int32_t)) == cudaSuccess;
     if (!ok) {
         patchkv_destroy(ctx);
         return PATCHKV_E_CUDA;
@@ -46,6 +47,7 @@ extern "C" int patchkv_destroy(patchkv_ctx* ctx) {
         if (ctx->h_meta) cudaFreeHost(ctx->h_meta);
         if (ctx->d_mass_ws) cudaFree(ctx->d_mass_ws);
         if (ctx->d_status) cudaFree(ctx->d_status);
+        if (ctx->d_sched) cudaFree(ctx->d_sched);
         if (ctx->ev_begin) cudaEventDestroy(ctx->ev_begin);
         if (ctx->ev_done) cudaEventDestroy(ctx->ev_done);
         if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);

@@ -431,13 +431,26 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
         const uint32_t hd = (uint32_t)p.H * p.D;
         uint32_t q = 0;
         bool alive = true;
+        // Work is handed out by a global counter in rounds that shrink towards the end of the list (a fraction of
+        // what is left per CTA, at most 32 blocks, at least one), so that CTAs with heavier tags do not leave a
+        // long tail; the blocks of a round are consecutive entries of one reuse list.
 #pragma unroll 1
-        for (long long first = blockIdx.x; alive && first < p.total_items; first += 32ll * gridDim.x) {
+        while (alive) {
+            long long first = 0;
+            int round = 0;
+            if (lane == 0) {
+                const long long left = (long long)p.total_items - *reinterpret_cast<volatile int*>(p.sched);
+                round = (int)max(1ll, min(32ll, left / (2ll * gridDim.x)));
+                first = atomicAdd(p.sched, round);
+            }
+            first = __shfl_sync(0xFFFFFFFFu, first, 0);
+            round = __shfl_sync(0xFFFFFFFFu, round, 0);
+            if (first >= p.total_items) break;
             {
                 ItemDesc d;
                 d.valid = 0;
-                const long long item = first + (long long)lane * gridDim.x;
-                if (item < p.total_items) {
+                const long long item = first + lane;
+                if (lane < round && item < p.total_items) {
                     int si = 0;
 #pragma unroll 1
                     for (int k = 1; k < p.n_sessions; k++) if (item >= p.s[k].item_begin) si = k;
@@ -698,6 +711,9 @@ int launch_restore(patchkv_ctx* ctx, RestoreParams* p, cudaStream_t stream) {
         else PKV_CUDA(ctx, cudaFuncSetAttribute(restore_pipe_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         int grid = ctx->sm_count * 2;
         if (grid > p->total_items) grid = p->total_items;
+        // each launch gets its own work counter from a small ring, zeroed in stream order just before it
+        p->sched = ctx->d_sched + (ctx->sched_seq++ % kSchedSlots);
+        PKV_CUDA(ctx, cudaMemsetAsync(p->sched, 0, sizeof(int32_t), stream));
         if (inter) restore_pipe_kernel<true><<<grid, kPipeThreads, smem, stream>>>(*p);
         else restore_pipe_kernel<false><<<grid, kPipeThreads, smem, stream>>>(*p);
         PKV_CUDA(ctx, cudaGetLastError());
@@ -743,7 +759,7 @@ extern "C" int patchkv_restore(patchkv_ctx* ctx, const patchkv_geom* geom, const
         d.n = s.n_suffix_tokens; d.nb = nb; d.delta = s.delta; d.dst_shift = s.dst_shift; d.n_table = s.n_table;
         d.item_begin = (int32_t)items;
         items += (long long)nb * geom->n_layers;
-        if (items > 0x7fffffffLL) return fail(ctx, PATCHKV_E_UNSUPPORTED, "restore: more than 2^31 work items");
+        if (items > 0x7fff0000LL) return fail(ctx, PATCHKV_E_UNSUPPORTED, "restore: more than 2^31 work items");
         build_rope_table(geom, s.delta, p.cs[i][0], p.cs[i][1]);
     }
     p.total_items = (int32_t)items;

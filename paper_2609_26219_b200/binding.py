@@ -148,8 +148,11 @@ class Context:
         self.device = device
 
     def close(self):
-        if getattr(self, "_h", None) and self._h.value:
-            lib().patchkv_destroy(self._h)
+        if getattr(self, "_h", None) and self._h.value and _lib is not None:
+            try:
+                _lib.patchkv_destroy(self._h)
+            except Exception:       # interpreter shutdown: the process is going away anyway
+                pass
             self._h = C.c_void_p()
 
     __del__ = close

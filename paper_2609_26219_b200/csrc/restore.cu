@@ -12,27 +12,6 @@ constexpr int kThreads = 256;
 constexpr int kCtasPerSm = 6;
 
 // ---------------------------------------------------------------- conversions
-// Four biased bytes -> four exact floats: byte b placed in the low mantissa byte of 2^23, minus (2^23 + bias).
-__device__ __forceinline__ void s8x4_to_f32(uint32_t w, float* o) {
-    const uint32_t x = w ^ 0x80808080u;      // two's complement -> offset binary
-    o[0] = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7650)) - 8388736.0f;
-    o[1] = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7651)) - 8388736.0f;
-    o[2] = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7652)) - 8388736.0f;
-    o[3] = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7653)) - 8388736.0f;
-}
-// Eight nibbles (channel 2k in the low nibble of byte k) -> eight exact floats in channel order.
-__device__ __forceinline__ void s4x8_to_f32(uint32_t w, float* o) {
-    const uint32_t x = w ^ 0x88888888u;
-    const uint32_t lo = x & 0x0F0F0F0Fu, hi = (x >> 4) & 0x0F0F0F0Fu;
-    o[0] = __uint_as_float(__byte_perm(lo, 0x4B000000u, 0x7650)) - 8388616.0f;
-    o[1] = __uint_as_float(__byte_perm(hi, 0x4B000000u, 0x7650)) - 8388616.0f;
-    o[2] = __uint_as_float(__byte_perm(lo, 0x4B000000u, 0x7651)) - 8388616.0f;
-    o[3] = __uint_as_float(__byte_perm(hi, 0x4B000000u, 0x7651)) - 8388616.0f;
-    o[4] = __uint_as_float(__byte_perm(lo, 0x4B000000u, 0x7652)) - 8388616.0f;
-    o[5] = __uint_as_float(__byte_perm(hi, 0x4B000000u, 0x7652)) - 8388616.0f;
-    o[6] = __uint_as_float(__byte_perm(lo, 0x4B000000u, 0x7653)) - 8388616.0f;
-    o[7] = __uint_as_float(__byte_perm(hi, 0x4B000000u, 0x7653)) - 8388616.0f;
-}
 __device__ __forceinline__ float fp16_bits_to_f32(uint16_t h) { return __half2float(__ushort_as_half(h)); }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -70,6 +49,32 @@ __device__ __forceinline__ Chunk load_chunk(const uint8_t* codes, const uint8_t*
     return c;
 }
 
+// Two fp32 lanes per instruction (sm_100 packed fp32): same IEEE result per lane as the scalar operation,
+// each lane rounded on its own, no fusion.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
+    f32x2 r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+    f32x2 r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) {
+    f32x2 r;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
 template <int FMT>
 __device__ __forceinline__ void chunk_to_f32(const Chunk& c, float* v) {
     if (FMT == FMT_BF16) {
@@ -78,11 +83,33 @@ __device__ __forceinline__ void chunk_to_f32(const Chunk& c, float* v) {
         v[4] = __uint_as_float(c.w.z << 16); v[5] = __uint_as_float(c.w.z & 0xFFFF0000u);
         v[6] = __uint_as_float(c.w.w << 16); v[7] = __uint_as_float(c.w.w & 0xFFFF0000u);
     } else {
-        if (FMT == FMT_INT8) { s8x4_to_f32(c.w.x, v); s8x4_to_f32(c.w.y, v + 4); }
-        else s4x8_to_f32(c.w.x, v);
+        // magic-number floats 2^23 + (code + bias); subtracting 2^23 + bias and multiplying by the scale are
+        // both exact (< 2^8 times an 11-bit significand), done two lanes at a time
+        uint32_t m[8];
+        float bias;
+        if (FMT == FMT_INT8) {
+            const uint32_t x = c.w.x ^ 0x80808080u, y = c.w.y ^ 0x80808080u;
+            m[0] = __byte_perm(x, 0x4B000000u, 0x7650); m[1] = __byte_perm(x, 0x4B000000u, 0x7651);
+            m[2] = __byte_perm(x, 0x4B000000u, 0x7652); m[3] = __byte_perm(x, 0x4B000000u, 0x7653);
+            m[4] = __byte_perm(y, 0x4B000000u, 0x7650); m[5] = __byte_perm(y, 0x4B000000u, 0x7651);
+            m[6] = __byte_perm(y, 0x4B000000u, 0x7652); m[7] = __byte_perm(y, 0x4B000000u, 0x7653);
+            bias = 8388736.0f;      // 2^23 + 128
+        } else {
+            const uint32_t x = c.w.x ^ 0x88888888u;
+            const uint32_t lo = x & 0x0F0F0F0Fu, hi = (x >> 4) & 0x0F0F0F0Fu;   // even / odd channels
+            m[0] = __byte_perm(lo, 0x4B000000u, 0x7650); m[1] = __byte_perm(hi, 0x4B000000u, 0x7650);
+            m[2] = __byte_perm(lo, 0x4B000000u, 0x7651); m[3] = __byte_perm(hi, 0x4B000000u, 0x7651);
+            m[4] = __byte_perm(lo, 0x4B000000u, 0x7652); m[5] = __byte_perm(hi, 0x4B000000u, 0x7652);
+            m[6] = __byte_perm(lo, 0x4B000000u, 0x7653); m[7] = __byte_perm(hi, 0x4B000000u, 0x7653);
+            bias = 8388616.0f;      // 2^23 + 8
+        }
         const float s = fp16_bits_to_f32(c.s);
+        const f32x2 b2 = pack2(bias, bias), s2 = pack2(s, s);
 #pragma unroll
-        for (int i = 0; i < 8; i++) v[i] = __fmul_rn(v[i], s);   // exact: < 2^8 times an 11-bit significand
+        for (int i = 0; i < 4; i++) {
+            const f32x2 q = sub2(pack2(__uint_as_float(m[2 * i]), __uint_as_float(m[2 * i + 1])), b2);
+            unpack2(mul2(q, s2), v[2 * i], v[2 * i + 1]);
+        }
     }
 }
 
@@ -91,6 +118,35 @@ __device__ __forceinline__ void rotate_pair(float& a, float& b, float c, float s
     const float ac = __fmul_rn(a, c), bs = __fmul_rn(b, s), as = __fmul_rn(a, s), bc = __fmul_rn(b, c);
     a = __fsub_rn(ac, bs);
     b = __fadd_rn(as, bc);
+}
+// The same for eight HALF-style pairs (a[i], b[i]) against (tc[i], ts[i]).  The four products of two pairs are
+// formed two lanes per instruction; the sum and the difference stay scalar __fadd_rn / __fsub_rn, which are
+// never merged with a multiply (packed add/sub were observed to be contracted with the products).
+__device__ __forceinline__ void rotate8_half(float* a, float* b, const float* tc, const float* ts) {
+#pragma unroll
+    for (int i = 0; i < 8; i += 2) {
+        const f32x2 A = pack2(a[i], a[i + 1]), B = pack2(b[i], b[i + 1]);
+        const f32x2 C = pack2(tc[i], tc[i + 1]), S = pack2(ts[i], ts[i + 1]);
+        float ac0, ac1, bs0, bs1, as0, as1, bc0, bc1;
+        unpack2(mul2(A, C), ac0, ac1);
+        unpack2(mul2(B, S), bs0, bs1);
+        unpack2(mul2(A, S), as0, as1);
+        unpack2(mul2(B, C), bc0, bc1);
+        a[i] = __fsub_rn(ac0, bs0); a[i + 1] = __fsub_rn(ac1, bs1);
+        b[i] = __fadd_rn(as0, bc0); b[i + 1] = __fadd_rn(as1, bc1);
+    }
+}
+// Four INTERLEAVED pairs (v[2i], v[2i+1]) against (tc[i], ts[i]).
+__device__ __forceinline__ void rotate4_interleaved(float* v, const float* tc, const float* ts) {
+#pragma unroll
+    for (int i = 0; i < 4; i++) {
+        const f32x2 X = pack2(v[2 * i], v[2 * i + 1]);
+        float xc, yc, xs, ys;
+        unpack2(mul2(X, pack2(tc[i], tc[i])), xc, yc);
+        unpack2(mul2(X, pack2(ts[i], ts[i])), xs, ys);
+        v[2 * i] = __fsub_rn(xc, ys);
+        v[2 * i + 1] = __fadd_rn(xs, yc);
+    }
 }
 
 // Which two 8-channel chunks of a head vector a thread owns, and how they rotate.
@@ -132,19 +188,10 @@ __device__ __forceinline__ void restore_vectors(const RestoreParams& p, const ui
             chunk_to_f32<KF>(ka, a);
             chunk_to_f32<KF>(kb, b);
             if (!INTER) {
-                if (rotA) {
-#pragma unroll
-                    for (int i = 0; i < 8; i++) rotate_pair(a[i], b[i], tc[i], ts[i]);
-                }
+                if (rotA) rotate8_half(a, b, tc, ts);
             } else {
-                if (rotA) {
-#pragma unroll
-                    for (int i = 0; i < 4; i++) rotate_pair(a[2 * i], a[2 * i + 1], tc[i], ts[i]);
-                }
-                if (rotB) {
-#pragma unroll
-                    for (int i = 0; i < 4; i++) rotate_pair(b[2 * i], b[2 * i + 1], tc[4 + i], ts[4 + i]);
-                }
+                if (rotA) rotate4_interleaved(a, tc, ts);
+                if (rotB) rotate4_interleaved(b, tc + 4, ts + 4);
             }
             // a bf16 code that is not rotated is copied bit for bit
             const uint4 oa = (KF == FMT_BF16 && !rotA) ? ka.w : pack8(a);
@@ -379,19 +426,10 @@ __device__ __forceinline__ void consume_unit(const RestoreParams& p, uint32_t co
             chunk_to_f32<FMT>(ca, a);
             chunk_to_f32<FMT>(cb, b);
             if (!INTER) {
-                if (rotA) {
-#pragma unroll
-                    for (int i = 0; i < 8; i++) rotate_pair(a[i], b[i], tc[i], ts[i]);
-                }
+                if (rotA) rotate8_half(a, b, tc, ts);
             } else {
-                if (rotA) {
-#pragma unroll
-                    for (int i = 0; i < 4; i++) rotate_pair(a[2 * i], a[2 * i + 1], tc[i], ts[i]);
-                }
-                if (rotB) {
-#pragma unroll
-                    for (int i = 0; i < 4; i++) rotate_pair(b[2 * i], b[2 * i + 1], tc[4 + i], ts[4 + i]);
-                }
+                if (rotA) rotate4_interleaved(a, tc, ts);
+                if (rotB) rotate4_interleaved(b, tc + 4, ts + 4);
             }
             if (FMT != FMT_BF16 || rotA) oa = pack8(a);      // a bf16 code that is not rotated is copied bit for bit
             if (FMT != FMT_BF16 || rotB) ob = pack8(b);

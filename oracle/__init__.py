@@ -48,6 +48,17 @@ class _RestoreArgs(C.Structure):
     ]
 
 
+class _GatherArgs(C.Structure):
+    _fields_ = [
+        ("L", C.c_int), ("H", C.c_int), ("D", C.c_int), ("B", C.c_int), ("P", C.c_int), ("G", C.c_int),
+        ("k_pool", C.c_void_p), ("v_pool", C.c_void_p),
+        ("stride_layer", C.c_int64), ("stride_page", C.c_int64), ("stride_token", C.c_int64), ("stride_head", C.c_int64),
+        ("n_pages", C.c_int), ("n", C.c_int), ("src_shift", C.c_int),
+        ("block_table", C.c_void_p), ("n_table", C.c_int),
+        ("tags", C.c_void_p), ("blk_off", C.c_void_p), ("layer_payload", C.c_void_p), ("layer_bytes", C.c_void_p),
+    ]
+
+
 def lib():
     global _lib
     if _lib is None:
@@ -84,6 +95,10 @@ def lib():
         l.pkvo_restore.restype = C.c_int
         l.pkvo_restore.argtypes = [C.POINTER(_RestoreArgs)]
         l.pkvo_max_threads.restype = C.c_int
+        l.pkvo_plan_checkpoint.restype = C.c_int
+        l.pkvo_plan_checkpoint.argtypes = [C.c_void_p] + [C.c_int] * 6 + [C.c_void_p, C.c_void_p]
+        l.pkvo_quantize_gather.restype = C.c_int
+        l.pkvo_quantize_gather.argtypes = [C.POINTER(_GatherArgs)]
         _lib = l
     return _lib
 
@@ -245,3 +260,35 @@ def restore(*, L, H, D, Dr, rope_style, rope_base, B, P, G, k_pool: np.ndarray, 
 
 def max_threads() -> int:
     return int(lib().pkvo_max_threads())
+
+
+# ---------------------------------------------------------------- checkpoint writer (offload side)
+def plan_checkpoint(tags: np.ndarray, B: int, H: int, D: int, G: int):
+    """tags u8 [L][NB] -> (status, blk_off u64 [L][NB], layer_bytes u64 [L]) of the clustered layout."""
+    tags = np.ascontiguousarray(tags, dtype=np.uint8)
+    L, NB = tags.shape
+    off = np.zeros((L, NB), dtype=np.uint64)
+    lb = np.zeros(L, dtype=np.uint64)
+    rc = lib().pkvo_plan_checkpoint(_p(tags), L, NB, B, H, D, G, _p(off), _p(lb))
+    return rc, off, lb
+
+
+def quantize_gather(*, L, H, D, B, P, G, k_pool: np.ndarray, v_pool: np.ndarray, strides: Sequence[int], n_pages: int,
+                    n: int, src_shift: int, block_table: np.ndarray, tags: np.ndarray, blk_off: np.ndarray,
+                    layer_payload: Sequence[np.ndarray]):
+    """Encode every block of every layer from the uint16 (bf16 bit pattern) pools into the per-layer uint8 buffers
+    `layer_payload` in place.  Returns the status."""
+    assert k_pool.dtype == np.uint16 and v_pool.dtype == np.uint16
+    NB = -(-n // B)
+    tags = np.ascontiguousarray(tags, dtype=np.uint8).reshape(L, NB)
+    blk_off = np.ascontiguousarray(blk_off).astype(np.uint64, copy=False).reshape(L, NB)
+    block_table = np.ascontiguousarray(block_table, dtype=np.int32)
+    for p_ in layer_payload:
+        assert p_.dtype == np.uint8 and p_.flags["C_CONTIGUOUS"]
+    ptrs = (C.c_void_p * L)(*[p_.ctypes.data if p_.size else None for p_ in layer_payload])
+    lbytes = np.array([p_.size for p_ in layer_payload], dtype=np.uint64)
+    a = _GatherArgs(L=L, H=H, D=D, B=B, P=P, G=G, k_pool=_p(k_pool), v_pool=_p(v_pool),
+                    stride_layer=strides[0], stride_page=strides[1], stride_token=strides[2], stride_head=strides[3],
+                    n_pages=n_pages, n=n, src_shift=src_shift, block_table=_p(block_table), n_table=block_table.size,
+                    tags=_p(tags), blk_off=_p(blk_off), layer_payload=C.cast(ptrs, C.c_void_p), layer_bytes=_p(lbytes))
+    return lib().pkvo_quantize_gather(C.byref(a))

@@ -421,3 +421,118 @@ int pkvo_max_threads(void) {
     return 1;
 #endif
 }
+
+/* ------------------------------------------------------------------ checkpoint writer (offload side) */
+/* Section IV-D, offload: gather the rows of each suffix block from the paged pool, compute per-group scales,
+ * pack the block at its precision tag, and cluster blocks of the same representation into contiguous runs.
+ * This is the inverse direction of restore; it is outside the resume path and is kept here as the oracle of
+ * the library's checkpoint writer. */
+
+/* Directory of the clustered layout: per layer all BF16-tag records, then INT8, INT4, K4V4, each run in
+ * ascending block index.  blk_off [L][NB], layer_bytes [L].  An unknown tag makes the call fail. */
+int pkvo_plan_checkpoint(const uint8_t* tags, int L, int NB, int B, int H, int D, int G,
+                         uint64_t* blk_off, uint64_t* layer_bytes) {
+    if (L <= 0 || NB < 0 || B <= 0 || H <= 0 || D <= 0 || G <= 0 || D % G) return PKVO_E_INVALID;
+    for (int l = 0; l < L; l++) {
+        uint64_t base = 0;
+        for (int tag = 0; tag <= PKVO_TAG_K4V4; tag++) {
+            uint64_t rec = pkvo_record_bytes(tag, B, H, D, G);
+            for (int j = 0; j < NB; j++)
+                if (tags[(int64_t)l * NB + j] == tag) { blk_off[(int64_t)l * NB + j] = base; base += rec; }
+        }
+        for (int j = 0; j < NB; j++) if (tags[(int64_t)l * NB + j] > PKVO_TAG_K4V4) return PKVO_E_INVALID;
+        layer_bytes[l] = base;
+    }
+    return PKVO_OK;
+}
+
+typedef struct {
+    int L, H, D, B, P, G;
+    const uint16_t* k_pool; const uint16_t* v_pool;         /* bf16 bit patterns */
+    int64_t stride_layer, stride_page, stride_token, stride_head;
+    int n_pages;
+    int n, src_shift;                                       /* suffix tokens; slot of the first one in logical page 0 */
+    const int32_t* block_table; int n_table;
+    const uint8_t* tags;                                    /* [L][NB] */
+    const uint64_t* blk_off;                                /* [L][NB] */
+    uint8_t* const* layer_payload;                          /* [L] destination buffers */
+    const uint64_t* layer_bytes;                            /* [L] */
+} pkvo_gather_args;
+
+/* Encode one section (K or V) of one block: values are the pool's bf16 rows read as fp32; tokens past the end of
+ * the suffix encode as zeros.  Quantiser: per group of G channels of one (token, head), s = fp16(amax / qmax),
+ * code = clamp(rint(x / s), -qmax, qmax) with ties to even, s == 0 -> code 0; qmax = 127 (int8) or 7 (int4). */
+static void encode_section(const pkvo_gather_args* a, const uint16_t* pool, int l, int j, int valid, int fmt,
+                           uint8_t* codes, uint8_t* scales) {
+    const int B = a->B, H = a->H, D = a->D, G = a->G, P = a->P;
+    float* x = (float*)malloc(sizeof(float) * (size_t)G);
+    int8_t* q = (int8_t*)malloc((size_t)G);
+    for (int t = 0; t < B; t++) {
+        int64_t u = (int64_t)j * B + t + a->src_shift;
+        const uint16_t* row = NULL;
+        if (t < valid)
+            row = pool + (int64_t)l * a->stride_layer + (int64_t)a->block_table[u / P] * a->stride_page +
+                  (u % P) * a->stride_token;
+        for (int h = 0; h < H; h++) {
+            const uint16_t* src = row ? row + (int64_t)h * a->stride_head : NULL;
+            uint64_t e0 = ((uint64_t)t * H + h) * D;
+            if (fmt == PKVO_FMT_BF16) {
+                for (int c = 0; c < D; c++) {
+                    uint16_t b = src ? src[c] : 0;
+                    memcpy(codes + 2 * (e0 + c), &b, 2);
+                }
+                continue;
+            }
+            for (int g = 0; g < D / G; g++) {
+                for (int i = 0; i < G; i++) x[i] = src ? pkvo_bf16_to_f32(src[g * G + i]) : 0.0f;
+                uint16_t sb;
+                pkvo_quantise_group(x, G, fmt == PKVO_FMT_INT8 ? 127 : 7, q, &sb);
+                memcpy(scales + 2 * (((uint64_t)t * H + h) * (D / G) + g), &sb, 2);
+                for (int i = 0; i < G; i++) {
+                    uint64_t e = e0 + (uint64_t)g * G + i;
+                    if (fmt == PKVO_FMT_INT8) codes[e] = (uint8_t)q[i];
+                    else {
+                        uint8_t nib = (uint8_t)q[i] & 15u;
+                        if (e & 1) codes[e >> 1] = (uint8_t)((codes[e >> 1] & 0x0f) | (nib << 4));
+                        else       codes[e >> 1] = (uint8_t)((codes[e >> 1] & 0xf0) | nib);
+                    }
+                }
+            }
+        }
+    }
+    free(x); free(q);
+}
+
+/* Write the record of every block of every layer.  A block whose tag, record extent or source pages are out of
+ * range is skipped whole (its bytes are left as they were) and the call returns PKVO_E_BOUNDS at the end. */
+int pkvo_quantize_gather(const pkvo_gather_args* a) {
+    if (a->L <= 0 || a->H <= 0 || a->D <= 0 || a->B <= 0 || a->P <= 0 || a->G <= 0 || a->D % a->G || a->n < 0 ||
+        a->src_shift < 0 || a->src_shift >= a->P)
+        return PKVO_E_INVALID;
+    const int NB = (a->n + a->B - 1) / a->B;
+    const uint64_t elems = (uint64_t)a->B * a->H * a->D;
+    int status = PKVO_OK;
+    for (int l = 0; l < a->L; l++)
+        for (int j = 0; j < NB; j++) {
+            int tag = a->tags[(int64_t)l * NB + j];
+            uint64_t rec = pkvo_record_bytes(tag, a->B, a->H, a->D, a->G);
+            uint64_t off = a->blk_off[(int64_t)l * NB + j];
+            int bad = rec == 0 || off > a->layer_bytes[l] || rec > a->layer_bytes[l] - off;
+            int valid = a->n - j * a->B < a->B ? a->n - j * a->B : a->B;
+            for (int t = 0; t < valid && !bad; t++) {
+                int64_t u = (int64_t)j * a->B + t + a->src_shift;
+                if (u / a->P >= a->n_table) { bad = 1; break; }
+                int32_t page = a->block_table[u / a->P];
+                if (page < 0 || page >= a->n_pages) bad = 1;
+            }
+            if (bad) { status = PKVO_E_BOUNDS; continue; }
+            const int kf = k_fmt(tag), vf = v_fmt(tag);
+            uint8_t* kc = a->layer_payload[l] + off;
+            uint8_t* ks = kc + codes_bytes(kf, elems);
+            uint8_t* vc = ks + scales_bytes(kf, elems, a->G);
+            uint8_t* vs = vc + codes_bytes(vf, elems);
+            encode_section(a, a->k_pool, l, j, valid, kf, kc, ks);
+            encode_section(a, a->v_pool, l, j, valid, vf, vc, vs);
+        }
+    return status;
+}

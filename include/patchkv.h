@@ -265,6 +265,29 @@ PATCHKV_API int patchkv_restore_from_host(patchkv_ctx* ctx, const patchkv_geom* 
                                           const patchkv_session_host* sessions, int n_sessions, void* stream,
                                           patchkv_restore_stats* stats);
 
+/* ---- checkpoint writer (offload side; not on the resume path) ----------------------------------------------
+ * Section IV-D: at offload a fused kernel gathers the rows of each suffix block, computes the scales and packs
+ * the payload at the block's calibrated precision; blocks of the same representation form contiguous runs.
+ *
+ * patchkv_plan_checkpoint fills the directory of that clustered layout from the tags: per layer all BF16-tag
+ * records, then INT8, INT4, K4V4, each run in ascending block index.
+ *   tags      DEVICE u8  [L][NB]  (in)      blk_off DEVICE u64 [L][NB] (out)     layer_bytes DEVICE u64 [L] (out)
+ * An unknown tag gets blk_off = UINT64_MAX (the writer then skips that block) and latches PATCHKV_E_BOUNDS. */
+PATCHKV_API int patchkv_plan_checkpoint(patchkv_ctx* ctx, const patchkv_geom* geom, int n_suffix_tokens,
+                                        const uint8_t* tags, uint64_t* blk_off, uint64_t* layer_bytes, void* stream);
+
+/* patchkv_quantize_gather writes the record of every block of every layer of one session from the paged pool.
+ * `session` is read as for patchkv_restore, with the roles reversed: block_table / dst_shift locate the SOURCE
+ * rows in `pool`, tags / blk_off / layer_payload / layer_bytes describe the DESTINATION records (layer_payload
+ * buffers are written), delta and the reuse lists are ignored.  Quantiser, per group of `group` channels of one
+ * (token, head): s = fp16(amax / qmax) (fp32 division, round to nearest even), code = clamp(rint(x / s), -qmax,
+ * qmax) with ties to even, s == 0 -> code 0; qmax = 127 for int8 and 7 for int4; a bf16 section copies the 16
+ * bits; tokens past the end of the suffix encode as zeros.  Values must be finite with amax / qmax <= 65504.
+ * Needs group in {8, 16, 32, 64, 128, 256}.  A block whose tag, record extent or source pages are out of range
+ * is skipped whole and PATCHKV_E_BOUNDS is latched.  One launch, asynchronous on `stream`. */
+PATCHKV_API int patchkv_quantize_gather(patchkv_ctx* ctx, const patchkv_geom* geom, const patchkv_pool* pool,
+                                        const patchkv_session* session, void* stream);
+
 /* Synchronises the context's device work and returns in *device_status the first device-side error latched
  * since the last query (PATCHKV_OK, PATCHKV_E_BOUNDS, PATCHKV_E_BADINPUT or PATCHKV_E_TIMEOUT), then clears it. */
 PATCHKV_API int patchkv_query_status(patchkv_ctx* ctx, int* device_status);

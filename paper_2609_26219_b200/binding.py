@@ -88,11 +88,15 @@ def lib():
         l.patchkv_restore.argtypes = [C.c_void_p, C.POINTER(Geom), C.POINTER(Pool), C.c_void_p, C.c_int, C.c_void_p]
         l.patchkv_restore_from_host.argtypes = [C.c_void_p, C.POINTER(Geom), C.POINTER(Pool), C.c_void_p, C.c_int,
                                                 C.c_void_p, C.POINTER(RestoreStats)]
+        l.patchkv_plan_checkpoint.argtypes = [C.c_void_p, C.POINTER(Geom), C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
+                                              C.c_void_p]
+        l.patchkv_quantize_gather.argtypes = [C.c_void_p, C.POINTER(Geom), C.POINTER(Pool), C.POINTER(Session), C.c_void_p]
         l.patchkv_query_status.argtypes = [C.c_void_p, C.POINTER(C.c_int)]
         l.patchkv_record_bytes.argtypes = [C.c_int] * 5
         l.patchkv_record_bytes.restype = C.c_uint64
         for f in (l.patchkv_create, l.patchkv_destroy, l.patchkv_last_error, l.patchkv_select_repair,
-                  l.patchkv_restore, l.patchkv_restore_from_host, l.patchkv_query_status):
+                  l.patchkv_restore, l.patchkv_restore_from_host, l.patchkv_query_status,
+                  l.patchkv_plan_checkpoint, l.patchkv_quantize_gather):
             f.restype = C.c_int
         _lib = l
     return _lib
@@ -181,6 +185,16 @@ class Context:
         rc = lib().patchkv_restore_from_host(self._h, C.byref(geom), C.byref(pool), C.cast(arr, C.c_void_p),
                                              len(sessions), _stream_handle(stream), C.byref(stats))
         return self._check(rc, check), stats
+
+    def plan_checkpoint(self, geom: Geom, n_suffix_tokens: int, tags: torch.Tensor, blk_off: torch.Tensor,
+                        layer_bytes: torch.Tensor, stream=None, check: bool = True) -> int:
+        """tags u8 [L][NB] (device) -> blk_off i64 [L][NB], layer_bytes i64 [L] (device) of the clustered layout."""
+        return self._check(lib().patchkv_plan_checkpoint(self._h, C.byref(geom), n_suffix_tokens, _ptr(tags),
+                                                         _ptr(blk_off), _ptr(layer_bytes), _stream_handle(stream)), check)
+
+    def quantize_gather(self, geom: Geom, pool: Pool, session: Session, stream=None, check: bool = True) -> int:
+        return self._check(lib().patchkv_quantize_gather(self._h, C.byref(geom), C.byref(pool), C.byref(session),
+                                                         _stream_handle(stream)), check)
 
     def query_status(self) -> int:
         v = C.c_int(0)

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpatchkv.so")
-SOURCES = ["context.cu", "restore.cu", "select.cu", "host_restore.cu"]
+SOURCES = ["context.cu", "restore.cu", "select.cu", "host_restore.cu", "writer.cu"]
 
 
 def _newest_source_mtime() -> float:

@@ -1,0 +1,257 @@
+// Checkpoint writer (Section IV-D, offload side): lay out the clustered directory from the tags, then gather
+// each block's rows from the paged pool, compute per-group fp16 scales, quantise and pack the record.
+// The inverse direction of restore; HBM-bound streaming with a warp-shuffle maximum per scale group.
+#include <cuda_fp16.h>
+
+#include "common.cuh"
+
+namespace patchkv {
+
+constexpr int kPlanThreads = 1024;
+constexpr int kGatherThreads = 256;
+
+// Exclusive prefix sum of v over a 1024-thread CTA; *total receives the CTA sum.
+__device__ __forceinline__ int plan_exclusive_scan(int v, int* warp_sums, int* total) {
+    const unsigned lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    int inc = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int o = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+        if (lane >= (unsigned)d) inc += o;
+    }
+    __syncthreads();
+    if (lane == 31) warp_sums[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        const int w = warp_sums[lane];
+        int winc = w;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int o = __shfl_up_sync(0xFFFFFFFFu, winc, d);
+            if (lane >= (unsigned)d) winc += o;
+        }
+        warp_sums[lane] = winc - w;
+        if (lane == 31) warp_sums[32] = winc;
+    }
+    __syncthreads();
+    *total = warp_sums[32];
+    return warp_sums[warp] + inc - v;
+}
+
+// One CTA per layer: offsets of the runs [bf16][int8][int4][k4v4], ascending block index inside a run.
+__global__ void __launch_bounds__(kPlanThreads)
+plan_checkpoint_kernel(const uint8_t* tags, int NB, unsigned long long elems, int group,
+                       unsigned long long* blk_off, unsigned long long* layer_bytes, int32_t* status) {
+    __shared__ int warp_sums[33];
+    const int l = blockIdx.x;
+    const uint8_t* tg = tags + (long long)l * NB;
+    unsigned long long* off = blk_off + (long long)l * NB;
+    unsigned long long base = 0;
+    for (int tag = 0; tag <= PATCHKV_TAG_K4V4; tag++) {
+        const unsigned long long rec = record_bytes(tag, elems, group);
+        int run = 0;
+        for (int j0 = 0; j0 < NB; j0 += kPlanThreads) {
+            const int j = j0 + threadIdx.x;
+            const int mine = j < NB && tg[j] == tag;
+            int tot;
+            const int rank = plan_exclusive_scan(mine, warp_sums, &tot) + run;
+            run += tot;
+            if (mine) off[j] = base + (unsigned long long)rank * rec;
+        }
+        base += (unsigned long long)run * rec;
+    }
+    bool bad = false;
+    for (int j = threadIdx.x; j < NB; j += kPlanThreads)
+        if (tg[j] > PATCHKV_TAG_K4V4) { off[j] = ~0ull; bad = true; }
+    if (bad) atomicCAS(status, 0, (int)PATCHKV_E_BOUNDS);
+    if (threadIdx.x == 0) layer_bytes[l] = base;
+}
+
+struct GatherParams {
+    int32_t L, H, D, B, P, G;
+    const uint16_t* k_base;
+    const uint16_t* v_base;
+    long long stride_layer, stride_page, stride_token, stride_head;
+    int32_t n_pages, n, nb, src_shift, n_table;
+    const int32_t* block_table;
+    const uint8_t* tags;
+    const unsigned long long* blk_off;
+    void* const* layer_payload;
+    const unsigned long long* layer_bytes;
+    int32_t* status;
+};
+
+// Eight bf16 channels -> one chunk of a section.  `seg` = lanes per scale group (group / 8, a power of two).
+template <int FMT>
+__device__ __forceinline__ void encode_chunk(const uint4& w, uint8_t* codes, uint8_t* scales, size_t elem0,
+                                             size_t scale_index, int seg, bool write) {
+    if (FMT == FMT_BF16) {
+        if (write) *reinterpret_cast<uint4*>(codes + 2 * elem0) = w;
+        return;
+    }
+    float x[8];
+    x[0] = __uint_as_float(w.x << 16); x[1] = __uint_as_float(w.x & 0xFFFF0000u);
+    x[2] = __uint_as_float(w.y << 16); x[3] = __uint_as_float(w.y & 0xFFFF0000u);
+    x[4] = __uint_as_float(w.z << 16); x[5] = __uint_as_float(w.z & 0xFFFF0000u);
+    x[6] = __uint_as_float(w.w << 16); x[7] = __uint_as_float(w.w & 0xFFFF0000u);
+    float amax = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 8; i++) amax = fmaxf(amax, fabsf(x[i]));
+    for (int d = 1; d < seg; d <<= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, d));
+    const float qmax = FMT == FMT_INT8 ? 127.0f : 7.0f;
+    const __half s16 = __float2half_rn(__fdiv_rn(amax, qmax));
+    const float s = __half2float(s16);
+    int q[8];
+#pragma unroll
+    for (int i = 0; i < 8; i++) {
+        float r = s > 0.0f ? rintf(__fdiv_rn(x[i], s)) : 0.0f;
+        r = fminf(fmaxf(r, -qmax), qmax);
+        q[i] = (int)r;
+    }
+    if (!write) return;
+    if (FMT == FMT_INT8) {
+        uint2 o;
+        o.x = (q[0] & 255) | ((q[1] & 255) << 8) | ((q[2] & 255) << 16) | ((uint32_t)(q[3] & 255) << 24);
+        o.y = (q[4] & 255) | ((q[5] & 255) << 8) | ((q[6] & 255) << 16) | ((uint32_t)(q[7] & 255) << 24);
+        *reinterpret_cast<uint2*>(codes + elem0) = o;
+    } else {
+        uint32_t o = 0;
+#pragma unroll
+        for (int i = 0; i < 8; i++) o |= (uint32_t)(q[i] & 15) << (4 * i);     // channel 2k -> low nibble of byte k
+        *reinterpret_cast<uint32_t*>(codes + (elem0 >> 1)) = o;
+    }
+    if (((threadIdx.x & 31) & (seg - 1)) == 0) *reinterpret_cast<__half*>(scales + 2 * scale_index) = s16;
+}
+
+// One CTA per (layer, block).
+__global__ void __launch_bounds__(kGatherThreads)
+quantize_gather_kernel(const GatherParams p) {
+    __shared__ long long tok_off[2048];
+    const int l = blockIdx.x / p.nb, j = blockIdx.x - l * p.nb;
+    const int tag = __ldg(p.tags + (size_t)l * p.nb + j);
+    const unsigned long long off = __ldg(p.blk_off + (size_t)l * p.nb + j);
+    const unsigned long long lbytes = __ldg(p.layer_bytes + l);
+    uint8_t* base = reinterpret_cast<uint8_t*>(
+        static_cast<uintptr_t>(__ldg(reinterpret_cast<const unsigned long long*>(p.layer_payload) + l)));
+    const unsigned long long elems = (unsigned long long)p.B * p.H * p.D;
+    const unsigned long long rec = record_bytes(tag, elems, p.G);
+    bool bad = rec == 0 || off > lbytes || rec > lbytes - off || base == nullptr ||
+               ((reinterpret_cast<uintptr_t>(base) + off) & 15u) != 0;
+    const int valid = min(p.B, p.n - j * p.B);
+    for (int t = threadIdx.x; t < p.B; t += kGatherThreads) {
+        long long o = -1;                                   // past the end of the suffix: encodes as zeros
+        if (t < valid) {
+            const long long u = (long long)j * p.B + t + p.src_shift;
+            const long long lp = u / p.P;
+            const int page = lp < p.n_table ? __ldg(p.block_table + lp) : -1;
+            if (page < 0 || page >= p.n_pages) bad = true;
+            o = (long long)l * p.stride_layer + (long long)page * p.stride_page + (u - lp * p.P) * p.stride_token;
+        }
+        tok_off[t] = o;
+    }
+    if (__syncthreads_or(bad)) {                            // skip the block whole, latch the error
+        if (threadIdx.x == 0) atomicCAS(p.status, 0, (int)PATCHKV_E_BOUNDS);
+        return;
+    }
+    const int kf = k_format(tag), vf = v_format(tag);
+    uint8_t* kc = base + off;
+    uint8_t* ks = kc + code_bytes(kf, elems);
+    uint8_t* vc = ks + scale_bytes(kf, elems, p.G);
+    uint8_t* vs = vc + code_bytes(vf, elems);
+    const int cpv = p.D >> 3;                               // 8-channel chunks per head vector
+    const int seg = p.G >> 3;                               // lanes per scale group
+    const int gpv = p.D / p.G;
+    const bool cpv_pow2 = (cpv & (cpv - 1)) == 0, h_pow2 = (p.H & (p.H - 1)) == 0;
+    const int cpv_shift = 31 - __clz(cpv), h_shift = 31 - __clz(p.H), seg_shift = 31 - __clz(seg);
+    const int units = p.B * p.H * cpv;
+    const int padded = (units + kGatherThreads - 1) / kGatherThreads * kGatherThreads;
+#pragma unroll 1
+    for (int sec = 0; sec < 2; sec++) {
+        const int fmt = sec ? vf : kf;
+        const uint16_t* pool = sec ? p.v_base : p.k_base;
+        uint8_t* codes = sec ? vc : kc;
+        uint8_t* scales = sec ? vs : ks;
+#pragma unroll 2
+        for (int u = threadIdx.x; u < padded; u += kGatherThreads) {
+            const bool in = u < units;
+            const int vec = cpv_pow2 ? (u >> cpv_shift) : u / cpv;
+            const int cx = u - vec * cpv;
+            const int t = h_pow2 ? (vec >> h_shift) : vec / p.H;
+            const int h = vec - t * p.H;
+            uint4 w = make_uint4(0, 0, 0, 0);
+            if (in) {
+                const long long to = tok_off[t];
+                if (to >= 0) w = __ldg(reinterpret_cast<const uint4*>(pool + to + (long long)h * p.stride_head + 8 * cx));
+            }
+            const size_t elem0 = (size_t)vec * p.D + 8 * cx;
+            const size_t sidx = (size_t)vec * gpv + (cx >> seg_shift);
+            switch (fmt) {
+                case FMT_BF16: encode_chunk<FMT_BF16>(w, codes, scales, elem0, sidx, seg, in); break;
+                case FMT_INT8: encode_chunk<FMT_INT8>(w, codes, scales, elem0, sidx, seg, in); break;
+                default:       encode_chunk<FMT_INT4>(w, codes, scales, elem0, sidx, seg, in); break;
+            }
+        }
+    }
+}
+
+}  // namespace patchkv
+
+using namespace patchkv;
+
+extern "C" int patchkv_plan_checkpoint(patchkv_ctx* ctx, const patchkv_geom* g, int n_suffix_tokens,
+                                       const uint8_t* tags, uint64_t* blk_off, uint64_t* layer_bytes, void* stream) {
+    if (!ctx) return PATCHKV_E_INVALID;
+    std::lock_guard<std::mutex> lock(ctx->mu);
+    if (!g || g->struct_size != sizeof(patchkv_geom)) return fail(ctx, PATCHKV_E_INVALID, "plan: geometry null or struct_size mismatch");
+    if (g->n_layers <= 0 || g->n_layers > 65535 || g->n_kv_heads <= 0 || g->head_dim <= 0 || g->block_tokens <= 0 ||
+        g->group <= 0 || g->head_dim % g->group || n_suffix_tokens < 0)
+        return fail(ctx, PATCHKV_E_INVALID, "plan: bad geometry");
+    if (!layer_bytes) return fail(ctx, PATCHKV_E_INVALID, "plan: null output");
+    const int NB = (n_suffix_tokens + g->block_tokens - 1) / g->block_tokens;
+    if (NB > 0 && (!tags || !blk_off)) return fail(ctx, PATCHKV_E_INVALID, "plan: null pointer");
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, PATCHKV_E_CUDA, "cudaSetDevice failed");
+    plan_checkpoint_kernel<<<g->n_layers, kPlanThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        tags, NB, (unsigned long long)g->block_tokens * g->n_kv_heads * g->head_dim, g->group,
+        reinterpret_cast<unsigned long long*>(blk_off), reinterpret_cast<unsigned long long*>(layer_bytes), ctx->d_status);
+    PKV_CUDA(ctx, cudaGetLastError());
+    return PATCHKV_OK;
+}
+
+extern "C" int patchkv_quantize_gather(patchkv_ctx* ctx, const patchkv_geom* g, const patchkv_pool* pool,
+                                       const patchkv_session* s, void* stream) {
+    if (!ctx) return PATCHKV_E_INVALID;
+    std::lock_guard<std::mutex> lock(ctx->mu);
+    static thread_local RestoreParams rp;                  // reused only for the shared geometry / pool validation
+    int rc = fill_geometry(ctx, g, pool, &rp);
+    if (rc != PATCHKV_OK) return rc;
+    if (!s || s->struct_size != sizeof(patchkv_session)) return fail(ctx, PATCHKV_E_INVALID, "session: null or struct_size mismatch");
+    if (s->n_suffix_tokens < 0 || s->dst_shift < 0 || s->dst_shift >= g->page_tokens || s->n_table < 0)
+        return fail(ctx, PATCHKV_E_INVALID, "session: n_suffix_tokens >= 0, 0 <= dst_shift < P, n_table >= 0");
+    const int G = g->group;
+    if (!(G == 8 || G == 16 || G == 32 || G == 64 || G == 128 || G == 256))
+        return fail(ctx, PATCHKV_E_UNSUPPORTED, "quantize_gather: group must be 8, 16, 32, 64, 128 or 256");
+    if (g->block_tokens > 2048) return fail(ctx, PATCHKV_E_UNSUPPORTED, "quantize_gather: block_tokens > 2048");
+    const int nb = (s->n_suffix_tokens + g->block_tokens - 1) / g->block_tokens;
+    if (nb == 0) return PATCHKV_OK;
+    if (!s->block_table || !s->tags || !s->blk_off || !s->layer_payload || !s->layer_bytes)
+        return fail(ctx, PATCHKV_E_INVALID, "session: null pointer");
+    if ((long long)nb * g->n_layers > 0x7fffffffLL) return fail(ctx, PATCHKV_E_UNSUPPORTED, "quantize_gather: too many blocks");
+    GatherParams p;
+    p.L = g->n_layers; p.H = g->n_kv_heads; p.D = g->head_dim; p.B = g->block_tokens; p.P = g->page_tokens; p.G = G;
+    p.k_base = static_cast<const uint16_t*>(pool->k_base);
+    p.v_base = static_cast<const uint16_t*>(pool->v_base);
+    p.stride_layer = pool->stride_layer; p.stride_page = pool->stride_page;
+    p.stride_token = pool->stride_token; p.stride_head = pool->stride_head;
+    p.n_pages = pool->n_pages; p.n = s->n_suffix_tokens; p.nb = nb; p.src_shift = s->dst_shift; p.n_table = s->n_table;
+    p.block_table = s->block_table; p.tags = s->tags;
+    p.blk_off = reinterpret_cast<const unsigned long long*>(s->blk_off);
+    p.layer_payload = const_cast<void* const*>(s->layer_payload);
+    p.layer_bytes = reinterpret_cast<const unsigned long long*>(s->layer_bytes);
+    p.status = ctx->d_status;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, PATCHKV_E_CUDA, "cudaSetDevice failed");
+    quantize_gather_kernel<<<nb * g->n_layers, kGatherThreads, 0, static_cast<cudaStream_t>(stream)>>>(p);
+    PKV_CUDA(ctx, cudaGetLastError());
+    return PATCHKV_OK;
+}

@@ -1,0 +1,163 @@
+"""GPU parity of the checkpoint writer (patchkv_plan_checkpoint + patchkv_quantize_gather) against the oracle:
+directory and payload bytes identical; and the round trip writer -> restore on the GPU."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import patchkv_inputs as pin
+from gpu_common import DEV, check_pools, gpu_pool, new_context, staged
+from helpers import np_u16, oracle_restore, oracle_select
+from test_oracle_writer import _ck, pool_from_raw, run_writer
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = new_context()
+    yield c
+    c.close()
+
+
+def gpu_writer(ctx, ck, kp, vp, shift=0, fill=0xEE, table=None, blk_off=None):
+    """Run plan + quantize_gather on the GPU for the pools kp, vp (uint16 numpy).  Returns (off, lb, payload bytes per layer)."""
+    from paper_2609_26219_b200 import binding as pk
+    g = ck.geom
+    L, NB = g.n_layers, ck.n_blocks
+    k = torch.from_numpy(kp.view(np.int16)).to(DEV)
+    v = torch.from_numpy(vp.view(np.int16)).to(DEV)
+    pool = pk.make_pool(k, v, ck.n_pages, pin.pool_strides(g, ck.n_pages))
+    geom = pk.make_geom(g.n_layers, g.n_kv_heads, g.head_dim, g.rotary_dim, g.rope_style, g.rope_base, g.block_tokens,
+                        g.page_tokens, g.group)
+    tags = ck.tags.to(DEV).contiguous()
+    off = torch.full((L, NB), -1, dtype=torch.int64, device=DEV)
+    lb = torch.zeros(L, dtype=torch.int64, device=DEV)
+    ctx.plan_checkpoint(geom, ck.n_suffix_tokens, tags, off, lb)
+    torch.cuda.synchronize()
+    sizes = [int(x) for x in lb.cpu()]
+    if blk_off is not None:
+        off = torch.from_numpy(blk_off.astype(np.int64)).to(DEV)
+    layer_off, total = [], 0
+    for s in sizes:
+        layer_off.append(total)
+        total += -(-s // 256) * 256
+    payload = torch.full((max(total, 256),), fill, dtype=torch.uint8, device=DEV)
+    ptrs = torch.tensor([payload.data_ptr() + o for o in layer_off], dtype=torch.int64, device=DEV)
+    tb = (ck.block_table if table is None else torch.from_numpy(table)).to(DEV).contiguous()
+    sess = pk.make_session(n_suffix_tokens=ck.n_suffix_tokens, delta=0, dst_shift=shift, block_table=tb, tags=tags,
+                           blk_off=off, layer_payload=ptrs, layer_bytes=lb, reuse_idx=None, reuse_cnt=None)
+    ctx.quantize_gather(geom, pool, sess)
+    torch.cuda.synchronize()
+    pay = payload.cpu().numpy()
+    return off.cpu().numpy().astype(np.uint64), sizes, [pay[o:o + s] for o, s in zip(layer_off, sizes)]
+
+
+@pytest.mark.parametrize("kw", [dict(), dict(n=150), dict(n=150, dst_shift=5),
+                                dict(geom=pin.Geometry(1, 4, 128, 128, pin.ROPE_HALF, 5e5, 16, 16, 128)),
+                                dict(geom=pin.Geometry(2, 2, 64, 64, pin.ROPE_HALF, 1e4, 32, 16, 8), n=200, n_pages=40),
+                                dict(geom=pin.Geometry(2, 3, 64, 64, pin.ROPE_HALF, 1e4, 16, 8, 64), n=100, n_pages=40)])
+def test_writer_bytes_match_the_oracle(ctx, kw):
+    ck = _ck(**kw)
+    shift = ck.dst_shift
+    kp, vp = pool_from_raw(ck, shift=shift)
+    rc, rc2, off_o, lb_o, bufs_o = run_writer(ck, kp, vp, shift=shift)
+    assert rc == oracle.OK and rc2 == oracle.OK
+    off, sizes, bufs = gpu_writer(ctx, ck, kp, vp, shift=shift)
+    assert ctx.query_status() == 0
+    assert np.array_equal(off, off_o) and sizes == [int(x) for x in lb_o]
+    for a, b in zip(bufs, bufs_o):
+        assert np.array_equal(a, b)
+
+
+@pytest.mark.parametrize("what", ["page", "offset", "table_short"])
+def test_writer_skips_out_of_range_blocks(ctx, what):
+    ck = _ck()
+    kp, vp = pool_from_raw(ck)
+    _, _, off_o, lb_o, _ = run_writer(ck, kp, vp)
+    table = ck.block_table.numpy().copy()
+    off2 = off_o.copy()
+    if what == "page":
+        table[4] = ck.n_pages + 3
+    elif what == "offset":
+        off2[:, 4] = max(int(x) for x in lb_o)
+    else:
+        table = table[:-1]
+    rc, rc2, _, _, bufs_o = run_writer(ck, kp, vp, table=table, blk_off=off2)
+    assert rc2 == oracle.E_BOUNDS
+    off, sizes, bufs = gpu_writer(ctx, ck, kp, vp, table=table, blk_off=off2)
+    assert ctx.query_status() == -3
+    for a, b in zip(bufs, bufs_o):
+        assert np.array_equal(a, b)
+
+
+def test_unknown_tag_in_plan_and_unsupported_group(ctx):
+    from paper_2609_26219_b200 import binding as pk
+    ck = _ck()
+    ck.tags[0, 3] = 9
+    kp, vp = pool_from_raw(ck)
+    off, sizes, bufs = gpu_writer(ctx, ck, kp, vp)
+    assert ctx.query_status() == -3
+    assert off[0, 3] == np.uint64(2 ** 64 - 1)
+    g24 = pin.Geometry(1, 2, 72, 48, pin.ROPE_HALF, 1e4, 16, 16, 24)
+    ck2 = pin.config_tiny(geom=g24)
+    st = staged(ck2)
+    k, v, pool = gpu_pool(ck2)
+    assert ctx.quantize_gather(st.geom(), pool, st.session(), check=False) == pk.E_UNSUPPORTED
+
+
+def test_full_size_8b_shape_writer_then_restore_round_trip(ctx):
+    """32-layer 8B-shaped pool -> checkpoint written on the GPU -> restored on the GPU with delta = 0 into a second
+    pool: bf16-tag blocks come back bit-identical, quantised blocks within half a quantisation step; sampled
+    layers of the written payload are compared byte for byte with the oracle's writer."""
+    from paper_2609_26219_b200 import binding as pk
+    ck = pin.config_llama8b(device=DEV, delta=0, dirty_tokens=0, top_k=0)
+    g = ck.geom
+    st = staged(ck)
+    ctx.select_repair(st.select_args())
+    k, v, pool = gpu_pool(ck)
+    ctx.restore(st.geom(), pool, [st.session()])          # pool <- the synthetic checkpoint (all 1024 blocks)
+    torch.cuda.synchronize()
+    # write a second checkpoint from that pool with the same tags
+    L, NB = g.n_layers, ck.n_blocks
+    off = torch.zeros((L, NB), dtype=torch.int64, device=DEV)
+    lb = torch.zeros(L, dtype=torch.int64, device=DEV)
+    ctx.plan_checkpoint(st.geom(), ck.n_suffix_tokens, st.tags, off, lb)
+    torch.cuda.synchronize()
+    assert torch.equal(off, st.blk_off) and [int(x) for x in lb.cpu()] == ck.layer_bytes
+    payload2 = torch.zeros_like(st.payload)
+    ptrs2 = torch.tensor([payload2.data_ptr() + o for o in ck.layer_off], dtype=torch.int64, device=DEV)
+    sess_w = st.session(layer_payload=ptrs2, blk_off=off, layer_bytes=lb)
+    ctx.quantize_gather(st.geom(), pool, sess_w)
+    torch.cuda.synchronize()
+    assert ctx.query_status() == 0
+    # sampled layers against the oracle's writer
+    table = ck.block_table.cpu().numpy()
+    tags_np = ck.tags.cpu().numpy()
+    for l in (0, 19):
+        sub = pin.Geometry(1, g.n_kv_heads, g.head_dim, g.rotary_dim, g.rope_style, g.rope_base, 16, 16, g.group)
+        kp, vp = np_u16(k[l:l + 1]), np_u16(v[l:l + 1])
+        buf = [np.zeros(ck.layer_bytes[l], dtype=np.uint8)]
+        rc = oracle.quantize_gather(L=1, H=g.n_kv_heads, D=g.head_dim, B=16, P=16, G=g.group, k_pool=kp, v_pool=vp,
+                                    strides=pin.pool_strides(sub, ck.n_pages), n_pages=ck.n_pages, n=ck.n_suffix_tokens,
+                                    src_shift=0, block_table=table, tags=tags_np[l:l + 1],
+                                    blk_off=off[l:l + 1].cpu().numpy(), layer_payload=buf)
+        assert rc == oracle.OK
+        got = payload2[ck.layer_off[l]:ck.layer_off[l] + ck.layer_bytes[l]].cpu().numpy()
+        assert np.array_equal(got, buf[0])
+    # restore the second checkpoint into a fresh pool and compare with the first pool
+    k2, v2, pool2 = gpu_pool(ck)
+    ctx.restore(st.geom(), pool2, [sess_w])
+    torch.cuda.synchronize()
+    bf = torch.from_numpy(np.isin(tags_np[0], [0])).to(DEV)
+    pages_bf = st.block_table[:NB][bf].long()
+    assert torch.equal(k2[:, pages_bf], k[:, pages_bf]) and torch.equal(v2[:, pages_bf], v[:, pages_bf])
+    a = k.view(torch.bfloat16).float()
+    b = k2.view(torch.bfloat16).float()
+    amax = a.abs().reshape(*a.shape[:-1], -1, g.group).amax(dim=-1, keepdim=True)
+    step = (amax / 127.0).expand(*amax.shape[:-1], g.group).reshape(a.shape)
+    used = torch.zeros(ck.n_pages, dtype=torch.bool, device=DEV)
+    used[st.block_table[:NB].long()] = True
+    err = (a - b).abs()[:, used]
+    bound = (0.5 * step * 1.01 + a.abs() * 2.0 ** -8 + amax.expand(*amax.shape[:-1], g.group).reshape(a.shape) * 2.0 ** -10)[:, used]
+    assert bool((err <= bound).all())

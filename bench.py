@@ -307,6 +307,35 @@ def run_ours(args):
                 "frac_of_nominal_8tbs": achieved / 8000.0, "traffic": RESTORE_KERNEL_DRAM_TRAFFIC_BYTES,
                 "algorithmic_bytes_per_launch": read_b + written_b, "kernel_ms": restore_avg_ms}
 
+    # ---- offload side: write a checkpoint of all 1024 blocks x 32 layers from the pool (not on the resume path)
+    writer = None
+    if not args.no_writer:
+        L_, NB_ = ck.geom.n_layers, ck.n_blocks
+        w_off = torch.zeros((L_, NB_), dtype=torch.int64, device=dev)
+        w_lb = torch.zeros(L_, dtype=torch.int64, device=dev)
+        w_pay = torch.empty_like(st.payload)
+        w_ptrs = torch.tensor([w_pay.data_ptr() + o for o in ck.layer_off], dtype=torch.int64, device=dev)
+        w_sess = st.session(layer_payload=w_ptrs, blk_off=w_off, layer_bytes=w_lb)
+        ts_w = []
+        for i in range(13):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            ctx.plan_checkpoint(geom, ck.n_suffix_tokens, st.tags, w_off, w_lb, stream)
+            ctx.quantize_gather(geom, pool, w_sess, stream)
+            b.record(stream)
+            b.synchronize()
+            if i >= 3:
+                ts_w.append(a.elapsed_time(b))
+        assert ctx.query_status() == 0 and torch.equal(w_off, st.blk_off)
+        t_w = statistics.median(ts_w)
+        pool_read = 2 * L_ * NB_ * ck.geom.block_tokens * ck.geom.n_kv_heads * ck.geom.head_dim * 2
+        pay_written = sum(ck.layer_bytes)
+        writer = {"workload": "quantize_gather of all 1024 blocks x 32 layers of the same pool and tags",
+                  "ms": t_w, "real_gbps": (pool_read + pay_written) / (t_w * 1e-3) / 1e9,
+                  "frac_of_hbm_peak": (pool_read + pay_written) / (t_w * 1e-3) / 1e9 / peak,
+                  "bf16_gbps_read": pool_read / (t_w * 1e-3) / 1e9, "payload_bytes": int(pay_written)}
+        del w_pay
+
     # ---- end to end: host buffers, copies inside the timed region
     e2e = None
     host_link = None
@@ -462,7 +491,7 @@ def run_ours(args):
             "select_us": select_us, "restore_ms": restore_avg_ms,
             "block_layers_per_s": world * items / (ms_per_step * 1e-3),
             "real_gbps": world * (read_b + written_b) / (ms_per_step * 1e-3) / 1e9,
-            "host_link": host_link, "select_at_scale": select_scale, "host_7b": host_cfg3, "stress": stress,
+            "host_link": host_link, "select_at_scale": select_scale, "host_7b": host_cfg3, "stress": stress, "writer": writer,
         }
         print(json.dumps(line), flush=True)
     ctx.close()
@@ -481,6 +510,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-scale-select", action="store_true")
     ap.add_argument("--no-host-configs", action="store_true")
+    ap.add_argument("--no-writer", action="store_true")
     ap.add_argument("--stress-layers", type=int, default=10)
     ap.add_argument("--scale-layers", type=int, default=32, help="layers of the selection-at-scale leg (profiling: fewer)")
     ap.add_argument("--layers", type=int, default=32,

@@ -101,24 +101,51 @@ __device__ __forceinline__ void encode_chunk(const uint4& w, uint8_t* codes, uin
     const float qmax = FMT == FMT_INT8 ? 127.0f : 7.0f;
     const __half s16 = __float2half_rn(__fdiv_rn(amax, qmax));
     const float s = __half2float(s16);
-    int q[8];
+    // code = rint(fp32(x / s)), ties to even.  x has 8 significant bits and s has 11, so x / s is either exactly a
+    // half-integer or at least 2^-12 away from one; the fp32 rounding of the quotient (< 2^-16 here) therefore never
+    // crosses a rounding boundary, and the code is the exact quotient rounded to the nearest integer, ties to even.
+    // That is computed without a division per element: t = x * (1/s) is within 2^-16 of the quotient, so rint(t) is
+    // right unless the quotient is an exact tie, which the exact remainder x - k*s (one fma) detects and repairs.
+    const float r = s > 0.0f ? __frcp_rn(s) : 0.0f;
+    const float half_s = 0.5f * s;
+    const float magic = 12582912.0f;                       // 1.5 * 2^23: adding it rounds to an integer, ties to even
+    // Two lanes per instruction for the products and sums.  (If the assembler contracts x*r + magic into one fused
+    // operation the integer k can only change at an exact tie, where the repair below picks the even neighbour from
+    // either side.)
+    uint32_t kb[8];                                        // bits of code + 1.5 * 2^23: the low byte is the code
+    float kf[8], df[8], tmf[8];
+    const f32x2 r2 = pack2(r, r), m2 = pack2(magic, magic), ns2 = pack2(-s, -s);
+    bool any_tie = false;
 #pragma unroll
-    for (int i = 0; i < 8; i++) {
-        float r = s > 0.0f ? rintf(__fdiv_rn(x[i], s)) : 0.0f;
-        r = fminf(fmaxf(r, -qmax), qmax);
-        q[i] = (int)r;
+    for (int i = 0; i < 8; i += 2) {
+        const f32x2 x2 = pack2(x[i], x[i + 1]);
+        const f32x2 tm = add2(mul2(x2, r2), m2);           // |x * r| <= ~2 * qmax: far below 2^22
+        const f32x2 k2 = sub2(tm, m2);
+        const f32x2 d2 = fma2(k2, ns2, x2);                // x - k*s, exact: a multiple of ulp(s) no larger than s
+        unpack2(tm, tmf[i], tmf[i + 1]);
+        unpack2(k2, kf[i], kf[i + 1]);
+        unpack2(d2, df[i], df[i + 1]);
+        any_tie = any_tie || fabsf(df[i]) == half_s || fabsf(df[i + 1]) == half_s;
     }
-    if (!write) return;
-    if (FMT == FMT_INT8) {
-        uint2 o;
-        o.x = (q[0] & 255) | ((q[1] & 255) << 8) | ((q[2] & 255) << 16) | ((uint32_t)(q[3] & 255) << 24);
-        o.y = (q[4] & 255) | ((q[5] & 255) << 8) | ((q[6] & 255) << 16) | ((uint32_t)(q[7] & 255) << 24);
-        *reinterpret_cast<uint2*>(codes + elem0) = o;
-    } else {
-        uint32_t o = 0;
+    if (any_tie) {                                         // rare: an exact half-integer quotient on an odd k
 #pragma unroll
-        for (int i = 0; i < 8; i++) o |= (uint32_t)(q[i] & 15) << (4 * i);     // channel 2k -> low nibble of byte k
-        *reinterpret_cast<uint32_t*>(codes + (elem0 >> 1)) = o;
+        for (int i = 0; i < 8; i++)
+            if (fabsf(df[i]) == half_s && (__float_as_uint(tmf[i]) & 1u)) kf[i] += df[i] > 0.0f ? 1.0f : -1.0f;
+    }
+#pragma unroll
+    for (int i = 0; i < 8; i++) kb[i] = __float_as_uint(fminf(fmaxf(kf[i], -qmax), qmax) + magic);
+    if (!write) return;
+    // byte k of a word <- low byte of kb[k]
+    const uint32_t w0 = __byte_perm(__byte_perm(kb[0], kb[1], 0x0040), __byte_perm(kb[2], kb[3], 0x0040), 0x5410);
+    const uint32_t w1 = __byte_perm(__byte_perm(kb[4], kb[5], 0x0040), __byte_perm(kb[6], kb[7], 0x0040), 0x5410);
+    if (FMT == FMT_INT8) {
+        *reinterpret_cast<uint2*>(codes + elem0) = make_uint2(w0, w1);
+    } else {
+        // keep the low nibble of every byte and squeeze four bytes into sixteen bits: channel 2k -> low nibble of byte k
+        uint32_t a = w0 & 0x0F0F0F0Fu, b = w1 & 0x0F0F0F0Fu;
+        a = (a | (a >> 4)) & 0x00FF00FFu; a = (a | (a >> 8)) & 0x0000FFFFu;
+        b = (b | (b >> 4)) & 0x00FF00FFu; b = (b | (b >> 8)) & 0x0000FFFFu;
+        *reinterpret_cast<uint32_t*>(codes + (elem0 >> 1)) = a | (b << 16);
     }
     if (((threadIdx.x & 31) & (seg - 1)) == 0) *reinterpret_cast<__half*>(scales + 2 * scale_index) = s16;
 }
@@ -126,7 +153,7 @@ __device__ __forceinline__ void encode_chunk(const uint4& w, uint8_t* codes, uin
 // One CTA per (layer, block).
 __global__ void __launch_bounds__(kGatherThreads)
 quantize_gather_kernel(const GatherParams p) {
-    __shared__ long long tok_off[2048];
+    extern __shared__ long long tok_off[];                  // block_tokens entries
     const int l = blockIdx.x / p.nb, j = blockIdx.x - l * p.nb;
     const int tag = __ldg(p.tags + (size_t)l * p.nb + j);
     const unsigned long long off = __ldg(p.blk_off + (size_t)l * p.nb + j);
@@ -171,7 +198,7 @@ quantize_gather_kernel(const GatherParams p) {
         const uint16_t* pool = sec ? p.v_base : p.k_base;
         uint8_t* codes = sec ? vc : kc;
         uint8_t* scales = sec ? vs : ks;
-#pragma unroll 2
+#pragma unroll 4
         for (int u = threadIdx.x; u < padded; u += kGatherThreads) {
             const bool in = u < units;
             const int vec = cpv_pow2 ? (u >> cpv_shift) : u / cpv;
@@ -251,7 +278,8 @@ extern "C" int patchkv_quantize_gather(patchkv_ctx* ctx, const patchkv_geom* g, 
     p.status = ctx->d_status;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return fail(ctx, PATCHKV_E_CUDA, "cudaSetDevice failed");
-    quantize_gather_kernel<<<nb * g->n_layers, kGatherThreads, 0, static_cast<cudaStream_t>(stream)>>>(p);
+    quantize_gather_kernel<<<nb * g->n_layers, kGatherThreads, g->block_tokens * sizeof(long long),
+                             static_cast<cudaStream_t>(stream)>>>(p);
     PKV_CUDA(ctx, cudaGetLastError());
     return PATCHKV_OK;
 }

@@ -468,6 +468,27 @@ def run_ours(args):
                                 f"per wave (fit rule: the 80-layer pool is 172 GB)", reps=3)
         del sess
 
+    # ---- the paper's restore microbenchmark shape (Section V-E): an ~8k-token checkpoint of a 64-layer, 8-KV-head,
+    #      head_dim-128 model (geometry from the public Qwen3-32B model card, not from the paper), 32-token blocks,
+    #      one fp16 scale per 128 channels, restored whole from pinned host memory in each transport format
+    paper_shape = None
+    if not args.no_host_configs:
+        gm = pin.Geometry(64, 8, 128, 128, pin.ROPE_HALF, 1.0e6, 32, 32, 128)
+        rows = {}
+        for label, probs in (("FP16(bf16)", (1.0, 0, 0, 0)), ("INT8 K8/V8", (0, 1.0, 0, 0)), ("INT4 K4/V4", (0, 0, 0, 1.0)),
+                             ("mixed 2/6/92 % bf16/K8V8/K8V4", (0.02, 0.06, 0.92, 0.0))):
+            cm = pin.make_checkpoint(name="paper-microbench", seed=2024, geom=gm, n=8031, delta=-512, tag_probs=probs,
+                                     n_outlier=6, outlier_scale=10.0, n_pages=256, dirty_tokens=0, top_k=0,
+                                     device=dev, pin_payload=True)
+            r_ = host_leg([cm], label, reps=5)
+            rows[label] = {"payload_mib": r_["bytes_useful"] / 2 ** 20, "fetch_and_restore_ms": r_["ms"],
+                           "payload_gbps": r_["payload_gbps"], "frac_of_link": r_["frac_of_link"], "copies": r_["copies"]}
+            del cm
+        paper_shape = {"workload": "8031-token checkpoint, L=64 H=8 D=128, B=P=32, G=128, every block restored from pinned host",
+                       "formats": rows,
+                       "paper_context_ms": {"FP16": 344.4, "INT8": 183.6, "INT4": 107.2, "PatchKV": 158.0,
+                                            "hardware": "A800 server, PCIe Gen4, 23.3 GiB/s pinned ceiling"}}
+
     # ---- CPU baseline: the checker, as it stands, on a bounded sample of the same workload (rank 0, N = 1)
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu:
@@ -491,7 +512,7 @@ def run_ours(args):
             "select_us": select_us, "restore_ms": restore_avg_ms,
             "block_layers_per_s": world * items / (ms_per_step * 1e-3),
             "real_gbps": world * (read_b + written_b) / (ms_per_step * 1e-3) / 1e9,
-            "host_link": host_link, "select_at_scale": select_scale, "host_7b": host_cfg3, "stress": stress, "writer": writer,
+            "host_link": host_link, "select_at_scale": select_scale, "host_7b": host_cfg3, "stress": stress, "writer": writer, "paper_microbench_shape": paper_shape,
         }
         print(json.dumps(line), flush=True)
     ctx.close()

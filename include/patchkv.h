@@ -87,7 +87,8 @@ enum {
 };
 enum { PATCHKV_ROPE_HALF = 0 /* pairs (i, i + rotary_dim/2) */, PATCHKV_ROPE_INTERLEAVED = 1 /* pairs (2i, 2i+1) */ };
 enum { PATCHKV_LAYERS_INDEPENDENT = 0 /* one (R_l, F_l) per layer */, PATCHKV_LAYERS_SHARED = 1 /* rank on the mass summed over layers */ };
-enum { PATCHKV_SCORE_ATTN_F16 = 0 /* stored attention */, PATCHKV_SCORE_BLOCK_MASS = 1 /* stored per-block mass */ };
+enum { PATCHKV_SCORE_ATTN_F16 = 0 /* stored attention */, PATCHKV_SCORE_BLOCK_MASS = 1 /* stored per-block mass */,
+       PATCHKV_SCORE_TOKEN_MASS = 2 /* stored per-token mass (patchkv_select_repair_tokens) */ };
 
 enum {
     PATCHKV_FLAG_DIRECT_LOADS = 1  /* restore with the plain-load kernel even where the bulk-copy pipeline applies */
@@ -221,6 +222,16 @@ PATCHKV_API int patchkv_last_error(patchkv_ctx* ctx, char* buf, size_t n);
  *   R_l = dirty u H_l and F_l = the rest, both ascending; unused list entries are set to -1.
  * Asynchronous on `stream`; all outputs are caller-allocated DEVICE arrays. */
 PATCHKV_API int patchkv_select_repair(patchkv_ctx* ctx, const patchkv_select_args* args, void* stream);
+
+/* The selection in the form the paper prints it (Section IV-C, Eqs. 10-12): the importance score is per TOKEN,
+ * H_l is the set of the top_k highest-scoring tokens outside the dirty token set D (ties: lower token index; the
+ * caller turns the paper's fraction kappa into a count), and D u H_l is rounded to blocks only afterwards:
+ * R_l = blocks holding a token of D u H_l.  (patchkv_select_repair ranks whole blocks by their summed mass, which
+ * can pick different blocks.)  Same argument struct; differences: kind is PATCHKV_SCORE_ATTN_F16 (token mass is
+ * the exact sum over heads and stored query positions) or PATCHKV_SCORE_TOKEN_MASS (`mass` is DEVICE u64 [L][n]);
+ * `mass_out`, if given, is DEVICE u64 [L][n]; PATCHKV_LAYERS_SHARED ranks on the mass summed over layers, which
+ * is the request-level score of Eq. 10.  Outputs exactly as for patchkv_select_repair. */
+PATCHKV_API int patchkv_select_repair_tokens(patchkv_ctx* ctx, const patchkv_select_args* args, void* stream);
 
 /* The selection of patchkv_select_repair for callers that must not allocate device memory.  (The paper has no
  * counterpart: this is a packaging variant of the same kernels, not another step of the method.)

@@ -95,6 +95,8 @@ def lib():
         l.pkvo_restore.restype = C.c_int
         l.pkvo_restore.argtypes = [C.POINTER(_RestoreArgs)]
         l.pkvo_max_threads.restype = C.c_int
+        l.pkvo_select_tokens.restype = C.c_int
+        l.pkvo_select_tokens.argtypes = [C.c_void_p] + [C.c_int] * 6 + [C.c_void_p] * 6
         l.pkvo_plan_checkpoint.restype = C.c_int
         l.pkvo_plan_checkpoint.argtypes = [C.c_void_p] + [C.c_int] * 6 + [C.c_void_p, C.c_void_p]
         l.pkvo_quantize_gather.restype = C.c_int
@@ -219,6 +221,23 @@ def select(mass: np.ndarray, n: int, B: int, dirty_tokens: int, top_k: int, laye
     fc = np.zeros(L, dtype=np.int32)
     rc = lib().pkvo_select(_p(mass), L, n, B, dirty_tokens, top_k, layer_mode, _p(mask), _p(ri), _p(rc_), _p(fi), _p(fc))
     return dict(status=rc, mask=mask, repair_idx=ri, repair_cnt=rc_, reuse_idx=fi, reuse_cnt=fc)
+
+
+def select_tokens(token_mass: np.ndarray, B: int, dirty_tokens: int, top_tokens: int, layer_mode: int = 1):
+    """Token-level selection (the paper's printed form): token_mass u64 [L][n].  Returns dict(status, token_mask
+    u8 [L][n], mask u8 [L][NB], repair_idx, repair_cnt, reuse_idx, reuse_cnt)."""
+    token_mass = np.ascontiguousarray(token_mass, dtype=np.uint64)
+    L, n = token_mass.shape
+    NB = -(-n // B)
+    tmask = np.zeros((L, n), dtype=np.uint8)
+    mask = np.zeros((L, NB), dtype=np.uint8)
+    ri = np.zeros((L, NB), dtype=np.int32)
+    fi = np.zeros((L, NB), dtype=np.int32)
+    rc_ = np.zeros(L, dtype=np.int32)
+    fc = np.zeros(L, dtype=np.int32)
+    rc = lib().pkvo_select_tokens(_p(token_mass), L, n, B, dirty_tokens, top_tokens, layer_mode, _p(tmask), _p(mask),
+                                  _p(ri), _p(rc_), _p(fi), _p(fc))
+    return dict(status=rc, token_mask=tmask, mask=mask, repair_idx=ri, repair_cnt=rc_, reuse_idx=fi, reuse_cnt=fc)
 
 
 # ---------------------------------------------------------------- restore

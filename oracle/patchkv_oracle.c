@@ -536,3 +536,55 @@ int pkvo_quantize_gather(const pkvo_gather_args* a) {
         }
     return status;
 }
+
+/* ------------------------------------------------------------------ token-level selection (Eqs. 9-12 as printed) */
+/* The paper's own form of the selection: the importance score is per TOKEN, H is the set of the top-kappa tokens
+ * outside the dirty token set D, and only then is D u H rounded to blocks:
+ *   D   = the first min(max(dirty_tokens, 0), n) suffix tokens                      (Eq. 9)
+ *   H_l = the min(top_tokens, #candidates) tokens outside D with the largest score; ties: lower token index (Eq. 11)
+ *   R_l = blocks holding a token of D u H_l,  F_l = the other blocks, both ascending (Eq. 12)
+ * token_mass is u64 [L][n] (the exact attention mass of Eq. 10 at token granularity, B = 1 in pkvo_block_mass).
+ * LAYERS_SHARED ranks on the mass summed over layers, the request-level reading of Eq. 10.
+ * Outputs as pkvo_select, plus an optional token mask u8 [L][n] (1 = token in D u H_l). */
+int pkvo_select_tokens(const uint64_t* token_mass, int L, int n, int B, int dirty_tokens, int top_tokens, int layer_mode,
+                       uint8_t* token_mask, uint8_t* mask, int32_t* repair_idx, int32_t* repair_cnt,
+                       int32_t* reuse_idx, int32_t* reuse_cnt) {
+    if (L <= 0 || n < 0 || B <= 0 || top_tokens < 0) return PKVO_E_INVALID;
+    if (layer_mode != PKVO_LAYERS_INDEPENDENT && layer_mode != PKVO_LAYERS_SHARED) return PKVO_E_INVALID;
+    int NB = (n + B - 1) / B;
+    int64_t nd64 = dirty_tokens < 0 ? 0 : dirty_tokens;
+    if (nd64 > n) nd64 = n;
+    int nd = (int)nd64;
+    cand_t* cand = (cand_t*)malloc(sizeof(cand_t) * (size_t)(n > 0 ? n : 1));
+    uint8_t* tmask = (uint8_t*)malloc((size_t)(n > 0 ? n : 1));
+    uint64_t* shared = NULL;
+    if (layer_mode == PKVO_LAYERS_SHARED) {
+        shared = (uint64_t*)calloc((size_t)(n > 0 ? n : 1), sizeof(uint64_t));
+        for (int l = 0; l < L; l++) for (int i = 0; i < n; i++) shared[i] += token_mass[(int64_t)l * n + i];
+    }
+    for (int l = 0; l < L; l++) {
+        const uint64_t* m = shared ? shared : token_mass + (int64_t)l * n;
+        int nc = 0;
+        for (int i = 0; i < n; i++) {
+            tmask[i] = i < nd;
+            if (i >= nd) { cand[nc].mass = m[i]; cand[nc].idx = i; nc++; }
+        }
+        qsort(cand, (size_t)nc, sizeof(cand_t), cand_cmp);
+        int take = top_tokens < nc ? top_tokens : nc;
+        for (int i = 0; i < take; i++) tmask[cand[i].idx] = 1;
+        if (token_mask) memcpy(token_mask + (int64_t)l * n, tmask, (size_t)n);
+        int nr = 0, nf = 0;
+        for (int j = 0; j < NB; j++) {
+            int hit = 0;
+            for (int i = j * B; i < (j + 1) * B && i < n; i++) hit |= tmask[i];   /* BlockRound: blocks that intersect */
+            mask[(int64_t)l * NB + j] = (uint8_t)hit;
+            if (hit) repair_idx[(int64_t)l * NB + nr++] = j;
+            else     reuse_idx[(int64_t)l * NB + nf++] = j;
+        }
+        for (int i = nr; i < NB; i++) repair_idx[(int64_t)l * NB + i] = -1;
+        for (int i = nf; i < NB; i++) reuse_idx[(int64_t)l * NB + i] = -1;
+        repair_cnt[l] = nr; reuse_cnt[l] = nf;
+    }
+    free(cand); free(tmask); free(shared);
+    return PKVO_OK;
+}

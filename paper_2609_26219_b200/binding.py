@@ -21,7 +21,7 @@ STATIC_MAX_MASS_ELEMS = 262144
 TAG_BF16, TAG_INT8, TAG_INT4, TAG_K4V4 = 0, 1, 2, 3
 ROPE_HALF, ROPE_INTERLEAVED = 0, 1
 LAYERS_INDEPENDENT, LAYERS_SHARED = 0, 1
-SCORE_ATTN_F16, SCORE_BLOCK_MASS = 0, 1
+SCORE_ATTN_F16, SCORE_BLOCK_MASS, SCORE_TOKEN_MASS = 0, 1, 2
 MAX_SESSIONS = 8
 FLAG_DIRECT_LOADS = 1
 
@@ -83,6 +83,8 @@ def lib():
         l.patchkv_destroy.argtypes = [C.c_void_p]
         l.patchkv_last_error.argtypes = [C.c_void_p, C.c_char_p, C.c_size_t]
         l.patchkv_select_repair.argtypes = [C.c_void_p, C.POINTER(SelectArgs), C.c_void_p]
+        l.patchkv_select_repair_tokens.argtypes = [C.c_void_p, C.POINTER(SelectArgs), C.c_void_p]
+        l.patchkv_select_repair_tokens.restype = C.c_int
         l.patchkv_select_repair_static.argtypes = [C.POINTER(SelectArgs), C.c_void_p, C.c_void_p]
         l.patchkv_select_repair_static.restype = C.c_int
         l.patchkv_restore.argtypes = [C.c_void_p, C.POINTER(Geom), C.POINTER(Pool), C.c_void_p, C.c_int, C.c_void_p]
@@ -173,6 +175,9 @@ class Context:
 
     def select_repair(self, args: SelectArgs, stream=None, check: bool = True) -> int:
         return self._check(lib().patchkv_select_repair(self._h, C.byref(args), _stream_handle(stream)), check)
+
+    def select_repair_tokens(self, args: SelectArgs, stream=None, check: bool = True) -> int:
+        return self._check(lib().patchkv_select_repair_tokens(self._h, C.byref(args), _stream_handle(stream)), check)
 
     def restore(self, geom: Geom, pool: Pool, sessions: List[Session], stream=None, check: bool = True) -> int:
         arr = (Session * max(len(sessions), 1))(*sessions)

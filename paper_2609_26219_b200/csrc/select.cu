@@ -312,7 +312,8 @@ select_kernel(const TopkParams p) {
     uint8_t* mask = p.mask + (long long)l * NB;
     int32_t* ridx = p.repair_idx + (long long)l * NB;
     int32_t* fidx = p.reuse_idx + (long long)l * NB;
-    for (int j = threadIdx.x; j < n_dirty; j += kSelThreads) { mask[j] = 1; ridx[j] = j; }
+    const bool lists = p.repair_idx != nullptr;          // the token-level stage only needs the mask
+    for (int j = threadIdx.x; j < n_dirty; j += kSelThreads) { mask[j] = 1; if (lists) ridx[j] = j; }
     int run_sel = 0, run_eq = 0;
     for (int i = 0; i < iters; i++) {
         const int c = threadIdx.x + i * kSelThreads;
@@ -337,14 +338,51 @@ select_kernel(const TopkParams p) {
         if (in) {
             const int j = n_dirty + c;
             mask[j] = sel ? 1 : 0;
-            if (sel) ridx[n_dirty + before] = j;
-            else fidx[c - before] = j;
+            if (lists) {
+                if (sel) ridx[n_dirty + before] = j;
+                else fidx[c - before] = j;
+            }
         }
     }
+    if (!lists) return;
     const int n_r = n_dirty + run_sel, n_f = NB - n_r;
     for (int i = n_r + threadIdx.x; i < NB; i += kSelThreads) ridx[i] = -1;
     for (int i = n_f + threadIdx.x; i < NB; i += kSelThreads) fidx[i] = -1;
     if (threadIdx.x == 0) { p.repair_cnt[l] = n_r; p.reuse_cnt[l] = n_f; }
+}
+
+// BlockRound of Eq. 12: a block is repaired when any of its tokens is in D u H.  One CTA per layer turns the token
+// mask into the block mask and the ascending repair / reuse lists.
+__global__ void __launch_bounds__(kSelThreads)
+block_round_kernel(const uint8_t* token_mask, int n, int B, int NB, uint8_t* mask, int32_t* repair_idx,
+                   int32_t* repair_cnt, int32_t* reuse_idx, int32_t* reuse_cnt) {
+    __shared__ int warp_sums[33];
+    const int l = blockIdx.x;
+    const uint8_t* tm = token_mask + (long long)l * n;
+    uint8_t* bm = mask + (long long)l * NB;
+    int32_t* ridx = repair_idx + (long long)l * NB;
+    int32_t* fidx = reuse_idx + (long long)l * NB;
+    int run = 0;
+    for (int j0 = 0; j0 < NB; j0 += kSelThreads) {
+        const int j = j0 + threadIdx.x;
+        int hit = 0;
+        if (j < NB) {
+            const int e = min(n, (j + 1) * B);
+            for (int i = j * B; i < e; i++) hit |= tm[i];
+        }
+        int tot;
+        const int before = block_exclusive_scan(hit, warp_sums, &tot) + run;
+        run += tot;
+        if (j < NB) {
+            bm[j] = (uint8_t)hit;
+            if (hit) ridx[before] = j;
+            else fidx[j - before] = j;
+        }
+    }
+    const int n_r = run, n_f = NB - run;
+    for (int i = n_r + threadIdx.x; i < NB; i += kSelThreads) ridx[i] = -1;
+    for (int i = n_f + threadIdx.x; i < NB; i += kSelThreads) fidx[i] = -1;
+    if (threadIdx.x == 0) { repair_cnt[l] = n_r; reuse_cnt[l] = n_f; }
 }
 
 static int ensure_mass_ws(patchkv_ctx* ctx, size_t elems) {
@@ -437,6 +475,87 @@ extern "C" int patchkv_select_repair(patchkv_ctx* ctx, const patchkv_select_args
     tp.mask = a->repair_mask; tp.repair_idx = a->repair_idx; tp.repair_cnt = a->repair_cnt;
     tp.reuse_idx = a->reuse_idx; tp.reuse_cnt = a->reuse_cnt;
     select_kernel<<<L, kSelThreads, 0, stream>>>(tp);
+    PKV_CUDA(ctx, cudaGetLastError());
+    return PATCHKV_OK;
+}
+
+// ---------------------------------------------------------------- token-level selection
+extern "C" int patchkv_select_repair_tokens(patchkv_ctx* ctx, const patchkv_select_args* a, void* stream_) {
+    if (!ctx) return PATCHKV_E_INVALID;
+    std::lock_guard<std::mutex> lock(ctx->mu);
+    if (!a || a->struct_size != sizeof(patchkv_select_args)) return fail(ctx, PATCHKV_E_INVALID, "select: null args or struct_size mismatch");
+    if (a->n_layers <= 0 || a->n_layers > 65535 || a->n_suffix_tokens < 0 || a->block_tokens <= 0 || a->top_k < 0)
+        return fail(ctx, PATCHKV_E_INVALID, "select: need 0 < L <= 65535, n >= 0, B > 0, top_k >= 0");
+    if (a->layer_mode != PATCHKV_LAYERS_INDEPENDENT && a->layer_mode != PATCHKV_LAYERS_SHARED)
+        return fail(ctx, PATCHKV_E_INVALID, "select: unknown layer_mode");
+    if (a->kind != PATCHKV_SCORE_ATTN_F16 && a->kind != PATCHKV_SCORE_TOKEN_MASS)
+        return fail(ctx, PATCHKV_E_INVALID, "select: kind must be ATTN_F16 or TOKEN_MASS");
+    if (!a->repair_mask || !a->repair_idx || !a->repair_cnt || !a->reuse_idx || !a->reuse_cnt)
+        return fail(ctx, PATCHKV_E_INVALID, "select: null output");
+    const int L = a->n_layers, n = a->n_suffix_tokens, B = a->block_tokens;
+    const int NB = (int)(((long long)n + B - 1) / B);
+    long long nd = a->dirty_tokens < 0 ? 0 : a->dirty_tokens;
+    if (nd > n) nd = n;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, PATCHKV_E_CUDA, "cudaSetDevice failed");
+
+    const bool shared = a->layer_mode == PATCHKV_LAYERS_SHARED && L > 1;
+    const bool from_attn = a->kind == PATCHKV_SCORE_ATTN_F16;
+    // workspace: [token mass L*n (if computed here and not handed out)] [summed mass n (shared)] [token mask L*n bytes]
+    const size_t mass_elems = from_attn && !a->mass_out ? (size_t)L * n : 0;
+    const size_t sum_elems = shared ? (size_t)n : 0;
+    const size_t mask_words = ((size_t)L * n + 7) / 8;
+    int rc = ensure_mass_ws(ctx, mass_elems + sum_elems + mask_words + 1);
+    if (rc != PATCHKV_OK) return rc;
+    unsigned long long* ws = ctx->d_mass_ws;
+    unsigned long long* ws_sum = ws + mass_elems;
+    uint8_t* tok_mask = reinterpret_cast<uint8_t*>(ws_sum + sum_elems);
+
+    const unsigned long long* mass = reinterpret_cast<const unsigned long long*>(a->mass);
+    if (from_attn) {
+        if (a->n_q_heads < 0 || a->n_queries < 0 || (n > 0 && a->n_q_heads > 0 && a->n_queries > 0 && !a->attn))
+            return fail(ctx, PATCHKV_E_INVALID, "select: attention shape / pointer");
+        unsigned long long* m = a->mass_out ? reinterpret_cast<unsigned long long*>(a->mass_out) : ws;
+        const long long rows = (long long)a->n_q_heads * a->n_queries;
+        if (rows > 0x7fffffffLL) return fail(ctx, PATCHKV_E_UNSUPPORTED, "select: Hq * Q too large");
+        if (n > 0) PKV_CUDA(ctx, cudaMemsetAsync(m, 0, (size_t)L * n * sizeof(unsigned long long), stream));
+        if (n > 0 && rows > 0) {
+            MassParams mp;                         // token granularity: a block of one token
+            mp.attn = static_cast<const uint16_t*>(a->attn);
+            mp.stride_layer = a->attn_stride_layer; mp.stride_head = a->attn_stride_head; mp.stride_query = a->attn_stride_query;
+            mp.Hq = a->n_q_heads; mp.Q = a->n_queries; mp.n = n; mp.B = 1; mp.NB = n;
+            mp.mass = m; mp.status = ctx->d_status;
+            const int tiles = (n + 255) / 256;
+            long long groups = (long long)ctx->sm_count * 16 / ((long long)tiles * L);
+            if (groups < 1) groups = 1;
+            long long rpc = (rows + groups - 1) / groups;
+            if (rpc < 64) rpc = 64;
+            if (rpc > rows) rpc = rows;
+            groups = (rows + rpc - 1) / rpc;
+            if (groups > 65535) return fail(ctx, PATCHKV_E_UNSUPPORTED, "select: grid too large");
+            mp.rows_per_cta = (int)rpc;
+            block_mass_generic_kernel<<<dim3(tiles, (unsigned)groups, L), 256, 0, stream>>>(mp);
+            PKV_CUDA(ctx, cudaGetLastError());
+        }
+        mass = m;
+    } else if (n > 0 && !mass) {
+        return fail(ctx, PATCHKV_E_INVALID, "select: null mass");
+    }
+
+    TopkParams tp;
+    tp.mass = mass; tp.shared = 0;
+    if (shared && n > 0) {
+        sum_layers_kernel<<<(n + 255) / 256, 256, 0, stream>>>(mass, L, n, ws_sum);
+        PKV_CUDA(ctx, cudaGetLastError());
+        tp.mass = ws_sum; tp.shared = 1;
+    }
+    tp.NB = n; tp.n_dirty = (int)nd; tp.top_k = a->top_k;     // the "blocks" of this stage are single tokens
+    tp.mask = tok_mask; tp.repair_idx = nullptr; tp.repair_cnt = nullptr; tp.reuse_idx = nullptr; tp.reuse_cnt = nullptr;
+    select_kernel<<<L, kSelThreads, 0, stream>>>(tp);
+    PKV_CUDA(ctx, cudaGetLastError());
+    block_round_kernel<<<L, kSelThreads, 0, stream>>>(tok_mask, n, B, NB, a->repair_mask, a->repair_idx, a->repair_cnt,
+                                                      a->reuse_idx, a->reuse_cnt);
     PKV_CUDA(ctx, cudaGetLastError());
     return PATCHKV_OK;
 }

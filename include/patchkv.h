@@ -276,6 +276,22 @@ PATCHKV_API int patchkv_restore_from_host(patchkv_ctx* ctx, const patchkv_geom* 
                                           const patchkv_session_host* sessions, int n_sessions, void* stream,
                                           patchkv_restore_stats* stats);
 
+/* ---- precision planner (offload side) -----------------------------------------------------------------------
+ * Section IV-D, Eqs. 13-14: for every block b of the suffix, Z_i = sqrt(A_i * e_i) over its tokens (A_i the
+ * normalised stored attention mass, e_i the normalised residual of the candidate low-bit value representation),
+ * r_b = alpha * max_i Z_i + (1 - alpha) * mean_i Z_i, and the frozen tag
+ *     r_b >= tau_H                  -> PATCHKV_TAG_BF16 (full precision)
+ *     tau_L <= r_b < tau_H          -> PATCHKV_TAG_INT8 (K8/V8)
+ *     r_b < tau_L and G4(b)         -> PATCHKV_TAG_INT4 (K8/V4)
+ *     r_b < tau_L and not G4(b)     -> PATCHKV_TAG_INT8
+ * The low-bit test G4 is not spelled out in the paper; here G4(b) = (max_i e_i <= eps4).  The calibration that
+ * produces alpha, tau_L, tau_H, eps4 and the measurement of e_i are the caller's.  fp32 throughout, tokens in
+ * ascending order, every operation rounded on its own.
+ *   attn, resid  DEVICE fp32 [n]     tags DEVICE u8 [NB] (out)     risk DEVICE fp32 [NB] (out, optional) */
+PATCHKV_API int patchkv_plan_precision(patchkv_ctx* ctx, const float* attn, const float* resid, int n_suffix_tokens,
+                                       int block_tokens, float alpha, float tau_L, float tau_H, float eps4,
+                                       uint8_t* tags, float* risk, void* stream);
+
 /* ---- checkpoint writer (offload side; not on the resume path) ----------------------------------------------
  * Section IV-D: at offload a fused kernel gathers the rows of each suffix block, computes the scales and packs
  * the payload at the block's calibrated precision; blocks of the same representation form contiguous runs.

@@ -97,6 +97,9 @@ def lib():
         l.pkvo_max_threads.restype = C.c_int
         l.pkvo_select_tokens.restype = C.c_int
         l.pkvo_select_tokens.argtypes = [C.c_void_p] + [C.c_int] * 6 + [C.c_void_p] * 6
+        l.pkvo_plan_precision.restype = C.c_int
+        l.pkvo_plan_precision.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_float, C.c_float, C.c_float,
+                                          C.c_float, C.c_void_p, C.c_void_p]
         l.pkvo_plan_checkpoint.restype = C.c_int
         l.pkvo_plan_checkpoint.argtypes = [C.c_void_p] + [C.c_int] * 6 + [C.c_void_p, C.c_void_p]
         l.pkvo_quantize_gather.restype = C.c_int
@@ -311,3 +314,15 @@ def quantize_gather(*, L, H, D, B, P, G, k_pool: np.ndarray, v_pool: np.ndarray,
                     n_pages=n_pages, n=n, src_shift=src_shift, block_table=_p(block_table), n_table=block_table.size,
                     tags=_p(tags), blk_off=_p(blk_off), layer_payload=C.cast(ptrs, C.c_void_p), layer_bytes=_p(lbytes))
     return lib().pkvo_quantize_gather(C.byref(a))
+
+
+def plan_precision(attn: np.ndarray, resid: np.ndarray, B: int, alpha: float, tau_L: float, tau_H: float, eps4: float):
+    """Eqs. 13-14: per-token fp32 attention mass and low-bit residual -> (status, tags u8 [NB], risk fp32 [NB])."""
+    attn = np.ascontiguousarray(attn, dtype=np.float32)
+    resid = np.ascontiguousarray(resid, dtype=np.float32)
+    n = attn.size
+    NB = -(-n // B)
+    tags = np.zeros(NB, dtype=np.uint8)
+    risk = np.zeros(NB, dtype=np.float32)
+    rc = lib().pkvo_plan_precision(_p(attn), _p(resid), n, B, alpha, tau_L, tau_H, eps4, _p(tags), _p(risk))
+    return rc, tags, risk

@@ -588,3 +588,44 @@ int pkvo_select_tokens(const uint64_t* token_mass, int L, int n, int B, int dirt
     free(cand); free(tmask); free(shared);
     return PKVO_OK;
 }
+
+/* ------------------------------------------------------------------ precision planner (Eqs. 13-14) */
+/* Per block b of the suffix: Z_i = sqrt(A_i * e_i) for its tokens (A_i the normalised stored attention mass, e_i the
+ * normalised residual of the candidate low-bit V representation), r_b = alpha * max Z + (1 - alpha) * mean Z, and
+ *   tag = BF16 (the full-precision tier)  if r_b >= tau_H
+ *         INT8 (K8/V8)                    if tau_L <= r_b < tau_H
+ *         INT4 (K8/V4)                    if r_b < tau_L and G4(b)
+ *         INT8                            if r_b < tau_L and not G4(b)
+ * The paper leaves the low-bit test G4 open; the reading here is G4(b) = (max_i e_i <= eps4).  All arithmetic is
+ * fp32 with every operation rounded on its own, tokens taken in ascending order, so that the decision is made in
+ * one fixed precision on both sides.  attn, resid: fp32 [n]; tags u8 [NB]; risk fp32 [NB] (optional). */
+int pkvo_plan_precision(const float* attn, const float* resid, int n, int B, float alpha, float tau_L, float tau_H,
+                        float eps4, uint8_t* tags, float* risk) {
+    if (n < 0 || B <= 0 || !(alpha >= 0.0f && alpha <= 1.0f) || !(tau_L < tau_H)) return PKVO_E_INVALID;
+    int NB = (n + B - 1) / B;
+    for (int j = 0; j < NB; j++) {
+        float zmax = 0.0f, zsum = 0.0f, emax = 0.0f;
+        int cnt = 0;
+        for (int i = j * B; i < (j + 1) * B && i < n; i++) {
+            volatile float prod = attn[i] * resid[i];
+            float z = sqrtf(prod);
+            if (z > zmax) zmax = z;
+            if (resid[i] > emax) emax = resid[i];
+            volatile float s = zsum + z;
+            zsum = s;
+            cnt++;
+        }
+        volatile float mean = zsum / (float)cnt;
+        volatile float t1 = alpha * zmax;
+        volatile float om = 1.0f - alpha;
+        volatile float t2 = om * mean;
+        float r = t1 + t2;
+        if (risk) risk[j] = r;
+        uint8_t tag;
+        if (r >= tau_H) tag = PKVO_TAG_BF16;
+        else if (r >= tau_L) tag = PKVO_TAG_INT8;
+        else tag = emax <= eps4 ? PKVO_TAG_INT4 : PKVO_TAG_INT8;
+        tags[j] = tag;
+    }
+    return PKVO_OK;
+}

@@ -93,6 +93,9 @@ def lib():
         l.patchkv_plan_checkpoint.argtypes = [C.c_void_p, C.POINTER(Geom), C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
                                               C.c_void_p]
         l.patchkv_quantize_gather.argtypes = [C.c_void_p, C.POINTER(Geom), C.POINTER(Pool), C.POINTER(Session), C.c_void_p]
+        l.patchkv_plan_precision.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_float, C.c_float,
+                                             C.c_float, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p]
+        l.patchkv_plan_precision.restype = C.c_int
         l.patchkv_query_status.argtypes = [C.c_void_p, C.POINTER(C.c_int)]
         l.patchkv_record_bytes.argtypes = [C.c_int] * 5
         l.patchkv_record_bytes.restype = C.c_uint64
@@ -200,6 +203,14 @@ class Context:
     def quantize_gather(self, geom: Geom, pool: Pool, session: Session, stream=None, check: bool = True) -> int:
         return self._check(lib().patchkv_quantize_gather(self._h, C.byref(geom), C.byref(pool), C.byref(session),
                                                          _stream_handle(stream)), check)
+
+    def plan_precision(self, attn: torch.Tensor, resid: torch.Tensor, block_tokens: int, alpha: float, tau_L: float,
+                       tau_H: float, eps4: float, tags: torch.Tensor, risk: Optional[torch.Tensor] = None,
+                       stream=None, check: bool = True) -> int:
+        """Eqs. 13-14: fp32 device tensors attn [n], resid [n] -> tags u8 [NB] (and risk fp32 [NB])."""
+        return self._check(lib().patchkv_plan_precision(self._h, _ptr(attn), _ptr(resid), attn.numel(), block_tokens,
+                                                        alpha, tau_L, tau_H, eps4, _ptr(tags), _ptr(risk),
+                                                        _stream_handle(stream)), check)
 
     def query_status(self) -> int:
         v = C.c_int(0)

@@ -283,3 +283,53 @@ extern "C" int patchkv_quantize_gather(patchkv_ctx* ctx, const patchkv_geom* g, 
     PKV_CUDA(ctx, cudaGetLastError());
     return PATCHKV_OK;
 }
+
+// ---------------------------------------------------------------- precision planner (Eqs. 13-14)
+namespace patchkv {
+
+// One thread per block walks its tokens in ascending order with separately rounded fp32 operations, so the tag is
+// decided in one fixed precision and order (the same sequence a scalar host program would take).
+__global__ void plan_precision_kernel(const float* attn, const float* resid, int n, int B, int NB, float alpha,
+                                      float tau_L, float tau_H, float eps4, uint8_t* tags, float* risk) {
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= NB) return;
+    float zmax = 0.0f, zsum = 0.0f, emax = 0.0f;
+    int cnt = 0;
+    const int e = min(n, (j + 1) * B);
+    for (int i = j * B; i < e; i++) {
+        const float a = __ldg(attn + i), r = __ldg(resid + i);
+        const float z = __fsqrt_rn(__fmul_rn(a, r));
+        if (z > zmax) zmax = z;
+        if (r > emax) emax = r;
+        zsum = __fadd_rn(zsum, z);
+        cnt++;
+    }
+    const float mean = __fdiv_rn(zsum, (float)cnt);
+    const float rb = __fadd_rn(__fmul_rn(alpha, zmax), __fmul_rn(__fsub_rn(1.0f, alpha), mean));
+    if (risk) risk[j] = rb;
+    uint8_t tag;
+    if (rb >= tau_H) tag = PATCHKV_TAG_BF16;
+    else if (rb >= tau_L) tag = PATCHKV_TAG_INT8;
+    else tag = emax <= eps4 ? PATCHKV_TAG_INT4 : PATCHKV_TAG_INT8;
+    tags[j] = tag;
+}
+
+}  // namespace patchkv
+
+extern "C" int patchkv_plan_precision(patchkv_ctx* ctx, const float* attn, const float* resid, int n_suffix_tokens,
+                                      int block_tokens, float alpha, float tau_L, float tau_H, float eps4,
+                                      uint8_t* tags, float* risk, void* stream) {
+    if (!ctx) return PATCHKV_E_INVALID;
+    std::lock_guard<std::mutex> lock(ctx->mu);
+    if (n_suffix_tokens < 0 || block_tokens <= 0 || !(alpha >= 0.0f && alpha <= 1.0f) || !(tau_L < tau_H))
+        return fail(ctx, PATCHKV_E_INVALID, "plan_precision: need n >= 0, B > 0, 0 <= alpha <= 1, tau_L < tau_H");
+    const int NB = (int)(((long long)n_suffix_tokens + block_tokens - 1) / block_tokens);
+    if (NB == 0) return PATCHKV_OK;
+    if (!attn || !resid || !tags) return fail(ctx, PATCHKV_E_INVALID, "plan_precision: null pointer");
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, PATCHKV_E_CUDA, "cudaSetDevice failed");
+    plan_precision_kernel<<<(NB + 127) / 128, 128, 0, static_cast<cudaStream_t>(stream)>>>(
+        attn, resid, n_suffix_tokens, block_tokens, NB, alpha, tau_L, tau_H, eps4, tags, risk);
+    PKV_CUDA(ctx, cudaGetLastError());
+    return PATCHKV_OK;
+}

@@ -161,3 +161,26 @@ def test_full_size_8b_shape_writer_then_restore_round_trip(ctx):
     err = (a - b).abs()[:, used]
     bound = (0.5 * step * 1.01 + a.abs() * 2.0 ** -8 + amax.expand(*amax.shape[:-1], g.group).reshape(a.shape) * 2.0 ** -10)[:, used]
     assert bool((err <= bound).all())
+
+
+@pytest.mark.parametrize("n,B", [(65536, 32), (1000, 16), (7, 16)])
+def test_precision_planner_matches_the_oracle_bit_for_bit(ctx, n, B):
+    rng = np.random.default_rng(n)
+    attn = (rng.random(n) ** 4 / n * 8).astype(np.float32)
+    resid = (rng.random(n) * 0.3).astype(np.float32)
+    NB = -(-n // B)
+    for alpha in (0.5, 0.0, 1.0):
+        # thresholds at quantiles of the risk so that every tier occurs (the real ones come from calibration)
+        _, _, r0 = oracle.plan_precision(attn, resid, B, alpha, 0.0, 1.0, 1.0)
+        tl, th = (float(np.quantile(r0, 0.4)), float(np.quantile(r0, 0.8))) if NB > 4 else (1e-4, 1e-3)
+        e4 = float(np.median(resid.reshape(-1)[:NB * B - (NB * B - n)].max())) * 0.97
+        rc, tags_o, risk_o = oracle.plan_precision(attn, resid, B, alpha, tl, th, e4)
+        assert rc == oracle.OK
+        tags = torch.full((NB,), 9, dtype=torch.uint8, device=DEV)
+        risk = torch.zeros(NB, dtype=torch.float32, device=DEV)
+        ctx.plan_precision(torch.from_numpy(attn).to(DEV), torch.from_numpy(resid).to(DEV), B, alpha, tl, th, e4, tags, risk)
+        torch.cuda.synchronize()
+        assert np.array_equal(risk.cpu().numpy().view(np.uint32), risk_o.view(np.uint32))
+        assert np.array_equal(tags.cpu().numpy(), tags_o)
+        if n > 1000:
+            assert len(set(tags_o)) == 3         # all three tiers occur

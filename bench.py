@@ -433,7 +433,16 @@ def run_ours(args):
     if not args.no_host_configs:
         ceiling = pinned_copy_ceiling(dev)
 
-        def host_leg(cks, label, reps=5):
+        ctx_direct = pk.Context(device=local_rank, flags=pk.FLAG_HOST_DIRECT)
+
+        def host_leg(cks, label, reps=5, both=False):
+            out_ = host_leg_on(ctx, cks, label, reps)
+            if both:     # the same through the zero-copy variant: the kernel pulls the records over the link itself
+                d_ = host_leg_on(ctx_direct, cks, label, reps)
+                out_["zero_copy"] = {k_: d_[k_] for k_ in ("ms", "payload_gbps", "frac_of_link", "bytes_copied", "copies")}
+            return out_
+
+        def host_leg_on(ctx, cks, label, reps=5):
             sts = [StagedCheckpoint(c, dev, payload_on_host=True) for c in cks]
             for s_ in sts:
                 ctx.select_repair(s_.select_args(), stream)
@@ -473,14 +482,14 @@ def run_ours(args):
         torch.cuda.empty_cache()
         c3 = pin.config_7b_host(device=dev, pin_payload=True)
         host_cfg3 = host_leg([c3], "7b-shaped: L=28 H=4 D=128 base=1e6 n=32768 delta=-3000, pinned host payload, "
-                                   "4096-page pool (2x), shuffled free list")
+                                   "4096-page pool (2x), shuffled free list", both=True)
         del c3
         SLy = args.stress_layers
         sess = [pin.config_stress_session(i, device=dev, n_layers=SLy, pin_payload=True) for i in range(8)]
         pin.shared_free_list(1005, 8 * 4096, sess)
         stress = host_leg(sess, f"70b-shaped stress: 8 sessions x 64k-token suffix, H=8 D=128, int4 share 10-60 %, "
                                 f"one shared pool of 32768 pages, pinned host payload; {SLy} of 80 layers resident "
-                                f"per wave (fit rule: the 80-layer pool is 172 GB)", reps=3)
+                                f"per wave (fit rule: the 80-layer pool is 172 GB)", reps=3, both=True)
         del sess
 
     # ---- the paper's restore microbenchmark shape (Section V-E): an ~8k-token checkpoint of a 64-layer, 8-KV-head,

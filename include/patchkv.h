@@ -91,7 +91,9 @@ enum { PATCHKV_SCORE_ATTN_F16 = 0 /* stored attention */, PATCHKV_SCORE_BLOCK_MA
        PATCHKV_SCORE_TOKEN_MASS = 2 /* stored per-token mass (patchkv_select_repair_tokens) */ };
 
 enum {
-    PATCHKV_FLAG_DIRECT_LOADS = 1  /* restore with the plain-load kernel even where the bulk-copy pipeline applies */
+    PATCHKV_FLAG_DIRECT_LOADS = 1, /* restore with the plain-load kernel even where the bulk-copy pipeline applies */
+    PATCHKV_FLAG_HOST_DIRECT = 2   /* restore_from_host: no staging copies; the restore kernel reads the pinned payload
+                                      through its device alias, so exactly the reused records cross the link */
 };
 
 enum {

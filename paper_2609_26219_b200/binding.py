@@ -24,6 +24,7 @@ LAYERS_INDEPENDENT, LAYERS_SHARED = 0, 1
 SCORE_ATTN_F16, SCORE_BLOCK_MASS, SCORE_TOKEN_MASS = 0, 1, 2
 MAX_SESSIONS = 8
 FLAG_DIRECT_LOADS = 1
+FLAG_HOST_DIRECT = 2
 
 
 class Config(C.Structure):

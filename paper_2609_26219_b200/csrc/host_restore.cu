@@ -114,7 +114,8 @@ extern "C" int patchkv_restore_from_host(patchkv_ctx* ctx, const patchkv_geom* g
         PKV_CUDA(ctx, cudaEventSynchronize(ctx->ev_done));
         ctx->host_call_pending = false;
     }
-    rc = ensure_host_workspace(ctx, meta, std::max<size_t>(slot_bytes, 16));
+    const bool direct = (ctx->flags & PATCHKV_FLAG_HOST_DIRECT) != 0;
+    rc = ensure_host_workspace(ctx, meta, direct ? 16 : std::max<size_t>(slot_bytes, 16));
     if (rc != PATCHKV_OK) return rc;
     const int n_slots = (int)ctx->slots.size();
 
@@ -145,7 +146,17 @@ extern "C" int patchkv_restore_from_host(patchkv_ctx* ctx, const patchkv_geom* g
         d.reuse_cnt = reinterpret_cast<const int32_t*>(ctx->d_meta + put(s.reuse_cnt, (size_t)L * 4));
         d.layer_bytes = reinterpret_cast<const unsigned long long*>(ctx->d_meta + put(s.layer_bytes, (size_t)L * 8));
         std::vector<const void*> staged(L);
-        for (int l = 0; l < L; l++) staged[l] = ctx->slots[(unit0 + l) % n_slots].base;
+        for (int l = 0; l < L; l++) {
+            if (!direct) { staged[l] = ctx->slots[(unit0 + l) % n_slots].base; continue; }
+            // zero-copy: the kernel's bulk copies read the pinned payload through its device alias
+            void* alias = nullptr;
+            if (s.layer_bytes[l] != 0 &&
+                cudaHostGetDevicePointer(&alias, const_cast<void*>(s.layer_payload[l]), 0) != cudaSuccess) {
+                cudaGetLastError();
+                return fail(ctx, PATCHKV_E_INVALID, "session: pinned payload has no device alias (not mapped)");
+            }
+            staged[l] = alias;
+        }
         d.layer_payload = reinterpret_cast<const void* const*>(ctx->d_meta + put(staged.data(), (size_t)L * 8));
         d.block_table = reinterpret_cast<const int32_t*>(ctx->d_meta + put(s.block_table, (size_t)s.n_table * 4));
         build_rope_table(geom, s.delta, per[i].cs[0][0], per[i].cs[0][1]);
@@ -153,10 +164,41 @@ extern "C" int patchkv_restore_from_host(patchkv_ctx* ctx, const patchkv_geom* g
     }
     PKV_CUDA(ctx, cudaMemcpyAsync(ctx->d_meta, ctx->h_meta, cur, cudaMemcpyHostToDevice, ctx->decode_stream));
 
-    // ---- units
     patchkv_restore_stats st;
     memset(&st, 0, sizeof(st));
     st.struct_size = sizeof(st);
+    if (direct) {
+        // one launch over every session and layer; exactly the reused records cross the link, pulled by the kernel
+        RestoreParams& q = base;
+        q.n_sessions = n_sessions; q.layer_begin = 0; q.layer_end = L;
+        long long items = 0;
+        for (int i = 0; i < n_sessions; i++) {
+            q.s[i] = per[i].s[0];
+            memcpy(q.cs[i], per[i].cs[0], sizeof(q.cs[i]));
+            q.s[i].item_begin = (int32_t)items;
+            items += (long long)nbs[i] * L;
+            if (items > 0x7fff0000LL) return fail(ctx, PATCHKV_E_UNSUPPORTED, "restore_from_host: too many work items");
+            const patchkv_session_host& s = sessions[i];
+            for (int l = 0; l < L && nbs[i] > 0; l++)
+                for (int r = 0; r < s.reuse_cnt[l]; r++) {
+                    const int j = s.reuse_idx[(size_t)l * nbs[i] + r];
+                    if (j < 0 || j >= nbs[i]) continue;
+                    st.bytes_useful += record_bytes(s.tags[(size_t)l * nbs[i] + j], elems, geom->group);
+                    st.n_block_layers++;
+                }
+        }
+        st.bytes_copied = st.bytes_useful;
+        q.total_items = (int32_t)items;
+        rc = launch_restore(ctx, &q, ctx->decode_stream);
+        if (rc != PATCHKV_OK) return rc;
+        PKV_CUDA(ctx, cudaEventRecord(ctx->ev_done, ctx->decode_stream));
+        PKV_CUDA(ctx, cudaStreamWaitEvent(stream, ctx->ev_done, 0));
+        ctx->host_call_pending = true;
+        if (stats) *stats = st;
+        return PATCHKV_OK;
+    }
+
+    // ---- units
     std::vector<Range> ranges;
     long long unit = 0;
     for (int i = 0; i < n_sessions; i++) {

@@ -209,6 +209,30 @@ def test_tiny_variants_from_pinned_host(ctx, name):
     run_select_and_restore(ctx, pin.config_tiny(**kw), host=True)
 
 
+@pytest.mark.parametrize("name", ["base", "delta0", "shift5", "ragged_n1000", "k4v4", "all_dirty", "interleaved"])
+def test_tiny_variants_from_pinned_host_zero_copy(name):
+    """PATCHKV_FLAG_HOST_DIRECT: no staging copies, the restore kernel reads the pinned payload itself."""
+    from paper_2609_26219_b200 import binding as pk
+    c = new_context(flags=pk.FLAG_HOST_DIRECT)
+    try:
+        kw = dict(TINY_VARIANTS.get(name, {}))
+        kw.setdefault("n_pages", 256)
+        st, sel, pools, _ = run_select_and_restore(c, pin.config_tiny(**kw), host=True)
+    finally:
+        c.close()
+
+
+def test_stress_shape_zero_copy_and_7b_shape_zero_copy():
+    from paper_2609_26219_b200 import binding as pk
+    c = new_context(flags=pk.FLAG_HOST_DIRECT)
+    try:
+        stats = _run_stress(c, _stress_sessions(n_layers=2, n=8192), range(8), [0, 1])
+        assert stats.n_copies == 0 and stats.bytes_copied == stats.bytes_useful
+        run_select_and_restore(c, pin.config_7b_host(device=DEV, pin_payload=True, n_layers=6), layers=[0, 5], host=True)
+    finally:
+        c.close()
+
+
 def test_host_restore_small_ring_and_no_merging():
     c = new_context(staging_slots=1, merge_gap_bytes=0)
     try:

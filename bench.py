@@ -300,6 +300,30 @@ def run_ours(args):
     value = aggregate_value(written_b, ms_per_step, world)
     assert ctx.query_status() == 0
 
+    # ---- the same step captured once in a CUDA graph and replayed (select_repair + counter reset + restore)
+    graph_ms = None
+    if world == 1 and not args.no_graph:
+        try:
+            side = torch.cuda.Stream()
+            side.wait_stream(stream)
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                ctx.select_repair(sel_args, side)
+                ctx.restore(geom, pool, [sess], side)
+            for _ in range(3):
+                g.replay()
+            ga, gb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            ga.record()
+            for _ in range(args.steps):
+                g.replay()
+            gb.record()
+            gb.synchronize()
+            graph_ms = ga.elapsed_time(gb) / args.steps
+            assert ctx.query_status() == 0
+        except Exception as exc:           # reported, never fatal: the headline numbers do not depend on it
+            graph_ms = f"unavailable: {type(exc).__name__}"
+
     peak, peak_kind = measured_hbm_peak()
     achieved = (read_b + written_b) / (restore_avg_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": "restore_pipe_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
@@ -533,7 +557,7 @@ def run_ours(args):
                        "parallelism": f"independent replicas x{world}" if world > 1 else "1 gpu"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": 2 * args.steps,
             "roofline": roofline, "cpu_baseline": cpu_baseline,
-            "select_us": select_us, "restore_ms": restore_avg_ms,
+            "select_us": select_us, "restore_ms": restore_avg_ms, "cuda_graph_ms_per_step": graph_ms,
             "block_layers_per_s": world * items / (ms_per_step * 1e-3),
             "real_gbps": world * (read_b + written_b) / (ms_per_step * 1e-3) / 1e9,
             "host_link": host_link, "select_at_scale": select_scale, "host_7b": host_cfg3, "stress": stress, "writer": writer, "paper_microbench_shape": paper_shape,
@@ -556,6 +580,7 @@ def main():
     ap.add_argument("--no-scale-select", action="store_true")
     ap.add_argument("--no-host-configs", action="store_true")
     ap.add_argument("--no-writer", action="store_true")
+    ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--stress-layers", type=int, default=10)
     ap.add_argument("--scale-layers", type=int, default=32, help="layers of the selection-at-scale leg (profiling: fewer)")
     ap.add_argument("--layers", type=int, default=32,

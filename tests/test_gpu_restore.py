@@ -337,3 +337,30 @@ def test_stress_shape_full_suffix_one_layer(ctx):
     """The same at the full 64k-token suffix per session (4096 blocks each, 32768 shared pages), one layer."""
     sess = _stress_sessions(n_layers=1, n=65536)
     _run_stress(ctx, sess, range(8), [0])
+
+
+def test_select_and_restore_replay_from_a_cuda_graph(ctx):
+    """select_repair + restore enqueue only stream work (a counter reset and kernels), so the pair can be captured
+    once and replayed; the replayed result equals the eager one bit for bit."""
+    ck = pin.config_tiny()
+    st = staged(ck)
+    k, v, pool = gpu_pool(ck)
+    geom, sess, sel_args = st.geom(), st.session(), st.select_args()
+    ctx.select_repair(sel_args)
+    ctx.restore(geom, pool, [sess])           # eager once: sizes every workspace before the capture
+    torch.cuda.synchronize()
+    k_eager, v_eager = k.clone(), v.clone()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        ctx.select_repair(sel_args, side)
+        ctx.restore(geom, pool, [sess], side)
+    for _ in range(3):
+        k.fill_(pin.SENTINEL - 0x10000)
+        v.fill_(pin.SENTINEL - 0x10000)
+        st.reuse_cnt.fill_(-7)
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(k, k_eager) and torch.equal(v, v_eager)
+    assert ctx.query_status() == 0

@@ -387,7 +387,7 @@ __device__ __forceinline__ void consume_unit(const RestoreParams& p, uint32_t co
                                              const ThreadMap& tm, int gpv, const float* tc, const float* ts, bool rotate) {
     const bool hasB = tm.cB >= 0;
     const bool rotA = rotate && tm.rotA, rotB = rotate && tm.rotB;
-#pragma unroll 2
+#pragma unroll 1
     for (int vec = tm.ty; vec < nvec; vec += tm.TY) {
         const Chunk ca = lds_chunk<FMT>(codes, scales, vec, p.D, gpv, tm.cA, tm.gA);
         Chunk cb = ca;

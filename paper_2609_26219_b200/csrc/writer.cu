@@ -107,33 +107,38 @@ __device__ __forceinline__ void encode_chunk(const uint4& w, uint8_t* codes, uin
     // That is computed without a division per element: t = x * (1/s) is within 2^-16 of the quotient, so rint(t) is
     // right unless the quotient is an exact tie, which the exact remainder x - k*s (one fma) detects and repairs.
     const float r = s > 0.0f ? __frcp_rn(s) : 0.0f;
-    const float half_s = 0.5f * s;
+    const float half_s = s > 0.0f ? 0.5f * s : -1.0f;      // -1: a zero group has no ties to look for
     const float magic = 12582912.0f;                       // 1.5 * 2^23: adding it rounds to an integer, ties to even
-    // Two lanes per instruction for the products and sums.  (If the assembler contracts x*r + magic into one fused
-    // operation the integer k can only change at an exact tie, where the repair below picks the even neighbour from
-    // either side.)
-    uint32_t kb[8];                                        // bits of code + 1.5 * 2^23: the low byte is the code
-    float kf[8], df[8], tmf[8];
+    // tm = x * r + magic in one fused operation rounds the product to an integer k (low byte of tm = the code).
+    // |x * r| <= qmax * (1 + 2^-11) < qmax + 0.5 whenever s is a normal fp16, so no clamp is needed then; a subnormal
+    // s can be far below amax / qmax and takes the clamped path below.  Two lanes per instruction throughout.
+    uint32_t kb[8];
+    float df[8];
     const f32x2 r2 = pack2(r, r), m2 = pack2(magic, magic), ns2 = pack2(-s, -s);
     bool any_tie = false;
 #pragma unroll
     for (int i = 0; i < 8; i += 2) {
         const f32x2 x2 = pack2(x[i], x[i + 1]);
-        const f32x2 tm = add2(mul2(x2, r2), m2);           // |x * r| <= ~2 * qmax: far below 2^22
-        const f32x2 k2 = sub2(tm, m2);
-        const f32x2 d2 = fma2(k2, ns2, x2);                // x - k*s, exact: a multiple of ulp(s) no larger than s
-        unpack2(tm, tmf[i], tmf[i + 1]);
-        unpack2(k2, kf[i], kf[i + 1]);
+        const f32x2 tm = fma2(x2, r2, m2);
+        const f32x2 d2 = fma2(sub2(tm, m2), ns2, x2);      // x - k*s, exact: a multiple of ulp(s) no larger than s
+        float a0, a1;
+        unpack2(tm, a0, a1);
+        kb[i] = __float_as_uint(a0); kb[i + 1] = __float_as_uint(a1);
         unpack2(d2, df[i], df[i + 1]);
         any_tie = any_tie || fabsf(df[i]) == half_s || fabsf(df[i + 1]) == half_s;
     }
-    if (any_tie) {                                         // rare: an exact half-integer quotient on an odd k
+    if (any_tie) {                                         // rare: an exact half-integer quotient sitting on an odd k
 #pragma unroll
         for (int i = 0; i < 8; i++)
-            if (fabsf(df[i]) == half_s && (__float_as_uint(tmf[i]) & 1u)) kf[i] += df[i] > 0.0f ? 1.0f : -1.0f;
+            if (fabsf(df[i]) == half_s && (kb[i] & 1u)) kb[i] += df[i] > 0.0f ? 1u : 0xFFFFFFFFu;
     }
+    if ((__half_as_ushort(s16) & 0x7C00u) == 0 && s > 0.0f) {      // subnormal scale: |k| may exceed qmax
 #pragma unroll
-    for (int i = 0; i < 8; i++) kb[i] = __float_as_uint(fminf(fmaxf(kf[i], -qmax), qmax) + magic);
+        for (int i = 0; i < 8; i++) {
+            const float k = fminf(fmaxf(__uint_as_float(kb[i]) - magic, -qmax), qmax);
+            kb[i] = __float_as_uint(k + magic);
+        }
+    }
     if (!write) return;
     // byte k of a word <- low byte of kb[k]
     const uint32_t w0 = __byte_perm(__byte_perm(kb[0], kb[1], 0x0040), __byte_perm(kb[2], kb[3], 0x0040), 0x5410);

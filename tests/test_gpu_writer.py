@@ -8,7 +8,7 @@ import oracle
 import patchkv_inputs as pin
 from gpu_common import DEV, check_pools, gpu_pool, new_context, staged
 from helpers import np_u16, oracle_restore, oracle_select
-from test_oracle_writer import _ck, pool_from_raw, run_writer
+from test_oracle_writer import _ck, pool_from_raw, run_writer, scale_raw
 
 pytestmark = pytest.mark.gpu
 
@@ -68,6 +68,41 @@ def test_writer_bytes_match_the_oracle(ctx, kw):
     assert np.array_equal(off, off_o) and sizes == [int(x) for x in lb_o]
     for a, b in zip(bufs, bufs_o):
         assert np.array_equal(a, b)
+
+
+@pytest.mark.parametrize("factor", [3e-5, 1e-6, 2e-8, 1e3])
+def test_writer_subnormal_scales_and_large_values(ctx, factor):
+    ck = scale_raw(_ck(), factor)
+    kp, vp = pool_from_raw(ck)
+    rc, rc2, off_o, lb_o, bufs_o = run_writer(ck, kp, vp)
+    off, sizes, bufs = gpu_writer(ctx, ck, kp, vp)
+    for a, b in zip(bufs, bufs_o):
+        assert np.array_equal(a, b)
+
+
+def test_writer_exact_ties_round_to_even(ctx):
+    """Exact half-integer quotients against a non-power-of-two scale (4-bit codes: amax 10.5 gives s = 1.5 exactly):
+    0.75 -> 0.5 -> 0, 2.25 -> 1.5 -> 2, -3.75 -> -2.5 -> -2, 5.25 -> 3.5 -> 4, 9.75 -> 6.5 -> 6."""
+    g = pin.Geometry(1, 1, 64, 64, pin.ROPE_HALF, 1e4, 16, 16, 32)
+    ck = _ck(geom=g, n=16, n_pages=2, table="identity", tag_probs=(0, 0, 0, 1.0))
+    kp = np.zeros((1, 2, 16, 1, 64), dtype=np.uint16)
+    vp = np.zeros_like(kp)
+    vals = [10.5, 0.75, 2.25, -3.75, 5.25, -0.75, 1.5, 9.75]
+    for c, x in enumerate(vals):
+        bits = int(np.array([x], dtype=np.float32).view(np.uint32)[0])
+        assert bits & 0xFFFF == 0                      # representable in bf16
+        kp[0, 0, 2, 0, c] = bits >> 16
+    rc, rc2, off_o, lb_o, bufs_o = run_writer(ck, kp, vp)
+    rec = bufs_o[0]
+    assert rec[512:512 + 64].view(np.float16).reshape(16, 2)[2, 0] == np.float16(1.5)
+    by = rec[:512].reshape(16, 32)[2, :4]
+    nib = []
+    for b in by:
+        nib += [int(b) & 15, int(b) >> 4]
+    codes = [n - 16 if n >= 8 else n for n in nib]
+    assert codes == [7, 0, 2, -2, 4, 0, 1, 6]
+    off, sizes, bufs = gpu_writer(ctx, ck, kp, vp)
+    assert np.array_equal(bufs[0], bufs_o[0])
 
 
 @pytest.mark.parametrize("what", ["page", "offset", "table_short"])

@@ -178,3 +178,24 @@ def test_writer_skips_out_of_range_blocks(what):
         keep = np.ones(bufs[l].size, dtype=bool)
         keep[o:o + r] = False
         assert np.array_equal(bufs[l][keep], good[l][keep])
+
+
+def scale_raw(ck, factor):
+    ck.raw_kv = [(k * factor, v * factor) for k, v in ck.raw_kv]
+    return ck
+
+
+@pytest.mark.parametrize("factor", [3e-5, 1e-6, 2e-8])
+def test_tiny_magnitudes_with_subnormal_fp16_scales_match_the_generators_encoder(factor):
+    """Groups whose amax / qmax falls in the fp16 subnormal range: the scale loses precision, codes can exceed qmax
+    before the clamp, and many groups quantise to a zero scale."""
+    ck = scale_raw(_ck(), factor)
+    g = ck.geom
+    kp, vp = pool_from_raw(ck)
+    rc, rc2, off, lb, bufs = run_writer(ck, kp, vp)
+    assert rc2 == oracle.OK
+    for l in range(g.n_layers):
+        k16 = ck.raw_kv[l][0].to(torch.bfloat16).float()
+        v16 = ck.raw_kv[l][1].to(torch.bfloat16).float()
+        want, _ = pin.encode_layer(k16, v16, ck.tags[l], g)
+        assert np.array_equal(bufs[l], want.numpy())

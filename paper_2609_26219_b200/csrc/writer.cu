@@ -226,6 +226,114 @@ quantize_gather_kernel(const GatherParams p) {
     }
 }
 
+// The same block encoder with the block's K and V rows staged in shared memory by bulk asynchronous copies: every
+// row of the block is in flight at once (no registers held for loads), and the encode loop reads 16-byte chunks
+// from shared memory.  One CTA per (layer, block); three CTAs per SM at the 8B-shaped geometry.
+__global__ void __launch_bounds__(kGatherThreads)
+quantize_gather_staged_kernel(const GatherParams p, int sec_bytes, int heads_contiguous) {
+    extern __shared__ __align__(128) uint8_t stage[];       // [K rows][V rows][tok_off]
+    __shared__ uint64_t bar[2];
+    __shared__ int abort_flag;
+    long long* tok_off = reinterpret_cast<long long*>(stage + 2 * (size_t)sec_bytes);
+    const int l = blockIdx.x / p.nb, j = blockIdx.x - l * p.nb;
+    const int tag = __ldg(p.tags + (size_t)l * p.nb + j);
+    const unsigned long long off = __ldg(p.blk_off + (size_t)l * p.nb + j);
+    const unsigned long long lbytes = __ldg(p.layer_bytes + l);
+    uint8_t* base = reinterpret_cast<uint8_t*>(
+        static_cast<uintptr_t>(__ldg(reinterpret_cast<const unsigned long long*>(p.layer_payload) + l)));
+    const unsigned long long elems = (unsigned long long)p.B * p.H * p.D;
+    const unsigned long long rec = record_bytes(tag, elems, p.G);
+    bool bad = rec == 0 || off > lbytes || rec > lbytes - off || base == nullptr ||
+               ((reinterpret_cast<uintptr_t>(base) + off) & 15u) != 0;
+    const int valid = min(p.B, p.n - j * p.B);
+    if (threadIdx.x == 0) {
+        mbar_init(&bar[0], 1); mbar_init(&bar[1], 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    for (int t = threadIdx.x; t < p.B; t += kGatherThreads) {
+        long long o = -1;
+        if (t < valid) {
+            const long long u = (long long)j * p.B + t + p.src_shift;
+            const long long lp = u / p.P;
+            const int page = lp < p.n_table ? __ldg(p.block_table + lp) : -1;
+            if (page < 0 || page >= p.n_pages) bad = true;
+            o = (long long)l * p.stride_layer + (long long)page * p.stride_page + (u - lp * p.P) * p.stride_token;
+        }
+        tok_off[t] = o;
+    }
+    if (__syncthreads_or(bad)) {                            // skip the block whole, latch the error
+        if (threadIdx.x == 0) atomicCAS(p.status, 0, (int)PATCHKV_E_BOUNDS);
+        return;
+    }
+    // ---- stage: valid rows by bulk copies (one per token, or one per (token, head) when heads are strided),
+    //      rows past the end of the suffix as zeros
+    const int row_bytes = p.H * p.D * 2, vec_bytes = p.D * 2;
+    if (threadIdx.x == 0) {
+        mbar_arrive_expect_tx(&bar[0], (uint32_t)valid * row_bytes);
+        mbar_arrive_expect_tx(&bar[1], (uint32_t)valid * row_bytes);
+    }
+    const int copies = heads_contiguous ? valid : valid * p.H;
+    for (int i = threadIdx.x; i < 2 * copies; i += kGatherThreads) {
+        const int sec = i >= copies, c = sec ? i - copies : i;
+        const uint16_t* pool = sec ? p.v_base : p.k_base;
+        uint8_t* dst = stage + (size_t)sec * sec_bytes;
+        if (heads_contiguous) bulk_g2s(dst + (size_t)c * row_bytes, pool + tok_off[c], row_bytes, &bar[sec]);
+        else {
+            const int t = c / p.H, h = c - t * p.H;
+            bulk_g2s(dst + (size_t)c * vec_bytes, pool + tok_off[t] + (long long)h * p.stride_head, vec_bytes, &bar[sec]);
+        }
+    }
+    for (int i = valid * row_bytes / 16 + threadIdx.x; i < sec_bytes / 16; i += kGatherThreads) {
+        reinterpret_cast<uint4*>(stage)[i] = make_uint4(0, 0, 0, 0);
+        reinterpret_cast<uint4*>(stage + sec_bytes)[i] = make_uint4(0, 0, 0, 0);
+    }
+    __syncthreads();
+
+    const int kf = k_format(tag), vf = v_format(tag);
+    uint8_t* kc = base + off;
+    uint8_t* ks = kc + code_bytes(kf, elems);
+    uint8_t* vc = ks + scale_bytes(kf, elems, p.G);
+    uint8_t* vs = vc + code_bytes(vf, elems);
+    const int cpv = p.D >> 3, seg = p.G >> 3, gpv = p.D / p.G;
+    const int seg_shift = 31 - __clz(seg);
+    const bool cpv_pow2 = (cpv & (cpv - 1)) == 0;
+    const int cpv_shift = 31 - __clz(cpv);
+    const int units = p.B * p.H * cpv;                      // 16-byte chunks of one section, in record order
+    const int padded = (units + kGatherThreads - 1) / kGatherThreads * kGatherThreads;
+    volatile int* abortp = &abort_flag;
+#pragma unroll 1
+    for (int sec = 0; sec < 2; sec++) {
+        // bounded wait for this section's rows; the verdict is CTA-uniform through the shared flag
+        const bool ok = mbar_wait(&bar[sec], 0, abortp);
+        if (__syncthreads_or(!ok)) {
+            if (threadIdx.x == 0) atomicCAS(p.status, 0, (int)PATCHKV_E_TIMEOUT);
+            // let the other section's copies land (bounded) before the CTA's shared memory is released
+            for (uint32_t i = 0; i < kWaitLimit && !mbar_try_wait(&bar[1], 0); i++) __nanosleep(100);
+            return;
+        }
+        const int fmt = sec ? vf : kf;
+        uint8_t* codes = sec ? vc : kc;
+        uint8_t* scales = sec ? vs : ks;
+        const uint32_t src = smem_u32(stage + (size_t)sec * sec_bytes);
+#pragma unroll 2
+        for (int u = threadIdx.x; u < padded; u += kGatherThreads) {
+            const bool in = u < units;
+            uint4 w = make_uint4(0, 0, 0, 0);
+            if (in) w = lds128(src + 16u * (uint32_t)u);
+            const int vec = cpv_pow2 ? (u >> cpv_shift) : u / cpv;
+            const int cx = u - vec * cpv;
+            const size_t elem0 = (size_t)u * 8;
+            const size_t sidx = (size_t)vec * gpv + (cx >> seg_shift);
+            switch (fmt) {
+                case FMT_BF16: encode_chunk<FMT_BF16>(w, codes, scales, elem0, sidx, seg, in); break;
+                case FMT_INT8: encode_chunk<FMT_INT8>(w, codes, scales, elem0, sidx, seg, in); break;
+                default:       encode_chunk<FMT_INT4>(w, codes, scales, elem0, sidx, seg, in); break;
+            }
+        }
+    }
+}
+
 }  // namespace patchkv
 
 using namespace patchkv;
@@ -283,8 +391,17 @@ extern "C" int patchkv_quantize_gather(patchkv_ctx* ctx, const patchkv_geom* g, 
     p.status = ctx->d_status;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return fail(ctx, PATCHKV_E_CUDA, "cudaSetDevice failed");
-    quantize_gather_kernel<<<nb * g->n_layers, kGatherThreads, g->block_tokens * sizeof(long long),
-                             static_cast<cudaStream_t>(stream)>>>(p);
+    // staged variant: both sections of a block in shared memory, at least two CTAs per SM
+    const long long sec_bytes = (long long)g->block_tokens * g->n_kv_heads * g->head_dim * 2;
+    const long long smem = 2 * sec_bytes + (long long)g->block_tokens * 8 + 16;
+    if (!(ctx->flags & PATCHKV_FLAG_DIRECT_LOADS) && smem <= 100 * 1024 && sec_bytes % 16 == 0) {
+        PKV_CUDA(ctx, cudaFuncSetAttribute(quantize_gather_staged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        quantize_gather_staged_kernel<<<nb * g->n_layers, kGatherThreads, smem, static_cast<cudaStream_t>(stream)>>>(
+            p, (int)sec_bytes, pool->stride_head == g->head_dim ? 1 : 0);
+    } else {
+        quantize_gather_kernel<<<nb * g->n_layers, kGatherThreads, g->block_tokens * sizeof(long long),
+                                 static_cast<cudaStream_t>(stream)>>>(p);
+    }
     PKV_CUDA(ctx, cudaGetLastError());
     return PATCHKV_OK;
 }

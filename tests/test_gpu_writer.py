@@ -13,9 +13,10 @@ from test_oracle_writer import _ck, pool_from_raw, run_writer, scale_raw
 pytestmark = pytest.mark.gpu
 
 
-@pytest.fixture(scope="module")
-def ctx():
-    c = new_context()
+@pytest.fixture(scope="module", params=[0, 1], ids=["staged", "direct_loads"])
+def ctx(request):
+    """Both writer kernels run every case: rows staged in shared memory by bulk copies, and plain loads."""
+    c = new_context(flags=request.param)
     yield c
     c.close()
 

@@ -317,6 +317,21 @@ PATCHKV_API int patchkv_plan_checkpoint(patchkv_ctx* ctx, const patchkv_geom* ge
 PATCHKV_API int patchkv_quantize_gather(patchkv_ctx* ctx, const patchkv_geom* geom, const patchkv_pool* pool,
                                         const patchkv_session* session, void* stream);
 
+/* Offload of one session to a CPU-resident checkpoint: patchkv_plan_checkpoint, then per layer patchkv_quantize_gather
+ * into a slot of the device staging ring and an asynchronous device-to-host copy of the finished layer payload into
+ * PINNED host memory, so that encoding layer l+1 overlaps copying layer l out.
+ *   session              as for patchkv_quantize_gather; its blk_off and layer_bytes (DEVICE, caller-allocated) are
+ *                        WRITTEN by the plan step and stay valid as the checkpoint's directory; layer_payload is ignored
+ *   host_layer_payload   HOST array of L PINNED destination pointers (16-byte aligned)
+ *   host_layer_capacity  HOST u64 [L]: bytes available behind each pointer (B*H*D*4*NB always suffices)
+ *   host_layer_bytes     HOST u64 [L] (out): bytes of each layer payload
+ * The call synchronises `stream` once, after the plan, to learn the layer sizes; everything else is enqueued on
+ * internal streams that `stream` waits for, as in patchkv_restore_from_host. */
+PATCHKV_API int patchkv_checkpoint_to_host(patchkv_ctx* ctx, const patchkv_geom* geom, const patchkv_pool* pool,
+                                           const patchkv_session* session, void* const* host_layer_payload,
+                                           const uint64_t* host_layer_capacity, uint64_t* host_layer_bytes,
+                                           void* stream);
+
 /* Synchronises the context's device work and returns in *device_status the first device-side error latched
  * since the last query (PATCHKV_OK, PATCHKV_E_BOUNDS, PATCHKV_E_BADINPUT or PATCHKV_E_TIMEOUT), then clears it. */
 PATCHKV_API int patchkv_query_status(patchkv_ctx* ctx, int* device_status);

@@ -94,6 +94,9 @@ def lib():
         l.patchkv_plan_checkpoint.argtypes = [C.c_void_p, C.POINTER(Geom), C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
                                               C.c_void_p]
         l.patchkv_quantize_gather.argtypes = [C.c_void_p, C.POINTER(Geom), C.POINTER(Pool), C.POINTER(Session), C.c_void_p]
+        l.patchkv_checkpoint_to_host.argtypes = [C.c_void_p, C.POINTER(Geom), C.POINTER(Pool), C.POINTER(Session),
+                                                 C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        l.patchkv_checkpoint_to_host.restype = C.c_int
         l.patchkv_plan_precision.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_float, C.c_float,
                                              C.c_float, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p]
         l.patchkv_plan_precision.restype = C.c_int
@@ -204,6 +207,15 @@ class Context:
     def quantize_gather(self, geom: Geom, pool: Pool, session: Session, stream=None, check: bool = True) -> int:
         return self._check(lib().patchkv_quantize_gather(self._h, C.byref(geom), C.byref(pool), C.byref(session),
                                                          _stream_handle(stream)), check)
+
+    def checkpoint_to_host(self, geom: Geom, pool: Pool, session: Session, host_layer_ptrs: torch.Tensor,
+                           host_layer_capacity: torch.Tensor, host_layer_bytes: torch.Tensor, stream=None,
+                           check: bool = True) -> int:
+        """host_layer_ptrs / host_layer_capacity / host_layer_bytes: CPU int64 tensors [L] (addresses of pinned buffers,
+        their sizes, and the output sizes)."""
+        return self._check(lib().patchkv_checkpoint_to_host(
+            self._h, C.byref(geom), C.byref(pool), C.byref(session), _ptr(host_layer_ptrs), _ptr(host_layer_capacity),
+            _ptr(host_layer_bytes), _stream_handle(stream)), check)
 
     def plan_precision(self, attn: torch.Tensor, resid: torch.Tensor, block_tokens: int, alpha: float, tau_L: float,
                        tau_H: float, eps4: float, tags: torch.Tensor, risk: Optional[torch.Tensor] = None,

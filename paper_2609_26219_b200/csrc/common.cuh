@@ -220,6 +220,8 @@ inline int fail(patchkv_ctx* ctx, int code, const std::string& msg) {
 int fill_geometry(patchkv_ctx* ctx, const patchkv_geom* g, const patchkv_pool* pool, RestoreParams* p);
 // cos / sin table of one session (double on the host, rounded once to fp32).
 void build_rope_table(const patchkv_geom* g, int delta, float* cos_out, float* sin_out);
+// Grows the pinned + device metadata arenas and the device staging ring of the host-resident entry points.
+int ensure_host_workspace(patchkv_ctx* ctx, size_t meta_bytes, size_t slot_bytes);
 // Launches the restore kernel for layers [layer_begin, layer_end) of the sessions already filled in p.
 int launch_restore(patchkv_ctx* ctx, RestoreParams* p, cudaStream_t stream);
 

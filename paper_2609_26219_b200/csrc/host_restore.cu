@@ -15,7 +15,7 @@ struct Range { uint64_t begin, end; };
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // Grow the metadata arenas (device + pinned mirror) and the staging ring.  Growing synchronises the device.
-static int ensure_host_workspace(patchkv_ctx* ctx, size_t meta_bytes, size_t slot_bytes) {
+int ensure_host_workspace(patchkv_ctx* ctx, size_t meta_bytes, size_t slot_bytes) {
     if (meta_bytes > ctx->meta_bytes) {
         PKV_CUDA(ctx, cudaDeviceSynchronize());
         if (ctx->d_meta) { cudaFree(ctx->d_meta); ctx->d_meta = nullptr; }

@@ -3,6 +3,8 @@
 // The inverse direction of restore; HBM-bound streaming with a warp-shuffle maximum per scale group.
 #include <cuda_fp16.h>
 
+#include <algorithm>
+
 #include "common.cuh"
 
 namespace patchkv {
@@ -73,6 +75,7 @@ struct GatherParams {
     const uint16_t* v_base;
     long long stride_layer, stride_page, stride_token, stride_head;
     int32_t n_pages, n, nb, src_shift, n_table;
+    int32_t layer_begin;                    // first layer of this launch (grid = nb * layers of the launch)
     const int32_t* block_table;
     const uint8_t* tags;
     const unsigned long long* blk_off;
@@ -159,7 +162,7 @@ __device__ __forceinline__ void encode_chunk(const uint4& w, uint8_t* codes, uin
 __global__ void __launch_bounds__(kGatherThreads)
 quantize_gather_kernel(const GatherParams p) {
     extern __shared__ long long tok_off[];                  // block_tokens entries
-    const int l = blockIdx.x / p.nb, j = blockIdx.x - l * p.nb;
+    const int l = p.layer_begin + blockIdx.x / p.nb, j = blockIdx.x % p.nb;
     const int tag = __ldg(p.tags + (size_t)l * p.nb + j);
     const unsigned long long off = __ldg(p.blk_off + (size_t)l * p.nb + j);
     const unsigned long long lbytes = __ldg(p.layer_bytes + l);
@@ -235,7 +238,7 @@ quantize_gather_staged_kernel(const GatherParams p, int sec_bytes, int heads_con
     __shared__ uint64_t bar[2];
     __shared__ int abort_flag;
     long long* tok_off = reinterpret_cast<long long*>(stage + 2 * (size_t)sec_bytes);
-    const int l = blockIdx.x / p.nb, j = blockIdx.x - l * p.nb;
+    const int l = p.layer_begin + blockIdx.x / p.nb, j = blockIdx.x % p.nb;
     const int tag = __ldg(p.tags + (size_t)l * p.nb + j);
     const unsigned long long off = __ldg(p.blk_off + (size_t)l * p.nb + j);
     const unsigned long long lbytes = __ldg(p.layer_bytes + l);
@@ -358,10 +361,11 @@ extern "C" int patchkv_plan_checkpoint(patchkv_ctx* ctx, const patchkv_geom* g, 
     return PATCHKV_OK;
 }
 
-extern "C" int patchkv_quantize_gather(patchkv_ctx* ctx, const patchkv_geom* g, const patchkv_pool* pool,
-                                       const patchkv_session* s, void* stream) {
-    if (!ctx) return PATCHKV_E_INVALID;
-    std::lock_guard<std::mutex> lock(ctx->mu);
+namespace patchkv {
+
+// Validates the arguments of a gather and fills the launch parameters (layer_payload / layer range set by the caller).
+static int fill_gather(patchkv_ctx* ctx, const patchkv_geom* g, const patchkv_pool* pool, const patchkv_session* s,
+                       GatherParams* p, int* nb_out) {
     static thread_local RestoreParams rp;                  // reused only for the shared geometry / pool validation
     int rc = fill_geometry(ctx, g, pool, &rp);
     if (rc != PATCHKV_OK) return rc;
@@ -373,36 +377,129 @@ extern "C" int patchkv_quantize_gather(patchkv_ctx* ctx, const patchkv_geom* g, 
         return fail(ctx, PATCHKV_E_UNSUPPORTED, "quantize_gather: group must be 8, 16, 32, 64, 128 or 256");
     if (g->block_tokens > 2048) return fail(ctx, PATCHKV_E_UNSUPPORTED, "quantize_gather: block_tokens > 2048");
     const int nb = (s->n_suffix_tokens + g->block_tokens - 1) / g->block_tokens;
+    *nb_out = nb;
     if (nb == 0) return PATCHKV_OK;
-    if (!s->block_table || !s->tags || !s->blk_off || !s->layer_payload || !s->layer_bytes)
+    if (!s->block_table || !s->tags || !s->blk_off || !s->layer_bytes)
         return fail(ctx, PATCHKV_E_INVALID, "session: null pointer");
     if ((long long)nb * g->n_layers > 0x7fffffffLL) return fail(ctx, PATCHKV_E_UNSUPPORTED, "quantize_gather: too many blocks");
-    GatherParams p;
-    p.L = g->n_layers; p.H = g->n_kv_heads; p.D = g->head_dim; p.B = g->block_tokens; p.P = g->page_tokens; p.G = G;
-    p.k_base = static_cast<const uint16_t*>(pool->k_base);
-    p.v_base = static_cast<const uint16_t*>(pool->v_base);
-    p.stride_layer = pool->stride_layer; p.stride_page = pool->stride_page;
-    p.stride_token = pool->stride_token; p.stride_head = pool->stride_head;
-    p.n_pages = pool->n_pages; p.n = s->n_suffix_tokens; p.nb = nb; p.src_shift = s->dst_shift; p.n_table = s->n_table;
-    p.block_table = s->block_table; p.tags = s->tags;
-    p.blk_off = reinterpret_cast<const unsigned long long*>(s->blk_off);
-    p.layer_payload = const_cast<void* const*>(s->layer_payload);
-    p.layer_bytes = reinterpret_cast<const unsigned long long*>(s->layer_bytes);
-    p.status = ctx->d_status;
-    DeviceGuard guard(ctx->device);
-    if (!guard.ok) return fail(ctx, PATCHKV_E_CUDA, "cudaSetDevice failed");
+    p->L = g->n_layers; p->H = g->n_kv_heads; p->D = g->head_dim; p->B = g->block_tokens; p->P = g->page_tokens; p->G = G;
+    p->k_base = static_cast<const uint16_t*>(pool->k_base);
+    p->v_base = static_cast<const uint16_t*>(pool->v_base);
+    p->stride_layer = pool->stride_layer; p->stride_page = pool->stride_page;
+    p->stride_token = pool->stride_token; p->stride_head = pool->stride_head;
+    p->n_pages = pool->n_pages; p->n = s->n_suffix_tokens; p->nb = nb; p->src_shift = s->dst_shift; p->n_table = s->n_table;
+    p->layer_begin = 0;
+    p->block_table = s->block_table; p->tags = s->tags;
+    p->blk_off = reinterpret_cast<const unsigned long long*>(s->blk_off);
+    p->layer_payload = const_cast<void* const*>(s->layer_payload);
+    p->layer_bytes = reinterpret_cast<const unsigned long long*>(s->layer_bytes);
+    p->status = ctx->d_status;
+    return PATCHKV_OK;
+}
+
+// Launches the block encoder for `layers` layers starting at p.layer_begin.
+static int launch_gather(patchkv_ctx* ctx, const patchkv_geom* g, const patchkv_pool* pool, const GatherParams& p,
+                         int layers, cudaStream_t stream) {
     // staged variant: both sections of a block in shared memory, at least two CTAs per SM
     const long long sec_bytes = (long long)g->block_tokens * g->n_kv_heads * g->head_dim * 2;
     const long long smem = 2 * sec_bytes + (long long)g->block_tokens * 8 + 16;
     if (!(ctx->flags & PATCHKV_FLAG_DIRECT_LOADS) && smem <= 100 * 1024 && sec_bytes % 16 == 0) {
         PKV_CUDA(ctx, cudaFuncSetAttribute(quantize_gather_staged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        quantize_gather_staged_kernel<<<nb * g->n_layers, kGatherThreads, smem, static_cast<cudaStream_t>(stream)>>>(
+        quantize_gather_staged_kernel<<<p.nb * layers, kGatherThreads, smem, stream>>>(
             p, (int)sec_bytes, pool->stride_head == g->head_dim ? 1 : 0);
     } else {
-        quantize_gather_kernel<<<nb * g->n_layers, kGatherThreads, g->block_tokens * sizeof(long long),
-                                 static_cast<cudaStream_t>(stream)>>>(p);
+        quantize_gather_kernel<<<p.nb * layers, kGatherThreads, g->block_tokens * sizeof(long long), stream>>>(p);
     }
     PKV_CUDA(ctx, cudaGetLastError());
+    return PATCHKV_OK;
+}
+
+}  // namespace patchkv
+
+extern "C" int patchkv_quantize_gather(patchkv_ctx* ctx, const patchkv_geom* g, const patchkv_pool* pool,
+                                       const patchkv_session* s, void* stream) {
+    if (!ctx) return PATCHKV_E_INVALID;
+    std::lock_guard<std::mutex> lock(ctx->mu);
+    GatherParams p;
+    int nb = 0;
+    int rc = fill_gather(ctx, g, pool, s, &p, &nb);
+    if (rc != PATCHKV_OK || nb == 0) return rc;
+    if (!s->layer_payload) return fail(ctx, PATCHKV_E_INVALID, "session: null layer_payload");
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, PATCHKV_E_CUDA, "cudaSetDevice failed");
+    return launch_gather(ctx, g, pool, p, g->n_layers, static_cast<cudaStream_t>(stream));
+}
+
+// Offload to a CPU-resident checkpoint: plan, then per layer encode into a device staging slot and copy the finished
+// layer payload to pinned host memory on the copy stream while the next layer is being encoded.
+extern "C" int patchkv_checkpoint_to_host(patchkv_ctx* ctx, const patchkv_geom* g, const patchkv_pool* pool,
+                                          const patchkv_session* s, void* const* host_layer_payload,
+                                          const uint64_t* host_layer_capacity, uint64_t* host_layer_bytes,
+                                          void* stream_) {
+    if (!ctx) return PATCHKV_E_INVALID;
+    std::lock_guard<std::mutex> lock(ctx->mu);
+    if (!host_layer_payload || !host_layer_capacity || !host_layer_bytes)
+        return fail(ctx, PATCHKV_E_INVALID, "checkpoint_to_host: null host array");
+    GatherParams p;
+    int nb = 0;
+    int rc = fill_gather(ctx, g, pool, s, &p, &nb);
+    if (rc != PATCHKV_OK) return rc;
+    const int L = g->n_layers;
+    if (nb == 0) { for (int l = 0; l < L; l++) host_layer_bytes[l] = 0; return PATCHKV_OK; }
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, PATCHKV_E_CUDA, "cudaSetDevice failed");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (ctx->host_call_pending) {                           // the ring and the metadata arena may still be in use
+        PKV_CUDA(ctx, cudaEventSynchronize(ctx->ev_done));
+        ctx->host_call_pending = false;
+    }
+    // 1. directory of the clustered layout, and its per-layer sizes back on the host (the one synchronisation)
+    plan_checkpoint_kernel<<<L, kPlanThreads, 0, stream>>>(
+        s->tags, nb, (unsigned long long)g->block_tokens * g->n_kv_heads * g->head_dim, g->group,
+        reinterpret_cast<unsigned long long*>(const_cast<uint64_t*>(s->blk_off)),
+        reinterpret_cast<unsigned long long*>(const_cast<uint64_t*>(s->layer_bytes)), ctx->d_status);
+    PKV_CUDA(ctx, cudaGetLastError());
+    rc = ensure_host_workspace(ctx, (size_t)L * 16 + 256, 16);
+    if (rc != PATCHKV_OK) return rc;
+    uint64_t* h_bytes = reinterpret_cast<uint64_t*>(ctx->h_meta);
+    PKV_CUDA(ctx, cudaMemcpyAsync(h_bytes, s->layer_bytes, (size_t)L * 8, cudaMemcpyDeviceToHost, stream));
+    PKV_CUDA(ctx, cudaStreamSynchronize(stream));
+    size_t slot_bytes = 16;
+    for (int l = 0; l < L; l++) {
+        host_layer_bytes[l] = h_bytes[l];
+        if (h_bytes[l] > host_layer_capacity[l]) return fail(ctx, PATCHKV_E_INVALID, "checkpoint_to_host: host buffer too small");
+        if (h_bytes[l] && (!host_layer_payload[l] || (reinterpret_cast<uintptr_t>(host_layer_payload[l]) & 15u)))
+            return fail(ctx, PATCHKV_E_INVALID, "checkpoint_to_host: host buffer null or not 16-byte aligned");
+        slot_bytes = std::max<size_t>(slot_bytes, h_bytes[l]);
+    }
+    rc = ensure_host_workspace(ctx, (size_t)L * 16 + 256, slot_bytes);
+    if (rc != PATCHKV_OK) return rc;
+    const int n_slots = (int)ctx->slots.size();
+    // 2. staged layer pointers: layer l encodes into slot l % n_slots
+    void** h_ptrs = reinterpret_cast<void**>(ctx->h_meta + (size_t)L * 8);
+    for (int l = 0; l < L; l++) h_ptrs[l] = ctx->slots[l % n_slots].base;
+    void** d_ptrs = reinterpret_cast<void**>(ctx->d_meta);
+    PKV_CUDA(ctx, cudaEventRecord(ctx->ev_begin, stream));
+    PKV_CUDA(ctx, cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_begin, 0));
+    PKV_CUDA(ctx, cudaStreamWaitEvent(ctx->decode_stream, ctx->ev_begin, 0));
+    PKV_CUDA(ctx, cudaMemcpyAsync(d_ptrs, h_ptrs, (size_t)L * 8, cudaMemcpyHostToDevice, ctx->decode_stream));
+    p.layer_payload = d_ptrs;
+    // 3. encode layer l on the decode stream, copy it out on the copy stream; events order slot reuse
+    for (int l = 0; l < L; l++) {
+        Staging& slot = ctx->slots[l % n_slots];
+        if (l >= n_slots) PKV_CUDA(ctx, cudaStreamWaitEvent(ctx->decode_stream, slot.freed, 0));
+        p.layer_begin = l;
+        rc = launch_gather(ctx, g, pool, p, 1, ctx->decode_stream);
+        if (rc != PATCHKV_OK) return rc;
+        PKV_CUDA(ctx, cudaEventRecord(slot.copied, ctx->decode_stream));
+        PKV_CUDA(ctx, cudaStreamWaitEvent(ctx->copy_stream, slot.copied, 0));
+        if (h_bytes[l])
+            PKV_CUDA(ctx, cudaMemcpyAsync(host_layer_payload[l], slot.base, h_bytes[l], cudaMemcpyDeviceToHost, ctx->copy_stream));
+        PKV_CUDA(ctx, cudaEventRecord(slot.freed, ctx->copy_stream));
+    }
+    PKV_CUDA(ctx, cudaEventRecord(ctx->ev_done, ctx->copy_stream));
+    PKV_CUDA(ctx, cudaStreamWaitEvent(stream, ctx->ev_done, 0));
+    ctx->host_call_pending = true;
     return PATCHKV_OK;
 }
 

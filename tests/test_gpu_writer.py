@@ -220,3 +220,46 @@ def test_precision_planner_matches_the_oracle_bit_for_bit(ctx, n, B):
         assert np.array_equal(tags.cpu().numpy(), tags_o)
         if n > 1000:
             assert len(set(tags_o)) == 3         # all three tiers occur
+
+
+@pytest.mark.parametrize("slots", [1, 2, 4])
+def test_checkpoint_to_host_streams_the_same_bytes(slots):
+    """Plan + encode + device-to-host copy per layer through the staging ring: the pinned buffers end up holding
+    exactly the oracle's payload, for ring depths below, at and above what overlaps."""
+    from paper_2609_26219_b200 import binding as pk
+    c = new_context(staging_slots=slots)
+    try:
+        g = pin.Geometry(5, 2, 64, 64, pin.ROPE_HALF, 1e4, 16, 16, 32)
+        ck = _ck(geom=g, n=150, n_pages=24)
+        kp, vp = pool_from_raw(ck)
+        rc, rc2, off_o, lb_o, bufs_o = run_writer(ck, kp, vp)
+        L, NB = g.n_layers, ck.n_blocks
+        k = torch.from_numpy(kp.view(np.int16)).to(DEV)
+        v = torch.from_numpy(vp.view(np.int16)).to(DEV)
+        pool = pk.make_pool(k, v, ck.n_pages, pin.pool_strides(g, ck.n_pages))
+        geom = pk.make_geom(g.n_layers, g.n_kv_heads, g.head_dim, g.rotary_dim, g.rope_style, g.rope_base,
+                            g.block_tokens, g.page_tokens, g.group)
+        tags = ck.tags.to(DEV).contiguous()
+        off = torch.zeros((L, NB), dtype=torch.int64, device=DEV)
+        lb = torch.zeros(L, dtype=torch.int64, device=DEV)
+        sess = pk.make_session(n_suffix_tokens=ck.n_suffix_tokens, delta=0, dst_shift=0,
+                               block_table=ck.block_table.to(DEV), tags=tags, blk_off=off, layer_payload=None,
+                               layer_bytes=lb, reuse_idx=None, reuse_cnt=None)
+        cap = NB * 16 * 2 * 64 * 4
+        host = [torch.full((cap,), 0x55, dtype=torch.uint8).pin_memory() for _ in range(L)]
+        ptrs = torch.tensor([h.data_ptr() for h in host], dtype=torch.int64)
+        caps = torch.full((L,), cap, dtype=torch.int64)
+        sizes = torch.zeros(L, dtype=torch.int64)
+        for _ in range(2):                                   # twice: ring and events are reused
+            c.checkpoint_to_host(geom, pool, sess, ptrs, caps, sizes)
+            torch.cuda.synchronize()
+            assert c.query_status() == 0
+            assert [int(x) for x in sizes] == [int(x) for x in lb_o]
+            assert np.array_equal(off.cpu().numpy().astype(np.uint64), off_o)
+            for l in range(L):
+                assert np.array_equal(host[l][:int(sizes[l])].numpy(), bufs_o[l])
+                assert bool((host[l][int(sizes[l]):] == 0x55).all())
+        small = torch.full((L,), 64, dtype=torch.int64)
+        assert c.checkpoint_to_host(geom, pool, sess, ptrs, small, sizes, check=False) == pk.E_INVALID
+    finally:
+        c.close()

@@ -562,11 +562,26 @@ def run_ours(args):
                                    "4096-page pool (2x), shuffled free list", both=True)
         del c3
         SLy = args.stress_layers
-        sess = [pin.config_stress_session(i, device=dev, n_layers=SLy, pin_payload=True) for i in range(8)]
-        pin.shared_free_list(1005, 8 * 4096, sess)
-        stress = host_leg(sess, f"70b-shaped stress: 8 sessions x 64k-token suffix, H=8 D=128, int4 share 10-60 %, "
-                                f"one shared pool of 32768 pages, pinned host payload; {SLy} of 80 layers resident "
-                                f"per wave (fit rule: the 80-layer pool is 172 GB)", reps=3, both=True)
+        waves = []
+        for w_ in range(args.stress_waves):          # each wave: SLy of the 80 layers, payload regenerated outside the timed region
+            sess = [pin.config_stress_session(i, device=dev, n_layers=SLy, pin_payload=True, seed=1005 + 17 * i + 1000 * w_)
+                    for i in range(8)]
+            pin.shared_free_list(1005, 8 * 4096, sess)
+            waves.append(host_leg(sess, "", reps=3, both=(w_ == 0)))
+            if w_ + 1 < args.stress_waves:
+                del sess
+        stress = dict(waves[0])
+        stress["workload"] = (f"70b-shaped stress: 8 sessions x 64k-token suffix, H=8 D=128, int4 share 10-60 %, one shared pool "
+                              f"of 32768 pages, pinned host payload; {SLy} of 80 layers resident per wave, {len(waves)} wave(s) "
+                              f"timed (fit rule: the 80-layer pool is 172 GB and its payload 103 GB of pinned memory)")
+        if len(waves) > 1:
+            tot_ms = sum(w["ms"] for w in waves)
+            tot_useful = sum(w["bytes_useful"] for w in waves)
+            stress.update(ms=tot_ms, bytes_useful=tot_useful, layers_covered=SLy * len(waves),
+                          payload_gbps=tot_useful / (tot_ms * 1e-3) / 1e9,
+                          frac_of_link=tot_useful / (tot_ms * 1e-3) / 1e9 / waves[0]["link_ceiling_gbps"],
+                          block_layers=sum(w["block_layers"] for w in waves),
+                          restored_kv_gbps_bf16_equiv=sum(w["restored_kv_gbps_bf16_equiv"] * w["ms"] for w in waves) / tot_ms)
         del sess
 
     # ---- the paper's restore microbenchmark shape (Section V-E): an ~8k-token checkpoint of a 64-layer, 8-KV-head,
@@ -635,6 +650,7 @@ def main():
     ap.add_argument("--no-writer", action="store_true")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--stress-layers", type=int, default=10)
+    ap.add_argument("--stress-waves", type=int, default=1, help="8 waves of 10 layers cover the full 80-layer stress config")
     ap.add_argument("--scale-layers", type=int, default=32, help="layers of the selection-at-scale leg (profiling: fewer)")
     ap.add_argument("--layers", type=int, default=32,
                     help="profiling only: fewer layers of the same workload (the bench line is quoted on 32)")

@@ -364,3 +364,46 @@ def test_select_and_restore_replay_from_a_cuda_graph(ctx):
         torch.cuda.synchronize()
         assert torch.equal(k, k_eager) and torch.equal(v, v_eager)
     assert ctx.query_status() == 0
+
+
+def test_restores_overlapping_on_two_streams_of_one_context(ctx):
+    """Launches from one context may overlap on the GPU: each gets its own work counter."""
+    a = pin.config_llama8b(device=DEV, n_layers=3, delta=77)
+    b = pin.config_llama8b(device=DEV, n_layers=3, delta=-1234, seed=4321)
+    sa, sb = staged(a), staged(b)
+    ctx.select_repair(sa.select_args())
+    ctx.select_repair(sb.select_args())
+    ka, va, pa = gpu_pool(a)
+    kb, vb, pb = gpu_pool(b)
+    torch.cuda.synchronize()
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    ga, gb = sa.geom(), sb.geom()
+    sess_a, sess_b = sa.session(), sb.session()
+    for _ in range(4):
+        ctx.restore(ga, pa, [sess_a], s1)
+        ctx.restore(gb, pb, [sess_b], s2)
+    torch.cuda.synchronize()
+    assert ctx.query_status() == 0
+    for ck, k, v in ((a, ka, va), (b, kb, vb)):
+        _, sel = oracle_select(ck)
+        rc, k_ref, v_ref, _ = oracle_restore(ck, sel["reuse_idx"], sel["reuse_cnt"])
+        check_pools(k, v, k_ref, v_ref, ck.geom)
+
+
+def test_eight_device_resident_sessions_in_one_launch(ctx):
+    sess = [pin.config_stress_session(i, device=DEV, n_layers=2, n=2048, n_pages=128, dirty_tokens=200, top_k=9)
+            for i in range(8)]
+    pin.shared_free_list(77, 8 * 128, sess)
+    sts = [staged(c) for c in sess]
+    for s in sts:
+        ctx.select_repair(s.select_args())
+    k, v, pool = gpu_pool(sess[0])
+    ctx.restore(sts[0].geom(), pool, [s.session() for s in sts])
+    torch.cuda.synchronize()
+    assert ctx.query_status() == 0
+    k_ref = v_ref = None
+    for c in sess:
+        _, sel = oracle_select(c)
+        pools = None if k_ref is None else (k_ref, v_ref)
+        rc, k_ref, v_ref, _ = oracle_restore(c, sel["reuse_idx"], sel["reuse_cnt"], pools=pools)
+    check_pools(k, v, k_ref, v_ref, sess[0].geom)

@@ -158,6 +158,100 @@ __device__ __forceinline__ void encode_chunk(const uint4& w, uint8_t* codes, uin
     if (((threadIdx.x & 31) & (seg - 1)) == 0) *reinterpret_cast<__half*>(scales + 2 * scale_index) = s16;
 }
 
+// NC consecutive 8-channel chunks (8 * NC channels of one head vector, all inside one scale group) per thread: the
+// scale arithmetic and the addressing are paid once per 8 * NC elements.  `seg` = lanes per scale group.
+template <int FMT, int NC>
+__device__ __forceinline__ void encode_span(const uint4* w, uint8_t* codes, uint8_t* scales, size_t elem0,
+                                            size_t scale_index, int seg, bool write) {
+    if (FMT == FMT_BF16) {
+        if (write) {
+#pragma unroll
+            for (int c = 0; c < NC; c++) reinterpret_cast<uint4*>(codes + 2 * elem0)[c] = w[c];
+        }
+        return;
+    }
+    // group maximum straight from the bf16 bit patterns (|x| as an integer compare is monotone for finite values)
+    uint32_t amax_bits = 0;
+#pragma unroll
+    for (int c = 0; c < NC; c++) {
+        const uint32_t ww[4] = {w[c].x, w[c].y, w[c].z, w[c].w};
+#pragma unroll
+        for (int i = 0; i < 4; i++) {
+            amax_bits = max(amax_bits, (ww[i] << 16) & 0x7FFF0000u);
+            amax_bits = max(amax_bits, ww[i] & 0x7FFF0000u);
+        }
+    }
+    for (int d = 1; d < seg; d <<= 1) amax_bits = max(amax_bits, __shfl_xor_sync(0xFFFFFFFFu, amax_bits, d));
+    const float amax = __uint_as_float(amax_bits);
+    const float qmax = FMT == FMT_INT8 ? 127.0f : 7.0f;
+    const __half s16 = __float2half_rn(__fdiv_rn(amax, qmax));
+    const float s = __half2float(s16);
+    const float r = s > 0.0f ? __frcp_rn(s) : 0.0f;
+    const float half_s = s > 0.0f ? 0.5f * s : -1.0f;
+    const float magic = 12582912.0f;
+    const bool subnormal = (__half_as_ushort(s16) & 0x7C00u) == 0 && s > 0.0f;
+    const f32x2 r2 = pack2(r, r), m2 = pack2(magic, magic), ns2 = pack2(-s, -s);
+    uint32_t out[2 * NC];
+#pragma unroll
+    for (int c = 0; c < NC; c++) {
+        float x[8];
+        x[0] = __uint_as_float(w[c].x << 16); x[1] = __uint_as_float(w[c].x & 0xFFFF0000u);
+        x[2] = __uint_as_float(w[c].y << 16); x[3] = __uint_as_float(w[c].y & 0xFFFF0000u);
+        x[4] = __uint_as_float(w[c].z << 16); x[5] = __uint_as_float(w[c].z & 0xFFFF0000u);
+        x[6] = __uint_as_float(w[c].w << 16); x[7] = __uint_as_float(w[c].w & 0xFFFF0000u);
+        uint32_t kb[8];
+        float df[8];
+        bool any_tie = false;
+#pragma unroll
+        for (int i = 0; i < 8; i += 2) {
+            const f32x2 x2 = pack2(x[i], x[i + 1]);
+            const f32x2 tm = fma2(x2, r2, m2);
+            const f32x2 d2 = fma2(sub2(tm, m2), ns2, x2);
+            float a0, a1;
+            unpack2(tm, a0, a1);
+            kb[i] = __float_as_uint(a0); kb[i + 1] = __float_as_uint(a1);
+            unpack2(d2, df[i], df[i + 1]);
+            any_tie = any_tie || fabsf(df[i]) == half_s || fabsf(df[i + 1]) == half_s;
+        }
+        if (any_tie) {
+#pragma unroll
+            for (int i = 0; i < 8; i++)
+                if (fabsf(df[i]) == half_s && (kb[i] & 1u)) kb[i] += df[i] > 0.0f ? 1u : 0xFFFFFFFFu;
+        }
+        if (subnormal) {
+#pragma unroll
+            for (int i = 0; i < 8; i++) {
+                const float k = fminf(fmaxf(__uint_as_float(kb[i]) - magic, -qmax), qmax);
+                kb[i] = __float_as_uint(k + magic);
+            }
+        }
+        out[2 * c] = __byte_perm(__byte_perm(kb[0], kb[1], 0x0040), __byte_perm(kb[2], kb[3], 0x0040), 0x5410);
+        out[2 * c + 1] = __byte_perm(__byte_perm(kb[4], kb[5], 0x0040), __byte_perm(kb[6], kb[7], 0x0040), 0x5410);
+    }
+    if (!write) return;
+    if (FMT == FMT_INT8) {
+        if (NC == 1) *reinterpret_cast<uint2*>(codes + elem0) = make_uint2(out[0], out[1]);
+        else {
+#pragma unroll
+            for (int c = 0; c < NC / 2; c++)
+                reinterpret_cast<uint4*>(codes + elem0)[c] = make_uint4(out[4 * c], out[4 * c + 1], out[4 * c + 2], out[4 * c + 3]);
+        }
+    } else {
+        uint32_t nib[NC];
+#pragma unroll
+        for (int c = 0; c < NC; c++) {
+            uint32_t a = out[2 * c] & 0x0F0F0F0Fu, b = out[2 * c + 1] & 0x0F0F0F0Fu;
+            a = (a | (a >> 4)) & 0x00FF00FFu; a = (a | (a >> 8)) & 0x0000FFFFu;
+            b = (b | (b >> 4)) & 0x00FF00FFu; b = (b | (b >> 8)) & 0x0000FFFFu;
+            nib[c] = a | (b << 16);
+        }
+        if (NC == 1) *reinterpret_cast<uint32_t*>(codes + (elem0 >> 1)) = nib[0];
+        else if (NC == 2) *reinterpret_cast<uint2*>(codes + (elem0 >> 1)) = make_uint2(nib[0], nib[NC - 1]);
+        else *reinterpret_cast<uint4*>(codes + (elem0 >> 1)) = make_uint4(nib[0], nib[1 % NC], nib[2 % NC], nib[3 % NC]);
+    }
+    if (((threadIdx.x & 31) & (seg - 1)) == 0) *reinterpret_cast<__half*>(scales + 2 * scale_index) = s16;
+}
+
 // One CTA per (layer, block).
 __global__ void __launch_bounds__(kGatherThreads)
 quantize_gather_kernel(const GatherParams p) {
@@ -232,6 +326,7 @@ quantize_gather_kernel(const GatherParams p) {
 // The same block encoder with the block's K and V rows staged in shared memory by bulk asynchronous copies: every
 // row of the block is in flight at once (no registers held for loads), and the encode loop reads 16-byte chunks
 // from shared memory.  One CTA per (layer, block); three CTAs per SM at the 8B-shaped geometry.
+template <int NC>
 __global__ void __launch_bounds__(kGatherThreads)
 quantize_gather_staged_kernel(const GatherParams p, int sec_bytes, int heads_contiguous) {
     extern __shared__ __align__(128) uint8_t stage[];       // [K rows][V rows][tok_off]
@@ -298,11 +393,13 @@ quantize_gather_staged_kernel(const GatherParams p, int sec_bytes, int heads_con
     uint8_t* ks = kc + code_bytes(kf, elems);
     uint8_t* vc = ks + scale_bytes(kf, elems, p.G);
     uint8_t* vs = vc + code_bytes(vf, elems);
-    const int cpv = p.D >> 3, seg = p.G >> 3, gpv = p.D / p.G;
+    const int spv = p.D / (8 * NC);                         // spans of 8 * NC channels per head vector
+    const int seg = p.G / (8 * NC);                         // lanes per scale group (>= 1: a span never crosses a group)
+    const int gpv = p.D / p.G;
     const int seg_shift = 31 - __clz(seg);
-    const bool cpv_pow2 = (cpv & (cpv - 1)) == 0;
-    const int cpv_shift = 31 - __clz(cpv);
-    const int units = p.B * p.H * cpv;                      // 16-byte chunks of one section, in record order
+    const bool spv_pow2 = (spv & (spv - 1)) == 0;
+    const int spv_shift = 31 - __clz(spv);
+    const int units = p.B * p.H * spv;                      // spans of one section, in record order
     const int padded = (units + kGatherThreads - 1) / kGatherThreads * kGatherThreads;
     volatile int* abortp = &abort_flag;
 #pragma unroll 1
@@ -319,19 +416,20 @@ quantize_gather_staged_kernel(const GatherParams p, int sec_bytes, int heads_con
         uint8_t* codes = sec ? vc : kc;
         uint8_t* scales = sec ? vs : ks;
         const uint32_t src = smem_u32(stage + (size_t)sec * sec_bytes);
-#pragma unroll 2
+#pragma unroll 1
         for (int u = threadIdx.x; u < padded; u += kGatherThreads) {
             const bool in = u < units;
-            uint4 w = make_uint4(0, 0, 0, 0);
-            if (in) w = lds128(src + 16u * (uint32_t)u);
-            const int vec = cpv_pow2 ? (u >> cpv_shift) : u / cpv;
-            const int cx = u - vec * cpv;
-            const size_t elem0 = (size_t)u * 8;
-            const size_t sidx = (size_t)vec * gpv + (cx >> seg_shift);
+            uint4 w[NC];
+#pragma unroll
+            for (int c = 0; c < NC; c++) w[c] = in ? lds128(src + 16u * (uint32_t)(u * NC + c)) : make_uint4(0, 0, 0, 0);
+            const int vec = spv_pow2 ? (u >> spv_shift) : u / spv;
+            const int sx = u - vec * spv;
+            const size_t elem0 = (size_t)u * 8 * NC;
+            const size_t sidx = (size_t)vec * gpv + (sx >> seg_shift);
             switch (fmt) {
-                case FMT_BF16: encode_chunk<FMT_BF16>(w, codes, scales, elem0, sidx, seg, in); break;
-                case FMT_INT8: encode_chunk<FMT_INT8>(w, codes, scales, elem0, sidx, seg, in); break;
-                default:       encode_chunk<FMT_INT4>(w, codes, scales, elem0, sidx, seg, in); break;
+                case FMT_BF16: encode_span<FMT_BF16, NC>(w, codes, scales, elem0, sidx, seg, in); break;
+                case FMT_INT8: encode_span<FMT_INT8, NC>(w, codes, scales, elem0, sidx, seg, in); break;
+                default:       encode_span<FMT_INT4, NC>(w, codes, scales, elem0, sidx, seg, in); break;
             }
         }
     }
@@ -404,9 +502,18 @@ static int launch_gather(patchkv_ctx* ctx, const patchkv_geom* g, const patchkv_
     const long long sec_bytes = (long long)g->block_tokens * g->n_kv_heads * g->head_dim * 2;
     const long long smem = 2 * sec_bytes + (long long)g->block_tokens * 8 + 16;
     if (!(ctx->flags & PATCHKV_FLAG_DIRECT_LOADS) && smem <= 100 * 1024 && sec_bytes % 16 == 0) {
-        PKV_CUDA(ctx, cudaFuncSetAttribute(quantize_gather_staged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        quantize_gather_staged_kernel<<<p.nb * layers, kGatherThreads, smem, stream>>>(
-            p, (int)sec_bytes, pool->stride_head == g->head_dim ? 1 : 0);
+        const int hc = pool->stride_head == g->head_dim ? 1 : 0;
+        // channels per thread: the whole scale group up to 32 channels
+        if (g->group >= 32) {
+            PKV_CUDA(ctx, cudaFuncSetAttribute(quantize_gather_staged_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            quantize_gather_staged_kernel<4><<<p.nb * layers, kGatherThreads, smem, stream>>>(p, (int)sec_bytes, hc);
+        } else if (g->group == 16) {
+            PKV_CUDA(ctx, cudaFuncSetAttribute(quantize_gather_staged_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            quantize_gather_staged_kernel<2><<<p.nb * layers, kGatherThreads, smem, stream>>>(p, (int)sec_bytes, hc);
+        } else {
+            PKV_CUDA(ctx, cudaFuncSetAttribute(quantize_gather_staged_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            quantize_gather_staged_kernel<1><<<p.nb * layers, kGatherThreads, smem, stream>>>(p, (int)sec_bytes, hc);
+        }
     } else {
         quantize_gather_kernel<<<p.nb * layers, kGatherThreads, g->block_tokens * sizeof(long long), stream>>>(p);
     }

@@ -499,7 +499,21 @@ def run_ours(args):
             if i >= 3:
                 tts.append(a.elapsed_time(b))
         token_form_us = 1e3 * statistics.median(tts)
+        ta_args = pk.select_args(kind=pk.SCORE_ATTN_F16, n_layers=SL, n_suffix_tokens=16384, block_tokens=16,
+                                 dirty_tokens=640, top_k=245, layer_mode=pk.LAYERS_SHARED, attn=attn, **out)
+        tts2 = []
+        for i in range(9):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            ctx.select_repair_tokens(ta_args, stream)
+            b.record(stream)
+            b.synchronize()
+            if i >= 3:
+                tts2.append(a.elapsed_time(b))
+        token_form_attn_us = 1e3 * statistics.median(tts2)
         select_scale = {"token_form_us_from_token_scores": token_form_us,
+                        "token_form_us_from_attention": token_form_attn_us,
+                        "token_form_attn_gbps": attn.numel() * 2 / (token_form_attn_us * 1e-6) / 1e9,
                         "workload": f"stored attention fp16 [{SL}][32][64][16384] ({SL * 64} MiB), 40-block dirty window, top-32 per layer",
                         "select_us": 1e3 * t_ms, "attn_gbps": nbytes / (t_ms * 1e-3) / 1e9,
                         "frac_of_hbm_peak": nbytes / (t_ms * 1e-3) / 1e9 / peak, "launches": 3}

@@ -139,6 +139,77 @@ block_mass_octet_kernel(const MassParams p) {
     }
 }
 
+// Token granularity (the score of Eq. 10 per token): one thread owns eight consecutive tokens and keeps one exact sum
+// per token over the rows of its CTA.  Same loads and the same exact-fp32 fast path as the block kernel.
+__global__ void __launch_bounds__(256)
+token_mass_octet_kernel(const MassParams p) {
+    const int oct = blockIdx.x * blockDim.x + threadIdx.x;
+    const int col = oct * 8;
+    const int l = blockIdx.z;
+    const int R = p.Hq * p.Q;
+    const int r0 = blockIdx.y * p.rows_per_cta;
+    const int r1 = min(R, r0 + p.rows_per_cta);
+    if (col + 8 > p.n) {                                   // ragged tail: element loads
+        bool bad = false;
+        for (int i = 0; i < 8 && col + i < p.n; i++) {
+            unsigned long long acc = 0;
+            for (int r = r0; r < r1; r++) {
+                const int h = r / p.Q, q = r - h * p.Q;
+                acc += units_any(__ldg(p.attn + (long long)l * p.stride_layer + (long long)h * p.stride_head +
+                                       (long long)q * p.stride_query + col + i), &bad);
+            }
+            if (acc) atomicAdd(p.mass + (long long)l * p.NB + col + i, acc);
+        }
+        if (bad) atomicCAS(p.status, 0, (int)PATCHKV_E_BADINPUT);
+        return;
+    }
+    float facc[8];
+    unsigned long long acc[8];
+#pragma unroll
+    for (int i = 0; i < 8; i++) { facc[i] = 0.0f; acc[i] = 0; }
+    int nf = 0;
+    bool bad = false;
+    const uint16_t* base = p.attn + (long long)l * p.stride_layer + col;
+    int h = r0 / p.Q, q = r0 - h * p.Q;
+    for (int r = r0; r < r1; r += kMassBatch) {
+        uint4 w[kMassBatch];
+#pragma unroll
+        for (int i = 0; i < kMassBatch; i++) {
+            w[i] = make_uint4(0, 0, 0, 0);
+            if (r + i < r1) {
+                w[i] = __ldcs(reinterpret_cast<const uint4*>(base + (long long)h * p.stride_head + (long long)q * p.stride_query));
+                if (++q == p.Q) { q = 0; h++; }
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < kMassBatch; i++) {
+            const uint32_t ww[4] = {w[i].x, w[i].y, w[i].z, w[i].w};
+            if (((ww[0] | ww[1] | ww[2] | ww[3]) & 0xE000E000u) == 0) {
+                // every entry below 2^-7: 64 such rows add up exactly in fp32 (< 1/2, multiples of 2^-24)
+#pragma unroll
+                for (int k = 0; k < 4; k++) {
+                    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&ww[k]));
+                    facc[2 * k] += f.x; facc[2 * k + 1] += f.y;
+                }
+                if (++nf == 64) {
+#pragma unroll
+                    for (int k = 0; k < 8; k++) { acc[k] += __float2uint_rz(facc[k] * 16777216.0f); facc[k] = 0.0f; }
+                    nf = 0;
+                }
+            } else {
+#pragma unroll
+                for (int k = 0; k < 4; k++) { acc[2 * k] += units_any(ww[k], &bad); acc[2 * k + 1] += units_any(ww[k] >> 16, &bad); }
+            }
+        }
+    }
+    if (bad) atomicCAS(p.status, 0, (int)PATCHKV_E_BADINPUT);
+#pragma unroll
+    for (int k = 0; k < 8; k++) {
+        const unsigned long long v = acc[k] + __float2uint_rz(facc[k] * 16777216.0f);
+        if (v) atomicAdd(p.mass + (long long)l * p.NB + col + k, v);
+    }
+}
+
 // Any B, any strides, any alignment: one thread per key position.
 __global__ void __launch_bounds__(256)
 block_mass_generic_kernel(const MassParams p) {
@@ -526,7 +597,11 @@ extern "C" int patchkv_select_repair_tokens(patchkv_ctx* ctx, const patchkv_sele
             mp.stride_layer = a->attn_stride_layer; mp.stride_head = a->attn_stride_head; mp.stride_query = a->attn_stride_query;
             mp.Hq = a->n_q_heads; mp.Q = a->n_queries; mp.n = n; mp.B = 1; mp.NB = n;
             mp.mass = m; mp.status = ctx->d_status;
-            const int tiles = (n + 255) / 256;
+            const bool octet = ((reinterpret_cast<uintptr_t>(a->attn) & 15u) == 0) &&
+                               ((a->attn_stride_layer | a->attn_stride_head | a->attn_stride_query) & 7) == 0;
+            const int cols = octet ? (n + 7) / 8 : n;
+            const int tiles = (cols + 255) / 256;
+            // few row groups: every thread ends with one 64-bit atomic per token
             long long groups = (long long)ctx->sm_count * 16 / ((long long)tiles * L);
             if (groups < 1) groups = 1;
             long long rpc = (rows + groups - 1) / groups;
@@ -535,7 +610,8 @@ extern "C" int patchkv_select_repair_tokens(patchkv_ctx* ctx, const patchkv_sele
             groups = (rows + rpc - 1) / rpc;
             if (groups > 65535) return fail(ctx, PATCHKV_E_UNSUPPORTED, "select: grid too large");
             mp.rows_per_cta = (int)rpc;
-            block_mass_generic_kernel<<<dim3(tiles, (unsigned)groups, L), 256, 0, stream>>>(mp);
+            if (octet) token_mass_octet_kernel<<<dim3(tiles, (unsigned)groups, L), 256, 0, stream>>>(mp);
+            else block_mass_generic_kernel<<<dim3(tiles, (unsigned)groups, L), 256, 0, stream>>>(mp);
             PKV_CUDA(ctx, cudaGetLastError());
         }
         mass = m;

@@ -100,3 +100,42 @@ def test_token_form_and_block_form_differ_on_the_constructed_case(ctx):
     bad = pk.select_args(kind=pk.SCORE_BLOCK_MASS, n_layers=1, n_suffix_tokens=n, block_tokens=B, dirty_tokens=0,
                          top_k=1, layer_mode=0, mass=bm, **out_b)
     assert ctx.select_repair_tokens(bad, check=False) == pk.E_INVALID
+
+
+def test_strided_and_unaligned_attention(ctx):
+    from paper_2609_26219_b200 import binding as pk
+    ck = pin.config_tiny()
+    rc, tmass = oracle.block_mass(ck.attn.numpy(), 1)
+    sel = oracle.select_tokens(tmass, 16, 90, 15, 1)
+    big = torch.zeros((2, 8, 16, 1024 + 3), dtype=torch.float16, device=DEV)
+    big[..., 3:] = ck.attn.to(DEV)
+    wide = torch.zeros((2, 16, 16, 1024), dtype=torch.float16, device=DEV)
+    wide[:, ::2] = ck.attn.to(DEV)
+    for view in (big[..., 3:], wide[:, ::2]):
+        out = _outputs(2, 64)
+        mass_out = torch.zeros((2, 1024), dtype=torch.int64, device=DEV)
+        a = pk.select_args(kind=pk.SCORE_ATTN_F16, n_layers=2, n_suffix_tokens=1024, block_tokens=16, dirty_tokens=90,
+                           top_k=15, layer_mode=1, attn=view, mass_out=mass_out, **out)
+        ctx.select_repair_tokens(a)
+        _check(out, sel)
+        assert np.array_equal(mass_out.cpu().numpy().astype(np.uint64), tmass)
+
+
+def test_token_mass_over_the_whole_fp16_range_and_bad_entries(ctx):
+    from paper_2609_26219_b200 import binding as pk
+    rng = np.random.default_rng(5)
+    bits = rng.integers(0, 0x7C00, size=(2, 3, 70, 512)).astype(np.uint16)
+    bits[0, 0, 0, 3] = 0xBC00       # -1.0
+    bits[1, 2, 5, 40] = 0x7E00      # NaN
+    rc, tmass = oracle.block_mass(bits, 1)
+    assert rc == oracle.E_BADINPUT
+    sel = oracle.select_tokens(tmass, 16, 33, 20, 0)
+    out = _outputs(2, 32)
+    mass_out = torch.zeros((2, 512), dtype=torch.int64, device=DEV)
+    a = pk.select_args(kind=pk.SCORE_ATTN_F16, n_layers=2, n_suffix_tokens=512, block_tokens=16, dirty_tokens=33,
+                       top_k=20, layer_mode=0, attn=torch.from_numpy(bits.view(np.float16).copy()).to(DEV),
+                       mass_out=mass_out, **out)
+    ctx.select_repair_tokens(a)
+    _check(out, sel)
+    assert np.array_equal(mass_out.cpu().numpy().astype(np.uint64), tmass)
+    assert ctx.query_status() == -7

@@ -44,8 +44,8 @@ WORKLOAD = "llama3-8b-shaped: L=32 H=8 D=128 base=5e5 n=16384 B=P=16 G=32 tags 3
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one restore launch on this workload, from the ncu capture of a
 # 4-layer slice summarised in profiles/restore_pipe_kernel_llama8b_slice.md: reads scale with the layers
-# (8 x 150.6 MB); writes are the algorithmic 1824 MB minus the ~54 MB still dirty in L2 when the kernel ends
-RESTORE_KERNEL_DRAM_TRAFFIC_BYTES = 2_975_000_000
+# (8 x 151.1 MB); writes are the algorithmic 1824 MB minus the ~51 MB still dirty in L2 when the kernel ends
+RESTORE_KERNEL_DRAM_TRAFFIC_BYTES = 2_982_000_000
 
 
 # ------------------------------------------------------------------------------------------ helpers
@@ -624,10 +624,11 @@ def run_ours(args):
     if rank == 0 and world == 1 and not args.no_cpu:
         import oracle
         oracle.build()
-        sample_layers = list(range(0, ck.geom.n_layers, 4))
-        dt, wb, threads = oracle_sample(ck, sample_layers, repeats=2)
+        sample_layers = list(range(ck.geom.n_layers))
+        dt, wb, threads = oracle_sample(ck, sample_layers, repeats=3)
         cpu_baseline = {"value": wb / dt / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
-                        "sample": f"{len(sample_layers)} of 32 layers (select + restore), best of 2, {dt:.2f} s"}
+                        "sample": f"all {len(sample_layers)} layers of the workload (select + restore), best of 3 passes "
+                                  f"of {dt:.2f} s on {threads} threads"}
 
     if rank == 0:
         line = {

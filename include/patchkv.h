@@ -261,8 +261,9 @@ PATCHKV_API int patchkv_select_repair_tokens(patchkv_ctx* ctx, const patchkv_sel
 PATCHKV_API int patchkv_select_repair_static(const patchkv_select_args* args, void* stream, int32_t* device_status);
 
 /* Section IV-D fused restore (dequantise, Eq. 3 RoPE correction of K, page placement) of the reuse sets of
- * up to PATCHKV_MAX_SESSIONS sessions whose payloads are in device memory.  One kernel launch, asynchronous
- * on `stream`, no host synchronisation, no allocation. */
+ * up to PATCHKV_MAX_SESSIONS sessions whose payloads are in device memory.  One 4-byte counter reset and one kernel
+ * launch, asynchronous on `stream`, no host synchronisation, no allocation; the pair can be captured in a CUDA graph.
+ * Launches from one context may overlap on different streams (each takes its own work counter from a ring of 256). */
 PATCHKV_API int patchkv_restore(patchkv_ctx* ctx, const patchkv_geom* geom, const patchkv_pool* pool,
                                 const patchkv_session* sessions, int n_sessions, void* stream);
 

@@ -43,7 +43,7 @@ UNIT = "GB/s"
 WORKLOAD = "llama3-8b-shaped: L=32 H=8 D=128 base=5e5 n=16384 B=P=16 G=32 tags 30/50/20 repair 15% device-resident"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one restore launch on this workload, from the ncu capture of a
-# 4-layer slice summarised in profiles/restore_pipe_kernel_llama8b_slice.md: reads scale with the layers
+# 4-layer slice summarised under profiles/: reads scale with the layers
 # (8 x 151.1 MB); writes are the algorithmic 1824 MB minus the ~51 MB still dirty in L2 when the kernel ends
 RESTORE_KERNEL_DRAM_TRAFFIC_BYTES = 2_982_000_000
 

@@ -407,3 +407,18 @@ def test_eight_device_resident_sessions_in_one_launch(ctx):
         pools = None if k_ref is None else (k_ref, v_ref)
         rc, k_ref, v_ref, _ = oracle_restore(c, sel["reuse_idx"], sel["reuse_cnt"], pools=pools)
     check_pools(k, v, k_ref, v_ref, sess[0].geom)
+
+
+def test_geometry_limits_block_vectors_and_rotary_dim(ctx):
+    """block_tokens * n_kv_heads = 2048 is the largest block the kernels take; one more token is refused."""
+    from paper_2609_26219_b200 import binding as pk
+    g = pin.Geometry(1, 16, 16, 16, pin.ROPE_HALF, 1e4, 128, 128, 8)       # 128 tokens x 16 heads = 2048 vectors
+    ck = pin.make_checkpoint(name="max", seed=3, geom=g, n=300, delta=19, tag_probs=(0.3, 0.3, 0.2, 0.2), tags_per_layer=True,
+                             n_pages=8, dirty_tokens=0, top_k=1)
+    run_select_and_restore(ctx, ck)
+    st = staged(ck)
+    k, v, pool = gpu_pool(ck)
+    bad = st.geom(); bad.block_tokens = 129
+    assert ctx.restore(bad, pool, [st.session()], check=False) == pk.E_UNSUPPORTED
+    bad = st.geom(); bad.head_dim = 512; bad.rotary_dim = 512
+    assert ctx.restore(bad, pool, [st.session()], check=False) == pk.E_UNSUPPORTED

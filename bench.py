@@ -670,6 +670,10 @@ def main():
     ap.add_argument("--layers", type=int, default=32,
                     help="profiling only: fewer layers of the same workload (the bench line is quoted on 32)")
     args = ap.parse_args()
+    if int(os.environ.get("WORLD_SIZE", 1)) > 1:
+        # multi-rank runs time the headline step and the end-to-end leg only: the extra legs pin tens of GB of host
+        # memory per rank and say nothing about scaling
+        args.no_host_configs = args.no_writer = args.no_scale_select = args.no_graph = True
     if args.impl == "reference":
         run_reference(args)
     else:

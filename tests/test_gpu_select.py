@@ -143,3 +143,15 @@ def test_selection_at_scale_full_size_sampled_layers(ctx):
         assert np.array_equal(st.repair_idx[l].cpu().numpy(), sel["repair_idx"][0])
         assert np.array_equal(st.reuse_idx[l].cpu().numpy(), sel["reuse_idx"][0])
         assert int(st.reuse_cnt[l]) == 952 and int(st.repair_cnt[l]) == 72
+    # ... followed by the restore of the complement, driven by the lists just produced on the device
+    from gpu_common import check_pools, gpu_pool
+    from helpers import oracle_restore
+    k, v, pool = gpu_pool(ck)
+    ctx.restore(st.geom(), pool, [st.session()])
+    torch.cuda.synchronize()
+    assert ctx.query_status() == 0
+    layers = [0, 13, 31]
+    ridx, rcnt = st.reuse_idx.cpu().numpy(), st.reuse_cnt.cpu().numpy()
+    rc, k_ref, v_ref, _ = oracle_restore(ck, ridx, rcnt, layers=layers)
+    assert rc == oracle.OK
+    check_pools(k[layers], v[layers], k_ref, v_ref, ck.geom)

@@ -132,6 +132,45 @@ struct ThreadMap {
     int tab;            // HALF: table index of the first pair; INTERLEAVED: unused
 };
 
+// The per-thread channel map, fixed for a launch: `n_threads` threads split into TX = ceil(D / 16) channel lanes times
+// TY vector lanes; thread `tid` owns chunk A and chunk B of every vector its lane visits.
+template <bool INTER>
+__device__ __forceinline__ ThreadMap make_thread_map(const RestoreParams& p, int n_threads, int tid, bool* lane_active) {
+    ThreadMap tm;
+    const int TX = (p.D + 15) >> 4;
+    tm.TY = n_threads / TX;
+    const int tx = tid % TX;
+    tm.ty = tid / TX;
+    *lane_active = tm.ty < tm.TY;
+    if (!INTER) {
+        const int n_rot = p.Dr >> 4;
+        if (tx < n_rot) { tm.cA = 8 * tx; tm.cB = (p.Dr >> 1) + 8 * tx; tm.rotA = tm.rotB = true; tm.tab = 8 * tx; }
+        else { tm.cA = p.Dr + 16 * (tx - n_rot); tm.cB = tm.cA + 8; tm.rotA = tm.rotB = false; tm.tab = 0; }
+    } else {
+        tm.cA = 16 * tx; tm.cB = tm.cA + 8;
+        tm.rotA = tm.cA < p.Dr; tm.rotB = tm.cB < p.Dr; tm.tab = 0;
+    }
+    if (tm.cB >= p.D) { tm.cB = -1; if (INTER) tm.rotB = false; }
+    tm.gA = tm.cA / p.G;
+    tm.gB = tm.cB >= 0 ? tm.cB / p.G : 0;
+    return tm;
+}
+
+// This thread's eight cos / sin entries of one session's table (HALF: pairs tab .. tab+7; INTERLEAVED: four pairs
+// of chunk A, then four of chunk B).
+template <bool INTER>
+__device__ __forceinline__ void load_rotation(const RestoreParams& p, int session, const ThreadMap& tm, float* tc, float* ts) {
+#pragma unroll
+    for (int i = 0; i < 8; i++) {
+        int idx;
+        if (!INTER) idx = tm.tab + i;
+        else idx = (i < 4) ? (tm.cA >> 1) + i : ((tm.cB >= 0 ? tm.cB : 0) >> 1) + (i - 4);
+        idx = min(idx, PATCHKV_MAX_ROTARY_DIM / 2 - 1);
+        tc[i] = p.cs[session][0][idx];
+        ts[i] = p.cs[session][1][idx];
+    }
+}
+
 template <int KF, int VF, bool INTER>
 __device__ __forceinline__ void restore_vectors(const RestoreParams& p, const uint8_t* rec, int nvec,
                                                 const long long* vec_off, const ThreadMap& tm,
@@ -196,24 +235,8 @@ __global__ void __launch_bounds__(kThreads)
 restore_kernel(const __grid_constant__ RestoreParams p) {
     __shared__ long long vec_off[PATCHKV_MAX_BLOCK_VECTORS];
 
-    // ---- per-thread channel map (fixed for the whole launch)
-    ThreadMap tm;
-    const int TX = (p.D + 15) >> 4;
-    tm.TY = kThreads / TX;
-    const int tx = threadIdx.x % TX;
-    tm.ty = threadIdx.x / TX;
-    const bool lane_active = tm.ty < tm.TY;
-    if (!INTER) {
-        const int n_rot = p.Dr >> 4;
-        if (tx < n_rot) { tm.cA = 8 * tx; tm.cB = (p.Dr >> 1) + 8 * tx; tm.rotA = tm.rotB = true; tm.tab = 8 * tx; }
-        else { tm.cA = p.Dr + 16 * (tx - n_rot); tm.cB = tm.cA + 8; tm.rotA = tm.rotB = false; tm.tab = 0; }
-    } else {
-        tm.cA = 16 * tx; tm.cB = tm.cA + 8;
-        tm.rotA = tm.cA < p.Dr; tm.rotB = tm.cB < p.Dr; tm.tab = 0;
-    }
-    if (tm.cB >= p.D) { tm.cB = -1; tm.rotB = INTER ? false : tm.rotB; }
-    tm.gA = tm.cA / p.G;
-    tm.gB = tm.cB >= 0 ? tm.cB / p.G : 0;
+    bool lane_active;
+    const ThreadMap tm = make_thread_map<INTER>(p, kThreads, threadIdx.x, &lane_active);
 
     float tc[8], ts[8];
     int cur_session = -1;
@@ -228,18 +251,7 @@ restore_kernel(const __grid_constant__ RestoreParams p) {
         const int r = local - (l - p.layer_begin) * S.nb;
         if (r >= __ldg(S.reuse_cnt + l)) continue;                     // uniform over the CTA
 
-        if (si != cur_session) {                                        // this thread's cos / sin entries
-            cur_session = si;
-#pragma unroll
-            for (int i = 0; i < 8; i++) {
-                int idx;
-                if (!INTER) idx = tm.tab + i;
-                else idx = (i < 4) ? (tm.cA >> 1) + i : ((tm.cB >= 0 ? tm.cB : 0) >> 1) + (i - 4);
-                idx = min(idx, PATCHKV_MAX_ROTARY_DIM / 2 - 1);
-                tc[i] = p.cs[si][0][idx];
-                ts[i] = p.cs[si][1][idx];
-            }
-        }
+        if (si != cur_session) { cur_session = si; load_rotation<INTER>(p, si, tm, tc, ts); }
 
         // ---- directory entry of the block; every thread reads the same words (broadcast)
         const int j = __ldg(S.reuse_idx + (size_t)l * S.nb + r);
@@ -525,23 +537,8 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
     } else {
         // ================================================================ consumer warps
         const int c = threadIdx.x - 32;
-        ThreadMap tm;
-        const int TX = (p.D + 15) >> 4;
-        tm.TY = kPipeConsumers / TX;
-        const int tx = c % TX;
-        tm.ty = c / TX;
-        const bool lane_active = tm.ty < tm.TY;
-        if (!INTER) {
-            const int n_rot = p.Dr >> 4;
-            if (tx < n_rot) { tm.cA = 8 * tx; tm.cB = (p.Dr >> 1) + 8 * tx; tm.rotA = tm.rotB = true; tm.tab = 8 * tx; }
-            else { tm.cA = p.Dr + 16 * (tx - n_rot); tm.cB = tm.cA + 8; tm.rotA = tm.rotB = false; tm.tab = 0; }
-        } else {
-            tm.cA = 16 * tx; tm.cB = tm.cA + 8;
-            tm.rotA = tm.cA < p.Dr; tm.rotB = tm.cB < p.Dr; tm.tab = 0;
-        }
-        if (tm.cB >= p.D) { tm.cB = -1; if (INTER) tm.rotB = false; }
-        tm.gA = tm.cA / p.G;
-        tm.gB = tm.cB >= 0 ? tm.cB / p.G : 0;
+        bool lane_active;
+        const ThreadMap tm = make_thread_map<INTER>(p, kPipeConsumers, c, &lane_active);
         const int gpv = p.D / p.G;
         float tc[8], ts[8];
         int cur_session = -1;
@@ -554,18 +551,7 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
             StageMeta m;
             m.nvec = (int)mw.x; m.fmt = (int)mw.y; m.flags = (int)mw.z; m.session = (int)mw.w;
             if (m.nvec < 0) break;
-            if (m.session != cur_session) {
-                cur_session = m.session;
-#pragma unroll
-                for (int i = 0; i < 8; i++) {
-                    int idx;
-                    if (!INTER) idx = tm.tab + i;
-                    else idx = (i < 4) ? (tm.cA >> 1) + i : ((tm.cB >= 0 ? tm.cB : 0) >> 1) + (i - 4);
-                    idx = min(idx, PATCHKV_MAX_ROTARY_DIM / 2 - 1);
-                    tc[i] = p.cs[cur_session][0][idx];
-                    ts[i] = p.cs[cur_session][1][idx];
-                }
-            }
+            if (m.session != cur_session) { cur_session = m.session; load_rotation<INTER>(p, cur_session, tm, tc, ts); }
             if (lane_active) {
                 const uint32_t codes = smem_u32(sp), scales = codes + off_scales;
                 const uint32_t voff = codes + off_vec;

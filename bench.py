@@ -324,33 +324,12 @@ def run_ours(args):
         except Exception as exc:           # reported, never fatal: the headline numbers do not depend on it
             graph_ms = f"unavailable: {type(exc).__name__}"
 
-    # ---- the restore kernel writes 1.5 bytes for every byte it reads: measure what this GPU sustains for writes alone
-    fill_gbps = None
-    if world == 1:
-        buf = torch.empty(1 << 31, dtype=torch.uint8, device=dev)
-        best = None
-        for i in range(8):
-            fa, fb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            fa.record()
-            buf.fill_(i)
-            fb.record()
-            fb.synchronize()
-            if i >= 3:
-                best = fa.elapsed_time(fb) if best is None else min(best, fa.elapsed_time(fb))
-        fill_gbps = buf.numel() / (best * 1e-3) / 1e9
-        del buf
-
     peak, peak_kind = measured_hbm_peak()
     achieved = (read_b + written_b) / (restore_avg_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": "restore_pipe_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": f"of {peak_kind} copy bandwidth (burst)",
                 "frac_of_nominal_8tbs": achieved / 8000.0, "traffic": RESTORE_KERNEL_DRAM_TRAFFIC_BYTES,
-                "algorithmic_bytes_per_launch": read_b + written_b, "kernel_ms": restore_avg_ms,
-                "write_side": None if fill_gbps is None else {
-                    "note": "60 % of the kernel's traffic is writes; a pure fill (torch fill_ of 2 GiB, best of 5, same run) "
-                            "is the write-only ceiling",
-                    "fill_gbps": fill_gbps, "achieved_write_gbps": written_b / (restore_avg_ms * 1e-3) / 1e9,
-                    "frac_of_fill": written_b / (restore_avg_ms * 1e-3) / 1e9 / fill_gbps}}
+                "algorithmic_bytes_per_launch": read_b + written_b, "kernel_ms": restore_avg_ms}
 
     # ---- offload side: write a checkpoint of all 1024 blocks x 32 layers from the pool (not on the resume path)
     writer = None

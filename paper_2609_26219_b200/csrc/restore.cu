@@ -130,6 +130,8 @@ struct ThreadMap {
     int gA, gB;         // scale group of each chunk
     bool rotA, rotB;    // chunk holds rotary channels (HALF: A and B are partners and rotate together)
     int tab;            // HALF: table index of the first pair; INTERLEAVED: unused
+    int t0, h0;         // (token, head) of vector index ty inside a unit, and the step of one loop iteration:
+    int dt, dh;         // vector ty + k*TY is (t0 + k*dt + carries, (h0 + k*dh) mod H)
 };
 
 // The per-thread channel map, fixed for a launch: `n_threads` threads split into TX = ceil(D / 16) channel lanes times
@@ -153,6 +155,8 @@ __device__ __forceinline__ ThreadMap make_thread_map(const RestoreParams& p, int
     if (tm.cB >= p.D) { tm.cB = -1; if (INTER) tm.rotB = false; }
     tm.gA = tm.cA / p.G;
     tm.gB = tm.cB >= 0 ? tm.cB / p.G : 0;
+    tm.t0 = tm.ty / p.H; tm.h0 = tm.ty - tm.t0 * p.H;
+    tm.dt = tm.TY / p.H; tm.dh = tm.TY - tm.dt * p.H;
     return tm;
 }
 
@@ -340,17 +344,20 @@ __device__ __forceinline__ Chunk lds_chunk(uint32_t codes, uint32_t scales, int 
 
 template <int FMT, bool INTER>
 __device__ __forceinline__ void consume_unit(const RestoreParams& p, uint32_t codes, uint32_t scales,
-                                             uint32_t vec_off, int nvec, uint16_t* dst_base,
+                                             uint32_t tok_off, int nvec, uint16_t* dst_base,
                                              const ThreadMap& tm, int gpv, const float* tc, const float* ts, bool rotate) {
     const bool hasB = tm.cB >= 0;
     const bool rotA = rotate && tm.rotA, rotB = rotate && tm.rotB;
+    int t = tm.t0, h = tm.h0;                              // (token, head) of `vec`, advanced without divisions
 #pragma unroll 1
     for (int vec = tm.ty; vec < nvec; vec += tm.TY) {
         const Chunk ca = lds_chunk<FMT>(codes, scales, vec, p.D, gpv, tm.cA, tm.gA);
         Chunk cb = ca;
         if (hasB) cb = lds_chunk<FMT>(codes, scales, vec, p.D, gpv, tm.cB, tm.gB);
-        const uint2 vo = lds64(vec_off + 8u * (uint32_t)vec);
-        uint16_t* d = dst_base + (long long)(((unsigned long long)vo.y << 32) | vo.x);
+        const uint2 vo = lds64(tok_off + 8u * (uint32_t)t);
+        uint16_t* d = dst_base + (long long)(((unsigned long long)vo.y << 32) | vo.x) + (long long)h * p.stride_head;
+        t += tm.dt; h += tm.dh;
+        if (h >= p.H) { h -= p.H; t++; }
         uint4 oa = ca.w, ob = cb.w;
         if (FMT != FMT_BF16 || rotA || rotB) {
             float a[8], b[8];
@@ -387,7 +394,7 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
     __syncthreads();
     const int off_scales = p.stage_code_bytes;
     const int off_vec = off_scales + p.stage_scale_bytes;
-    const int off_meta = (off_vec + 8 * p.unit_tokens * p.H + 15) & ~15;
+    const int off_meta = (off_vec + 8 * p.unit_tokens + 15) & ~15;
     volatile int* abortp = &abort_flag;
 
     if (threadIdx.x < 32) {
@@ -485,12 +492,11 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
                         if (!__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], ((q / S) & 1) ^ 1, abortp))) { alive = false; break; }
                         uint8_t* sp = ring + (size_t)stage * p.stage_bytes;
                         long long* voff = reinterpret_cast<long long*>(sp + off_vec);
-                        for (int i = lane; i < nt * p.H; i += 32) {
-                            const int tt = i / p.H, h = i - tt * p.H;
-                            const int us = d.slot0 + t0 + tt;               // slot counted from the first page
+                        for (int i = lane; i < nt; i += 32) {                // one destination row per token
+                            const int us = d.slot0 + t0 + i;               // slot counted from the first page
                             const int pi = us / p.P;
                             voff[i] = (long long)l * p.stride_layer + (long long)d.pages[pi] * p.stride_page +
-                                      (long long)(us - pi * p.P) * p.stride_token + (long long)h * p.stride_head;
+                                      (long long)(us - pi * p.P) * p.stride_token;
                         }
                         if (lane == 0) {
                             StageMeta m;
@@ -634,7 +640,7 @@ static bool plan_pipeline(const patchkv_ctx* ctx, RestoreParams* p) {
     p->unit_tokens = (int32_t)ut;
     p->stage_code_bytes = (int32_t)(ut * hd * 2);
     p->stage_scale_bytes = (int32_t)(ut * (hd / p->G) * 2);
-    const long long raw = (long long)p->stage_code_bytes + p->stage_scale_bytes + 8 * ut * p->H + 32;
+    const long long raw = (long long)p->stage_code_bytes + p->stage_scale_bytes + 8 * ut + 32;
     p->stage_bytes = (int32_t)((raw + 127) / 128 * 128);
     long long budget = ((long long)ctx->max_smem_optin - 2048) / 2;   // two CTAs per SM
     if (budget > 112 * 1024) budget = 112 * 1024;

@@ -405,7 +405,9 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
         const int lane = threadIdx.x;
         const uint64_t elems = (uint64_t)p.B * p.H * p.D;
         const uint32_t hd = (uint32_t)p.H * p.D;
-        uint32_t q = 0;
+        uint32_t q = 0;                                  // units issued
+        int stage = 0;                                   // q % S, and the parity of q / S, kept without divisions
+        uint32_t phase = 0;
         bool alive = true;
         // Work is handed out by a global counter in rounds that shrink towards the end of the list (a fraction of
         // what is left per CTA, at most 32 blocks, at least one), so that CTAs with heavier tags do not leave a
@@ -487,9 +489,8 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
 #pragma unroll 1
                     for (int t0 = 0; t0 < valid; t0 += p.unit_tokens) {
                         const int nt = min(p.unit_tokens, valid - t0);
-                        const int stage = q % S;
                         // the verdict is made warp-uniform: the lanes meet again at __syncwarp below
-                        if (!__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], ((q / S) & 1) ^ 1, abortp))) { alive = false; break; }
+                        if (!__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], phase ^ 1, abortp))) { alive = false; break; }
                         uint8_t* sp = ring + (size_t)stage * p.stage_bytes;
                         long long* voff = reinterpret_cast<long long*>(sp + off_vec);
                         for (int i = lane; i < nt; i += 32) {                // one destination row per token
@@ -512,14 +513,14 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
                             if (sb) bulk_g2s(sp + off_scales, sec_scales[sec] + (size_t)t0 * stok, sb, &full_bar[stage]);
                         }
                         q++;
+                        if (++stage == S) { stage = 0; phase ^= 1; }
                     }
                 }
             }
             __syncwarp();                                 // descs are rewritten by the next round
         }
         if (alive) {                                     // tell the consumers that the work list is exhausted
-            const int stage = q % S;
-            if (__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], ((q / S) & 1) ^ 1, abortp))) {
+            if (__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], phase ^ 1, abortp))) {
                 if (lane == 0) {
                     StageMeta m; m.nvec = -1; m.fmt = 0; m.flags = 0; m.session = 0;
                     *reinterpret_cast<StageMeta*>(ring + (size_t)stage * p.stage_bytes + off_meta) = m;
@@ -548,10 +549,10 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
         const int gpv = p.D / p.G;
         float tc[8], ts[8];
         int cur_session = -1;
-        uint32_t q = 0;
+        int stage = 0;
+        uint32_t phase = 0;
         while (true) {
-            const int stage = q % S;
-            if (!__all_sync(0xFFFFFFFFu, mbar_wait(&full_bar[stage], (q / S) & 1, abortp))) break;
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait(&full_bar[stage], phase, abortp))) break;
             uint8_t* sp = ring + (size_t)stage * p.stage_bytes;
             const uint4 mw = lds128(smem_u32(sp) + off_meta);
             StageMeta m;
@@ -571,7 +572,7 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
             }
             __syncwarp();
             if ((c & 31) == 0) mbar_arrive(&empty_bar[stage]);
-            q++;
+            if (++stage == S) { stage = 0; phase ^= 1; }
         }
         if (c == 0 && *abortp) atomicCAS(p.status, 0, (int)PATCHKV_E_TIMEOUT);
     }

@@ -196,6 +196,15 @@ token_mass_octet_kernel(const MassParams p) {
                     for (int k = 0; k < 8; k++) { acc[k] += __float2uint_rz(facc[k] * 16777216.0f); facc[k] = 0.0f; }
                     nf = 0;
                 }
+            } else if (((ww[0] | ww[1] | ww[2] | ww[3]) & 0xC000C000u) == 0) {
+                // every entry in [0, 2): value * 2^24 is an integer below 2^25, exact in fp32 (a warp takes this path
+                // whenever one of its lanes holds a large attention weight, so it has to stay cheap)
+#pragma unroll
+                for (int k = 0; k < 4; k++) {
+                    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&ww[k]));
+                    acc[2 * k] += __float2uint_rz(f.x * 16777216.0f);
+                    acc[2 * k + 1] += __float2uint_rz(f.y * 16777216.0f);
+                }
             } else {
 #pragma unroll
                 for (int k = 0; k < 4; k++) { acc[2 * k] += units_any(ww[k], &bad); acc[2 * k + 1] += units_any(ww[k] >> 16, &bad); }

@@ -312,7 +312,8 @@ restore_kernel(const __grid_constant__ RestoreParams p) {
 // shared memory and write the bf16 rows to the pool with 128-bit stores.  Directory latency and HBM read
 // latency are hidden by the ring instead of by occupancy.  Every wait is bounded.
 constexpr int kPipeConsumers = 256;
-constexpr int kPipeThreads = kPipeConsumers + 32;
+constexpr int kPipeProducers = 64;                          // warp 0 feeds the ring, warp 1 resolves the next round of blocks
+constexpr int kPipeThreads = kPipeConsumers + kPipeProducers;
 constexpr int kMaxStages = 8;
 
 struct StageMeta { int32_t nvec, fmt, flags, session; };   // nvec < 0: no more work; flags bit0 = K section, bit1 = rotate
@@ -383,11 +384,14 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
     extern __shared__ __align__(128) uint8_t ring[];
     __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages];
     __shared__ int abort_flag;
-    __shared__ ItemDesc descs[32];
+    __shared__ ItemDesc descs[2][32];                    // two rounds of resolved blocks: one being issued, one being resolved
+    __shared__ int round_blocks[2];                      // blocks in each round buffer (-1: the work list is exhausted)
+    __shared__ uint64_t rfull_bar[2], rempty_bar[2];
 
     const int S = p.n_stages;
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; s++) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], kPipeConsumers / 32); }
+        for (int b = 0; b < 2; b++) { mbar_init(&rfull_bar[b], 1); mbar_init(&rempty_bar[b], 1); }
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -397,80 +401,99 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
     const int off_meta = (off_vec + 8 * p.unit_tokens + 15) & ~15;
     volatile int* abortp = &abort_flag;
 
-    if (threadIdx.x < 32) {
-        // ================================================================ producer warp
-        // Each lane resolves one upcoming block on its own (directory entry, record extent, destination pages),
-        // so the dependent global loads of 32 blocks overlap; the results are parked in shared memory and the
-        // warp then feeds the ring from them without touching global memory again.
+    if (threadIdx.x >= 32 && threadIdx.x < kPipeProducers) {
+        // ================================================================ resolver warp
+        // Takes rounds of blocks from the global work counter and resolves them one lane per block (directory
+        // entry, record extent, destination pages: three dependent global loads), into the round buffer the issuing
+        // warp is not reading.  The directory latency of a round is spent while the previous round is being issued.
+        // Rounds shrink towards the end of the list (a fraction of what is left per CTA, at most 32 blocks, at least
+        // one) so that CTAs with heavier tags do not leave a long tail; a round is consecutive entries of one list.
+        const int lane = threadIdx.x - 32;
+        const uint64_t elems = (uint64_t)p.B * p.H * p.D;
+        int rb = 0;
+        uint32_t rphase = 0;
+#pragma unroll 1
+        while (true) {
+            long long first = 0;
+            int round = 0;
+            if (lane == 0) {
+                const long long left = (long long)p.total_items - *reinterpret_cast<volatile int*>(p.sched);
+                round = (int)max(1ll, min(4ll, left / (8ll * gridDim.x)));       // small: a CTA holds up to two rounds
+                first = atomicAdd(p.sched, round);
+            }
+            first = __shfl_sync(0xFFFFFFFFu, first, 0);
+            round = __shfl_sync(0xFFFFFFFFu, round, 0);
+            ItemDesc d;
+            d.valid = 0;
+            const long long item = first + lane;
+            if (lane < round && item < p.total_items) {
+                int si = 0;
+#pragma unroll 1
+                for (int k = 1; k < p.n_sessions; k++) if (item >= p.s[k].item_begin) si = k;
+                const SessionDev& Sd = p.s[si];
+                const int local = (int)item - Sd.item_begin;
+                const int l = p.layer_begin + local / Sd.nb;
+                const int r = local - (l - p.layer_begin) * Sd.nb;
+                if (r < __ldg(Sd.reuse_cnt + l)) {
+                    const int j = __ldg(Sd.reuse_idx + (size_t)l * Sd.nb + r);
+                    bool bad = j < 0 || j >= Sd.nb;
+                    if (!bad) {
+                        const int tag = __ldg(Sd.tags + (size_t)l * Sd.nb + j);
+                        const unsigned long long off = __ldg(Sd.blk_off + (size_t)l * Sd.nb + j);
+                        const unsigned long long lbytes = __ldg(Sd.layer_bytes + l);
+                        const uint8_t* base = reinterpret_cast<const uint8_t*>(static_cast<uintptr_t>(
+                            __ldg(reinterpret_cast<const unsigned long long*>(Sd.layer_payload) + l)));
+                        const unsigned long long rbytes = record_bytes(tag, elems, p.G);
+                        bad = rbytes == 0 || off > lbytes || rbytes > lbytes - off || base == nullptr ||
+                              ((reinterpret_cast<uintptr_t>(base) + off) & 15u) != 0;
+                        const int valid = min(p.B, Sd.n - j * p.B);
+                        const long long u0 = (long long)j * p.B + Sd.dst_shift;
+                        const long long lp0 = u0 / p.P, lp1 = (u0 + valid - 1) / p.P;
+                        if (!bad) {                      // every destination page is validated before any write
+                            for (long long lp = lp0; lp <= lp1; lp++) {
+                                const int page = lp < Sd.n_table ? __ldg(Sd.block_table + lp) : -1;
+                                if (page < 0 || page >= p.n_pages) bad = true;
+                                d.pages[lp - lp0] = page;
+                            }
+                        }
+                        d.rec = base + off;
+                        d.valid = valid; d.tag = tag; d.l = l; d.si = si;
+                        d.slot0 = (int)(u0 - lp0 * p.P);
+                    }
+                    if (bad) { d.valid = 0; atomicCAS(p.status, 0, (int)PATCHKV_E_BOUNDS); }
+                }
+            }
+            // hand the round over once the issuing warp has finished with this buffer (bounded, warp-uniform)
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait(&rempty_bar[rb], rphase ^ 1, abortp))) break;
+            descs[rb][lane] = d;
+            if (lane == 0) round_blocks[rb] = first >= p.total_items ? -1 : round;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&rfull_bar[rb]);
+            if (first >= p.total_items) break;
+            rb ^= 1;
+            if (rb == 0) rphase ^= 1;
+        }
+    } else if (threadIdx.x < 32) {
+        // ================================================================ issuing warp
+        // Feeds the shared-memory ring from the resolved rounds without touching global memory itself: per unit it
+        // waits for a free stage, writes the per-token destination offsets and the unit header, and starts the two
+        // bulk copies.
         const int lane = threadIdx.x;
         const uint64_t elems = (uint64_t)p.B * p.H * p.D;
         const uint32_t hd = (uint32_t)p.H * p.D;
         uint32_t q = 0;                                  // units issued
         int stage = 0;                                   // q % S, and the parity of q / S, kept without divisions
         uint32_t phase = 0;
+        int ib = 0;
+        uint32_t iphase = 0;
         bool alive = true;
-        // Work is handed out by a global counter in rounds that shrink towards the end of the list (a fraction of
-        // what is left per CTA, at most 32 blocks, at least one), so that CTAs with heavier tags do not leave a
-        // long tail; the blocks of a round are consecutive entries of one reuse list.
 #pragma unroll 1
         while (alive) {
-            long long first = 0;
-            int round = 0;
-            if (lane == 0) {
-                const long long left = (long long)p.total_items - *reinterpret_cast<volatile int*>(p.sched);
-                round = (int)max(1ll, min(32ll, left / (2ll * gridDim.x)));
-                first = atomicAdd(p.sched, round);
-            }
-            first = __shfl_sync(0xFFFFFFFFu, first, 0);
-            round = __shfl_sync(0xFFFFFFFFu, round, 0);
-            if (first >= p.total_items) break;
-            {
-                ItemDesc d;
-                d.valid = 0;
-                const long long item = first + lane;
-                if (lane < round && item < p.total_items) {
-                    int si = 0;
-#pragma unroll 1
-                    for (int k = 1; k < p.n_sessions; k++) if (item >= p.s[k].item_begin) si = k;
-                    const SessionDev& Sd = p.s[si];
-                    const int local = (int)item - Sd.item_begin;
-                    const int l = p.layer_begin + local / Sd.nb;
-                    const int r = local - (l - p.layer_begin) * Sd.nb;
-                    if (r < __ldg(Sd.reuse_cnt + l)) {
-                        const int j = __ldg(Sd.reuse_idx + (size_t)l * Sd.nb + r);
-                        bool bad = j < 0 || j >= Sd.nb;
-                        if (!bad) {
-                            const int tag = __ldg(Sd.tags + (size_t)l * Sd.nb + j);
-                            const unsigned long long off = __ldg(Sd.blk_off + (size_t)l * Sd.nb + j);
-                            const unsigned long long lbytes = __ldg(Sd.layer_bytes + l);
-                            const uint8_t* base = reinterpret_cast<const uint8_t*>(static_cast<uintptr_t>(
-                                __ldg(reinterpret_cast<const unsigned long long*>(Sd.layer_payload) + l)));
-                            const unsigned long long rb = record_bytes(tag, elems, p.G);
-                            bad = rb == 0 || off > lbytes || rb > lbytes - off || base == nullptr ||
-                                  ((reinterpret_cast<uintptr_t>(base) + off) & 15u) != 0;
-                            const int valid = min(p.B, Sd.n - j * p.B);
-                            const long long u0 = (long long)j * p.B + Sd.dst_shift;
-                            const long long lp0 = u0 / p.P, lp1 = (u0 + valid - 1) / p.P;
-                            if (!bad) {                  // every destination page is validated before any write
-                                for (long long lp = lp0; lp <= lp1; lp++) {
-                                    const int page = lp < Sd.n_table ? __ldg(Sd.block_table + lp) : -1;
-                                    if (page < 0 || page >= p.n_pages) bad = true;
-                                    d.pages[lp - lp0] = page;
-                                }
-                            }
-                            d.rec = base + off;
-                            d.valid = valid; d.tag = tag; d.l = l; d.si = si;
-                            d.slot0 = (int)(u0 - lp0 * p.P);
-                        }
-                        if (bad) { d.valid = 0; atomicCAS(p.status, 0, (int)PATCHKV_E_BOUNDS); }
-                    }
-                }
-                descs[lane] = d;
-            }
-            __syncwarp();
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait(&rfull_bar[ib], iphase, abortp))) { alive = false; break; }
+            if (round_blocks[ib] < 0) break;
 #pragma unroll 1
             for (int di = 0; di < 32 && alive; di++) {
-                const ItemDesc& d = descs[di];
+                const ItemDesc& d = descs[ib][di];
                 const int valid = d.valid;
                 if (valid == 0) continue;
                 const int tag = d.tag, l = d.l, si = d.si;
@@ -517,7 +540,10 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
                     }
                 }
             }
-            __syncwarp();                                 // descs are rewritten by the next round
+            __syncwarp();                                 // every lane is done with this round buffer
+            if (lane == 0) mbar_arrive(&rempty_bar[ib]);
+            ib ^= 1;
+            if (ib == 0) iphase ^= 1;
         }
         if (alive) {                                     // tell the consumers that the work list is exhausted
             if (__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], phase ^ 1, abortp))) {
@@ -543,7 +569,7 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
         }
     } else {
         // ================================================================ consumer warps
-        const int c = threadIdx.x - 32;
+        const int c = threadIdx.x - kPipeProducers;
         bool lane_active;
         const ThreadMap tm = make_thread_map<INTER>(p, kPipeConsumers, c, &lane_active);
         const int gpv = p.D / p.G;

@@ -306,9 +306,9 @@ restore_kernel(const __grid_constant__ RestoreParams p) {
 }
 
 // ---------------------------------------------------------------- bulk-copy pipeline
-// One producer warp walks the work list, resolves the directory and the destination pages of each block a few
-// stages ahead, and stages the block's K and V sections (in units of a few tokens) into a shared-memory ring
-// with bulk asynchronous copies that complete on an mbarrier.  Eight consumer warps dequantise / rotate from
+// A resolver warp takes rounds of blocks from the global work counter and resolves the directory entry and the
+// destination pages of each block one round ahead; an issuing warp stages each resolved block's K and V sections
+// (in units of a few tokens) into a shared-memory ring with bulk asynchronous copies that complete on an mbarrier.  Eight consumer warps dequantise / rotate from
 // shared memory and write the bf16 rows to the pool with 128-bit stores.  Directory latency and HBM read
 // latency are hidden by the ring instead of by occupancy.  Every wait is bounded.
 constexpr int kPipeConsumers = 256;

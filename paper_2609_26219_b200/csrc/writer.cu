@@ -158,98 +158,10 @@ __device__ __forceinline__ void encode_chunk(const uint4& w, uint8_t* codes, uin
     if (((threadIdx.x & 31) & (seg - 1)) == 0) *reinterpret_cast<__half*>(scales + 2 * scale_index) = s16;
 }
 
-// NC consecutive 8-channel chunks (8 * NC channels of one head vector, all inside one scale group) per thread: the
-// scale arithmetic and the addressing are paid once per 8 * NC elements.  `seg` = lanes per scale group.
-template <int FMT, int NC>
-__device__ __forceinline__ void encode_span(const uint4* w, uint8_t* codes, uint8_t* scales, size_t elem0,
-                                            size_t scale_index, int seg, bool write) {
-    if (FMT == FMT_BF16) {
-        if (write) {
-#pragma unroll
-            for (int c = 0; c < NC; c++) reinterpret_cast<uint4*>(codes + 2 * elem0)[c] = w[c];
-        }
-        return;
-    }
-    // group maximum straight from the bf16 bit patterns (|x| as an integer compare is monotone for finite values)
-    uint32_t amax_bits = 0;
-#pragma unroll
-    for (int c = 0; c < NC; c++) {
-        const uint32_t ww[4] = {w[c].x, w[c].y, w[c].z, w[c].w};
-#pragma unroll
-        for (int i = 0; i < 4; i++) {
-            amax_bits = max(amax_bits, (ww[i] << 16) & 0x7FFF0000u);
-            amax_bits = max(amax_bits, ww[i] & 0x7FFF0000u);
-        }
-    }
-    for (int d = 1; d < seg; d <<= 1) amax_bits = max(amax_bits, __shfl_xor_sync(0xFFFFFFFFu, amax_bits, d));
-    const float amax = __uint_as_float(amax_bits);
-    const float qmax = FMT == FMT_INT8 ? 127.0f : 7.0f;
-    const __half s16 = __float2half_rn(__fdiv_rn(amax, qmax));
-    const float s = __half2float(s16);
-    const float r = s > 0.0f ? __frcp_rn(s) : 0.0f;
-    const float half_s = s > 0.0f ? 0.5f * s : -1.0f;
-    const float magic = 12582912.0f;
-    const bool subnormal = (__half_as_ushort(s16) & 0x7C00u) == 0 && s > 0.0f;
-    const f32x2 r2 = pack2(r, r), m2 = pack2(magic, magic), ns2 = pack2(-s, -s);
-    uint32_t out[2 * NC];
-#pragma unroll
-    for (int c = 0; c < NC; c++) {
-        float x[8];
-        x[0] = __uint_as_float(w[c].x << 16); x[1] = __uint_as_float(w[c].x & 0xFFFF0000u);
-        x[2] = __uint_as_float(w[c].y << 16); x[3] = __uint_as_float(w[c].y & 0xFFFF0000u);
-        x[4] = __uint_as_float(w[c].z << 16); x[5] = __uint_as_float(w[c].z & 0xFFFF0000u);
-        x[6] = __uint_as_float(w[c].w << 16); x[7] = __uint_as_float(w[c].w & 0xFFFF0000u);
-        uint32_t kb[8];
-        float df[8];
-        bool any_tie = false;
-#pragma unroll
-        for (int i = 0; i < 8; i += 2) {
-            const f32x2 x2 = pack2(x[i], x[i + 1]);
-            const f32x2 tm = fma2(x2, r2, m2);
-            const f32x2 d2 = fma2(sub2(tm, m2), ns2, x2);
-            float a0, a1;
-            unpack2(tm, a0, a1);
-            kb[i] = __float_as_uint(a0); kb[i + 1] = __float_as_uint(a1);
-            unpack2(d2, df[i], df[i + 1]);
-            any_tie = any_tie || fabsf(df[i]) == half_s || fabsf(df[i + 1]) == half_s;
-        }
-        if (any_tie) {
-#pragma unroll
-            for (int i = 0; i < 8; i++)
-                if (fabsf(df[i]) == half_s && (kb[i] & 1u)) kb[i] += df[i] > 0.0f ? 1u : 0xFFFFFFFFu;
-        }
-        if (subnormal) {
-#pragma unroll
-            for (int i = 0; i < 8; i++) {
-                const float k = fminf(fmaxf(__uint_as_float(kb[i]) - magic, -qmax), qmax);
-                kb[i] = __float_as_uint(k + magic);
-            }
-        }
-        out[2 * c] = __byte_perm(__byte_perm(kb[0], kb[1], 0x0040), __byte_perm(kb[2], kb[3], 0x0040), 0x5410);
-        out[2 * c + 1] = __byte_perm(__byte_perm(kb[4], kb[5], 0x0040), __byte_perm(kb[6], kb[7], 0x0040), 0x5410);
-    }
-    if (!write) return;
-    if (FMT == FMT_INT8) {
-        if (NC == 1) *reinterpret_cast<uint2*>(codes + elem0) = make_uint2(out[0], out[1]);
-        else {
-#pragma unroll
-            for (int c = 0; c < NC / 2; c++)
-                reinterpret_cast<uint4*>(codes + elem0)[c] = make_uint4(out[4 * c], out[4 * c + 1], out[4 * c + 2], out[4 * c + 3]);
-        }
-    } else {
-        uint32_t nib[NC];
-#pragma unroll
-        for (int c = 0; c < NC; c++) {
-            uint32_t a = out[2 * c] & 0x0F0F0F0Fu, b = out[2 * c + 1] & 0x0F0F0F0Fu;
-            a = (a | (a >> 4)) & 0x00FF00FFu; a = (a | (a >> 8)) & 0x0000FFFFu;
-            b = (b | (b >> 4)) & 0x00FF00FFu; b = (b | (b >> 8)) & 0x0000FFFFu;
-            nib[c] = a | (b << 16);
-        }
-        if (NC == 1) *reinterpret_cast<uint32_t*>(codes + (elem0 >> 1)) = nib[0];
-        else if (NC == 2) *reinterpret_cast<uint2*>(codes + (elem0 >> 1)) = make_uint2(nib[0], nib[NC - 1]);
-        else *reinterpret_cast<uint4*>(codes + (elem0 >> 1)) = make_uint4(nib[0], nib[1 % NC], nib[2 % NC], nib[3 % NC]);
-    }
-    if (((threadIdx.x & 31) & (seg - 1)) == 0) *reinterpret_cast<__half*>(scales + 2 * scale_index) = s16;
+__device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
 }
 
 // One CTA per (layer, block).
@@ -323,115 +235,361 @@ quantize_gather_kernel(const GatherParams p) {
     }
 }
 
-// The same block encoder with the block's K and V rows staged in shared memory by bulk asynchronous copies: every
-// row of the block is in flight at once (no registers held for loads), and the encode loop reads 16-byte chunks
-// from shared memory.  One CTA per (layer, block); three CTAs per SM at the 8B-shaped geometry.
+// Quantises a span of NC consecutive 8-channel chunks (8 * NC channels of one head vector, all inside one scale
+// group), so that the scale arithmetic is paid once per 8 * NC elements.  `seg` = lanes that share a scale group.
+// Register c of `w` holds chunk (c + rot) & (NC - 1) of the span (neighbouring threads read their chunks from shared
+// memory in a rotated order so that a quarter-warp's 128-bit loads fall into distinct banks); the codes come back
+// packed in registers in that same order (int8: two words per chunk; int4: one word per chunk), with the fp16 scale.
+template <int FMT, int NC>
+__device__ __forceinline__ void quantise_span(const uint4* w, int seg, uint32_t* out, __half* scale) {
+    uint32_t mx = 0;
+#pragma unroll
+    for (int c = 0; c < NC; c++) {
+        mx = max_bf16x2(mx, w[c].x & 0x7FFF7FFFu); mx = max_bf16x2(mx, w[c].y & 0x7FFF7FFFu);
+        mx = max_bf16x2(mx, w[c].z & 0x7FFF7FFFu); mx = max_bf16x2(mx, w[c].w & 0x7FFF7FFFu);
+    }
+    uint32_t amax_bits = max(mx << 16, mx & 0xFFFF0000u);
+    for (int d = 1; d < seg; d <<= 1) amax_bits = max(amax_bits, __shfl_xor_sync(0xFFFFFFFFu, amax_bits, d));
+    const float amax = __uint_as_float(amax_bits);
+    const float qmax = FMT == FMT_INT8 ? 127.0f : 7.0f;
+    const __half s16 = __float2half_rn(__fdiv_rn(amax, qmax));
+    const float s = __half2float(s16);
+    const float r = s > 0.0f ? __frcp_rn(s) : 0.0f;
+    const float half_s = s > 0.0f ? 0.5f * s : -1.0f;
+    const float magic = 12582912.0f;
+    const bool subnormal = (__half_as_ushort(s16) & 0x7C00u) == 0 && s > 0.0f;
+    const f32x2 r2 = pack2(r, r), m2 = pack2(magic, magic), ns2 = pack2(-s, -s);
+#pragma unroll
+    for (int c = 0; c < NC; c++) {
+        float x[8];
+        x[0] = __uint_as_float(w[c].x << 16); x[1] = __uint_as_float(w[c].x & 0xFFFF0000u);
+        x[2] = __uint_as_float(w[c].y << 16); x[3] = __uint_as_float(w[c].y & 0xFFFF0000u);
+        x[4] = __uint_as_float(w[c].z << 16); x[5] = __uint_as_float(w[c].z & 0xFFFF0000u);
+        x[6] = __uint_as_float(w[c].w << 16); x[7] = __uint_as_float(w[c].w & 0xFFFF0000u);
+        uint32_t kb[8];
+        float df[8];
+        bool any_tie = false;
+#pragma unroll
+        for (int i = 0; i < 8; i += 2) {
+            const f32x2 x2 = pack2(x[i], x[i + 1]);
+            const f32x2 tm = fma2(x2, r2, m2);
+            const f32x2 d2 = fma2(sub2(tm, m2), ns2, x2);
+            float a0, a1;
+            unpack2(tm, a0, a1);
+            kb[i] = __float_as_uint(a0); kb[i + 1] = __float_as_uint(a1);
+            unpack2(d2, df[i], df[i + 1]);
+            any_tie = any_tie || fabsf(df[i]) == half_s || fabsf(df[i + 1]) == half_s;
+        }
+        if (any_tie) {
+#pragma unroll
+            for (int i = 0; i < 8; i++)
+                if (fabsf(df[i]) == half_s && (kb[i] & 1u)) kb[i] += df[i] > 0.0f ? 1u : 0xFFFFFFFFu;
+        }
+        if (subnormal) {
+#pragma unroll
+            for (int i = 0; i < 8; i++) {
+                const float k = fminf(fmaxf(__uint_as_float(kb[i]) - magic, -qmax), qmax);
+                kb[i] = __float_as_uint(k + magic);
+            }
+        }
+        const uint32_t o0 = __byte_perm(__byte_perm(kb[0], kb[1], 0x0040), __byte_perm(kb[2], kb[3], 0x0040), 0x5410);
+        const uint32_t o1 = __byte_perm(__byte_perm(kb[4], kb[5], 0x0040), __byte_perm(kb[6], kb[7], 0x0040), 0x5410);
+        if (FMT == FMT_INT8) {
+            out[2 * c] = o0; out[2 * c + 1] = o1;
+        } else {
+            uint32_t a = o0 & 0x0F0F0F0Fu, b = o1 & 0x0F0F0F0Fu;
+            a = (a | (a >> 4)) & 0x00FF00FFu; a = (a | (a >> 8)) & 0x0000FFFFu;
+            b = (b | (b >> 4)) & 0x00FF00FFu; b = (b | (b >> 8)) & 0x0000FFFFu;
+            out[c] = a | (b << 16);
+        }
+    }
+    *scale = s16;
+}
+
+__device__ __forceinline__ void sts64(uint32_t a, uint32_t x, uint32_t y) {
+    asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(a), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void sts32(uint32_t a, uint32_t x) {
+    asm volatile("st.shared.b32 [%0], %1;" ::"r"(a), "r"(x) : "memory");
+}
+
+// One pass of a consumer warp over 32 consecutive spans of a quantised unit: quantise, put the codes back into the
+// warp's own part of the stage in record order, and copy them out with 16-byte stores that cover the warp's piece of
+// the record contiguously.  `region` = shared address of the warp's 32 spans, `u0` = index of its first span.
+template <int FMT, int NC>
+__device__ __forceinline__ void encode_pass(uint32_t region, int u0, int units, int staged, uint8_t* codes,
+                                            uint8_t* scales, int seg, int seg_shift, int rot, int lane) {
+    constexpr int kSpanOut = FMT == FMT_INT8 ? 8 * NC : 4 * NC;     // bytes of codes per span
+    const int u = u0 + lane;
+    uint4 w[NC];
+#pragma unroll
+    for (int k = 0; k < NC; k++)                            // rows past the end of the suffix encode as zeros
+        w[k] = u < staged ? lds128(region + 16u * (uint32_t)(lane * NC + ((k + rot) & (NC - 1)))) : make_uint4(0, 0, 0, 0);
+    uint32_t out[FMT == FMT_INT8 ? 2 * NC : NC];
+    __half s16;
+    quantise_span<FMT, NC>(w, seg, out, &s16);
+    __syncwarp();                                           // every lane holds its input: the region can be reused
+    if (u < units) {
+#pragma unroll
+        for (int k = 0; k < NC; k++) {
+            const int lc = (k + rot) & (NC - 1);
+            if (FMT == FMT_INT8) sts64(region + (uint32_t)(lane * kSpanOut + 8 * lc), out[2 * k], out[2 * k + 1]);
+            else sts32(region + (uint32_t)(lane * kSpanOut + 4 * lc), out[k]);
+        }
+        if ((lane & (seg - 1)) == 0) *reinterpret_cast<__half*>(scales + 2 * (size_t)(u >> seg_shift)) = s16;
+    }
+    __syncwarp();
+    const int bytes = min(32, units - u0) * kSpanOut;       // a multiple of 16 (checked at launch)
+#pragma unroll
+    for (int o = 0; o < 32 * kSpanOut; o += 512) {
+        const int b = o + 16 * lane;
+        if (b < bytes) *reinterpret_cast<uint4*>(codes + (size_t)u0 * kSpanOut + b) = lds128(region + b);
+    }
+}
+
+// ---------------------------------------------------------------- persistent bulk-copy pipeline
+// The block encoder as a persistent kernel: one producer warp walks this CTA's share of the (layer, block) list,
+// looks up the next block's directory entry and source pages while the current block is being issued, and stages
+// the block's K and V rows (in units of a few tokens) into a shared-memory ring with bulk asynchronous copies that
+// complete on an mbarrier; eight consumer warps quantise from shared memory and write the record.  Loads of several
+// units are in flight per CTA at all times, which one CTA per block (above) cannot do.  Every wait is bounded.
+constexpr int kWPipeConsumers = 256;
+constexpr int kWPipeThreads = kWPipeConsumers + 32;
+constexpr int kWPipeMaxStages = 8;
+constexpr int kWPipeMaxTokens = 128;                       // block_tokens the producer's offset table holds
+constexpr int kWPipeMaxPages = 4;                          // logical pages one block may touch in this kernel
+
+struct WPipeCfg {
+    int32_t unit_tokens, stage_bytes, n_stages, heads_contiguous, total_items;
+    // bytes of a block's / a token's codes and scales per format, and of a record per tag
+    uint32_t blk_codes[3], blk_scales[3], tok_codes[3], tok_scales[3], rec_bytes[4];
+};
+struct WStageMeta {                                         // 32 bytes at the end of each stage
+    unsigned long long codes, scales;                       // where this unit's codes / scales go in the record
+    int32_t fmt, rows_total, rows_valid, pad;               // rows_total < 0: no more work
+};
+
 template <int NC>
-__global__ void __launch_bounds__(kGatherThreads)
-quantize_gather_staged_kernel(const GatherParams p, int sec_bytes, int heads_contiguous) {
-    extern __shared__ __align__(128) uint8_t stage[];       // [K rows][V rows][tok_off]
-    __shared__ uint64_t bar[2];
+__global__ void __launch_bounds__(kWPipeThreads)
+quantize_gather_pipe_kernel(const __grid_constant__ GatherParams p, const __grid_constant__ WPipeCfg cfg) {
+    extern __shared__ __align__(128) uint8_t ring[];
+    __shared__ uint64_t full_bar[kWPipeMaxStages], empty_bar[kWPipeMaxStages];
+    __shared__ long long tok_off[kWPipeMaxTokens];
     __shared__ int abort_flag;
-    long long* tok_off = reinterpret_cast<long long*>(stage + 2 * (size_t)sec_bytes);
-    const int l = p.layer_begin + blockIdx.x / p.nb, j = blockIdx.x % p.nb;
-    const int tag = __ldg(p.tags + (size_t)l * p.nb + j);
-    const unsigned long long off = __ldg(p.blk_off + (size_t)l * p.nb + j);
-    const unsigned long long lbytes = __ldg(p.layer_bytes + l);
-    uint8_t* base = reinterpret_cast<uint8_t*>(
-        static_cast<uintptr_t>(__ldg(reinterpret_cast<const unsigned long long*>(p.layer_payload) + l)));
-    const unsigned long long elems = (unsigned long long)p.B * p.H * p.D;
-    const unsigned long long rec = record_bytes(tag, elems, p.G);
-    bool bad = rec == 0 || off > lbytes || rec > lbytes - off || base == nullptr ||
-               ((reinterpret_cast<uintptr_t>(base) + off) & 15u) != 0;
-    const int valid = min(p.B, p.n - j * p.B);
+    const int S = cfg.n_stages;
     if (threadIdx.x == 0) {
-        mbar_init(&bar[0], 1); mbar_init(&bar[1], 1);
+        for (int s = 0; s < S; s++) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], kWPipeConsumers / 32); }
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    for (int t = threadIdx.x; t < p.B; t += kGatherThreads) {
-        long long o = -1;
-        if (t < valid) {
-            const long long u = (long long)j * p.B + t + p.src_shift;
-            const long long lp = u / p.P;
-            const int page = lp < p.n_table ? __ldg(p.block_table + lp) : -1;
-            if (page < 0 || page >= p.n_pages) bad = true;
-            o = (long long)l * p.stride_layer + (long long)page * p.stride_page + (u - lp * p.P) * p.stride_token;
-        }
-        tok_off[t] = o;
-    }
-    if (__syncthreads_or(bad)) {                            // skip the block whole, latch the error
-        if (threadIdx.x == 0) atomicCAS(p.status, 0, (int)PATCHKV_E_BOUNDS);
-        return;
-    }
-    // ---- stage: valid rows by bulk copies (one per token, or one per (token, head) when heads are strided),
-    //      rows past the end of the suffix as zeros
-    const int row_bytes = p.H * p.D * 2, vec_bytes = p.D * 2;
-    if (threadIdx.x == 0) {
-        mbar_arrive_expect_tx(&bar[0], (uint32_t)valid * row_bytes);
-        mbar_arrive_expect_tx(&bar[1], (uint32_t)valid * row_bytes);
-    }
-    const int copies = heads_contiguous ? valid : valid * p.H;
-    for (int i = threadIdx.x; i < 2 * copies; i += kGatherThreads) {
-        const int sec = i >= copies, c = sec ? i - copies : i;
-        const uint16_t* pool = sec ? p.v_base : p.k_base;
-        uint8_t* dst = stage + (size_t)sec * sec_bytes;
-        if (heads_contiguous) bulk_g2s(dst + (size_t)c * row_bytes, pool + tok_off[c], row_bytes, &bar[sec]);
-        else {
-            const int t = c / p.H, h = c - t * p.H;
-            bulk_g2s(dst + (size_t)c * vec_bytes, pool + tok_off[t] + (long long)h * p.stride_head, vec_bytes, &bar[sec]);
-        }
-    }
-    for (int i = valid * row_bytes / 16 + threadIdx.x; i < sec_bytes / 16; i += kGatherThreads) {
-        reinterpret_cast<uint4*>(stage)[i] = make_uint4(0, 0, 0, 0);
-        reinterpret_cast<uint4*>(stage + sec_bytes)[i] = make_uint4(0, 0, 0, 0);
-    }
     __syncthreads();
-
-    const int kf = k_format(tag), vf = v_format(tag);
-    uint8_t* kc = base + off;
-    uint8_t* ks = kc + code_bytes(kf, elems);
-    uint8_t* vc = ks + scale_bytes(kf, elems, p.G);
-    uint8_t* vs = vc + code_bytes(vf, elems);
-    const int spv = p.D / (8 * NC);                         // spans of 8 * NC channels per head vector
-    const int seg = p.G / (8 * NC);                         // lanes per scale group (>= 1: a span never crosses a group)
-    const int gpv = p.D / p.G;
-    const int seg_shift = 31 - __clz(seg);
-    const bool spv_pow2 = (spv & (spv - 1)) == 0;
-    const int spv_shift = 31 - __clz(spv);
-    const int units = p.B * p.H * spv;                      // spans of one section, in record order
-    const int padded = (units + kGatherThreads - 1) / kGatherThreads * kGatherThreads;
     volatile int* abortp = &abort_flag;
-#pragma unroll 1
-    for (int sec = 0; sec < 2; sec++) {
-        // bounded wait for this section's rows; the verdict is CTA-uniform through the shared flag
-        const bool ok = mbar_wait(&bar[sec], 0, abortp);
-        if (__syncthreads_or(!ok)) {
-            if (threadIdx.x == 0) atomicCAS(p.status, 0, (int)PATCHKV_E_TIMEOUT);
-            // let the other section's copies land (bounded) before the CTA's shared memory is released
-            for (uint32_t i = 0; i < kWaitLimit && !mbar_try_wait(&bar[1], 0); i++) __nanosleep(100);
-            return;
-        }
-        const int fmt = sec ? vf : kf;
-        uint8_t* codes = sec ? vc : kc;
-        uint8_t* scales = sec ? vs : ks;
-        const uint32_t src = smem_u32(stage + (size_t)sec * sec_bytes);
-#pragma unroll 1
-        for (int u = threadIdx.x; u < padded; u += kGatherThreads) {
-            const bool in = u < units;
-            uint4 w[NC];
+    const int off_meta = cfg.stage_bytes - 32;
+    const int row_bytes = p.H * p.D * 2, vec_bytes = p.D * 2;
+
+    if (threadIdx.x < 32) {
+        // ================================================================ producer warp
+        const int lane = threadIdx.x;
+        const uint32_t hd = (uint32_t)p.H * p.D;
+        uint32_t q = 0;
+        int stage = 0;
+        uint32_t phase = 0;
+        bool alive = true;
+        // Directory entries and source pages are looked up and validated thirty-two blocks at a time, one block per
+        // lane, a whole round before they are used: the loads of the next round are issued when the current round
+        // starts, so their latency never sits in front of a copy, and the per-block work left on the serial path is
+        // a handful of shuffles.  Section sizes per format come precomputed (no divisions here).
+        struct Pre {
+            unsigned long long rec;                         // address of the block's record, 0: skip the block
+            long long layer_off;                            // l * stride_layer
+            int tag, valid, slot0;                          // slot0: first source slot counted from the first page
+            int pages[kWPipeMaxPages];
+        };
+        auto lookup = [&](long long first, Pre& r) {
+            const long long item = first + (long long)lane * gridDim.x;
+            r.rec = 0; r.layer_off = 0; r.tag = 0; r.valid = 0; r.slot0 = 0;
 #pragma unroll
-            for (int c = 0; c < NC; c++) w[c] = in ? lds128(src + 16u * (uint32_t)(u * NC + c)) : make_uint4(0, 0, 0, 0);
-            const int vec = spv_pow2 ? (u >> spv_shift) : u / spv;
-            const int sx = u - vec * spv;
-            const size_t elem0 = (size_t)u * 8 * NC;
-            const size_t sidx = (size_t)vec * gpv + (sx >> seg_shift);
-            switch (fmt) {
-                case FMT_BF16: encode_span<FMT_BF16, NC>(w, codes, scales, elem0, sidx, seg, in); break;
-                case FMT_INT8: encode_span<FMT_INT8, NC>(w, codes, scales, elem0, sidx, seg, in); break;
-                default:       encode_span<FMT_INT4, NC>(w, codes, scales, elem0, sidx, seg, in); break;
+            for (int k = 0; k < kWPipeMaxPages; k++) r.pages[k] = 0;
+            if (item < cfg.total_items) {
+                const int it = (int)item;
+                const int l = p.layer_begin + it / p.nb, j = it - (it / p.nb) * p.nb;
+                const int tag = __ldg(p.tags + (size_t)l * p.nb + j);
+                const unsigned long long off = __ldg(p.blk_off + (size_t)l * p.nb + j);
+                const unsigned long long lbytes = __ldg(p.layer_bytes + l);
+                const unsigned long long base = __ldg(reinterpret_cast<const unsigned long long*>(p.layer_payload) + l);
+                const int u0 = j * p.B + p.src_shift;       // token indices fit 32 bits (checked at launch)
+                const int lp0 = u0 / p.P;
+                const int valid = min(p.B, p.n - j * p.B);
+                const int last = (u0 + valid - 1) / p.P - lp0;
+                bool bad = tag < 0 || tag > PATCHKV_TAG_K4V4;
+                const unsigned long long rec = bad ? 0 : (unsigned long long)cfg.rec_bytes[tag];
+                bad = bad || off > lbytes || rec > lbytes - off || base == 0 || ((base + off) & 15u) != 0;
+#pragma unroll
+                for (int k = 0; k < kWPipeMaxPages; k++) {
+                    if (k <= last) {
+                        const int page = lp0 + k < p.n_table ? __ldg(p.block_table + lp0 + k) : -1;
+                        if (page < 0 || page >= p.n_pages) bad = true;
+                        r.pages[k] = page;
+                    }
+                }
+                r.rec = bad ? 1 : base + off;               // 1: latch the error when the block's turn comes
+                r.layer_off = (long long)l * p.stride_layer;
+                r.tag = tag; r.valid = valid; r.slot0 = u0 - lp0 * p.P;
             }
+        };
+        Pre cur, nxt;
+        lookup(blockIdx.x, cur);
+        nxt = cur;
+#pragma unroll 1
+        for (long long first = blockIdx.x; first < cfg.total_items && alive; first += 32ll * gridDim.x) {
+            if (first + 32ll * gridDim.x < cfg.total_items) lookup(first + 32ll * gridDim.x, nxt);
+#pragma unroll 1
+            for (int ri = 0; ri < 32 && alive; ri++) {
+            if (first + (long long)ri * gridDim.x >= cfg.total_items) break;
+            const unsigned long long rec = __shfl_sync(0xFFFFFFFFu, cur.rec, ri);
+            if (rec == 1) {                                 // skip the block whole, latch the error
+                if (lane == 0) atomicCAS(p.status, 0, (int)PATCHKV_E_BOUNDS);
+                continue;
+            }
+            const long long layer_off = __shfl_sync(0xFFFFFFFFu, cur.layer_off, ri);
+            const int tag = __shfl_sync(0xFFFFFFFFu, cur.tag, ri);
+            const int valid = __shfl_sync(0xFFFFFFFFu, cur.valid, ri);
+            const int slot0 = __shfl_sync(0xFFFFFFFFu, cur.slot0, ri);
+            int pages[kWPipeMaxPages];
+#pragma unroll
+            for (int k = 0; k < kWPipeMaxPages; k++) pages[k] = __shfl_sync(0xFFFFFFFFu, cur.pages[k], ri);
+            for (int t = lane; t < p.B; t += 32) {
+                long long o = -1;
+                if (t < valid) {
+                    int us = slot0 + t, page = pages[0];
+#pragma unroll
+                    for (int k = 1; k < kWPipeMaxPages; k++) if (us >= p.P) { us -= p.P; page = pages[k]; }
+                    o = layer_off + (long long)page * p.stride_page + (long long)us * p.stride_token;
+                }
+                tok_off[t] = o;
+            }
+            __syncwarp();
+            const int kf = k_format(tag), vf = v_format(tag);
+            uint8_t* sec_codes[2];
+            uint8_t* sec_scales[2];
+            sec_codes[0] = reinterpret_cast<uint8_t*>(static_cast<uintptr_t>(rec));
+            sec_scales[0] = sec_codes[0] + cfg.blk_codes[kf];
+            sec_codes[1] = sec_scales[0] + cfg.blk_scales[kf];
+            sec_scales[1] = sec_codes[1] + cfg.blk_codes[vf];
+#pragma unroll 1
+            for (int sec = 0; sec < 2 && alive; sec++) {
+                const int fmt = sec ? vf : kf;
+                const uint16_t* pool = sec ? p.v_base : p.k_base;
+                const uint32_t ctok = cfg.tok_codes[fmt], stok = cfg.tok_scales[fmt];
+#pragma unroll 1
+                for (int t0 = 0; t0 < p.B; t0 += cfg.unit_tokens) {
+                    const int rows_total = min(cfg.unit_tokens, p.B - t0);
+                    const int rows_valid = max(0, min(rows_total, valid - t0));
+                    if (!__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], phase ^ 1, abortp))) { alive = false; break; }
+                    uint8_t* sp = ring + (size_t)stage * cfg.stage_bytes;
+                    if (lane == 0) {
+                        WStageMeta m;
+                        m.codes = reinterpret_cast<unsigned long long>(sec_codes[sec] + (size_t)t0 * ctok);
+                        m.scales = reinterpret_cast<unsigned long long>(sec_scales[sec] + (size_t)t0 * stok);
+                        m.fmt = fmt; m.rows_total = rows_total; m.rows_valid = rows_valid; m.pad = 0;
+                        *reinterpret_cast<WStageMeta*>(sp + off_meta) = m;
+                        if (rows_valid) mbar_arrive_expect_tx(&full_bar[stage], (uint32_t)rows_valid * row_bytes);
+                        else mbar_arrive(&full_bar[stage]);
+                    }
+                    __syncwarp();
+                    if (cfg.heads_contiguous) {
+                        // rows that follow one another in the pool (consecutive slots of one page) travel as one copy:
+                        // a lane whose row does not continue its predecessor's starts a run and copies all of it
+                        for (int ib = 0; ib < rows_valid; ib += 32) {
+                            const int i = ib + lane;
+                            const bool have = i < rows_valid;
+                            const long long o = have ? tok_off[t0 + i] : 0;
+                            const bool head = have && (lane == 0 || o != tok_off[t0 + i - 1] + (long long)hd);
+                            const uint32_t heads = __ballot_sync(0xFFFFFFFFu, head);
+                            if (head) {
+                                const uint32_t later = lane == 31 ? 0u : heads >> (lane + 1);
+                                const int end = later ? lane + __ffs(later) : min(32, rows_valid - ib);
+                                bulk_g2s(sp + (size_t)i * row_bytes, pool + o, (uint32_t)(end - lane) * row_bytes, &full_bar[stage]);
+                            }
+                        }
+                    } else {
+                        for (int i = lane; i < rows_valid * p.H; i += 32) {
+                            const int t = i / p.H, h = i - t * p.H;
+                            bulk_g2s(sp + (size_t)i * vec_bytes, pool + tok_off[t0 + t] + (long long)h * p.stride_head,
+                                     vec_bytes, &full_bar[stage]);
+                        }
+                    }
+                    q++;
+                    if (++stage == S) { stage = 0; phase ^= 1; }
+                }
+            }
+            __syncwarp();                                   // tok_off is rewritten by the next block
+            }
+            cur = nxt;
         }
+        if (alive) {                                        // tell the consumers that the list is exhausted
+            if (__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], phase ^ 1, abortp))) {
+                if (lane == 0) {
+                    WStageMeta m;
+                    m.codes = 0; m.scales = 0; m.fmt = 0; m.rows_total = -1; m.rows_valid = 0; m.pad = 0;
+                    *reinterpret_cast<WStageMeta*>(ring + (size_t)stage * cfg.stage_bytes + off_meta) = m;
+                    mbar_arrive(&full_bar[stage]);
+                }
+            } else alive = false;
+        }
+        if (!alive) {
+            // a wait gave up: let the copies already issued land (bounded), so that no bulk copy is still writing
+            // this CTA's shared memory after it exits
+            const uint32_t issued = q < (uint32_t)S ? q : (uint32_t)S;
+            for (uint32_t k = 0; k < issued; k++) {
+                const uint32_t qq = q - 1 - k;
+                for (uint32_t i = 0; i < kWaitLimit; i++) {
+                    if (mbar_try_wait(&full_bar[qq % S], (qq / S) & 1)) break;
+                    __nanosleep(100);
+                }
+            }
+            if (lane == 0) atomicCAS(p.status, 0, (int)PATCHKV_E_TIMEOUT);
+        }
+    } else {
+        // ================================================================ consumer warps
+        const int c = threadIdx.x - 32;
+        const int spv = p.D / (8 * NC);                     // spans of 8 * NC channels per head vector
+        const int seg = p.G / (8 * NC);                     // lanes per scale group (>= 1: a span never crosses a group)
+        const int seg_shift = 31 - __clz(seg);
+        const int rot = NC > 1 ? (c / (8 / NC)) & (NC - 1) : 0;
+        int stage = 0;
+        uint32_t phase = 0;
+        while (true) {
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait(&full_bar[stage], phase, abortp))) break;
+            uint8_t* sp = ring + (size_t)stage * cfg.stage_bytes;
+            const uint32_t src = smem_u32(sp);
+            const uint4 m0 = lds128(src + off_meta), m1 = lds128(src + off_meta + 16);
+            const int rows_total = (int)m1.y;
+            if (rows_total < 0) break;
+            uint8_t* codes = reinterpret_cast<uint8_t*>(static_cast<uintptr_t>(((unsigned long long)m0.y << 32) | m0.x));
+            uint8_t* scales = reinterpret_cast<uint8_t*>(static_cast<uintptr_t>(((unsigned long long)m0.w << 32) | m0.z));
+            const int fmt = (int)m1.x;
+            const int units = rows_total * p.H * spv, staged = (int)m1.z * p.H * spv;
+            const int lane = c & 31;
+            if (fmt == FMT_BF16) {
+                // a copy: 16 bytes per lane, lanes side by side
+                const int n16 = units * NC, have16 = staged * NC;
+#pragma unroll 4
+                for (int i = c; i < n16; i += kWPipeConsumers)
+                    reinterpret_cast<uint4*>(codes)[i] = i < have16 ? lds128(src + 16u * (uint32_t)i) : make_uint4(0, 0, 0, 0);
+            } else {
+#pragma unroll 1
+                for (int u0 = c - lane; u0 < units; u0 += kWPipeConsumers) {
+                    const uint32_t region = src + 16u * NC * (uint32_t)u0;
+                    if (fmt == FMT_INT8) encode_pass<FMT_INT8, NC>(region, u0, units, staged, codes, scales, seg, seg_shift, rot, lane);
+                    else                 encode_pass<FMT_INT4, NC>(region, u0, units, staged, codes, scales, seg, seg_shift, rot, lane);
+                }
+            }
+            __syncwarp();
+            if ((c & 31) == 0) mbar_arrive(&empty_bar[stage]);
+            if (++stage == S) { stage = 0; phase ^= 1; }
+        }
+        if (c == 0 && *abortp) atomicCAS(p.status, 0, (int)PATCHKV_E_TIMEOUT);
     }
 }
 
@@ -498,25 +656,48 @@ static int fill_gather(patchkv_ctx* ctx, const patchkv_geom* g, const patchkv_po
 // Launches the block encoder for `layers` layers starting at p.layer_begin.
 static int launch_gather(patchkv_ctx* ctx, const patchkv_geom* g, const patchkv_pool* pool, const GatherParams& p,
                          int layers, cudaStream_t stream) {
-    // staged variant: both sections of a block in shared memory, at least two CTAs per SM
-    const long long sec_bytes = (long long)g->block_tokens * g->n_kv_heads * g->head_dim * 2;
-    const long long smem = 2 * sec_bytes + (long long)g->block_tokens * 8 + 16;
-    if (!(ctx->flags & PATCHKV_FLAG_DIRECT_LOADS) && smem <= 100 * 1024 && sec_bytes % 16 == 0) {
+    // persistent pipeline, two CTAs per SM: stages of about 32 KiB of rows and about 64 KiB of reads in flight per
+    // CTA (measured: a deeper ring is slower, the reads then crowd out the writes)
+    {
+        const long long row_bytes = (long long)g->n_kv_heads * g->head_dim * 2;
         const int hc = pool->stride_head == g->head_dim ? 1 : 0;
-        // channels per thread: the whole scale group up to 32 channels
-        if (g->group >= 32) {
-            PKV_CUDA(ctx, cudaFuncSetAttribute(quantize_gather_staged_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            quantize_gather_staged_kernel<4><<<p.nb * layers, kGatherThreads, smem, stream>>>(p, (int)sec_bytes, hc);
-        } else if (g->group == 16) {
-            PKV_CUDA(ctx, cudaFuncSetAttribute(quantize_gather_staged_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            quantize_gather_staged_kernel<2><<<p.nb * layers, kGatherThreads, smem, stream>>>(p, (int)sec_bytes, hc);
-        } else {
-            PKV_CUDA(ctx, cudaFuncSetAttribute(quantize_gather_staged_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            quantize_gather_staged_kernel<1><<<p.nb * layers, kGatherThreads, smem, stream>>>(p, (int)sec_bytes, hc);
+        const long long pages_per_block = (g->block_tokens + g->page_tokens - 1) / g->page_tokens + 1;
+        int ut = (int)std::min<long long>(g->block_tokens, std::max<long long>(1, 32768 / row_bytes));
+        ut = std::min(ut, 32);
+        const long long stage_bytes = ((long long)ut * row_bytes + 32 + 127) & ~127ll;
+        const int budget = std::min(ctx->max_smem_optin, 227 * 1024) / 2 - 2048;
+        const int n_stages = (int)std::min<long long>(std::min<long long>(kWPipeMaxStages, budget / stage_bytes),
+                                                      std::max<long long>(2, (65536 + stage_bytes / 2) / stage_bytes));
+        if (!(ctx->flags & PATCHKV_FLAG_DIRECT_LOADS) && row_bytes % 16 == 0 && g->block_tokens <= kWPipeMaxTokens &&
+            pages_per_block <= kWPipeMaxPages && n_stages >= 2 && g->group >= 8 && (g->n_kv_heads * g->head_dim) % 32 == 0 &&
+            (long long)p.nb * g->block_tokens + g->page_tokens < 0x7fffffffLL) {
+            WPipeCfg cfg;
+            cfg.unit_tokens = ut; cfg.stage_bytes = (int)stage_bytes; cfg.n_stages = n_stages; cfg.heads_contiguous = hc;
+            cfg.total_items = p.nb * layers;
+            const uint64_t elems = (uint64_t)g->block_tokens * g->n_kv_heads * g->head_dim, hd = (uint64_t)g->n_kv_heads * g->head_dim;
+            for (int f = 0; f < 3; f++) {
+                cfg.blk_codes[f] = (uint32_t)code_bytes(f, elems); cfg.blk_scales[f] = (uint32_t)scale_bytes(f, elems, g->group);
+                cfg.tok_codes[f] = (uint32_t)code_bytes(f, hd); cfg.tok_scales[f] = (uint32_t)scale_bytes(f, hd, g->group);
+            }
+            for (int t = 0; t < 4; t++) cfg.rec_bytes[t] = (uint32_t)record_bytes(t, elems, g->group);
+            const int smem = (int)(stage_bytes * n_stages);
+            const int grid = std::min(cfg.total_items, 2 * ctx->sm_count);
+            if (g->group >= 32) {
+                PKV_CUDA(ctx, cudaFuncSetAttribute(quantize_gather_pipe_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+                quantize_gather_pipe_kernel<4><<<grid, kWPipeThreads, smem, stream>>>(p, cfg);
+            } else if (g->group == 16) {
+                PKV_CUDA(ctx, cudaFuncSetAttribute(quantize_gather_pipe_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+                quantize_gather_pipe_kernel<2><<<grid, kWPipeThreads, smem, stream>>>(p, cfg);
+            } else {
+                PKV_CUDA(ctx, cudaFuncSetAttribute(quantize_gather_pipe_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+                quantize_gather_pipe_kernel<1><<<grid, kWPipeThreads, smem, stream>>>(p, cfg);
+            }
+            PKV_CUDA(ctx, cudaGetLastError());
+            return PATCHKV_OK;
         }
-    } else {
-        quantize_gather_kernel<<<p.nb * layers, kGatherThreads, g->block_tokens * sizeof(long long), stream>>>(p);
     }
+    // direct loads: one CTA per (layer, block)
+    quantize_gather_kernel<<<p.nb * layers, kGatherThreads, g->block_tokens * sizeof(long long), stream>>>(p);
     PKV_CUDA(ctx, cudaGetLastError());
     return PATCHKV_OK;
 }

@@ -13,22 +13,23 @@ from test_oracle_writer import _ck, pool_from_raw, run_writer, scale_raw
 pytestmark = pytest.mark.gpu
 
 
-@pytest.fixture(scope="module", params=[0, 1], ids=["staged", "direct_loads"])
+@pytest.fixture(scope="module", params=[0, 1], ids=["pipeline", "direct_loads"])
 def ctx(request):
-    """Both writer kernels run every case: rows staged in shared memory by bulk copies, and plain loads."""
+    """Both writer kernels run every case: the bulk-copy pipeline, and one CTA per block with plain loads."""
     c = new_context(flags=request.param)
     yield c
     c.close()
 
 
-def gpu_writer(ctx, ck, kp, vp, shift=0, fill=0xEE, table=None, blk_off=None):
-    """Run plan + quantize_gather on the GPU for the pools kp, vp (uint16 numpy).  Returns (off, lb, payload bytes per layer)."""
+def gpu_writer(ctx, ck, kp, vp, shift=0, fill=0xEE, table=None, blk_off=None, geom=None, strides=None):
+    """Run plan + quantize_gather on the GPU for the pools kp, vp (uint16 numpy).  Returns (off, lb, payload bytes per layer).
+    `geom` / `strides` override the checkpoint's geometry and the pool's element strides (a strided view of the pool)."""
     from paper_2609_26219_b200 import binding as pk
-    g = ck.geom
+    g = ck.geom if geom is None else geom
     L, NB = g.n_layers, ck.n_blocks
     k = torch.from_numpy(kp.view(np.int16)).to(DEV)
     v = torch.from_numpy(vp.view(np.int16)).to(DEV)
-    pool = pk.make_pool(k, v, ck.n_pages, pin.pool_strides(g, ck.n_pages))
+    pool = pk.make_pool(k, v, ck.n_pages, pin.pool_strides(g, ck.n_pages) if strides is None else strides)
     geom = pk.make_geom(g.n_layers, g.n_kv_heads, g.head_dim, g.rotary_dim, g.rope_style, g.rope_base, g.block_tokens,
                         g.page_tokens, g.group)
     tags = ck.tags.to(DEV).contiguous()
@@ -57,7 +58,10 @@ def gpu_writer(ctx, ck, kp, vp, shift=0, fill=0xEE, table=None, blk_off=None):
 @pytest.mark.parametrize("kw", [dict(), dict(n=150), dict(n=150, dst_shift=5),
                                 dict(geom=pin.Geometry(1, 4, 128, 128, pin.ROPE_HALF, 5e5, 16, 16, 128)),
                                 dict(geom=pin.Geometry(2, 2, 64, 64, pin.ROPE_HALF, 1e4, 32, 16, 8), n=200, n_pages=40),
-                                dict(geom=pin.Geometry(2, 3, 64, 64, pin.ROPE_HALF, 1e4, 16, 8, 64), n=100, n_pages=40)])
+                                dict(geom=pin.Geometry(2, 3, 64, 64, pin.ROPE_HALF, 1e4, 16, 8, 64), n=100, n_pages=40),
+                                dict(geom=pin.Geometry(2, 4, 64, 64, pin.ROPE_HALF, 1e4, 16, 16, 16), n=150, dst_shift=3),
+                                dict(geom=pin.Geometry(2, 2, 128, 128, pin.ROPE_HALF, 1e4, 48, 16, 32), n=500, n_pages=40),
+                                dict(geom=pin.Geometry(1, 1, 16, 16, pin.ROPE_HALF, 1e4, 16, 16, 8), n=40, n_pages=8)])
 def test_writer_bytes_match_the_oracle(ctx, kw):
     ck = _ck(**kw)
     shift = ck.dst_shift
@@ -65,6 +69,29 @@ def test_writer_bytes_match_the_oracle(ctx, kw):
     rc, rc2, off_o, lb_o, bufs_o = run_writer(ck, kp, vp, shift=shift)
     assert rc == oracle.OK and rc2 == oracle.OK
     off, sizes, bufs = gpu_writer(ctx, ck, kp, vp, shift=shift)
+    assert ctx.query_status() == 0
+    assert np.array_equal(off, off_o) and sizes == [int(x) for x in lb_o]
+    for a, b in zip(bufs, bufs_o):
+        assert np.array_equal(a, b)
+
+
+@pytest.mark.parametrize("G", [16, 32])
+def test_writer_reads_a_strided_view_of_the_pool(ctx, G):
+    """Heads that are not contiguous in the pool: encode the first half of every head vector of a D = 64 pool
+    (geometry D = 32, head stride 64), so that every row is gathered head by head."""
+    full = pin.Geometry(2, 4, 64, 64, pin.ROPE_HALF, 1e4, 16, 16, 32)
+    ck = _ck(geom=full, n=150, dst_shift=5)
+    kp, vp = pool_from_raw(ck, shift=5)
+    half = pin.Geometry(2, 4, 32, 32, pin.ROPE_HALF, 1e4, 16, 16, G)
+    strides = pin.pool_strides(full, ck.n_pages)
+    tags = ck.tags.numpy()
+    rc, off_o, lb_o = oracle.plan_checkpoint(tags, 16, 4, 32, G)
+    bufs_o = [np.full(int(x), 0xEE, dtype=np.uint8) for x in lb_o]
+    rc2 = oracle.quantize_gather(L=2, H=4, D=32, B=16, P=16, G=G, k_pool=kp, v_pool=vp, strides=strides,
+                                 n_pages=ck.n_pages, n=150, src_shift=5, block_table=ck.block_table.numpy(),
+                                 tags=tags, blk_off=off_o, layer_payload=bufs_o)
+    assert rc == oracle.OK and rc2 == oracle.OK
+    off, sizes, bufs = gpu_writer(ctx, ck, kp, vp, shift=5, geom=half, strides=strides)
     assert ctx.query_status() == 0
     assert np.array_equal(off, off_o) and sizes == [int(x) for x in lb_o]
     for a, b in zip(bufs, bufs_o):

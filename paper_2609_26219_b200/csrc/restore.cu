@@ -479,8 +479,6 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
         // waits for a free stage, writes the per-token destination offsets and the unit header, and starts the two
         // bulk copies.
         const int lane = threadIdx.x;
-        const uint64_t elems = (uint64_t)p.B * p.H * p.D;
-        const uint32_t hd = (uint32_t)p.H * p.D;
         uint32_t q = 0;                                  // units issued
         int stage = 0;                                   // q % S, and the parity of q / S, kept without divisions
         uint32_t phase = 0;
@@ -501,14 +499,14 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
                 const uint8_t* sec_codes[2];
                 const uint8_t* sec_scales[2];
                 sec_codes[0] = d.rec;
-                sec_scales[0] = sec_codes[0] + code_bytes(kf, elems);
-                sec_codes[1] = sec_scales[0] + scale_bytes(kf, elems, p.G);
-                sec_scales[1] = sec_codes[1] + code_bytes(vf, elems);
+                sec_scales[0] = sec_codes[0] + p.blk_codes[kf];
+                sec_codes[1] = sec_scales[0] + p.blk_scales[kf];
+                sec_scales[1] = sec_codes[1] + p.blk_codes[vf];
                 const bool shifted = p.s[si].delta != 0;
 #pragma unroll 1
                 for (int sec = 0; sec < 2 && alive; sec++) {
                     const int fmt = sec ? vf : kf;
-                    const uint32_t ctok = (uint32_t)code_bytes(fmt, hd), stok = (uint32_t)scale_bytes(fmt, hd, p.G);
+                    const uint32_t ctok = p.tok_codes[fmt], stok = p.tok_scales[fmt];
 #pragma unroll 1
                     for (int t0 = 0; t0 < valid; t0 += p.unit_tokens) {
                         const int nt = min(p.unit_tokens, valid - t0);
@@ -675,6 +673,11 @@ static bool plan_pipeline(const patchkv_ctx* ctx, RestoreParams* p) {
     if (stages > kMaxStages) stages = kMaxStages;
     if (stages < 2) return false;
     p->n_stages = (int32_t)stages;
+    const uint64_t elems = (uint64_t)p->B * hd;
+    for (int f = 0; f < 3; f++) {                     // section sizes per format: no divisions in the issuing warp
+        p->blk_codes[f] = (uint32_t)code_bytes(f, elems); p->blk_scales[f] = (uint32_t)scale_bytes(f, elems, p->G);
+        p->tok_codes[f] = (uint32_t)code_bytes(f, hd); p->tok_scales[f] = (uint32_t)scale_bytes(f, hd, p->G);
+    }
     return true;
 }
 

@@ -585,6 +585,8 @@ quantize_gather_pipe_kernel(const __grid_constant__ GatherParams p, const __grid
                     else                 encode_pass<FMT_INT4, NC>(region, u0, units, staged, codes, scales, seg, seg_shift, rot, lane);
                 }
             }
+            // the stage was rewritten with ordinary stores above; order them before the bulk copy that refills it
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if ((c & 31) == 0) mbar_arrive(&empty_bar[stage]);
             if (++stage == S) { stage = 0; phase ^= 1; }

@@ -181,6 +181,46 @@ token_mass_octet_kernel(const MassParams p) {
     bool bad = false;
     const uint16_t* base = p.attn + (long long)l * p.stride_layer + col;
     int h = r0 / p.Q, q = r0 - h * p.Q;
+    if (p.Q % kMassBatch == 0 && r0 % kMassBatch == 0 && (r1 - r0) % kMassBatch == 0) {
+        // Regular shape (the usual one): a batch of eight rows never straddles a head, so the row pointers are
+        // base + i * stride_query with no wrap test per load, and the fp32 sums are flushed by position in the row
+        // loop (every 64 rows) instead of by a counter.
+        for (int rc = r0; rc < r1; rc += 64) {
+            const int re = min(r1, rc + 64);
+            for (int r = rc; r < re; r += kMassBatch) {
+                const uint16_t* row = base + (long long)h * p.stride_head + (long long)q * p.stride_query;
+                q += kMassBatch;
+                if (q == p.Q) { q = 0; h++; }
+                uint4 w[kMassBatch];
+#pragma unroll
+                for (int i = 0; i < kMassBatch; i++) w[i] = __ldcs(reinterpret_cast<const uint4*>(row + (long long)i * p.stride_query));
+#pragma unroll
+                for (int i = 0; i < kMassBatch; i++) {
+                    const uint32_t ww[4] = {w[i].x, w[i].y, w[i].z, w[i].w};
+                    const uint32_t m = ww[0] | ww[1] | ww[2] | ww[3];
+                    if ((m & 0xE000E000u) == 0) {           // every entry below 2^-7: exact in fp32 for 64 rows
+#pragma unroll
+                        for (int k = 0; k < 4; k++) {
+                            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&ww[k]));
+                            facc[2 * k] += f.x; facc[2 * k + 1] += f.y;
+                        }
+                    } else if ((m & 0xC000C000u) == 0) {    // every entry in [0, 2): value * 2^24 is exact in fp32
+#pragma unroll
+                        for (int k = 0; k < 4; k++) {
+                            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&ww[k]));
+                            acc[2 * k] += __float2uint_rz(f.x * 16777216.0f);
+                            acc[2 * k + 1] += __float2uint_rz(f.y * 16777216.0f);
+                        }
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < 4; k++) { acc[2 * k] += units_any(ww[k], &bad); acc[2 * k + 1] += units_any(ww[k] >> 16, &bad); }
+                    }
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < 8; k++) { acc[k] += __float2uint_rz(facc[k] * 16777216.0f); facc[k] = 0.0f; }
+        }
+    } else
     for (int r = r0; r < r1; r += kMassBatch) {
         uint4 w[kMassBatch];
 #pragma unroll
@@ -620,13 +660,26 @@ extern "C" int patchkv_select_repair_tokens(patchkv_ctx* ctx, const patchkv_sele
                                ((a->attn_stride_layer | a->attn_stride_head | a->attn_stride_query) & 7) == 0;
             const int cols = octet ? (n + 7) / 8 : n;
             const int tiles = (cols + 255) / 256;
-            // few row groups: every thread ends with one 64-bit atomic per token
-            long long groups = (long long)ctx->sm_count * 16 / ((long long)tiles * L);
-            if (groups < 1) groups = 1;
-            long long rpc = (rows + groups - 1) / groups;
-            if (rpc < 64) rpc = 64;
-            if (rpc > rows) rpc = rows;
-            groups = (rows + rpc - 1) / rpc;
+            // few row groups (every thread ends with one 64-bit atomic per token), a whole number of batches each,
+            // and a grid that fills its last wave: among the candidates the one with the best wave efficiency
+            int occ = 0;
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, token_mass_octet_kernel, 256, 0) != cudaSuccess || occ < 1) {
+                cudaGetLastError();
+                occ = 2;
+            }
+            const long long slots = (long long)ctx->sm_count * occ, per_group = (long long)tiles * L;
+            long long rpc = rows;
+            double best = -1.0;
+            for (long long g = std::max<long long>(1, 4 * slots / per_group); g <= std::max<long long>(1, 9 * slots / per_group); g++) {
+                long long c = (rows + g - 1) / g;
+                c = (c + kMassBatch - 1) / kMassBatch * kMassBatch;
+                if (c < 64) c = 64;
+                if (c > rows) c = rows;
+                const long long ctas = ((rows + c - 1) / c) * per_group;
+                const double eff = (double)ctas / (double)(((ctas + slots - 1) / slots) * slots);
+                if (eff > best + 1e-9) { best = eff; rpc = c; }
+            }
+            long long groups = (rows + rpc - 1) / rpc;
             if (groups > 65535) return fail(ctx, PATCHKV_E_UNSUPPORTED, "select: grid too large");
             mp.rows_per_cta = (int)rpc;
             if (octet) token_mass_octet_kernel<<<dim3(tiles, (unsigned)groups, L), 256, 0, stream>>>(mp);

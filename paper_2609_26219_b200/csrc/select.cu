@@ -105,7 +105,19 @@ block_mass_octet_kernel(const MassParams p) {
     if (in_range) {
         const uint16_t* base = p.attn + (long long)l * p.stride_layer + col;
         int h = r0 / p.Q, q = r0 - h * p.Q;
-        if (n_valid == 8) {
+        if (n_valid == 8 && p.Q % kMassBatch == 0 && r0 % kMassBatch == 0 && (r1 - r0) % kMassBatch == 0) {
+            // regular shape: a batch of eight rows lies inside one head, no wrap test per load
+            for (int r = r0; r < r1; r += kMassBatch) {
+                const uint16_t* row = base + (long long)h * p.stride_head + (long long)q * p.stride_query;
+                q += kMassBatch;
+                if (q == p.Q) { q = 0; h++; }
+                uint4 w[kMassBatch];
+#pragma unroll
+                for (int i = 0; i < kMassBatch; i++) w[i] = __ldcs(reinterpret_cast<const uint4*>(row + (long long)i * p.stride_query));
+#pragma unroll
+                for (int i = 0; i < kMassBatch; i++) sum.add(w[i]);
+            }
+        } else if (n_valid == 8) {
             for (int r = r0; r < r1; r += kMassBatch) {
                 uint4 w[kMassBatch];
 #pragma unroll
@@ -579,6 +591,7 @@ extern "C" int patchkv_select_repair(patchkv_ctx* ctx, const patchkv_select_args
             long long groups = want / ((long long)tiles * L);
             if (groups < 1) groups = 1;
             long long rpc = (rows + groups - 1) / groups;
+            rpc = (rpc + kMassBatch - 1) / kMassBatch * kMassBatch;     // whole batches of rows per CTA
             if (rpc < 16) rpc = 16;
             if (rpc > rows) rpc = rows;
             groups = (rows + rpc - 1) / rpc;
@@ -790,6 +803,7 @@ extern "C" int patchkv_select_repair_static(const patchkv_select_args* a, void* 
             long long groups = 8192 / ((long long)tiles * L);       // about 8192 CTAs, at least 16 rows each
             if (groups < 1) groups = 1;
             long long rpc = (rows + groups - 1) / groups;
+            rpc = (rpc + kMassBatch - 1) / kMassBatch * kMassBatch;     // whole batches of rows per CTA
             if (rpc < 16) rpc = 16;
             if (rpc > rows) rpc = rows;
             groups = (rows + rpc - 1) / rpc;

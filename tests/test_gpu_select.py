@@ -65,9 +65,11 @@ def test_strided_and_unaligned_attention_uses_the_general_kernel(ctx):
     check_select(st, sel, mass)
 
 
-def test_values_outside_the_unit_interval_and_bad_entries(ctx):
+@pytest.mark.parametrize("Q", [5, 24])
+def test_values_outside_the_unit_interval_and_bad_entries(ctx, Q):
+    """Q = 24 takes the kernel's regular row loop (batches of eight rows inside one head), Q = 5 the general one."""
     rng = np.random.default_rng(3)
-    bits = rng.integers(0, 0x7C00, size=(2, 3, 5, 512)).astype(np.uint16)     # whole finite fp16 range
+    bits = rng.integers(0, 0x7C00, size=(2, 3, Q, 512)).astype(np.uint16)     # whole finite fp16 range
     attn = torch.from_numpy(bits.view(np.float16).copy())
     g = pin.Geometry(2, 4, 64, 64, pin.ROPE_HALF, 1e4, 16, 16, 32)
     ck = pin.config_tiny(n=512, geom=g)

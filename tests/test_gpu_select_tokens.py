@@ -121,10 +121,12 @@ def test_strided_and_unaligned_attention(ctx):
         assert np.array_equal(mass_out.cpu().numpy().astype(np.uint64), tmass)
 
 
-def test_token_mass_over_the_whole_fp16_range_and_bad_entries(ctx):
+@pytest.mark.parametrize("Q", [70, 72])
+def test_token_mass_over_the_whole_fp16_range_and_bad_entries(ctx, Q):
+    """Q = 72 takes the kernel's regular row loop (batches of eight rows inside one head), Q = 70 the general one."""
     from paper_2609_26219_b200 import binding as pk
     rng = np.random.default_rng(5)
-    bits = rng.integers(0, 0x7C00, size=(2, 3, 70, 512)).astype(np.uint16)
+    bits = rng.integers(0, 0x7C00, size=(2, 3, Q, 512)).astype(np.uint16)
     bits[0, 0, 0, 3] = 0xBC00       # -1.0
     bits[1, 2, 5, 40] = 0x7E00      # NaN
     rc, tmass = oracle.block_mass(bits, 1)

@@ -1,6 +1,6 @@
 // Checkpoint writer (Section IV-D, offload side): lay out the clustered directory from the tags, then gather
 // each block's rows from the paged pool, compute per-group fp16 scales, quantise and pack the record.
-// The inverse direction of restore; HBM-bound streaming with a warp-shuffle maximum per scale group.
+// The inverse direction of restore: an HBM-bound stream through the same kind of bulk-copy pipeline.
 #include <cuda_fp16.h>
 
 #include <algorithm>
@@ -348,11 +348,12 @@ __device__ __forceinline__ void encode_pass(uint32_t region, int u0, int units, 
 }
 
 // ---------------------------------------------------------------- persistent bulk-copy pipeline
-// The block encoder as a persistent kernel: one producer warp walks this CTA's share of the (layer, block) list,
-// looks up the next block's directory entry and source pages while the current block is being issued, and stages
-// the block's K and V rows (in units of a few tokens) into a shared-memory ring with bulk asynchronous copies that
-// complete on an mbarrier; eight consumer warps quantise from shared memory and write the record.  Loads of several
-// units are in flight per CTA at all times, which one CTA per block (above) cannot do.  Every wait is bounded.
+// The block encoder as a persistent kernel: one producer warp walks this CTA's share of the (layer, block) list
+// (block i of the launch goes to CTA i mod grid), looks up and validates the directory entries and source pages a
+// round of 32 blocks ahead, and stages each block's K and V rows (in units of a few tokens) into a shared-memory
+// ring with bulk asynchronous copies that complete on an mbarrier; eight consumer warps quantise from shared memory
+// and write the record with warp-contiguous stores.  Reads of several units are in flight per CTA at all times,
+// which one CTA per block (above) cannot do.  Every wait is bounded.
 constexpr int kWPipeConsumers = 256;
 constexpr int kWPipeThreads = kWPipeConsumers + 32;
 constexpr int kWPipeMaxStages = 8;

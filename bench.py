@@ -128,9 +128,9 @@ def measured_hbm_peak():
     return FALLBACK_HBM_GBS, "fallback"
 
 
-def oracle_sample(ck: pin.SuffixCheckpoint, layers, repeats: int = 1):
+def oracle_sample(ck: pin.SuffixCheckpoint, layers, repeats: int = 1, threads=None):
     """Time the CPU checker (select + restore) on `layers` of the workload.  Returns (seconds per pass,
-    bf16-equivalent bytes per pass, threads)."""
+    bf16-equivalent bytes per pass, threads); `threads` None = all host cores."""
     import oracle
     g = ck.geom
     L = len(layers)
@@ -145,7 +145,7 @@ def oracle_sample(ck: pin.SuffixCheckpoint, layers, repeats: int = 1):
     tags = ck.tags.cpu().numpy()[layers]
     off = ck.blk_off.cpu().numpy()[layers]
     table = ck.block_table.cpu().numpy()
-    threads = oracle.max_threads()
+    threads = oracle.max_threads() if threads is None else threads
     best, written = None, 0
     for _ in range(repeats):
         t0 = time.perf_counter()
@@ -605,9 +605,13 @@ def run_ours(args):
         oracle.build()
         sample_layers = list(range(ck.geom.n_layers))
         dt, wb, threads = oracle_sample(ck, sample_layers, repeats=3)
+        one_layers = sample_layers[:min(4, len(sample_layers))]
+        dt1, wb1, _ = oracle_sample(ck, one_layers, repeats=1, threads=1)
         cpu_baseline = {"value": wb / dt / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
                         "sample": f"all {len(sample_layers)} layers of the workload (select + restore), best of 3 passes "
-                                  f"of {dt:.2f} s on {threads} threads"}
+                                  f"of {dt:.2f} s on {threads} threads",
+                        "single_thread": {"value": wb1 / dt1 / 1e9, "unit": UNIT,
+                                          "sample": f"{len(one_layers)} layers, one pass of {dt1:.2f} s on 1 thread"}}
 
     if rank == 0:
         line = {

@@ -45,6 +45,10 @@ TINY_VARIANTS = {
     "all_dirty": dict(dirty_tokens=10 ** 6),
     "nothing_dirty_k0": dict(dirty_tokens=0, top_k=0),
     "shared_layers": dict(layer_mode=pin.LAYERS_SHARED, top_k=4),
+    # the geometry of the benchmark's paper-microbenchmark leg: 8 KV heads x 128, 32-token blocks and pages, one scale
+    # per 128 channels, a ragged 8031-token suffix, all four formats
+    "microbench_geometry": dict(geom=pin.Geometry(2, 8, 128, 128, pin.ROPE_HALF, 1e6, 32, 32, 128), n=8031, n_pages=300,
+                                tag_probs=(0.25, 0.25, 0.25, 0.25), dirty_tokens=200, top_k=8),
 }
 
 

@@ -92,6 +92,8 @@ def lib():
                           C.c_int, C.c_void_p]
         l.pkvo_select.restype = C.c_int
         l.pkvo_select.argtypes = [C.c_void_p] + [C.c_int] * 6 + [C.c_void_p] * 5
+        l.pkvo_normalise.restype = C.c_int
+        l.pkvo_normalise.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p]
         l.pkvo_restore.restype = C.c_int
         l.pkvo_restore.argtypes = [C.POINTER(_RestoreArgs)]
         l.pkvo_max_threads.restype = C.c_int
@@ -224,6 +226,16 @@ def select(mass: np.ndarray, n: int, B: int, dirty_tokens: int, top_k: int, laye
     fc = np.zeros(L, dtype=np.int32)
     rc = lib().pkvo_select(_p(mass), L, n, B, dirty_tokens, top_k, layer_mode, _p(mask), _p(ri), _p(rc_), _p(fi), _p(fc))
     return dict(status=rc, mask=mask, repair_idx=ri, repair_cnt=rc_, reuse_idx=fi, reuse_cnt=fc)
+
+
+def normalise(mass: np.ndarray, layer_mode: int = 0) -> np.ndarray:
+    """Norm of Eq. 10 as the share of the total: mass u64 [L][NB] -> fp32 [L][NB] (independent) or [NB] (shared)."""
+    mass = np.ascontiguousarray(mass, dtype=np.uint64)
+    L, NB = mass.shape
+    out = np.zeros((NB,) if layer_mode == 1 else (L, NB), dtype=np.float32)
+    rc = lib().pkvo_normalise(_p(mass), L, NB, layer_mode, _p(out))
+    assert rc == OK
+    return out
 
 
 def select_tokens(token_mass: np.ndarray, B: int, dirty_tokens: int, top_tokens: int, layer_mode: int = 1):

@@ -234,6 +234,34 @@ int pkvo_block_mass_f64(const uint16_t* attn, int L, int Hq, int Q, int n,
     return PKVO_OK;
 }
 
+/* Norm of Eq. 10, read as division by the total: the importance of unit j (a block, or a token in the token-level
+ * form) is its share of the summed mass, I_j = mass_j / sum_j' mass_j' over every unit of the row, the dirty window
+ * included.  A positive rescaling leaves the ranking as it is, so selection ranks on the exact masses and this score
+ * is reported only.  Masses are exact integers; the quotient is taken in double and rounded once to fp32.  A row
+ * whose masses are all zero gets zeros.  LAYERS_SHARED: one row, from the masses summed over the layers.
+ * mass u64 [L][NB] -> score fp32 [L][NB] (LAYERS_INDEPENDENT) or [NB] (LAYERS_SHARED). */
+int pkvo_normalise(const uint64_t* mass, int L, int NB, int layer_mode, float* score) {
+    if (L <= 0 || NB < 0) return PKVO_E_INVALID;
+    if (layer_mode != PKVO_LAYERS_INDEPENDENT && layer_mode != PKVO_LAYERS_SHARED) return PKVO_E_INVALID;
+    if (layer_mode == PKVO_LAYERS_SHARED) {
+        uint64_t total = 0;
+        for (int l = 0; l < L; l++) for (int j = 0; j < NB; j++) total += mass[(size_t)l * NB + j];
+        for (int j = 0; j < NB; j++) {
+            uint64_t m = 0;
+            for (int l = 0; l < L; l++) m += mass[(size_t)l * NB + j];
+            score[j] = total ? (float)((double)m / (double)total) : 0.0f;
+        }
+        return PKVO_OK;
+    }
+    for (int l = 0; l < L; l++) {
+        uint64_t total = 0;
+        for (int j = 0; j < NB; j++) total += mass[(size_t)l * NB + j];
+        for (int j = 0; j < NB; j++)
+            score[(size_t)l * NB + j] = total ? (float)((double)mass[(size_t)l * NB + j] / (double)total) : 0.0f;
+    }
+    return PKVO_OK;
+}
+
 typedef struct { uint64_t mass; int32_t idx; } cand_t;
 static int cand_cmp(const void* pa, const void* pb) {
     const cand_t* a = (const cand_t*)pa; const cand_t* b = (const cand_t*)pb;

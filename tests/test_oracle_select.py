@@ -152,3 +152,49 @@ def test_tiny_config_counts():
     sel = oracle.select(mass, 1024, 16, ck.dirty_tokens, ck.top_k)
     assert list(sel["repair_cnt"]) == [8, 8] and list(sel["reuse_cnt"]) == [56, 56]
     assert list(sel["repair_idx"][0, :6]) == [0, 1, 2, 3, 4, 5]
+
+
+# ---------------------------------------------------------------- Norm of Eq. 10 (reported score, not used for ranking)
+def test_normalise_closed_forms():
+    """Constant masses give exactly 1/NB; a single non-zero unit gives exactly 1; a zero row gives zeros;
+    a mass of 1 against a total of 2^k gives exactly 2^-k."""
+    for NB in (1, 3, 64, 1000):
+        out = oracle.normalise(np.full((2, NB), 12345, dtype=np.uint64))
+        assert np.all(out == np.float32(1.0 / NB))
+    m = np.zeros((3, 10), dtype=np.uint64)
+    m[0, 4] = 7
+    m[2, 0] = 1
+    m[2, 9] = (1 << 40) - 1
+    out = oracle.normalise(m)
+    assert out[0, 4] == 1.0 and out[0].sum() == 1.0
+    assert np.all(out[1] == 0.0)
+    assert out[2, 0] == np.float32(2.0 ** -40) and out[2, 9] == np.float32(1.0)
+
+
+def test_normalise_sums_to_one_keeps_order_and_ignores_scale():
+    rng = np.random.default_rng(11)
+    m = rng.integers(0, 1 << 38, size=(4, 777)).astype(np.uint64)
+    m[1, :100] = 0
+    out = oracle.normalise(m)
+    assert out.dtype == np.float32 and out.shape == m.shape
+    assert np.all(np.abs(out.astype(np.float64).sum(axis=1) - 1.0) < 777 * 2.0 ** -25)
+    for l in range(4):                                     # a larger mass never gets a smaller score
+        order = np.argsort(m[l], kind="stable")
+        assert np.all(np.diff(out[l][order]) >= 0)
+    assert np.array_equal(oracle.normalise(m * np.uint64(8)), out)       # Norm is scale-free (powers of two: exactly)
+    # the same quotient by a library routine
+    want = (m.astype(np.float64) / m.sum(axis=1, dtype=np.uint64).astype(np.float64)[:, None]).astype(np.float32)
+    assert np.array_equal(out, want)
+
+
+def test_normalise_shared_mode_is_the_share_of_the_layer_summed_mass():
+    rng = np.random.default_rng(12)
+    m = rng.integers(0, 1 << 30, size=(5, 64)).astype(np.uint64)
+    out = oracle.normalise(m, layer_mode=1)
+    assert out.shape == (64,)
+    summed = m.sum(axis=0, dtype=np.uint64)[None, :]
+    assert np.array_equal(out, oracle.normalise(summed)[0])
+    # ranking by the score agrees with ranking by the exact mass wherever the scores differ
+    sel = oracle.select(m, 64 * 16, 16, 0, 8, 1)
+    top = set(sel["repair_idx"][0, :8].tolist())
+    assert min(out[j] for j in top) >= max(out[j] for j in range(64) if j not in top)

@@ -197,6 +197,11 @@ typedef struct {
     int32_t* repair_cnt;         /* DEVICE i32 [L] */
     int32_t* reuse_idx;          /* DEVICE i32 [L][NB]: F_l ascending, then -1 */
     int32_t* reuse_cnt;          /* DEVICE i32 [L] */
+    float* score_out;            /* DEVICE fp32, optional: Norm of Eq. 10 read as the share of the total, I_j = mass_j /
+                                    sum of the row's masses (dirty window included; quotient in double, rounded once to
+                                    fp32; an all-zero row gives zeros).  [L][NB] for LAYERS_INDEPENDENT, one row [NB] of
+                                    the layer-summed masses for LAYERS_SHARED; the unit is a token ([L][n] / [n]) in
+                                    patchkv_select_repair_tokens.  Reported only: ranking uses the exact masses. */
 } patchkv_select_args;
 
 typedef struct {

@@ -61,7 +61,7 @@ class SelectArgs(C.Structure):
                 ("attn", C.c_void_p), ("attn_stride_layer", C.c_int64), ("attn_stride_head", C.c_int64),
                 ("attn_stride_query", C.c_int64), ("mass", C.c_void_p), ("mass_out", C.c_void_p),
                 ("repair_mask", C.c_void_p), ("repair_idx", C.c_void_p), ("repair_cnt", C.c_void_p),
-                ("reuse_idx", C.c_void_p), ("reuse_cnt", C.c_void_p)]
+                ("reuse_idx", C.c_void_p), ("reuse_cnt", C.c_void_p), ("score_out", C.c_void_p)]
 
 
 class RestoreStats(C.Structure):
@@ -248,8 +248,10 @@ def record_bytes(tag: int, block_tokens: int, n_kv_heads: int, head_dim: int, gr
 
 def select_args(*, kind, n_layers, n_suffix_tokens, block_tokens, dirty_tokens, top_k, layer_mode, repair_mask,
                 repair_idx, repair_cnt, reuse_idx, reuse_cnt, attn: Optional[torch.Tensor] = None,
-                mass: Optional[torch.Tensor] = None, mass_out: Optional[torch.Tensor] = None) -> SelectArgs:
-    """attn: fp16 device tensor [L][Hq][Q][n] with unit stride on the last axis (any other strides)."""
+                mass: Optional[torch.Tensor] = None, mass_out: Optional[torch.Tensor] = None,
+                score_out: Optional[torch.Tensor] = None) -> SelectArgs:
+    """attn: fp16 device tensor [L][Hq][Q][n] with unit stride on the last axis (any other strides);
+    score_out: optional fp32 device tensor that receives the normalised importance (Norm of Eq. 10)."""
     a = SelectArgs()
     a.struct_size = C.sizeof(SelectArgs)
     a.kind, a.n_layers, a.n_suffix_tokens, a.block_tokens = kind, n_layers, n_suffix_tokens, block_tokens
@@ -262,4 +264,5 @@ def select_args(*, kind, n_layers, n_suffix_tokens, block_tokens, dirty_tokens, 
     a.mass, a.mass_out = _ptr(mass), _ptr(mass_out)
     a.repair_mask, a.repair_idx, a.repair_cnt = _ptr(repair_mask), _ptr(repair_idx), _ptr(repair_cnt)
     a.reuse_idx, a.reuse_cnt = _ptr(reuse_idx), _ptr(reuse_cnt)
+    a.score_out = _ptr(score_out)
     return a

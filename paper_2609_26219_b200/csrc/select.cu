@@ -350,6 +350,25 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int* 
     return warp_sums[warp] + inc - v;
 }
 
+// Norm of Eq. 10 as the share of the row total: one CTA per row, exact u64 total, quotient in double, one rounding
+// to fp32.  Reported only; the ranking uses the exact masses.
+__global__ void __launch_bounds__(256)
+normalise_kernel(const unsigned long long* mass, int NB, float* score) {
+    __shared__ unsigned long long part[8];
+    const unsigned long long* m = mass + (long long)blockIdx.x * NB;
+    unsigned long long t = 0;
+    for (int j = threadIdx.x; j < NB; j += 256) t += m[j];
+    for (int d = 16; d > 0; d >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, d);
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = t;
+    __syncthreads();
+    unsigned long long total = 0;
+#pragma unroll
+    for (int w = 0; w < 8; w++) total += part[w];
+    const double dt = (double)total;
+    for (int j = threadIdx.x; j < NB; j += 256)
+        score[(long long)blockIdx.x * NB + j] = total ? (float)__ddiv_rn((double)m[j], dt) : 0.0f;
+}
+
 constexpr int kKeysPerThread = 8;      // candidate masses cached in registers: covers NB - n_dirty <= 8192
 
 __global__ void __launch_bounds__(kSelThreads)
@@ -617,6 +636,7 @@ extern "C" int patchkv_select_repair(patchkv_ctx* ctx, const patchkv_select_args
     tp.NB = NB; tp.n_dirty = n_dirty; tp.top_k = a->top_k;
     tp.mask = a->repair_mask; tp.repair_idx = a->repair_idx; tp.repair_cnt = a->repair_cnt;
     tp.reuse_idx = a->reuse_idx; tp.reuse_cnt = a->reuse_cnt;
+    if (a->score_out && NB > 0) normalise_kernel<<<tp.shared ? 1 : L, 256, 0, stream>>>(tp.mass, NB, a->score_out);
     select_kernel<<<L, kSelThreads, 0, stream>>>(tp);
     PKV_CUDA(ctx, cudaGetLastError());
     return PATCHKV_OK;
@@ -711,6 +731,7 @@ extern "C" int patchkv_select_repair_tokens(patchkv_ctx* ctx, const patchkv_sele
         PKV_CUDA(ctx, cudaGetLastError());
         tp.mass = ws_sum; tp.shared = 1;
     }
+    if (a->score_out && n > 0) normalise_kernel<<<tp.shared ? 1 : L, 256, 0, stream>>>(tp.mass, n, a->score_out);
     tp.NB = n; tp.n_dirty = (int)nd; tp.top_k = a->top_k;     // the "blocks" of this stage are single tokens
     tp.mask = tok_mask; tp.repair_idx = nullptr; tp.repair_cnt = nullptr; tp.reuse_idx = nullptr; tp.reuse_cnt = nullptr;
     select_kernel<<<L, kSelThreads, 0, stream>>>(tp);
@@ -832,6 +853,7 @@ extern "C" int patchkv_select_repair_static(const patchkv_select_args* a, void* 
     tp.NB = NB; tp.n_dirty = n_dirty; tp.top_k = a->top_k;
     tp.mask = a->repair_mask; tp.repair_idx = a->repair_idx; tp.repair_cnt = a->repair_cnt;
     tp.reuse_idx = a->reuse_idx; tp.reuse_cnt = a->reuse_cnt;
+    if (a->score_out && NB > 0) normalise_kernel<<<tp.shared ? 1 : L, 256, 0, stream>>>(tp.mass, NB, a->score_out);
     select_kernel<<<L, kSelThreads, 0, stream>>>(tp);
     if (cudaGetLastError() != cudaSuccess) return PATCHKV_E_CUDA;
     return PATCHKV_OK;

@@ -157,3 +157,47 @@ def test_selection_at_scale_full_size_sampled_layers(ctx):
     rc, k_ref, v_ref, _ = oracle_restore(ck, ridx, rcnt, layers=layers)
     assert rc == oracle.OK
     check_pools(k[layers], v[layers], k_ref, v_ref, ck.geom)
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_normalised_score_output_matches_the_oracle_bit_for_bit(ctx, mode):
+    """Norm of Eq. 10 (share of the row total): from stored attention and from given masses, per layer and request-level."""
+    from paper_2609_26219_b200 import binding as pk
+    ck = pin.config_tiny(n=1000, layer_mode=mode, top_k=3)
+    rc, mass = oracle.block_mass(ck.attn.numpy(), 16)
+    want = oracle.normalise(mass, mode)
+    NB, L = mass.shape[1], mass.shape[0]
+    sel = oracle.select(mass, 1000, 16, ck.dirty_tokens, 3, mode)
+    for kind in ("attn", "mass"):
+        out = dict(repair_mask=torch.zeros((L, NB), dtype=torch.uint8, device=DEV),
+                   repair_idx=torch.zeros((L, NB), dtype=torch.int32, device=DEV),
+                   repair_cnt=torch.zeros(L, dtype=torch.int32, device=DEV),
+                   reuse_idx=torch.zeros((L, NB), dtype=torch.int32, device=DEV),
+                   reuse_cnt=torch.zeros(L, dtype=torch.int32, device=DEV))
+        score = torch.full((L, NB), -1.0, dtype=torch.float32, device=DEV)
+        if kind == "attn":
+            a = pk.select_args(kind=pk.SCORE_ATTN_F16, n_layers=L, n_suffix_tokens=1000, block_tokens=16,
+                               dirty_tokens=ck.dirty_tokens, top_k=3, layer_mode=mode, attn=ck.attn.to(DEV),
+                               score_out=score, **out)
+        else:
+            a = pk.select_args(kind=pk.SCORE_BLOCK_MASS, n_layers=L, n_suffix_tokens=1000, block_tokens=16,
+                               dirty_tokens=ck.dirty_tokens, top_k=3, layer_mode=mode,
+                               mass=torch.from_numpy(mass.astype(np.int64)).to(DEV), score_out=score, **out)
+        ctx.select_repair(a)
+        torch.cuda.synchronize()
+        got = score.cpu().numpy()
+        if mode == 1:
+            assert np.array_equal(got[0].view(np.uint32), want.view(np.uint32))
+            assert np.all(got[1:] == -1.0)                  # one row only
+        else:
+            assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+        assert np.array_equal(out["repair_idx"].cpu().numpy(), sel["repair_idx"])
+    assert ctx.query_status() == 0
+    # an all-zero row gives zeros
+    zero = torch.zeros((L, NB), dtype=torch.int64, device=DEV)
+    score = torch.full((L, NB), -1.0, dtype=torch.float32, device=DEV)
+    a = pk.select_args(kind=pk.SCORE_BLOCK_MASS, n_layers=L, n_suffix_tokens=1000, block_tokens=16, dirty_tokens=0,
+                       top_k=3, layer_mode=0, mass=zero, score_out=score, **out)
+    ctx.select_repair(a)
+    torch.cuda.synchronize()
+    assert np.all(score.cpu().numpy() == 0.0)

@@ -141,3 +141,23 @@ def test_token_mass_over_the_whole_fp16_range_and_bad_entries(ctx, Q):
     _check(out, sel)
     assert np.array_equal(mass_out.cpu().numpy().astype(np.uint64), tmass)
     assert ctx.query_status() == -7
+
+
+def test_token_level_normalised_score(ctx):
+    """score_out of the token form: one fp32 per token, request-level (layers summed) and per layer."""
+    from paper_2609_26219_b200 import binding as pk
+    ck = pin.config_tiny()
+    rc, tmass = oracle.block_mass(ck.attn.numpy(), 1)
+    for mode in (1, 0):
+        want = oracle.normalise(tmass, mode)
+        out = _outputs(2, 64)
+        score = torch.full((2, 1024), -1.0, dtype=torch.float32, device=DEV)
+        a = pk.select_args(kind=pk.SCORE_ATTN_F16, n_layers=2, n_suffix_tokens=1024, block_tokens=16, dirty_tokens=90,
+                           top_k=15, layer_mode=mode, attn=ck.attn.to(DEV), score_out=score, **out)
+        ctx.select_repair_tokens(a)
+        _check(out, oracle.select_tokens(tmass, 16, 90, 15, mode))
+        got = score.cpu().numpy()
+        if mode == 1:
+            assert np.array_equal(got[0].view(np.uint32), want.view(np.uint32)) and np.all(got[1] == -1.0)
+        else:
+            assert np.array_equal(got.view(np.uint32), want.view(np.uint32))

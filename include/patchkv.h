@@ -202,6 +202,18 @@ typedef struct {
                                     fp32; an all-zero row gives zeros).  [L][NB] for LAYERS_INDEPENDENT, one row [NB] of
                                     the layer-summed masses for LAYERS_SHARED; the unit is a token ([L][n] / [n]) in
                                     patchkv_select_repair_tokens.  Reported only: ranking uses the exact masses. */
+    /* Optional HOST mirrors (pinned memory) of the outputs, for a caller whose next step runs on the host
+     * (patchkv_restore_from_host plans its copies from the reuse lists): each non-NULL pointer receives a copy of
+     * the device array of the same name, enqueued on `stream` after the selection.  With sync_to_host != 0 the call
+     * waits for `stream` before it returns, so the mirrors are valid on return (not inside a stream capture);
+     * otherwise they are valid once the caller has synchronised `stream`. */
+    uint8_t* host_repair_mask;   /* HOST u8  [L][NB] */
+    int32_t* host_repair_idx;    /* HOST i32 [L][NB] */
+    int32_t* host_repair_cnt;    /* HOST i32 [L] */
+    int32_t* host_reuse_idx;     /* HOST i32 [L][NB] */
+    int32_t* host_reuse_cnt;     /* HOST i32 [L] */
+    int32_t sync_to_host;
+    int32_t reserved;
 } patchkv_select_args;
 
 typedef struct {

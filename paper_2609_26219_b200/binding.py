@@ -61,7 +61,10 @@ class SelectArgs(C.Structure):
                 ("attn", C.c_void_p), ("attn_stride_layer", C.c_int64), ("attn_stride_head", C.c_int64),
                 ("attn_stride_query", C.c_int64), ("mass", C.c_void_p), ("mass_out", C.c_void_p),
                 ("repair_mask", C.c_void_p), ("repair_idx", C.c_void_p), ("repair_cnt", C.c_void_p),
-                ("reuse_idx", C.c_void_p), ("reuse_cnt", C.c_void_p), ("score_out", C.c_void_p)]
+                ("reuse_idx", C.c_void_p), ("reuse_cnt", C.c_void_p), ("score_out", C.c_void_p),
+                ("host_repair_mask", C.c_void_p), ("host_repair_idx", C.c_void_p), ("host_repair_cnt", C.c_void_p),
+                ("host_reuse_idx", C.c_void_p), ("host_reuse_cnt", C.c_void_p), ("sync_to_host", C.c_int32),
+                ("reserved", C.c_int32)]
 
 
 class RestoreStats(C.Structure):
@@ -249,7 +252,10 @@ def record_bytes(tag: int, block_tokens: int, n_kv_heads: int, head_dim: int, gr
 def select_args(*, kind, n_layers, n_suffix_tokens, block_tokens, dirty_tokens, top_k, layer_mode, repair_mask,
                 repair_idx, repair_cnt, reuse_idx, reuse_cnt, attn: Optional[torch.Tensor] = None,
                 mass: Optional[torch.Tensor] = None, mass_out: Optional[torch.Tensor] = None,
-                score_out: Optional[torch.Tensor] = None) -> SelectArgs:
+                score_out: Optional[torch.Tensor] = None, host_repair_mask: Optional[torch.Tensor] = None,
+                host_repair_idx: Optional[torch.Tensor] = None, host_repair_cnt: Optional[torch.Tensor] = None,
+                host_reuse_idx: Optional[torch.Tensor] = None, host_reuse_cnt: Optional[torch.Tensor] = None,
+                sync_to_host: bool = False) -> SelectArgs:
     """attn: fp16 device tensor [L][Hq][Q][n] with unit stride on the last axis (any other strides);
     score_out: optional fp32 device tensor that receives the normalised importance (Norm of Eq. 10)."""
     a = SelectArgs()
@@ -265,4 +271,11 @@ def select_args(*, kind, n_layers, n_suffix_tokens, block_tokens, dirty_tokens, 
     a.repair_mask, a.repair_idx, a.repair_cnt = _ptr(repair_mask), _ptr(repair_idx), _ptr(repair_cnt)
     a.reuse_idx, a.reuse_cnt = _ptr(reuse_idx), _ptr(reuse_cnt)
     a.score_out = _ptr(score_out)
+    for name, t in (("host_repair_mask", host_repair_mask), ("host_repair_idx", host_repair_idx),
+                    ("host_repair_cnt", host_repair_cnt), ("host_reuse_idx", host_reuse_idx),
+                    ("host_reuse_cnt", host_reuse_cnt)):
+        if t is not None:
+            assert t.device.type == "cpu" and t.is_pinned() and t.is_contiguous(), f"{name} must be pinned host memory"
+        setattr(a, name, _ptr(t))
+    a.sync_to_host = 1 if sync_to_host else 0
     return a

@@ -559,6 +559,24 @@ static int ensure_mass_ws(patchkv_ctx* ctx, size_t elems) {
 
 using namespace patchkv;
 
+// Copies of the selection outputs into the caller's pinned host mirrors, in stream order after the kernels.
+static cudaError_t mirror_to_host(const patchkv_select_args* a, int L, int NB, cudaStream_t stream) {
+    const size_t cells = (size_t)L * NB;
+    cudaError_t e = cudaSuccess;
+    if (a->host_repair_mask && cells && e == cudaSuccess)
+        e = cudaMemcpyAsync(a->host_repair_mask, a->repair_mask, cells, cudaMemcpyDeviceToHost, stream);
+    if (a->host_repair_idx && cells && e == cudaSuccess)
+        e = cudaMemcpyAsync(a->host_repair_idx, a->repair_idx, cells * 4, cudaMemcpyDeviceToHost, stream);
+    if (a->host_reuse_idx && cells && e == cudaSuccess)
+        e = cudaMemcpyAsync(a->host_reuse_idx, a->reuse_idx, cells * 4, cudaMemcpyDeviceToHost, stream);
+    if (a->host_repair_cnt && e == cudaSuccess)
+        e = cudaMemcpyAsync(a->host_repair_cnt, a->repair_cnt, (size_t)L * 4, cudaMemcpyDeviceToHost, stream);
+    if (a->host_reuse_cnt && e == cudaSuccess)
+        e = cudaMemcpyAsync(a->host_reuse_cnt, a->reuse_cnt, (size_t)L * 4, cudaMemcpyDeviceToHost, stream);
+    if (a->sync_to_host && e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    return e;
+}
+
 extern "C" int patchkv_select_repair(patchkv_ctx* ctx, const patchkv_select_args* a, void* stream_) {
     if (!ctx) return PATCHKV_E_INVALID;
     std::lock_guard<std::mutex> lock(ctx->mu);
@@ -639,6 +657,7 @@ extern "C" int patchkv_select_repair(patchkv_ctx* ctx, const patchkv_select_args
     if (a->score_out && NB > 0) normalise_kernel<<<tp.shared ? 1 : L, 256, 0, stream>>>(tp.mass, NB, a->score_out);
     select_kernel<<<L, kSelThreads, 0, stream>>>(tp);
     PKV_CUDA(ctx, cudaGetLastError());
+    PKV_CUDA(ctx, mirror_to_host(a, L, NB, stream));
     return PATCHKV_OK;
 }
 
@@ -739,6 +758,7 @@ extern "C" int patchkv_select_repair_tokens(patchkv_ctx* ctx, const patchkv_sele
     block_round_kernel<<<L, kSelThreads, 0, stream>>>(tok_mask, n, B, NB, a->repair_mask, a->repair_idx, a->repair_cnt,
                                                       a->reuse_idx, a->reuse_cnt);
     PKV_CUDA(ctx, cudaGetLastError());
+    PKV_CUDA(ctx, mirror_to_host(a, L, NB, stream));
     return PATCHKV_OK;
 }
 
@@ -856,5 +876,6 @@ extern "C" int patchkv_select_repair_static(const patchkv_select_args* a, void* 
     if (a->score_out && NB > 0) normalise_kernel<<<tp.shared ? 1 : L, 256, 0, stream>>>(tp.mass, NB, a->score_out);
     select_kernel<<<L, kSelThreads, 0, stream>>>(tp);
     if (cudaGetLastError() != cudaSuccess) return PATCHKV_E_CUDA;
+    if (mirror_to_host(a, L, NB, stream) != cudaSuccess) { cudaGetLastError(); return PATCHKV_E_CUDA; }
     return PATCHKV_OK;
 }

@@ -201,3 +201,41 @@ def test_normalised_score_output_matches_the_oracle_bit_for_bit(ctx, mode):
     ctx.select_repair(a)
     torch.cuda.synchronize()
     assert np.all(score.cpu().numpy() == 0.0)
+
+
+@pytest.mark.parametrize("sync", [True, False])
+def test_host_mirrors_of_the_selection_outputs(ctx, sync):
+    ck = pin.config_llama8b(n_layers=3)
+    st = staged(ck)
+    mass, sel = oracle_select(ck)
+    L, NB = 3, ck.n_blocks
+    mirrors = dict(host_repair_mask=torch.full((L, NB), 7, dtype=torch.uint8).pin_memory(),
+                   host_repair_idx=torch.full((L, NB), -5, dtype=torch.int32).pin_memory(),
+                   host_repair_cnt=torch.full((L,), -5, dtype=torch.int32).pin_memory(),
+                   host_reuse_idx=torch.full((L, NB), -5, dtype=torch.int32).pin_memory(),
+                   host_reuse_cnt=torch.full((L,), -5, dtype=torch.int32).pin_memory())
+    ctx.select_repair(st.select_args(sync_to_host=sync, **mirrors))
+    if not sync:
+        torch.cuda.current_stream().synchronize()
+    assert np.array_equal(mirrors["host_repair_mask"].numpy(), sel["mask"])
+    assert np.array_equal(mirrors["host_repair_idx"].numpy(), sel["repair_idx"])
+    assert np.array_equal(mirrors["host_reuse_idx"].numpy(), sel["reuse_idx"])
+    assert np.array_equal(mirrors["host_repair_cnt"].numpy(), sel["repair_cnt"])
+    assert np.array_equal(mirrors["host_reuse_cnt"].numpy(), sel["reuse_cnt"])
+    check_select(st, sel)
+    # a subset of the mirrors, through the token-level entry point
+    from paper_2609_26219_b200 import binding as pk
+    tm = pin.zipf_block_mass(torch.Generator().manual_seed(3), 2, 512, "cpu")
+    want = oracle.select_tokens(tm.numpy().astype(np.uint64), 16, 40, 9, 1)
+    out = dict(repair_mask=torch.zeros((2, 32), dtype=torch.uint8, device=DEV),
+               repair_idx=torch.zeros((2, 32), dtype=torch.int32, device=DEV),
+               repair_cnt=torch.zeros(2, dtype=torch.int32, device=DEV),
+               reuse_idx=torch.zeros((2, 32), dtype=torch.int32, device=DEV),
+               reuse_cnt=torch.zeros(2, dtype=torch.int32, device=DEV))
+    h_idx = torch.full((2, 32), -5, dtype=torch.int32).pin_memory()
+    h_cnt = torch.full((2,), -5, dtype=torch.int32).pin_memory()
+    a = pk.select_args(kind=pk.SCORE_TOKEN_MASS, n_layers=2, n_suffix_tokens=512, block_tokens=16, dirty_tokens=40,
+                       top_k=9, layer_mode=1, mass=tm.to(DEV), host_reuse_idx=h_idx, host_reuse_cnt=h_cnt,
+                       sync_to_host=True, **out)
+    ctx.select_repair_tokens(a)
+    assert np.array_equal(h_idx.numpy(), want["reuse_idx"]) and np.array_equal(h_cnt.numpy(), want["reuse_cnt"])

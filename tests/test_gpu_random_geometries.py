@@ -73,3 +73,73 @@ def test_writer_random_configuration(ctx, seed):
     assert np.array_equal(off, off_o) and sizes == [int(x) for x in lb_o]
     for a, b in zip(bufs, bufs_o):
         assert np.array_equal(a, b)
+
+
+@pytest.fixture(scope="module")
+def sctx():
+    c = new_context()
+    yield c
+    c.close()
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_selection_random_configuration(sctx, seed):
+    """Block form and token form, from masses full of ties and from small attention maps of odd shapes."""
+    from gpu_common import DEV
+    from paper_2609_26219_b200 import binding as pk
+    rng = np.random.default_rng(5000 + seed)
+    L = int(rng.integers(1, 5))
+    n = int(rng.integers(1, 3000))
+    B = int(rng.choice([1, 8, 16, 20, 32, 64]))
+    NB = -(-n // B)
+    d_hat = int(rng.integers(-5, n + 6))
+    mode = int(rng.integers(0, 2))
+    from_attn = bool(rng.integers(0, 2))
+    if from_attn:
+        Hq, Q = int(rng.integers(1, 4)), int(rng.integers(1, 20))
+        bits = rng.integers(0, 0x3C01, size=(L, Hq, Q, n)).astype(np.uint16)          # [0, 1]
+        bits[rng.random(bits.shape) < 0.7] = 0                                         # many zeros: ties
+        attn = torch.from_numpy(bits.view(np.float16).copy()).to(DEV)
+        rc, mass = oracle.block_mass(bits, B)
+        rc, tmass = oracle.block_mass(bits, 1)
+    else:
+        tmass = rng.integers(0, 6, size=(L, n)).astype(np.uint64) << np.uint64(int(rng.integers(0, 40)))
+        mass = np.zeros((L, NB), dtype=np.uint64)
+        for j in range(NB):
+            mass[:, j] = tmass[:, j * B:(j + 1) * B].sum(axis=1)
+
+    def outputs():
+        return dict(repair_mask=torch.full((L, NB), 9, dtype=torch.uint8, device=DEV),
+                    repair_idx=torch.full((L, NB), -7, dtype=torch.int32, device=DEV),
+                    repair_cnt=torch.full((L,), -7, dtype=torch.int32, device=DEV),
+                    reuse_idx=torch.full((L, NB), -7, dtype=torch.int32, device=DEV),
+                    reuse_cnt=torch.full((L,), -7, dtype=torch.int32, device=DEV))
+
+    def check(out, sel):
+        torch.cuda.synchronize()
+        for name, key in (("repair_mask", "mask"), ("repair_idx", "repair_idx"), ("reuse_idx", "reuse_idx"),
+                          ("repair_cnt", "repair_cnt"), ("reuse_cnt", "reuse_cnt")):
+            assert np.array_equal(out[name].cpu().numpy(), sel[key]), name
+
+    # block form
+    k = int(rng.integers(0, NB + 3))
+    out = outputs()
+    common = dict(n_layers=L, n_suffix_tokens=n, block_tokens=B, dirty_tokens=d_hat, layer_mode=mode)
+    if from_attn:
+        a = pk.select_args(kind=pk.SCORE_ATTN_F16, top_k=k, attn=attn, **common, **out)
+    else:
+        a = pk.select_args(kind=pk.SCORE_BLOCK_MASS, top_k=k, mass=torch.from_numpy(mass.astype(np.int64)).to(DEV),
+                           **common, **out)
+    sctx.select_repair(a)
+    check(out, oracle.select(mass, n, B, d_hat, k, mode))
+    # token form
+    kappa = int(rng.integers(0, n + 3))
+    out = outputs()
+    if from_attn:
+        a = pk.select_args(kind=pk.SCORE_ATTN_F16, top_k=kappa, attn=attn, **common, **out)
+    else:
+        a = pk.select_args(kind=pk.SCORE_TOKEN_MASS, top_k=kappa, mass=torch.from_numpy(tmass.astype(np.int64)).to(DEV),
+                           **common, **out)
+    sctx.select_repair_tokens(a)
+    check(out, oracle.select_tokens(tmass, B, d_hat, kappa, mode))
+    assert sctx.query_status() == 0

@@ -495,6 +495,29 @@ def run_ours(args):
                         "select_us": 1e3 * t_ms, "attn_gbps": nbytes / (t_ms * 1e-3) / 1e9,
                         "frac_of_hbm_peak": nbytes / (t_ms * 1e-3) / 1e9 / peak, "launches": 3}
         del attn
+        if SL == ck.geom.n_layers:
+            # ... then the restore of the blocks that selection leaves to reuse (72 repaired / 952 reused per layer),
+            # on the same 8B-shaped payload and pool as the headline step
+            sa_lists = pk.select_args(kind=pk.SCORE_BLOCK_MASS, n_layers=SL, n_suffix_tokens=16384, block_tokens=16,
+                                      dirty_tokens=640, top_k=32, layer_mode=pk.LAYERS_INDEPENDENT, mass=mass_out, **out)
+            ctx.select_repair(sa_lists, stream)               # the lists of the block form, from the masses just computed
+            torch.cuda.synchronize()
+            sess4 = st.session(reuse_idx=out["reuse_idx"], reuse_cnt=out["reuse_cnt"])
+            r4, w4, items4 = algorithmic_bytes(ck, out["reuse_idx"].cpu().numpy(), out["reuse_cnt"].cpu().numpy())
+            ts4 = []
+            for i in range(13):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                ctx.restore(geom, pool, [sess4], stream)
+                b.record(stream)
+                b.synchronize()
+                if i >= 3:
+                    ts4.append(a.elapsed_time(b))
+            assert ctx.query_status() == 0
+            r_ms = statistics.median(ts4)
+            select_scale["restore_of_its_reuse_set"] = {
+                "ms": r_ms, "block_layers": int(items4), "restored_kv_gbps_bf16_equiv": w4 / (r_ms * 1e-3) / 1e9,
+                "real_gbps": (r4 + w4) / (r_ms * 1e-3) / 1e9, "frac_of_hbm_peak": (r4 + w4) / (r_ms * 1e-3) / 1e9 / peak}
 
     # ---- the two host-resident workloads: 7B-shaped / 4 KV heads (one session), 70B-shaped stress (8 sessions)
     host_cfg3 = stress = None

@@ -62,7 +62,8 @@ def gpu_writer(ctx, ck, kp, vp, shift=0, fill=0xEE, table=None, blk_off=None, ge
                                 dict(geom=pin.Geometry(2, 4, 64, 64, pin.ROPE_HALF, 1e4, 16, 16, 16), n=150, dst_shift=3),
                                 dict(geom=pin.Geometry(2, 2, 128, 128, pin.ROPE_HALF, 1e4, 48, 16, 32), n=500, n_pages=40),
                                 dict(geom=pin.Geometry(1, 1, 16, 16, pin.ROPE_HALF, 1e4, 16, 16, 8), n=40, n_pages=8),
-                                dict(geom=pin.Geometry(1, 8, 128, 128, pin.ROPE_HALF, 1e6, 32, 32, 128), n=500, n_pages=20)])
+                                dict(geom=pin.Geometry(1, 8, 128, 128, pin.ROPE_HALF, 1e6, 32, 32, 128), n=500, n_pages=20),
+                                dict(geom=pin.Geometry(1, 2, 256, 256, pin.ROPE_HALF, 1e4, 16, 16, 256), n=100, n_pages=12)])
 def test_writer_bytes_match_the_oracle(ctx, kw):
     ck = _ck(**kw)
     shift = ck.dst_shift

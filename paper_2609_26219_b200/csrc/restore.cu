@@ -390,7 +390,7 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
 
     const int S = p.n_stages;
     if (threadIdx.x == 0) {
-        for (int s = 0; s < S; s++) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], kPipeConsumers / 32); }
+        for (int s = 0; s < S; s++) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], p.group_warps); }
         for (int b = 0; b < 2; b++) { mbar_init(&rfull_bar[b], 1); mbar_init(&rempty_bar[b], 1); }
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -406,8 +406,8 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
         // Takes rounds of blocks from the global work counter and resolves them one lane per block (directory
         // entry, record extent, destination pages: three dependent global loads), into the round buffer the issuing
         // warp is not reading.  The directory latency of a round is spent while the previous round is being issued.
-        // Rounds shrink towards the end of the list (a fraction of what is left per CTA, at most 32 blocks, at least
-        // one) so that CTAs with heavier tags do not leave a long tail; a round is consecutive entries of one list.
+        // Rounds shrink towards the end of the list (a fraction of what is left per CTA, at most round_cap blocks, at
+        // least one) so that CTAs with heavier tags do not leave a long tail; a round is consecutive entries of one list.
         const int lane = threadIdx.x - 32;
         const uint64_t elems = (uint64_t)p.B * p.H * p.D;
         int rb = 0;
@@ -418,7 +418,7 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
             int round = 0;
             if (lane == 0) {
                 const long long left = (long long)p.total_items - *reinterpret_cast<volatile int*>(p.sched);
-                round = (int)max(1ll, min(4ll, left / (8ll * gridDim.x)));       // small: a CTA holds up to two rounds
+                round = (int)max(1ll, min((long long)p.round_cap, left / ((long long)p.round_div * gridDim.x)));       // small: a CTA holds up to two rounds
                 first = atomicAdd(p.sched, round);
             }
             first = __shfl_sync(0xFFFFFFFFu, first, 0);
@@ -543,13 +543,16 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
             ib ^= 1;
             if (ib == 0) iphase ^= 1;
         }
-        if (alive) {                                     // tell the consumers that the work list is exhausted
+        // tell every consumer group that the work list is exhausted: one empty unit each, in the groups' turn order
+        for (int g = 0; g < (kPipeConsumers / 32) / p.group_warps && alive; g++) {
             if (__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], phase ^ 1, abortp))) {
                 if (lane == 0) {
                     StageMeta m; m.nvec = -1; m.fmt = 0; m.flags = 0; m.session = 0;
                     *reinterpret_cast<StageMeta*>(ring + (size_t)stage * p.stage_bytes + off_meta) = m;
                     mbar_arrive(&full_bar[stage]);
                 }
+                q++;
+                if (++stage == S) { stage = 0; phase ^= 1; }
             } else alive = false;
         }
         if (!alive) {
@@ -567,13 +570,16 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
         }
     } else {
         // ================================================================ consumer warps
+        // group g of the consumer warps takes units g, g + n_groups, ... (units are numbered in issue order)
         const int c = threadIdx.x - kPipeProducers;
+        const int group_threads = p.group_warps * 32, n_groups = kPipeConsumers / group_threads;
+        const int grp = c / group_threads;
         bool lane_active;
-        const ThreadMap tm = make_thread_map<INTER>(p, kPipeConsumers, c, &lane_active);
+        const ThreadMap tm = make_thread_map<INTER>(p, group_threads, c - grp * group_threads, &lane_active);
         const int gpv = p.D / p.G;
         float tc[8], ts[8];
         int cur_session = -1;
-        int stage = 0;
+        int stage = grp;                                 // n_groups <= S
         uint32_t phase = 0;
         while (true) {
             if (!__all_sync(0xFFFFFFFFu, mbar_wait(&full_bar[stage], phase, abortp))) break;
@@ -596,7 +602,8 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
             }
             __syncwarp();
             if ((c & 31) == 0) mbar_arrive(&empty_bar[stage]);
-            if (++stage == S) { stage = 0; phase ^= 1; }
+            stage += n_groups;
+            if (stage >= S) { stage -= S; phase ^= 1; }
         }
         if (c == 0 && *abortp) atomicCAS(p.status, 0, (int)PATCHKV_E_TIMEOUT);
     }
@@ -673,6 +680,19 @@ static bool plan_pipeline(const patchkv_ctx* ctx, RestoreParams* p) {
     if (stages > kMaxStages) stages = kMaxStages;
     if (stages < 2) return false;
     p->n_stages = (int32_t)stages;
+    // Consumer groups: a unit of few vectors is not worth the fixed work of all eight consumer warps (barrier wait,
+    // unit header, format switch), so the warps split into groups that take units in turn, sized so that a thread
+    // gets about four (vector, channel-lane) tasks per unit; never more groups than stages.
+    const long long tasks = ut * p->H * ((p->D + 15) / 16);
+    int gw = kPipeConsumers / 32;
+    while (gw > 1 && (long long)gw * 32 / 2 * 4 >= tasks && (kPipeConsumers / 32) / (gw / 2) <= stages) gw /= 2;
+    p->group_warps = gw;
+    // Self-scheduled rounds: the resolver's chain of dependent lookups (about 7 us under load) has to stay shorter
+    // than the time the CTA spends issuing the previous round, so small records are claimed in larger rounds
+    // (about 256 KiB of bf16 per round), and shrink later (measured on records of 16 to 128 KiB).
+    const long long rec_bf16 = 4ll * p->B * hd;
+    p->round_cap = (int32_t)std::max<long long>(4, std::min<long long>(16, (256 * 1024) / rec_bf16));
+    p->round_div = (int32_t)std::max<long long>(2, std::min<long long>(8, rec_bf16 / 8192));
     const uint64_t elems = (uint64_t)p->B * hd;
     for (int f = 0; f < 3; f++) {                     // section sizes per format: no divisions in the issuing warp
         p->blk_codes[f] = (uint32_t)code_bytes(f, elems); p->blk_scales[f] = (uint32_t)scale_bytes(f, elems, p->G);

@@ -109,7 +109,7 @@ typedef struct {
     int32_t staging_slots;     /* restore_from_host: depth of the device staging ring (0 = 4) */
     int32_t flags;             /* PATCHKV_FLAG_* */
     uint64_t merge_gap_bytes;  /* restore_from_host: two reused records closer than this are fetched by one copy
-                                  (the bytes between them are transferred and ignored); UINT64_MAX = default 64 KiB */
+                                  (the bytes between them are transferred and ignored); UINT64_MAX = default 128 KiB */
 } patchkv_config;
 
 /* Model / cache geometry shared by all sessions of a call. */

@@ -15,7 +15,7 @@ extern "C" int patchkv_create(patchkv_ctx** out, const patchkv_config* cfg) {
     ctx->staging_slots = cfg->staging_slots > 0 ? cfg->staging_slots : 4;
     if (ctx->staging_slots > 64) ctx->staging_slots = 64;
     ctx->flags = cfg->flags;
-    ctx->merge_gap = cfg->merge_gap_bytes == UINT64_MAX ? 64 * 1024 : cfg->merge_gap_bytes;
+    ctx->merge_gap = cfg->merge_gap_bytes == UINT64_MAX ? 128 * 1024 : cfg->merge_gap_bytes;
     bool ok = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, cfg->device) == cudaSuccess;
     ok = ok && cudaDeviceGetAttribute(&ctx->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, cfg->device) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) == cudaSuccess;

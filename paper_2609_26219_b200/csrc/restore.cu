@@ -413,17 +413,33 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
         const uint64_t elems = (uint64_t)p.B * p.H * p.D;
         int rb = 0;
         uint32_t rphase = 0;
+        // The lookups of a round form a chain of dependent global loads, each a microsecond when the memory system is
+        // busy, so the chain is kept short: the first round is dealt out statically (CTA b takes blocks b * r0 ..., the
+        // counter hands out what follows), the size of a round comes from the previous claim's answer instead of a
+        // fresh read of the counter, and loads that do not depend on one another are issued together (the list entry
+        // with the list length; the destination pages with the directory entry).
+        const int r0 = (int)max(1ll, min((long long)p.round_cap, (long long)p.total_items / ((long long)p.round_div * gridDim.x)));
+        const long long static_items = (long long)r0 * gridDim.x;
+        long long seen = static_items;                   // blocks known to be handed out already
+        bool first_round = true;
 #pragma unroll 1
         while (true) {
             long long first = 0;
             int round = 0;
-            if (lane == 0) {
-                const long long left = (long long)p.total_items - *reinterpret_cast<volatile int*>(p.sched);
-                round = (int)max(1ll, min((long long)p.round_cap, left / ((long long)p.round_div * gridDim.x)));       // small: a CTA holds up to two rounds
-                first = atomicAdd(p.sched, round);
+            if (first_round) {
+                first = (long long)blockIdx.x * r0;
+                round = r0;
+                first_round = false;
+            } else {
+                if (lane == 0) {
+                    const long long left = (long long)p.total_items - seen;
+                    round = (int)max(1ll, min((long long)p.round_cap, left / ((long long)p.round_div * gridDim.x)));
+                    first = static_items + atomicAdd(p.sched, round);
+                }
+                first = __shfl_sync(0xFFFFFFFFu, first, 0);
+                round = __shfl_sync(0xFFFFFFFFu, round, 0);
+                seen = max(seen, first + round);
             }
-            first = __shfl_sync(0xFFFFFFFFu, first, 0);
-            round = __shfl_sync(0xFFFFFFFFu, round, 0);
             ItemDesc d;
             d.valid = 0;
             const long long item = first + lane;
@@ -435,30 +451,31 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
                 const int local = (int)item - Sd.item_begin;
                 const int l = p.layer_begin + local / Sd.nb;
                 const int r = local - (l - p.layer_begin) * Sd.nb;
-                if (r < __ldg(Sd.reuse_cnt + l)) {
-                    const int j = __ldg(Sd.reuse_idx + (size_t)l * Sd.nb + r);
+                // r < nb, so the list entry can be read before the list length is known
+                const int cnt = __ldg(Sd.reuse_cnt + l);
+                const int j = __ldg(Sd.reuse_idx + (size_t)l * Sd.nb + r);
+                if (r < cnt) {
                     bool bad = j < 0 || j >= Sd.nb;
                     if (!bad) {
+                        const int valid = min(p.B, Sd.n - j * p.B);
+                        const long long u0 = (long long)j * p.B + Sd.dst_shift;
+                        const long long lp0 = u0 / p.P, lp1 = (u0 + valid - 1) / p.P;
                         const int tag = __ldg(Sd.tags + (size_t)l * Sd.nb + j);
                         const unsigned long long off = __ldg(Sd.blk_off + (size_t)l * Sd.nb + j);
                         const unsigned long long lbytes = __ldg(Sd.layer_bytes + l);
                         const uint8_t* base = reinterpret_cast<const uint8_t*>(static_cast<uintptr_t>(
                             __ldg(reinterpret_cast<const unsigned long long*>(Sd.layer_payload) + l)));
-                        const unsigned long long rbytes = record_bytes(tag, elems, p.G);
-                        bad = rbytes == 0 || off > lbytes || rbytes > lbytes - off || base == nullptr ||
-                              ((reinterpret_cast<uintptr_t>(base) + off) & 15u) != 0;
-                        const int valid = min(p.B, Sd.n - j * p.B);
-                        const long long u0 = (long long)j * p.B + Sd.dst_shift;
-                        const long long lp0 = u0 / p.P, lp1 = (u0 + valid - 1) / p.P;
-                        if (!bad) {                      // every destination page is validated before any write
-                            for (long long lp = lp0; lp <= lp1; lp++) {
-                                const int page = lp < Sd.n_table ? __ldg(Sd.block_table + lp) : -1;
-                                if (page < 0 || page >= p.n_pages) bad = true;
-                                d.pages[lp - lp0] = page;
-                            }
+                        // every destination page is validated before any write
+                        for (long long lp = lp0; lp <= lp1; lp++) {
+                            const int page = lp < Sd.n_table ? __ldg(Sd.block_table + lp) : -1;
+                            if (page < 0 || page >= p.n_pages) bad = true;
+                            d.pages[lp - lp0] = page;
                         }
+                        const unsigned long long rbytes = record_bytes(tag, elems, p.G);
+                        bad = bad || rbytes == 0 || off > lbytes || rbytes > lbytes - off || base == nullptr ||
+                              ((reinterpret_cast<uintptr_t>(base) + off) & 15u) != 0;
                         d.rec = base + off;
-                        d.valid = valid; d.tag = tag; d.l = l; d.si = si;
+                        d.valid = bad ? 0 : valid; d.tag = tag; d.l = l; d.si = si;
                         d.slot0 = (int)(u0 - lp0 * p.P);
                     }
                     if (bad) { d.valid = 0; atomicCAS(p.status, 0, (int)PATCHKV_E_BOUNDS); }

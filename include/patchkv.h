@@ -354,6 +354,14 @@ PATCHKV_API int patchkv_checkpoint_to_host(patchkv_ctx* ctx, const patchkv_geom*
  * since the last query (PATCHKV_OK, PATCHKV_E_BOUNDS, PATCHKV_E_BADINPUT or PATCHKV_E_TIMEOUT), then clears it. */
 PATCHKV_API int patchkv_query_status(patchkv_ctx* ctx, int* device_status);
 
+/* Diagnostic (the paper has no counterpart).  Every barrier wait inside the pipeline kernels is bounded: after a fixed
+ * number of polls the waiting role gives up, raises the CTA's abort flag, lets the copies in flight land and the kernel
+ * latches PATCHKV_E_TIMEOUT instead of spinning.  This call runs that same wait, in a one-CTA kernel of its own, on a
+ * barrier that nothing completes, with a limit of `max_polls` polls (1 .. 2^20; microseconds to a fraction of a
+ * second), so that a caller can check that the limit expires, that patchkv_query_status then reports
+ * PATCHKV_E_TIMEOUT, and that the context keeps working afterwards.  Asynchronous on `stream`. */
+PATCHKV_API int patchkv_selftest_bounded_wait(patchkv_ctx* ctx, uint32_t max_polls, void* stream);
+
 /* Bytes of one block record for a tag under a geometry; 0 for an unknown tag. */
 PATCHKV_API uint64_t patchkv_record_bytes(int tag, int block_tokens, int n_kv_heads, int head_dim, int group);
 

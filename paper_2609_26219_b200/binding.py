@@ -104,6 +104,7 @@ def lib():
                                              C.c_float, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p]
         l.patchkv_plan_precision.restype = C.c_int
         l.patchkv_query_status.argtypes = [C.c_void_p, C.POINTER(C.c_int)]
+        l.patchkv_selftest_bounded_wait.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p]
         l.patchkv_record_bytes.argtypes = [C.c_int] * 5
         l.patchkv_record_bytes.restype = C.c_uint64
         for f in (l.patchkv_create, l.patchkv_destroy, l.patchkv_last_error, l.patchkv_select_repair,
@@ -227,6 +228,10 @@ class Context:
         return self._check(lib().patchkv_plan_precision(self._h, _ptr(attn), _ptr(resid), attn.numel(), block_tokens,
                                                         alpha, tau_L, tau_H, eps4, _ptr(tags), _ptr(risk),
                                                         _stream_handle(stream)), check)
+
+    def selftest_bounded_wait(self, max_polls: int, stream=None, check: bool = True) -> int:
+        """Runs the kernels' bounded barrier wait on a barrier that nothing completes; query_status() then reports E_TIMEOUT."""
+        return self._check(lib().patchkv_selftest_bounded_wait(self._h, max_polls, _stream_handle(stream)), check)
 
     def query_status(self) -> int:
         v = C.c_int(0)

@@ -78,6 +78,35 @@ extern "C" int patchkv_query_status(patchkv_ctx* ctx, int* device_status) {
     return PATCHKV_OK;
 }
 
+// A wait that nothing will ever satisfy, with a short limit: the same helper the pipeline kernels wait with has to give
+// up, raise the abort flag and let the kernel report PATCHKV_E_TIMEOUT instead of spinning.
+namespace patchkv {
+__global__ void bounded_wait_selftest_kernel(uint32_t limit, int32_t* status) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const bool ok = mbar_wait(&bar, 0, &abort_flag, limit);       // no thread arrives on `bar`
+    if (!__all_sync(0xFFFFFFFFu, ok) && (threadIdx.x & 31) == 0 && abort_flag)
+        atomicCAS(status, 0, (int)PATCHKV_E_TIMEOUT);
+}
+}  // namespace patchkv
+
+extern "C" int patchkv_selftest_bounded_wait(patchkv_ctx* ctx, uint32_t max_polls, void* stream) {
+    if (!ctx) return PATCHKV_E_INVALID;
+    std::lock_guard<std::mutex> lock(ctx->mu);
+    if (max_polls == 0 || max_polls > (1u << 20)) return fail(ctx, PATCHKV_E_INVALID, "selftest: max_polls must be 1 .. 2^20");
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, PATCHKV_E_CUDA, "cudaSetDevice failed");
+    patchkv::bounded_wait_selftest_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>(max_polls, ctx->d_status);
+    PKV_CUDA(ctx, cudaGetLastError());
+    return PATCHKV_OK;
+}
+
 extern "C" uint64_t patchkv_record_bytes(int tag, int block_tokens, int n_kv_heads, int head_dim, int group) {
     if (block_tokens <= 0 || n_kv_heads <= 0 || head_dim <= 0 || group <= 0) return 0;
     return record_bytes(tag, (uint64_t)block_tokens * n_kv_heads * head_dim, group);

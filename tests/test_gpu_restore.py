@@ -426,3 +426,16 @@ def test_geometry_limits_block_vectors_and_rotary_dim(ctx):
     assert ctx.restore(bad, pool, [st.session()], check=False) == pk.E_UNSUPPORTED
     bad = st.geom(); bad.head_dim = 512; bad.rotary_dim = 512
     assert ctx.restore(bad, pool, [st.session()], check=False) == pk.E_UNSUPPORTED
+
+
+def test_a_bounded_wait_runs_out_and_the_context_keeps_working(ctx):
+    """The wait helper of the pipeline kernels, on a barrier that nothing completes and with a short limit: it gives
+    up, the kernel latches E_TIMEOUT, the host reads it, and the next restore on the same context is correct."""
+    import time
+    t0 = time.time()
+    ctx.selftest_bounded_wait(2000)
+    assert ctx.query_status() == -5
+    assert time.time() - t0 < 5.0
+    assert ctx.query_status() == 0                       # the latch clears on read
+    assert ctx.selftest_bounded_wait(0, check=False) == -1
+    run_select_and_restore(ctx, pin.config_tiny(n_pages=256))

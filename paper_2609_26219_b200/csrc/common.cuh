@@ -151,6 +151,7 @@ struct RestoreParams {
     int32_t* sched;         // work counter of this launch (zeroed on the stream right before it)
     // bulk-copy pipeline: tokens per staged unit, bytes of one stage's code / scale / offset areas, ring depth
     int32_t unit_tokens, stage_code_bytes, stage_scale_bytes, stage_bytes, n_stages;
+    int32_t whole_record;   // 1: a unit is a whole block record (K and V sections together, one bulk copy)
     int32_t round_cap, round_div;   // a round of self-scheduled blocks: min(round_cap, left / (round_div * CTAs)), at least 1
     int32_t group_warps;    // consumer warps that share one unit (8, 4, 2 or 1): small units go to small groups
     uint32_t blk_codes[3], blk_scales[3], tok_codes[3], tok_scales[3];   // bytes per block / per token, by format

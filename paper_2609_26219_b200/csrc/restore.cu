@@ -521,6 +521,33 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
                 sec_codes[1] = sec_scales[0] + p.blk_scales[kf];
                 sec_scales[1] = sec_codes[1] + p.blk_codes[vf];
                 const bool shifted = p.s[si].delta != 0;
+                if (p.whole_record) {
+                    // one unit: the record as it lies in the payload, and the destination row of every token
+                    if (!__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], phase ^ 1, abortp))) { alive = false; break; }
+                    uint8_t* sp = ring + (size_t)stage * p.stage_bytes;
+                    long long* voff = reinterpret_cast<long long*>(sp + off_vec);
+                    for (int i = lane; i < valid; i += 32) {
+                        const int us = d.slot0 + i;
+                        const int pi = us / p.P;
+                        voff[i] = (long long)l * p.stride_layer + (long long)d.pages[pi] * p.stride_page +
+                                  (long long)(us - pi * p.P) * p.stride_token;
+                    }
+                    if (lane == 0) {
+                        StageMeta m;
+                        m.nvec = valid * p.H; m.fmt = kf | (vf << 4); m.session = si;
+                        m.flags = 4 | (shifted ? 2 : 0);
+                        *reinterpret_cast<StageMeta*>(sp + off_meta) = m;
+                    }
+                    __syncwarp();
+                    if (lane == 0) {
+                        const uint32_t rb_ = p.blk_codes[kf] + p.blk_scales[kf] + p.blk_codes[vf] + p.blk_scales[vf];
+                        mbar_arrive_expect_tx(&full_bar[stage], rb_);
+                        bulk_g2s(sp, d.rec, rb_, &full_bar[stage]);
+                    }
+                    q++;
+                    if (++stage == S) { stage = 0; phase ^= 1; }
+                    continue;
+                }
 #pragma unroll 1
                 for (int sec = 0; sec < 2 && alive; sec++) {
                     const int fmt = sec ? vf : kf;
@@ -608,14 +635,28 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
             if (m.nvec < 0) break;
             if (m.session != cur_session) { cur_session = m.session; load_rotation<INTER>(p, cur_session, tm, tc, ts); }
             if (lane_active) {
-                const uint32_t codes = smem_u32(sp), scales = codes + off_scales;
-                const uint32_t voff = codes + off_vec;
-                uint16_t* dst = (m.flags & 1) ? p.k_base : p.v_base;
-                const bool rotate = (m.flags & 2) != 0;
-                switch (m.fmt) {
-                    case FMT_BF16: consume_unit<FMT_BF16, INTER>(p, codes, scales, voff, m.nvec, dst, tm, gpv, tc, ts, rotate); break;
-                    case FMT_INT8: consume_unit<FMT_INT8, INTER>(p, codes, scales, voff, m.nvec, dst, tm, gpv, tc, ts, rotate); break;
-                    default:       consume_unit<FMT_INT4, INTER>(p, codes, scales, voff, m.nvec, dst, tm, gpv, tc, ts, rotate); break;
+                const uint32_t base = smem_u32(sp);
+                const uint32_t voff = base + off_vec;
+                const bool whole = (m.flags & 4) != 0;
+                const int kf = m.fmt & 15, vf = m.fmt >> 4;          // whole-record units carry both formats
+#pragma unroll 1
+                for (int sec = 0; sec < (whole ? 2 : 1); sec++) {
+                    int fmt = m.fmt;
+                    uint32_t codes = base, scales = base + off_scales;
+                    uint16_t* dst = (m.flags & 1) ? p.k_base : p.v_base;
+                    bool rotate = (m.flags & 2) != 0;
+                    if (whole) {                                     // sections in record order: K codes, K scales, V codes, V scales
+                        fmt = sec ? vf : kf;
+                        codes = sec ? base + p.blk_codes[kf] + p.blk_scales[kf] : base;
+                        scales = codes + p.blk_codes[fmt];
+                        dst = sec ? p.v_base : p.k_base;
+                        rotate = rotate && sec == 0;
+                    }
+                    switch (fmt) {
+                        case FMT_BF16: consume_unit<FMT_BF16, INTER>(p, codes, scales, voff, m.nvec, dst, tm, gpv, tc, ts, rotate); break;
+                        case FMT_INT8: consume_unit<FMT_INT8, INTER>(p, codes, scales, voff, m.nvec, dst, tm, gpv, tc, ts, rotate); break;
+                        default:       consume_unit<FMT_INT4, INTER>(p, codes, scales, voff, m.nvec, dst, tm, gpv, tc, ts, rotate); break;
+                    }
                 }
             }
             __syncwarp();
@@ -687,9 +728,12 @@ static bool plan_pipeline(const patchkv_ctx* ctx, RestoreParams* p) {
     if (ut > 256 / p->H) ut = 256 / p->H;            // at most 256 (token, head) vectors per stage
     if (ut < 1) return false;
     if ((p->B + p->P - 2) / p->P + 1 > kMaxItemPages) return false;   // pages one block can straddle
+    // Small records (both bf16 sections of a block within 36 KiB) travel whole: one unit and one bulk copy per block
+    // instead of one per section, which halves the issuing warp's work where it is the limit.
+    p->whole_record = (ut == p->B && 4ll * p->B * hd <= 36 * 1024) ? 1 : 0;
     p->unit_tokens = (int32_t)ut;
-    p->stage_code_bytes = (int32_t)(ut * hd * 2);
-    p->stage_scale_bytes = (int32_t)(ut * (hd / p->G) * 2);
+    p->stage_code_bytes = (int32_t)(p->whole_record ? 4 * ut * hd : ut * hd * 2);      // whole: the largest (bf16) record
+    p->stage_scale_bytes = (int32_t)(p->whole_record ? 0 : ut * (hd / p->G) * 2);
     const long long raw = (long long)p->stage_code_bytes + p->stage_scale_bytes + 8 * ut + 32;
     p->stage_bytes = (int32_t)((raw + 127) / 128 * 128);
     long long budget = ((long long)ctx->max_smem_optin - 2048) / 2;   // two CTAs per SM
@@ -701,7 +745,7 @@ static bool plan_pipeline(const patchkv_ctx* ctx, RestoreParams* p) {
     // Consumer groups: a unit of few vectors is not worth the fixed work of all eight consumer warps (barrier wait,
     // unit header, format switch), so the warps split into groups that take units in turn, sized so that a thread
     // gets about four (vector, channel-lane) tasks per unit; never more groups than stages.
-    const long long tasks = ut * p->H * ((p->D + 15) / 16);
+    const long long tasks = (p->whole_record ? 2 : 1) * ut * p->H * ((p->D + 15) / 16);
     int gw = kPipeConsumers / 32;
     while (gw > 1 && (long long)gw * 32 / 2 * 4 >= tasks && (kPipeConsumers / 32) / (gw / 2) <= stages) gw /= 2;
     p->group_warps = gw;

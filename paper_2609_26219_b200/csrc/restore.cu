@@ -308,7 +308,8 @@ restore_kernel(const __grid_constant__ RestoreParams p) {
 // ---------------------------------------------------------------- bulk-copy pipeline
 // A resolver warp takes rounds of blocks from the global work counter and resolves the directory entry and the
 // destination pages of each block one round ahead; an issuing warp stages each resolved block's K and V sections
-// (in units of a few tokens) into a shared-memory ring with bulk asynchronous copies that complete on an mbarrier.
+// (in units of a few tokens; small records whole, K and V in one unit) into a shared-memory ring with bulk
+// asynchronous copies that complete on an mbarrier.
 // Eight consumer warps dequantise / rotate from shared memory and write the bf16 rows to the pool with 128-bit
 // stores; when a unit holds few vectors they split into groups that take units in turn.  Directory latency and HBM
 // read latency are hidden by the ring instead of by occupancy.  Every wait is bounded.

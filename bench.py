@@ -163,6 +163,13 @@ def oracle_sample(ck: pin.SuffixCheckpoint, layers, repeats: int = 1, threads=No
     return best, written, threads
 
 
+def leg_failed(exc: Exception) -> dict:
+    """What an optional leg reports when it raised (out of pinned memory on a small box, say): the headline line is
+    still printed, with the reason in place of the leg's figures."""
+    print(f"bench: optional leg failed: {exc!r}", file=sys.stderr)
+    return {"error": repr(exc)[:300]}
+
+
 def dist_env():
     return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
 
@@ -334,305 +341,335 @@ def run_ours(args):
     # ---- offload side: write a checkpoint of all 1024 blocks x 32 layers from the pool (not on the resume path)
     writer = None
     if not args.no_writer:
-        L_, NB_ = ck.geom.n_layers, ck.n_blocks
-        w_off = torch.zeros((L_, NB_), dtype=torch.int64, device=dev)
-        w_lb = torch.zeros(L_, dtype=torch.int64, device=dev)
-        w_pay = torch.empty_like(st.payload)
-        w_ptrs = torch.tensor([w_pay.data_ptr() + o for o in ck.layer_off], dtype=torch.int64, device=dev)
-        w_sess = st.session(layer_payload=w_ptrs, blk_off=w_off, layer_bytes=w_lb)
-        ts_w = []
-        for i in range(13):
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            ctx.plan_checkpoint(geom, ck.n_suffix_tokens, st.tags, w_off, w_lb, stream)
-            ctx.quantize_gather(geom, pool, w_sess, stream)
-            b.record(stream)
-            b.synchronize()
-            if i >= 3:
-                ts_w.append(a.elapsed_time(b))
-        assert ctx.query_status() == 0 and torch.equal(w_off, st.blk_off)
-        t_w = statistics.median(ts_w)
-        pool_read = 2 * L_ * NB_ * ck.geom.block_tokens * ck.geom.n_kv_heads * ck.geom.head_dim * 2
-        pay_written = sum(ck.layer_bytes)
-        # the same checkpoint streamed to pinned host memory (encode layer l+1 while layer l is copied out)
-        cap_ = max(ck.layer_bytes)
-        hbufs = [torch.empty(cap_, dtype=torch.uint8).pin_memory() for _ in range(L_)]
-        hptrs = torch.tensor([h_.data_ptr() for h_ in hbufs], dtype=torch.int64)
-        hcaps = torch.full((L_,), cap_, dtype=torch.int64)
-        hsizes = torch.zeros(L_, dtype=torch.int64)
-        ts_h = []
-        for i in range(6):
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            torch.cuda.synchronize()
-            a.record(stream)
-            ctx.checkpoint_to_host(geom, pool, w_sess, hptrs, hcaps, hsizes, stream)
-            b.record(stream)
-            b.synchronize()
-            if i >= 2:
-                ts_h.append(a.elapsed_time(b))
-        assert ctx.query_status() == 0 and int(hsizes.sum()) == pay_written
-        src_ = torch.empty(1 << 30, dtype=torch.uint8, device=dev)
-        dst_ = torch.empty(1 << 30, dtype=torch.uint8).pin_memory()
-        d2h_best = None
-        for i in range(6):
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record()
-            dst_.copy_(src_, non_blocking=True)
-            b.record()
-            b.synchronize()
-            d2h_best = a.elapsed_time(b) if d2h_best is None else min(d2h_best, a.elapsed_time(b))
-        d2h_ceiling = (1 << 30) / (d2h_best * 1e-3) / 1e9
-        t_h = statistics.median(ts_h)
-        del hbufs, src_, dst_
-        writer = {"to_host": {"ms": t_h, "payload_gbps": pay_written / (t_h * 1e-3) / 1e9,
-                              "d2h_ceiling_gbps": d2h_ceiling, "frac_of_link": pay_written / (t_h * 1e-3) / 1e9 / d2h_ceiling},
-                  "workload": "quantize_gather of all 1024 blocks x 32 layers of the same pool and tags",
-                  "ms": t_w, "real_gbps": (pool_read + pay_written) / (t_w * 1e-3) / 1e9,
-                  "frac_of_hbm_peak": (pool_read + pay_written) / (t_w * 1e-3) / 1e9 / peak,
-                  "bf16_gbps_read": pool_read / (t_w * 1e-3) / 1e9, "payload_bytes": int(pay_written)}
-        del w_pay
+        try:
+            L_, NB_ = ck.geom.n_layers, ck.n_blocks
+            w_off = torch.zeros((L_, NB_), dtype=torch.int64, device=dev)
+            w_lb = torch.zeros(L_, dtype=torch.int64, device=dev)
+            w_pay = torch.empty_like(st.payload)
+            w_ptrs = torch.tensor([w_pay.data_ptr() + o for o in ck.layer_off], dtype=torch.int64, device=dev)
+            w_sess = st.session(layer_payload=w_ptrs, blk_off=w_off, layer_bytes=w_lb)
+            ts_w = []
+            for i in range(13):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                ctx.plan_checkpoint(geom, ck.n_suffix_tokens, st.tags, w_off, w_lb, stream)
+                ctx.quantize_gather(geom, pool, w_sess, stream)
+                b.record(stream)
+                b.synchronize()
+                if i >= 3:
+                    ts_w.append(a.elapsed_time(b))
+            assert ctx.query_status() == 0 and torch.equal(w_off, st.blk_off)
+            t_w = statistics.median(ts_w)
+            pool_read = 2 * L_ * NB_ * ck.geom.block_tokens * ck.geom.n_kv_heads * ck.geom.head_dim * 2
+            pay_written = sum(ck.layer_bytes)
+            # the same checkpoint streamed to pinned host memory (encode layer l+1 while layer l is copied out)
+            cap_ = max(ck.layer_bytes)
+            hbufs = [torch.empty(cap_, dtype=torch.uint8).pin_memory() for _ in range(L_)]
+            hptrs = torch.tensor([h_.data_ptr() for h_ in hbufs], dtype=torch.int64)
+            hcaps = torch.full((L_,), cap_, dtype=torch.int64)
+            hsizes = torch.zeros(L_, dtype=torch.int64)
+            ts_h = []
+            for i in range(6):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                a.record(stream)
+                ctx.checkpoint_to_host(geom, pool, w_sess, hptrs, hcaps, hsizes, stream)
+                b.record(stream)
+                b.synchronize()
+                if i >= 2:
+                    ts_h.append(a.elapsed_time(b))
+            assert ctx.query_status() == 0 and int(hsizes.sum()) == pay_written
+            src_ = torch.empty(1 << 30, dtype=torch.uint8, device=dev)
+            dst_ = torch.empty(1 << 30, dtype=torch.uint8).pin_memory()
+            d2h_best = None
+            for i in range(6):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                dst_.copy_(src_, non_blocking=True)
+                b.record()
+                b.synchronize()
+                d2h_best = a.elapsed_time(b) if d2h_best is None else min(d2h_best, a.elapsed_time(b))
+            d2h_ceiling = (1 << 30) / (d2h_best * 1e-3) / 1e9
+            t_h = statistics.median(ts_h)
+            del hbufs, src_, dst_
+            writer = {"to_host": {"ms": t_h, "payload_gbps": pay_written / (t_h * 1e-3) / 1e9,
+                                  "d2h_ceiling_gbps": d2h_ceiling, "frac_of_link": pay_written / (t_h * 1e-3) / 1e9 / d2h_ceiling},
+                      "workload": "quantize_gather of all 1024 blocks x 32 layers of the same pool and tags",
+                      "ms": t_w, "real_gbps": (pool_read + pay_written) / (t_w * 1e-3) / 1e9,
+                      "frac_of_hbm_peak": (pool_read + pay_written) / (t_w * 1e-3) / 1e9 / peak,
+                      "bf16_gbps_read": pool_read / (t_w * 1e-3) / 1e9, "payload_bytes": int(pay_written)}
+            del w_pay
+        except Exception as exc:                          # an optional leg must not cost the bench line
+            if world > 1:
+                raise
+            writer = leg_failed(exc)
 
     # ---- end to end: host buffers, copies inside the timed region
     e2e = None
     host_link = None
     if not args.no_e2e:
-        ceiling = pinned_copy_ceiling(dev)
-        hst = StagedCheckpoint(ck, dev, payload_on_host=True)
-        mass_host = ck.mass.cpu().pin_memory()
-        idx_host = torch.empty_like(hst.reuse_idx, device="cpu").pin_memory()
-        cnt_host = torch.empty_like(hst.reuse_cnt, device="cpu").pin_memory()
-        hsel = hst.select_args(host_reuse_idx=idx_host, host_reuse_cnt=cnt_host, sync_to_host=True)
-        hs = hst.host_session(reuse_idx=idx_host, reuse_cnt=cnt_host)
-        dir_bytes = ck.tags.numel() + ck.blk_off.numel() * 8 + idx_host.numel() * 4 + cnt_host.numel() * 4 + \
-            ck.block_table.numel() * 4 + 16 * ck.geom.n_layers
-        e2e_steps = max(3, min(args.steps, 10))
-        times, copied = [], 0
-        for i in range(3 + e2e_steps):
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            torch.cuda.synchronize()
-            barrier(world)
-            a.record(stream)
-            hst.mass.copy_(mass_host, non_blocking=True)                 # stored block masses: host -> device
-            ctx.select_repair(hsel, stream)                               # lists also land in the pinned mirrors:
-            rc, stats = ctx.restore_from_host(geom, pool, [hs], stream)   # the host planner reads them
-            b.record(stream)
-            status = ctx.query_status()                                   # reads the device status word back
-            assert status == 0
-            if i >= 3:
-                times.append(max_over_ranks(a.elapsed_time(b), world, dev))
-                copied = stats.bytes_copied
-        e_ms = sum(times) / len(times)
-        e2e = {"value": world * written_b / (e_ms * 1e-3) / 1e9, "unit": UNIT,
-               "h2d_bytes_per_step": int(copied + mass_host.numel() * 8 + dir_bytes),
-               "d2h_bytes_per_step": int(idx_host.numel() * 4 + cnt_host.numel() * 4 + 4),
-               "ms_per_step": e_ms, "steps": len(times),
-               "path": "pinned masses H2D, select_repair with pinned host mirrors of the lists (D2H, waited for), "
-                       "restore_from_host (pinned payload), status D2H"}
-        host_link = {"ceiling_gbps": ceiling, "ceiling": "1 GiB pinned cudaMemcpyAsync H2D, best of 10, same run",
-                     "payload_gbps": read_b / (e_ms * 1e-3) / 1e9, "frac": read_b / (e_ms * 1e-3) / 1e9 / ceiling,
-                     "bytes_copied": int(copied), "bytes_useful": int(read_b), "copies": int(stats.n_copies)}
+        try:
+            ceiling = pinned_copy_ceiling(dev)
+            hst = StagedCheckpoint(ck, dev, payload_on_host=True)
+            mass_host = ck.mass.cpu().pin_memory()
+            idx_host = torch.empty_like(hst.reuse_idx, device="cpu").pin_memory()
+            cnt_host = torch.empty_like(hst.reuse_cnt, device="cpu").pin_memory()
+            hsel = hst.select_args(host_reuse_idx=idx_host, host_reuse_cnt=cnt_host, sync_to_host=True)
+            hs = hst.host_session(reuse_idx=idx_host, reuse_cnt=cnt_host)
+            dir_bytes = ck.tags.numel() + ck.blk_off.numel() * 8 + idx_host.numel() * 4 + cnt_host.numel() * 4 + \
+                ck.block_table.numel() * 4 + 16 * ck.geom.n_layers
+            e2e_steps = max(3, min(args.steps, 10))
+            times, copied = [], 0
+            for i in range(3 + e2e_steps):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                barrier(world)
+                a.record(stream)
+                hst.mass.copy_(mass_host, non_blocking=True)                 # stored block masses: host -> device
+                ctx.select_repair(hsel, stream)                               # lists also land in the pinned mirrors:
+                rc, stats = ctx.restore_from_host(geom, pool, [hs], stream)   # the host planner reads them
+                b.record(stream)
+                status = ctx.query_status()                                   # reads the device status word back
+                assert status == 0
+                if i >= 3:
+                    times.append(max_over_ranks(a.elapsed_time(b), world, dev))
+                    copied = stats.bytes_copied
+            e_ms = sum(times) / len(times)
+            e2e = {"value": world * written_b / (e_ms * 1e-3) / 1e9, "unit": UNIT,
+                   "h2d_bytes_per_step": int(copied + mass_host.numel() * 8 + dir_bytes),
+                   "d2h_bytes_per_step": int(idx_host.numel() * 4 + cnt_host.numel() * 4 + 4),
+                   "ms_per_step": e_ms, "steps": len(times),
+                   "path": "pinned masses H2D, select_repair with pinned host mirrors of the lists (D2H, waited for), "
+                           "restore_from_host (pinned payload), status D2H"}
+            host_link = {"ceiling_gbps": ceiling, "ceiling": "1 GiB pinned cudaMemcpyAsync H2D, best of 10, same run",
+                         "payload_gbps": read_b / (e_ms * 1e-3) / 1e9, "frac": read_b / (e_ms * 1e-3) / 1e9 / ceiling,
+                         "bytes_copied": int(copied), "bytes_useful": int(read_b), "copies": int(stats.n_copies)}
+        except Exception as exc:                          # an optional leg must not cost the bench line
+            if world > 1:
+                raise
+            e2e = leg_failed(exc)
 
     # ---- selection at scale: stored attention [32][32][64][16384] fp16 (2 GiB) -> masses -> lists
     select_scale = None
     if not args.no_scale_select:
-        torch.cuda.empty_cache()
-        gen = torch.Generator(device=dev)
-        gen.manual_seed(1004)
-        SL = args.scale_layers
-        attn = pin.zipf_attention(gen, SL, 32, 64, 16384, dev)
-        NBs = 1024
-        out = dict(repair_mask=torch.empty((SL, NBs), dtype=torch.uint8, device=dev),
-                   repair_idx=torch.empty((SL, NBs), dtype=torch.int32, device=dev),
-                   repair_cnt=torch.empty(SL, dtype=torch.int32, device=dev),
-                   reuse_idx=torch.empty((SL, NBs), dtype=torch.int32, device=dev),
-                   reuse_cnt=torch.empty(SL, dtype=torch.int32, device=dev))
-        mass_out = torch.empty((SL, NBs), dtype=torch.int64, device=dev)
-        sa = pk.select_args(kind=pk.SCORE_ATTN_F16, n_layers=SL, n_suffix_tokens=16384, block_tokens=16,
-                            dirty_tokens=640, top_k=32, layer_mode=pk.LAYERS_INDEPENDENT, attn=attn,
-                            mass_out=mass_out, **out)
-        ts = []
-        for i in range(13):
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            ctx.select_repair(sa, stream)
-            b.record(stream)
-            b.synchronize()
-            if i >= 3:
-                ts.append(a.elapsed_time(b))
-        assert ctx.query_status() == 0 and int(out["reuse_cnt"][0]) == 952
-        t_ms = statistics.median(ts)
-        nbytes = attn.numel() * 2
-        # the paper's token-level form from stored per-token scores: top 1.5 % of the suffix tokens, request-level
-        tmass = pin.zipf_block_mass(gen, SL, 16384, dev)
-        st_args = pk.select_args(kind=pk.SCORE_TOKEN_MASS, n_layers=SL, n_suffix_tokens=16384, block_tokens=16,
-                                 dirty_tokens=640, top_k=245, layer_mode=pk.LAYERS_SHARED, mass=tmass, **out)
-        tts = []
-        for i in range(13):
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            ctx.select_repair_tokens(st_args, stream)
-            b.record(stream)
-            b.synchronize()
-            if i >= 3:
-                tts.append(a.elapsed_time(b))
-        token_form_us = 1e3 * statistics.median(tts)
-        ta_args = pk.select_args(kind=pk.SCORE_ATTN_F16, n_layers=SL, n_suffix_tokens=16384, block_tokens=16,
-                                 dirty_tokens=640, top_k=245, layer_mode=pk.LAYERS_SHARED, attn=attn, **out)
-        tts2 = []
-        for i in range(9):
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            ctx.select_repair_tokens(ta_args, stream)
-            b.record(stream)
-            b.synchronize()
-            if i >= 3:
-                tts2.append(a.elapsed_time(b))
-        token_form_attn_us = 1e3 * statistics.median(tts2)
-        select_scale = {"token_form_us_from_token_scores": token_form_us,
-                        "token_form_us_from_attention": token_form_attn_us,
-                        "token_form_attn_gbps": attn.numel() * 2 / (token_form_attn_us * 1e-6) / 1e9,
-                        "workload": f"stored attention fp16 [{SL}][32][64][16384] ({SL * 64} MiB), 40-block dirty window, top-32 per layer",
-                        "select_us": 1e3 * t_ms, "attn_gbps": nbytes / (t_ms * 1e-3) / 1e9,
-                        "frac_of_hbm_peak": nbytes / (t_ms * 1e-3) / 1e9 / peak, "launches": 3}
-        del attn
-        if SL == ck.geom.n_layers:
-            # ... then the restore of the blocks that selection leaves to reuse (72 repaired / 952 reused per layer),
-            # on the same 8B-shaped payload and pool as the headline step
-            sa_lists = pk.select_args(kind=pk.SCORE_BLOCK_MASS, n_layers=SL, n_suffix_tokens=16384, block_tokens=16,
-                                      dirty_tokens=640, top_k=32, layer_mode=pk.LAYERS_INDEPENDENT, mass=mass_out, **out)
-            ctx.select_repair(sa_lists, stream)               # the lists of the block form, from the masses just computed
-            torch.cuda.synchronize()
-            sess4 = st.session(reuse_idx=out["reuse_idx"], reuse_cnt=out["reuse_cnt"])
-            r4, w4, items4 = algorithmic_bytes(ck, out["reuse_idx"].cpu().numpy(), out["reuse_cnt"].cpu().numpy())
-            ts4 = []
+        try:
+            torch.cuda.empty_cache()
+            gen = torch.Generator(device=dev)
+            gen.manual_seed(1004)
+            SL = args.scale_layers
+            attn = pin.zipf_attention(gen, SL, 32, 64, 16384, dev)
+            NBs = 1024
+            out = dict(repair_mask=torch.empty((SL, NBs), dtype=torch.uint8, device=dev),
+                       repair_idx=torch.empty((SL, NBs), dtype=torch.int32, device=dev),
+                       repair_cnt=torch.empty(SL, dtype=torch.int32, device=dev),
+                       reuse_idx=torch.empty((SL, NBs), dtype=torch.int32, device=dev),
+                       reuse_cnt=torch.empty(SL, dtype=torch.int32, device=dev))
+            mass_out = torch.empty((SL, NBs), dtype=torch.int64, device=dev)
+            sa = pk.select_args(kind=pk.SCORE_ATTN_F16, n_layers=SL, n_suffix_tokens=16384, block_tokens=16,
+                                dirty_tokens=640, top_k=32, layer_mode=pk.LAYERS_INDEPENDENT, attn=attn,
+                                mass_out=mass_out, **out)
+            ts = []
             for i in range(13):
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 a.record(stream)
-                ctx.restore(geom, pool, [sess4], stream)
+                ctx.select_repair(sa, stream)
                 b.record(stream)
                 b.synchronize()
                 if i >= 3:
-                    ts4.append(a.elapsed_time(b))
-            assert ctx.query_status() == 0
-            r_ms = statistics.median(ts4)
-            select_scale["restore_of_its_reuse_set"] = {
-                "ms": r_ms, "block_layers": int(items4), "restored_kv_gbps_bf16_equiv": w4 / (r_ms * 1e-3) / 1e9,
-                "real_gbps": (r4 + w4) / (r_ms * 1e-3) / 1e9, "frac_of_hbm_peak": (r4 + w4) / (r_ms * 1e-3) / 1e9 / peak}
+                    ts.append(a.elapsed_time(b))
+            assert ctx.query_status() == 0 and int(out["reuse_cnt"][0]) == 952
+            t_ms = statistics.median(ts)
+            nbytes = attn.numel() * 2
+            # the paper's token-level form from stored per-token scores: top 1.5 % of the suffix tokens, request-level
+            tmass = pin.zipf_block_mass(gen, SL, 16384, dev)
+            st_args = pk.select_args(kind=pk.SCORE_TOKEN_MASS, n_layers=SL, n_suffix_tokens=16384, block_tokens=16,
+                                     dirty_tokens=640, top_k=245, layer_mode=pk.LAYERS_SHARED, mass=tmass, **out)
+            tts = []
+            for i in range(13):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                ctx.select_repair_tokens(st_args, stream)
+                b.record(stream)
+                b.synchronize()
+                if i >= 3:
+                    tts.append(a.elapsed_time(b))
+            token_form_us = 1e3 * statistics.median(tts)
+            ta_args = pk.select_args(kind=pk.SCORE_ATTN_F16, n_layers=SL, n_suffix_tokens=16384, block_tokens=16,
+                                     dirty_tokens=640, top_k=245, layer_mode=pk.LAYERS_SHARED, attn=attn, **out)
+            tts2 = []
+            for i in range(9):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                ctx.select_repair_tokens(ta_args, stream)
+                b.record(stream)
+                b.synchronize()
+                if i >= 3:
+                    tts2.append(a.elapsed_time(b))
+            token_form_attn_us = 1e3 * statistics.median(tts2)
+            select_scale = {"token_form_us_from_token_scores": token_form_us,
+                            "token_form_us_from_attention": token_form_attn_us,
+                            "token_form_attn_gbps": attn.numel() * 2 / (token_form_attn_us * 1e-6) / 1e9,
+                            "workload": f"stored attention fp16 [{SL}][32][64][16384] ({SL * 64} MiB), 40-block dirty window, top-32 per layer",
+                            "select_us": 1e3 * t_ms, "attn_gbps": nbytes / (t_ms * 1e-3) / 1e9,
+                            "frac_of_hbm_peak": nbytes / (t_ms * 1e-3) / 1e9 / peak, "launches": 3}
+            del attn
+            if SL == ck.geom.n_layers:
+                # ... then the restore of the blocks that selection leaves to reuse (72 repaired / 952 reused per layer),
+                # on the same 8B-shaped payload and pool as the headline step
+                sa_lists = pk.select_args(kind=pk.SCORE_BLOCK_MASS, n_layers=SL, n_suffix_tokens=16384, block_tokens=16,
+                                          dirty_tokens=640, top_k=32, layer_mode=pk.LAYERS_INDEPENDENT, mass=mass_out, **out)
+                ctx.select_repair(sa_lists, stream)               # the lists of the block form, from the masses just computed
+                torch.cuda.synchronize()
+                sess4 = st.session(reuse_idx=out["reuse_idx"], reuse_cnt=out["reuse_cnt"])
+                r4, w4, items4 = algorithmic_bytes(ck, out["reuse_idx"].cpu().numpy(), out["reuse_cnt"].cpu().numpy())
+                ts4 = []
+                for i in range(13):
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record(stream)
+                    ctx.restore(geom, pool, [sess4], stream)
+                    b.record(stream)
+                    b.synchronize()
+                    if i >= 3:
+                        ts4.append(a.elapsed_time(b))
+                assert ctx.query_status() == 0
+                r_ms = statistics.median(ts4)
+                select_scale["restore_of_its_reuse_set"] = {
+                    "ms": r_ms, "block_layers": int(items4), "restored_kv_gbps_bf16_equiv": w4 / (r_ms * 1e-3) / 1e9,
+                    "real_gbps": (r4 + w4) / (r_ms * 1e-3) / 1e9, "frac_of_hbm_peak": (r4 + w4) / (r_ms * 1e-3) / 1e9 / peak}
+        except Exception as exc:                          # an optional leg must not cost the bench line
+            if world > 1:
+                raise
+            select_scale = leg_failed(exc)
 
     # ---- the two host-resident workloads: 7B-shaped / 4 KV heads (one session), 70B-shaped stress (8 sessions)
     host_cfg3 = stress = None
     if not args.no_host_configs:
-        ceiling = pinned_copy_ceiling(dev)
-
-        ctx_direct = pk.Context(device=local_rank, flags=pk.FLAG_HOST_DIRECT)
-
-        def host_leg(cks, label, reps=5, both=False):
-            out_ = host_leg_on(ctx, cks, label, reps)
-            if both:     # the same through the zero-copy variant: the kernel pulls the records over the link itself
-                d_ = host_leg_on(ctx_direct, cks, label, reps)
-                out_["zero_copy"] = {k_: d_[k_] for k_ in ("ms", "payload_gbps", "frac_of_link", "bytes_copied", "copies")}
-            return out_
-
-        def host_leg_on(ctx, cks, label, reps=5):
-            sts = [StagedCheckpoint(c, dev, payload_on_host=True) for c in cks]
-            for s_ in sts:
-                ctx.select_repair(s_.select_args(), stream)
-            torch.cuda.synchronize()
-            hk, hv, hpool = device_pool(cks[0], dev)
-            hgeom = sts[0].geom()
-            hss = [s_.host_session() for s_ in sts]
-            useful = written = items_h = 0
-            for c, s_ in zip(cks, sts):
-                r_, w_, i_ = algorithmic_bytes(c, s_.reuse_idx.cpu().numpy(), s_.reuse_cnt.cpu().numpy())
-                useful, written, items_h = useful + r_, written + w_, items_h + i_
-            ts_, stats_ = [], None
-            for i in range(2 + reps):
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                torch.cuda.synchronize()
-                a.record(stream)
-                rc_, stats_ = ctx.restore_from_host(hgeom, hpool, hss, stream)
-                b.record(stream)
-                b.synchronize()
-                if i >= 2:
-                    ts_.append(a.elapsed_time(b))
-            assert ctx.query_status() == 0 and stats_.bytes_useful == useful
-            t_ms = statistics.median(ts_)
-            out_ = {"workload": label, "ms": t_ms, "restored_kv_gbps_bf16_equiv": written / (t_ms * 1e-3) / 1e9,
-                    "payload_gbps": useful / (t_ms * 1e-3) / 1e9, "link_ceiling_gbps": ceiling,
-                    "frac_of_link": useful / (t_ms * 1e-3) / 1e9 / ceiling, "bytes_useful": int(useful),
-                    "bytes_copied": int(stats_.bytes_copied), "copies": int(stats_.n_copies),
-                    "block_layers": int(items_h), "block_layers_per_s": items_h / (t_ms * 1e-3)}
-            del sts, hk, hv, hss
-            torch.cuda.empty_cache()
-            return out_
-
         try:
-            del st, k, v
-        except NameError:
-            pass
-        torch.cuda.empty_cache()
-        c3 = pin.config_7b_host(device=dev, pin_payload=True)
-        host_cfg3 = host_leg([c3], "7b-shaped: L=28 H=4 D=128 base=1e6 n=32768 delta=-3000, pinned host payload, "
-                                   "4096-page pool (2x), shuffled free list", both=True)
-        del c3
-        SLy = args.stress_layers
-        waves = []
-        for w_ in range(args.stress_waves):          # each wave: SLy of the 80 layers, payload regenerated outside the timed region
-            sess = [pin.config_stress_session(i, device=dev, n_layers=SLy, pin_payload=True, seed=1005 + 17 * i + 1000 * w_)
-                    for i in range(8)]
-            pin.shared_free_list(1005, 8 * 4096, sess)
-            waves.append(host_leg(sess, "", reps=3, both=(w_ == 0)))
-            if w_ + 1 < args.stress_waves:
-                del sess
-        stress = dict(waves[0])
-        stress["workload"] = (f"70b-shaped stress: 8 sessions x 64k-token suffix, H=8 D=128, int4 share 10-60 %, one shared pool "
-                              f"of 32768 pages, pinned host payload; {SLy} of 80 layers resident per wave, {len(waves)} wave(s) "
-                              f"timed (fit rule: the 80-layer pool is 172 GB and its payload 103 GB of pinned memory)")
-        if len(waves) > 1:
-            tot_ms = sum(w["ms"] for w in waves)
-            tot_useful = sum(w["bytes_useful"] for w in waves)
-            stress.update(ms=tot_ms, bytes_useful=tot_useful, layers_covered=SLy * len(waves),
-                          payload_gbps=tot_useful / (tot_ms * 1e-3) / 1e9,
-                          frac_of_link=tot_useful / (tot_ms * 1e-3) / 1e9 / waves[0]["link_ceiling_gbps"],
-                          block_layers=sum(w["block_layers"] for w in waves),
-                          restored_kv_gbps_bf16_equiv=sum(w["restored_kv_gbps_bf16_equiv"] * w["ms"] for w in waves) / tot_ms)
-        del sess
+            ceiling = pinned_copy_ceiling(dev)
+
+            ctx_direct = pk.Context(device=local_rank, flags=pk.FLAG_HOST_DIRECT)
+
+            def host_leg(cks, label, reps=5, both=False):
+                out_ = host_leg_on(ctx, cks, label, reps)
+                if both:     # the same through the zero-copy variant: the kernel pulls the records over the link itself
+                    d_ = host_leg_on(ctx_direct, cks, label, reps)
+                    out_["zero_copy"] = {k_: d_[k_] for k_ in ("ms", "payload_gbps", "frac_of_link", "bytes_copied", "copies")}
+                return out_
+
+            def host_leg_on(ctx, cks, label, reps=5):
+                sts = [StagedCheckpoint(c, dev, payload_on_host=True) for c in cks]
+                for s_ in sts:
+                    ctx.select_repair(s_.select_args(), stream)
+                torch.cuda.synchronize()
+                hk, hv, hpool = device_pool(cks[0], dev)
+                hgeom = sts[0].geom()
+                hss = [s_.host_session() for s_ in sts]
+                useful = written = items_h = 0
+                for c, s_ in zip(cks, sts):
+                    r_, w_, i_ = algorithmic_bytes(c, s_.reuse_idx.cpu().numpy(), s_.reuse_cnt.cpu().numpy())
+                    useful, written, items_h = useful + r_, written + w_, items_h + i_
+                ts_, stats_ = [], None
+                for i in range(2 + reps):
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    torch.cuda.synchronize()
+                    a.record(stream)
+                    rc_, stats_ = ctx.restore_from_host(hgeom, hpool, hss, stream)
+                    b.record(stream)
+                    b.synchronize()
+                    if i >= 2:
+                        ts_.append(a.elapsed_time(b))
+                assert ctx.query_status() == 0 and stats_.bytes_useful == useful
+                t_ms = statistics.median(ts_)
+                out_ = {"workload": label, "ms": t_ms, "restored_kv_gbps_bf16_equiv": written / (t_ms * 1e-3) / 1e9,
+                        "payload_gbps": useful / (t_ms * 1e-3) / 1e9, "link_ceiling_gbps": ceiling,
+                        "frac_of_link": useful / (t_ms * 1e-3) / 1e9 / ceiling, "bytes_useful": int(useful),
+                        "bytes_copied": int(stats_.bytes_copied), "copies": int(stats_.n_copies),
+                        "block_layers": int(items_h), "block_layers_per_s": items_h / (t_ms * 1e-3)}
+                del sts, hk, hv, hss
+                torch.cuda.empty_cache()
+                return out_
+
+            try:
+                del st, k, v
+            except NameError:
+                pass
+            torch.cuda.empty_cache()
+            c3 = pin.config_7b_host(device=dev, pin_payload=True)
+            host_cfg3 = host_leg([c3], "7b-shaped: L=28 H=4 D=128 base=1e6 n=32768 delta=-3000, pinned host payload, "
+                                       "4096-page pool (2x), shuffled free list", both=True)
+            del c3
+            SLy = args.stress_layers
+            waves = []
+            for w_ in range(args.stress_waves):          # each wave: SLy of the 80 layers, payload regenerated outside the timed region
+                sess = [pin.config_stress_session(i, device=dev, n_layers=SLy, pin_payload=True, seed=1005 + 17 * i + 1000 * w_)
+                        for i in range(8)]
+                pin.shared_free_list(1005, 8 * 4096, sess)
+                waves.append(host_leg(sess, "", reps=3, both=(w_ == 0)))
+                if w_ + 1 < args.stress_waves:
+                    del sess
+            stress = dict(waves[0])
+            stress["workload"] = (f"70b-shaped stress: 8 sessions x 64k-token suffix, H=8 D=128, int4 share 10-60 %, one shared pool "
+                                  f"of 32768 pages, pinned host payload; {SLy} of 80 layers resident per wave, {len(waves)} wave(s) "
+                                  f"timed (fit rule: the 80-layer pool is 172 GB and its payload 103 GB of pinned memory)")
+            if len(waves) > 1:
+                tot_ms = sum(w["ms"] for w in waves)
+                tot_useful = sum(w["bytes_useful"] for w in waves)
+                stress.update(ms=tot_ms, bytes_useful=tot_useful, layers_covered=SLy * len(waves),
+                              payload_gbps=tot_useful / (tot_ms * 1e-3) / 1e9,
+                              frac_of_link=tot_useful / (tot_ms * 1e-3) / 1e9 / waves[0]["link_ceiling_gbps"],
+                              block_layers=sum(w["block_layers"] for w in waves),
+                              restored_kv_gbps_bf16_equiv=sum(w["restored_kv_gbps_bf16_equiv"] * w["ms"] for w in waves) / tot_ms)
+            del sess
+        except Exception as exc:                          # an optional leg must not cost the bench line
+            if world > 1:
+                raise
+            host_cfg3 = leg_failed(exc)
 
     # ---- the paper's restore microbenchmark shape (Section V-E): an ~8k-token checkpoint of a 64-layer, 8-KV-head,
     #      head_dim-128 model (geometry from the public Qwen3-32B model card, not from the paper), 32-token blocks,
     #      one fp16 scale per 128 channels, restored whole from pinned host memory in each transport format
     paper_shape = None
     if not args.no_host_configs:
-        gm = pin.Geometry(64, 8, 128, 128, pin.ROPE_HALF, 1.0e6, 32, 32, 128)
-        rows = {}
-        for label, probs in (("FP16(bf16)", (1.0, 0, 0, 0)), ("INT8 K8/V8", (0, 1.0, 0, 0)), ("INT4 K4/V4", (0, 0, 0, 1.0)),
-                             ("mixed 2/6/92 % bf16/K8V8/K8V4", (0.02, 0.06, 0.92, 0.0))):
-            cm = pin.make_checkpoint(name="paper-microbench", seed=2024, geom=gm, n=8031, delta=-512, tag_probs=probs,
-                                     n_outlier=6, outlier_scale=10.0, n_pages=256, dirty_tokens=0, top_k=0,
-                                     device=dev, pin_payload=True)
-            r_ = host_leg([cm], label, reps=5)
-            rows[label] = {"payload_mib": r_["bytes_useful"] / 2 ** 20, "fetch_and_restore_ms": r_["ms"],
-                           "payload_gbps": r_["payload_gbps"], "frac_of_link": r_["frac_of_link"], "copies": r_["copies"]}
-            del cm
-        paper_shape = {"workload": "8031-token checkpoint, L=64 H=8 D=128, B=P=32, G=128, every block restored from pinned host",
-                       "formats": rows,
-                       "paper_context_ms": {"FP16": 344.4, "INT8": 183.6, "INT4": 107.2, "PatchKV": 158.0,
-                                            "hardware": "A800 server, PCIe Gen4, 23.3 GiB/s pinned ceiling"}}
+        try:
+            gm = pin.Geometry(64, 8, 128, 128, pin.ROPE_HALF, 1.0e6, 32, 32, 128)
+            rows = {}
+            for label, probs in (("FP16(bf16)", (1.0, 0, 0, 0)), ("INT8 K8/V8", (0, 1.0, 0, 0)), ("INT4 K4/V4", (0, 0, 0, 1.0)),
+                                 ("mixed 2/6/92 % bf16/K8V8/K8V4", (0.02, 0.06, 0.92, 0.0))):
+                cm = pin.make_checkpoint(name="paper-microbench", seed=2024, geom=gm, n=8031, delta=-512, tag_probs=probs,
+                                         n_outlier=6, outlier_scale=10.0, n_pages=256, dirty_tokens=0, top_k=0,
+                                         device=dev, pin_payload=True)
+                r_ = host_leg([cm], label, reps=5)
+                rows[label] = {"payload_mib": r_["bytes_useful"] / 2 ** 20, "fetch_and_restore_ms": r_["ms"],
+                               "payload_gbps": r_["payload_gbps"], "frac_of_link": r_["frac_of_link"], "copies": r_["copies"]}
+                del cm
+            paper_shape = {"workload": "8031-token checkpoint, L=64 H=8 D=128, B=P=32, G=128, every block restored from pinned host",
+                           "formats": rows,
+                           "paper_context_ms": {"FP16": 344.4, "INT8": 183.6, "INT4": 107.2, "PatchKV": 158.0,
+                                                "hardware": "A800 server, PCIe Gen4, 23.3 GiB/s pinned ceiling"}}
+        except Exception as exc:                          # an optional leg must not cost the bench line
+            if world > 1:
+                raise
+            paper_shape = leg_failed(exc)
 
     # ---- CPU baseline: the checker, as it stands, on a bounded sample of the same workload (rank 0, N = 1)
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu:
-        import oracle
-        oracle.build()
-        sample_layers = list(range(ck.geom.n_layers))
-        dt, wb, threads = oracle_sample(ck, sample_layers, repeats=3)
-        one_layers = sample_layers[:min(4, len(sample_layers))]
-        dt1, wb1, _ = oracle_sample(ck, one_layers, repeats=1, threads=1)
-        cpu_baseline = {"value": wb / dt / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
-                        "sample": f"all {len(sample_layers)} layers of the workload (select + restore), best of 3 passes "
-                                  f"of {dt:.2f} s on {threads} threads",
-                        "single_thread": {"value": wb1 / dt1 / 1e9, "unit": UNIT,
-                                          "sample": f"{len(one_layers)} layers, one pass of {dt1:.2f} s on 1 thread"}}
+        try:
+            import oracle
+            oracle.build()
+            sample_layers = list(range(ck.geom.n_layers))
+            dt, wb, threads = oracle_sample(ck, sample_layers, repeats=3)
+            one_layers = sample_layers[:min(4, len(sample_layers))]
+            dt1, wb1, _ = oracle_sample(ck, one_layers, repeats=1, threads=1)
+            cpu_baseline = {"value": wb / dt / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
+                            "sample": f"all {len(sample_layers)} layers of the workload (select + restore), best of 3 passes "
+                                      f"of {dt:.2f} s on {threads} threads",
+                            "single_thread": {"value": wb1 / dt1 / 1e9, "unit": UNIT,
+                                              "sample": f"{len(one_layers)} layers, one pass of {dt1:.2f} s on 1 thread"}}
+        except Exception as exc:                          # an optional leg must not cost the bench line
+            if world > 1:
+                raise
+            cpu_baseline = leg_failed(exc)
 
     if rank == 0:
         line = {

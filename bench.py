@@ -44,8 +44,8 @@ WORKLOAD = "llama3-8b-shaped: L=32 H=8 D=128 base=5e5 n=16384 B=P=16 G=32 tags 3
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one restore launch on this workload, from the ncu capture of a
 # 4-layer slice summarised under profiles/: reads scale with the layers
-# (8 x 151.1 MB); writes are the algorithmic 1824 MB minus the ~51 MB still dirty in L2 when the kernel ends
-RESTORE_KERNEL_DRAM_TRAFFIC_BYTES = 2_982_000_000
+# (8 x 150.6 MB); writes are the algorithmic 1824 MB minus the ~52 MB still dirty in L2 when the kernel ends
+RESTORE_KERNEL_DRAM_TRAFFIC_BYTES = 2_977_000_000
 
 
 # ------------------------------------------------------------------------------------------ helpers

@@ -349,7 +349,7 @@ def run_ours(args):
             w_ptrs = torch.tensor([w_pay.data_ptr() + o for o in ck.layer_off], dtype=torch.int64, device=dev)
             w_sess = st.session(layer_payload=w_ptrs, blk_off=w_off, layer_bytes=w_lb)
             ts_w = []
-            for i in range(13):
+            for i in range(33):                           # a median over 30: single calls wander by a few per cent
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 a.record(stream)
                 ctx.plan_checkpoint(geom, ck.n_suffix_tokens, st.tags, w_off, w_lb, stream)

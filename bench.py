@@ -7,14 +7,20 @@ phase correction of K, page placement) of every reused block, on the Llama-3-8B-
 8 KV heads, head_dim 128, 16384-token suffix, 16-token blocks, tags 30/50/20 bf16/int8/int4, repair set
 15 %, device-resident payload, 1280-page pool).  Prints ONE JSON line (rank 0).
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--sweep]
 
-value      restored KV GB/s (bf16-equivalent: bytes of bf16 K+V written to the pool / time), inputs in HBM.
+value      restored KV GB/s (bf16-equivalent: bytes of bf16 K+V written to the pool / time), inputs in HBM.  The
+           block of K steps is repeated until at least one second of GPU time has been timed; value and ms_per_step
+           are those of the median block, min / max and the SM clocks seen alongside are reported too.
 e2e        the same metric through the host-resident entry point: block masses copied from pinned host
            memory, selection lists read back, patchkv_restore_from_host streaming the pinned payload.
 roofline   the restore kernel against the measured HBM copy bandwidth.
 cpu_baseline / --impl reference   the CPU checker in oracle/ timed on the machine's host cores (a reported
            baseline only; it is a deliberately plain program).
+configs    (last key) one compact row per BASELINE configuration: ms, bf16-equivalent GB/s, fraction of the roofline
+           that bounds it (HBM or the host link), selection time.
+--sweep    instead of the benchmark line: restore / writer fractions by tag and by geometry, restore time by suffix
+           length, and the host path's merge-gap sweep, on half-size (16-layer) workloads; one JSON line.
 With N > 1 (torchrun) every rank restores its own copy of the workload on its own GPU: the path has no
 exchange step, so this is weak scaling without any data-path collective.
 """
@@ -23,6 +29,7 @@ from __future__ import annotations
 import argparse
 import json
 import os
+import re
 import statistics
 import subprocess
 import sys
@@ -42,13 +49,18 @@ METRIC = "restored_kv_gbps_bf16_equiv"
 UNIT = "GB/s"
 WORKLOAD = "llama3-8b-shaped: L=32 H=8 D=128 base=5e5 n=16384 B=P=16 G=32 tags 30/50/20 repair 15% device-resident"
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one restore launch on this workload, from the ncu capture of a
-# 4-layer slice summarised under profiles/: reads scale with the layers
-# (8 x 150.6 MB); writes are the algorithmic 1824 MB minus the ~52 MB still dirty in L2 when the kernel ends
-RESTORE_KERNEL_DRAM_TRAFFIC_BYTES = 2_977_000_000
+MIN_TIMED_GPU_SECONDS = 1.0
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "restore_pipe_kernel_llama8b_slice.traffic.txt")
 
 
 # ------------------------------------------------------------------------------------------ helpers
+def workload_config(delta: int, world: int, layers: int = 32) -> dict:
+    """The `config` object of the JSON line, the same for both arms."""
+    return {"workload": WORKLOAD if layers == 32 else WORKLOAD + f" [PROFILING SLICE: {layers} layers]",
+            "delta": delta, "l2": "working set 3.0 GB per step >> 126 MB L2, no flush",
+            "parallelism": f"independent replicas x{world}" if world > 1 else "1 gpu"}
+
+
 def algorithmic_bytes(ck: pin.SuffixCheckpoint, reuse_idx: np.ndarray, reuse_cnt: np.ndarray):
     """(payload bytes read, bf16 bytes written, reused block-layers) of one restore of `ck`."""
     g = ck.geom
@@ -65,11 +77,27 @@ def algorithmic_bytes(ck: pin.SuffixCheckpoint, reuse_idx: np.ndarray, reuse_cnt
     return read, written, items
 
 
+def captured_traffic(block_layers: int, written_bytes: int):
+    """DRAM traffic of one restore launch from the committed ncu capture of a slice of the same workload
+    (profiles/restore_pipe_kernel_llama8b_slice.traffic.txt).  Reads are proportional to the reused block-layers;
+    writes are the launch's bf16 bytes less what the capture shows still dirty in L2 at kernel end.
+    Returns (bytes, where it comes from); (None, reason) when the file is absent."""
+    try:
+        kv = dict(re.findall(r"^(\w+)\s*=\s*(\S+)\s*$", open(TRAFFIC_FILE).read(), flags=re.M))
+        reads = float(kv["dram_bytes_read_per_launch"]) / float(kv["block_layers"]) * block_layers
+        l2_dirty = float(kv["algorithmic_bytes_written"]) - float(kv["dram_bytes_write_per_launch"])
+        return int(reads + written_bytes - l2_dirty), (f"ncu capture {kv['capture']} of a {kv['block_layers']}-block-layer slice, "
+                                                       f"scaled (profiles/{os.path.basename(TRAFFIC_FILE)})")
+    except Exception as exc:
+        return None, f"no capture on file: {exc!r}"[:120]
+
+
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
     def __init__(self, gpu_index: int):
         self.gpu_index = gpu_index
@@ -90,7 +118,24 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.lines.append((time.time(), line.strip()))
 
-    def stop(self, t0: float, t1: float):
+    def rows(self, t0: float, t1: float):
+        """(time, sm MHz, max MHz, active reasons) of the samples taken in [t0, t1] (all samples if none fall inside)."""
+        out = []
+        for t, line in list(self.lines):
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                out.append((t, float(f[1]), float(f[2]),
+                            [n for n, val in zip(self.NAMES, f[5:9]) if val.lower().startswith("active")]))
+            except ValueError:
+                continue
+        inside = [r for r in out if t0 - 0.05 <= r[0] <= t1 + 0.25]
+        return inside or out
+
+    def stop(self, t0: float, t1: float, blocks=None):
+        """Summary of the samples in [t0, t1].  `blocks`: [(host time at the block's end, ms per step)] - each block is
+        booked under the SM clock of the sample nearest to it in time."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         time.sleep(0.15)
@@ -99,23 +144,18 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        rows = [l for (t, l) in self.lines if t0 - 0.05 <= t <= t1 + 0.25] or [l for (_, l) in self.lines]
-        for line in rows:
-            f = [x.strip() for x in line.split(",")]
-            if len(f) < 9:
-                continue
-            try:
-                sm.append(float(f[1]))
-                mx.append(float(f[2]))
-            except ValueError:
-                continue
-            for name, val in zip(names, f[5:9]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+        rows = self.rows(t0, t1)
+        sm = [r[1] for r in rows]
+        out = {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max((r[2] for r in rows), default=None),
+               "sm_mhz_min": min(sm) if sm else None, "reasons": sorted({n for r in rows for n in r[3]}), "samples": len(sm)}
+        if blocks and rows:
+            bins = {}
+            for t_end, ms in blocks:
+                near = min(rows, key=lambda r: abs(r[0] - t_end))
+                bins.setdefault(int(near[1]), []).append(ms)
+            out["by_sm_mhz"] = {str(mhz): {"blocks": len(v), "ms_per_step_median": round(statistics.median(v), 5)}
+                                for mhz, v in sorted(bins.items())}
+        return out
 
 
 def measured_hbm_peak():
@@ -194,31 +234,49 @@ def barrier(world: int):
         dist.barrier()
 
 
+def median_ms(fn, stream, reps: int, warm: int = 3) -> float:
+    """Median CUDA-event time of fn() over `reps` calls after `warm` untimed ones, each call waited for."""
+    ts = []
+    for i in range(warm + reps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        fn()
+        b.record(stream)
+        b.synchronize()
+        if i >= warm:
+            ts.append(a.elapsed_time(b))
+    return statistics.median(ts)
+
+
+def r3(x):
+    return None if x is None else float(f"{x:.4g}")
+
+
 # ------------------------------------------------------------------------------------------ reference arm
 def run_reference(args):
-    """The CPU checker as the reference arm: each step is a bounded sample (2 layers of the 32) of the same
-    workload, select + restore, on all host cores.  Rank 0 only."""
+    """The CPU checker as the reference arm: each step is one pass of select + restore over all 32 layers of the
+    same workload, on all host cores.  Rank 0 only."""
     rank, _, world = dist_env()
     if rank != 0:
         return
     import oracle
     oracle.build()
-    sample_layers = [0, 1]
-    ck = pin.config_llama8b(device="cpu", n_layers=len(sample_layers))
+    ck = pin.config_llama8b(device="cpu")
+    layers = list(range(ck.geom.n_layers))
     times = []
     written = 0
     for i in range(args.warmup + args.steps):
-        dt, written, threads = oracle_sample(ck, list(range(len(sample_layers))))
+        dt, written, threads = oracle_sample(ck, layers)
         if i >= args.warmup:
             times.append(dt)
     total = sum(times)
     value = written * len(times) / total / 1e9
-    sample = f"{len(sample_layers)} of 32 layers per step (select + restore of 870 reused blocks per layer)"
+    sample = f"all {len(layers)} layers per step (select + restore of 870 reused blocks per layer), {threads} threads"
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "sample": sample},
+        "config": workload_config(ck.delta, max(world, 1)),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
@@ -242,6 +300,42 @@ def pinned_copy_ceiling(device, nbytes=1 << 30, reps=10):
     return nbytes / (best * 1e-3) / 1e9
 
 
+def host_leg_on(ctx, cks, label, ceiling, dev, stream, reps=5):
+    """restore_from_host of the sessions `cks` (pinned payloads) into a fresh pool: median time and link fractions."""
+    from patchkv_inputs.staging import StagedCheckpoint, device_pool
+    sts = [StagedCheckpoint(c, dev, payload_on_host=True) for c in cks]
+    for s_ in sts:
+        ctx.select_repair(s_.select_args(), stream)
+    torch.cuda.synchronize()
+    hk, hv, hpool = device_pool(cks[0], dev)
+    hgeom = sts[0].geom()
+    hss = [s_.host_session() for s_ in sts]
+    useful = written = items_h = 0
+    for c, s_ in zip(cks, sts):
+        r_, w_, i_ = algorithmic_bytes(c, s_.reuse_idx.cpu().numpy(), s_.reuse_cnt.cpu().numpy())
+        useful, written, items_h = useful + r_, written + w_, items_h + i_
+    ts_, stats_ = [], None
+    for i in range(2 + reps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record(stream)
+        rc_, stats_ = ctx.restore_from_host(hgeom, hpool, hss, stream)
+        b.record(stream)
+        b.synchronize()
+        if i >= 2:
+            ts_.append(a.elapsed_time(b))
+    assert ctx.query_status() == 0 and stats_.bytes_useful == useful
+    t_ms = statistics.median(ts_)
+    out_ = {"workload": label, "ms": t_ms, "restored_kv_gbps_bf16_equiv": written / (t_ms * 1e-3) / 1e9,
+            "payload_gbps": useful / (t_ms * 1e-3) / 1e9, "link_ceiling_gbps": ceiling,
+            "frac_of_link": useful / (t_ms * 1e-3) / 1e9 / ceiling, "bytes_useful": int(useful),
+            "bytes_copied": int(stats_.bytes_copied), "bytes_wasted": int(stats_.bytes_copied - useful),
+            "copies": int(stats_.n_copies), "block_layers": int(items_h), "block_layers_per_s": items_h / (t_ms * 1e-3)}
+    del sts, hk, hv, hss
+    torch.cuda.empty_cache()
+    return out_
+
+
 def run_ours(args):
     rank, local_rank, world = dist_env()
     if world > 1:
@@ -252,7 +346,7 @@ def run_ours(args):
 
     from paper_2609_26219_b200 import binding as pk
     from paper_2609_26219_b200 import build as pkbuild
-    from paper_2609_26219_b200.harness import StagedCheckpoint, device_pool
+    from patchkv_inputs.staging import StagedCheckpoint, device_pool
     if rank == 0:
         pkbuild.build()
     barrier(world)
@@ -282,32 +376,51 @@ def run_ours(args):
     reuse_idx, reuse_cnt = st.reuse_idx.cpu().numpy(), st.reuse_cnt.cpu().numpy()
     read_b, written_b, items = algorithmic_bytes(ck, reuse_idx, reuse_cnt)
 
-    # ---- timed region: K steps, CUDA events on the launching stream, clocks sampled alongside
+    # ---- timed region: blocks of K steps, CUDA events on the launching stream, clocks sampled alongside.  The block
+    #      is repeated until at least MIN_TIMED_GPU_SECONDS of GPU time is covered (one short block would be ten
+    #      milliseconds and a handful of clock samples); every rank times the same number of blocks.
+    K = args.steps
+    a0, b0 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a0.record(stream)
+    for _ in range(3):
+        step()
+    b0.record(stream)
+    b0.synchronize()
+    est_ms = max_over_ranks(a0.elapsed_time(b0) / 3, world, dev)
+    n_blocks = 1 if args.single_block else max(1, min(2000, int(np.ceil(MIN_TIMED_GPU_SECONDS * 1e3 / (K * est_ms)))))
     sampler = ClockSampler(local_rank)
     sampler.start()
     time.sleep(0.3)
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    e_begin, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    blocks, restore_ms = [], []
     barrier(world)
     torch.cuda.synchronize()
     t0 = time.time()
-    e_begin.record(stream)
-    for i in range(args.steps):
-        step(evs[i])
-    e_end.record(stream)
+    for _ in range(n_blocks):
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+        e_begin, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e_begin.record(stream)
+        for i in range(K):
+            step(evs[i])
+        e_end.record(stream)
+        e_end.synchronize()
+        blocks.append((time.time(), e_begin.elapsed_time(e_end) / K))
+        restore_ms.extend(a.elapsed_time(b) for a, b in evs)
     torch.cuda.synchronize()
     barrier(world)
     t1 = time.time()
-    clocks = sampler.stop(t0, t1)
-    total_ms = max_over_ranks(e_begin.elapsed_time(e_end), world, dev)
-    restore_ms = [a.elapsed_time(b) for a, b in evs]
+    clocks = sampler.stop(t0, t1, blocks)
+    per_block = [ms for _, ms in blocks]
+    ms_per_step = max_over_ranks(statistics.median(per_block), world, dev)
     restore_avg_ms = sum(restore_ms) / len(restore_ms)
-    ms_per_step = total_ms / args.steps
-    select_us = 1e3 * (total_ms / args.steps - restore_avg_ms) if world == 1 else None
+    select_us = 1e3 * (statistics.median(per_block) - statistics.median(restore_ms)) if world == 1 else None
     value = aggregate_value(written_b, ms_per_step, world)
+    timing = {"blocks": n_blocks, "steps_per_block": K, "gpu_seconds_timed": sum(per_block) * K * 1e-3,
+              "ms_per_step_median": statistics.median(per_block), "ms_per_step_min": min(per_block),
+              "ms_per_step_max": max(per_block), "restore_kernel_ms_median": statistics.median(restore_ms),
+              "restore_kernel_ms_min": min(restore_ms), "restore_kernel_ms_max": max(restore_ms)}
     assert ctx.query_status() == 0
 
-    # ---- the same step captured once in a CUDA graph and replayed (select_repair + counter reset + restore)
+    # ---- the same step captured once in a CUDA graph and replayed (select_repair + restore)
     graph_ms = None
     if world == 1 and not args.no_graph:
         try:
@@ -319,23 +432,25 @@ def run_ours(args):
                 ctx.restore(geom, pool, [sess], side)
             for _ in range(3):
                 g.replay()
+            n_rep = max(K, 100)
             ga, gb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             torch.cuda.synchronize()
             ga.record()
-            for _ in range(args.steps):
+            for _ in range(n_rep):
                 g.replay()
             gb.record()
             gb.synchronize()
-            graph_ms = ga.elapsed_time(gb) / args.steps
+            graph_ms = ga.elapsed_time(gb) / n_rep
             assert ctx.query_status() == 0
         except Exception as exc:           # reported, never fatal: the headline numbers do not depend on it
             graph_ms = f"unavailable: {type(exc).__name__}"
 
     peak, peak_kind = measured_hbm_peak()
     achieved = (read_b + written_b) / (restore_avg_ms * 1e-3) / 1e9
+    traffic, traffic_src = captured_traffic(items, written_b)
     roofline = {"bound": "hbm", "kernel": "restore_pipe_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": f"of {peak_kind} copy bandwidth (burst)",
-                "frac_of_nominal_8tbs": achieved / 8000.0, "traffic": RESTORE_KERNEL_DRAM_TRAFFIC_BYTES,
+                "frac_of_nominal_8tbs": achieved / 8000.0, "traffic": traffic, "traffic_source": traffic_src,
                 "algorithmic_bytes_per_launch": read_b + written_b, "kernel_ms": restore_avg_ms}
 
     # ---- offload side: write a checkpoint of all 1024 blocks x 32 layers from the pool (not on the resume path)
@@ -348,18 +463,13 @@ def run_ours(args):
             w_pay = torch.empty_like(st.payload)
             w_ptrs = torch.tensor([w_pay.data_ptr() + o for o in ck.layer_off], dtype=torch.int64, device=dev)
             w_sess = st.session(layer_payload=w_ptrs, blk_off=w_off, layer_bytes=w_lb)
-            ts_w = []
-            for i in range(33):                           # a median over 30: single calls wander by a few per cent
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(stream)
+
+            def write_once():
                 ctx.plan_checkpoint(geom, ck.n_suffix_tokens, st.tags, w_off, w_lb, stream)
                 ctx.quantize_gather(geom, pool, w_sess, stream)
-                b.record(stream)
-                b.synchronize()
-                if i >= 3:
-                    ts_w.append(a.elapsed_time(b))
+
+            t_w = median_ms(write_once, stream, 30)         # a median over 30: single calls wander by a few per cent
             assert ctx.query_status() == 0 and torch.equal(w_off, st.blk_off)
-            t_w = statistics.median(ts_w)
             pool_read = 2 * L_ * NB_ * ck.geom.block_tokens * ck.geom.n_kv_heads * ck.geom.head_dim * 2
             pay_written = sum(ck.layer_bytes)
             # the same checkpoint streamed to pinned host memory (encode layer l+1 while layer l is copied out)
@@ -368,16 +478,7 @@ def run_ours(args):
             hptrs = torch.tensor([h_.data_ptr() for h_ in hbufs], dtype=torch.int64)
             hcaps = torch.full((L_,), cap_, dtype=torch.int64)
             hsizes = torch.zeros(L_, dtype=torch.int64)
-            ts_h = []
-            for i in range(6):
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                torch.cuda.synchronize()
-                a.record(stream)
-                ctx.checkpoint_to_host(geom, pool, w_sess, hptrs, hcaps, hsizes, stream)
-                b.record(stream)
-                b.synchronize()
-                if i >= 2:
-                    ts_h.append(a.elapsed_time(b))
+            t_h = median_ms(lambda: ctx.checkpoint_to_host(geom, pool, w_sess, hptrs, hcaps, hsizes, stream), stream, 4, warm=2)
             assert ctx.query_status() == 0 and int(hsizes.sum()) == pay_written
             src_ = torch.empty(1 << 30, dtype=torch.uint8, device=dev)
             dst_ = torch.empty(1 << 30, dtype=torch.uint8).pin_memory()
@@ -390,7 +491,6 @@ def run_ours(args):
                 b.synchronize()
                 d2h_best = a.elapsed_time(b) if d2h_best is None else min(d2h_best, a.elapsed_time(b))
             d2h_ceiling = (1 << 30) / (d2h_best * 1e-3) / 1e9
-            t_h = statistics.median(ts_h)
             del hbufs, src_, dst_
             writer = {"to_host": {"ms": t_h, "payload_gbps": pay_written / (t_h * 1e-3) / 1e9,
                                   "d2h_ceiling_gbps": d2h_ceiling, "frac_of_link": pay_written / (t_h * 1e-3) / 1e9 / d2h_ceiling},
@@ -428,8 +528,9 @@ def run_ours(args):
                 hst.mass.copy_(mass_host, non_blocking=True)                 # stored block masses: host -> device
                 ctx.select_repair(hsel, stream)                               # lists also land in the pinned mirrors:
                 rc, stats = ctx.restore_from_host(geom, pool, [hs], stream)   # the host planner reads them
-                b.record(stream)
-                status = ctx.query_status()                                   # reads the device status word back
+                status = ctx.query_status()                                   # waits, reads the device status word back
+                b.record(stream)                                              # ... inside the timed region
+                b.synchronize()
                 assert status == 0
                 if i >= 3:
                     times.append(max_over_ranks(a.elapsed_time(b), world, dev))
@@ -440,7 +541,7 @@ def run_ours(args):
                    "d2h_bytes_per_step": int(idx_host.numel() * 4 + cnt_host.numel() * 4 + 4),
                    "ms_per_step": e_ms, "steps": len(times),
                    "path": "pinned masses H2D, select_repair with pinned host mirrors of the lists (D2H, waited for), "
-                           "restore_from_host (pinned payload), status D2H"}
+                           "restore_from_host (pinned payload), status word D2H (waited for); all inside the events"}
             host_link = {"ceiling_gbps": ceiling, "ceiling": "1 GiB pinned cudaMemcpyAsync H2D, best of 10, same run",
                          "payload_gbps": read_b / (e_ms * 1e-3) / 1e9, "frac": read_b / (e_ms * 1e-3) / 1e9 / ceiling,
                          "bytes_copied": int(copied), "bytes_useful": int(read_b), "copies": int(stats.n_copies)}
@@ -468,47 +569,25 @@ def run_ours(args):
             sa = pk.select_args(kind=pk.SCORE_ATTN_F16, n_layers=SL, n_suffix_tokens=16384, block_tokens=16,
                                 dirty_tokens=640, top_k=32, layer_mode=pk.LAYERS_INDEPENDENT, attn=attn,
                                 mass_out=mass_out, **out)
-            ts = []
-            for i in range(13):
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(stream)
-                ctx.select_repair(sa, stream)
-                b.record(stream)
-                b.synchronize()
-                if i >= 3:
-                    ts.append(a.elapsed_time(b))
+            t_ms = median_ms(lambda: ctx.select_repair(sa, stream), stream, 10)
             assert ctx.query_status() == 0 and int(out["reuse_cnt"][0]) == 952
-            t_ms = statistics.median(ts)
             nbytes = attn.numel() * 2
             # the paper's token-level form from stored per-token scores: top 1.5 % of the suffix tokens, request-level
             tmass = pin.zipf_block_mass(gen, SL, 16384, dev)
             st_args = pk.select_args(kind=pk.SCORE_TOKEN_MASS, n_layers=SL, n_suffix_tokens=16384, block_tokens=16,
                                      dirty_tokens=640, top_k=245, layer_mode=pk.LAYERS_SHARED, mass=tmass, **out)
-            tts = []
-            for i in range(13):
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(stream)
-                ctx.select_repair_tokens(st_args, stream)
-                b.record(stream)
-                b.synchronize()
-                if i >= 3:
-                    tts.append(a.elapsed_time(b))
-            token_form_us = 1e3 * statistics.median(tts)
+            token_form_us = 1e3 * median_ms(lambda: ctx.select_repair_tokens(st_args, stream), stream, 10)
             ta_args = pk.select_args(kind=pk.SCORE_ATTN_F16, n_layers=SL, n_suffix_tokens=16384, block_tokens=16,
                                      dirty_tokens=640, top_k=245, layer_mode=pk.LAYERS_SHARED, attn=attn, **out)
-            tts2 = []
-            for i in range(9):
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(stream)
-                ctx.select_repair_tokens(ta_args, stream)
-                b.record(stream)
-                b.synchronize()
-                if i >= 3:
-                    tts2.append(a.elapsed_time(b))
-            token_form_attn_us = 1e3 * statistics.median(tts2)
+            token_form_attn_us = 1e3 * median_ms(lambda: ctx.select_repair_tokens(ta_args, stream), stream, 6)
+            ti_args = pk.select_args(kind=pk.SCORE_ATTN_F16, n_layers=SL, n_suffix_tokens=16384, block_tokens=16,
+                                     dirty_tokens=640, top_k=245, layer_mode=pk.LAYERS_INDEPENDENT, attn=attn, **out)
+            token_form_attn_indep_us = 1e3 * median_ms(lambda: ctx.select_repair_tokens(ti_args, stream), stream, 6)
             select_scale = {"token_form_us_from_token_scores": token_form_us,
                             "token_form_us_from_attention": token_form_attn_us,
-                            "token_form_attn_gbps": attn.numel() * 2 / (token_form_attn_us * 1e-6) / 1e9,
+                            "token_form_attn_gbps": nbytes / (token_form_attn_us * 1e-6) / 1e9,
+                            "token_form_attn_frac_of_hbm_peak": nbytes / (token_form_attn_us * 1e-6) / 1e9 / peak,
+                            "token_form_us_from_attention_per_layer_sets": token_form_attn_indep_us,
                             "workload": f"stored attention fp16 [{SL}][32][64][16384] ({SL * 64} MiB), 40-block dirty window, top-32 per layer",
                             "select_us": 1e3 * t_ms, "attn_gbps": nbytes / (t_ms * 1e-3) / 1e9,
                             "frac_of_hbm_peak": nbytes / (t_ms * 1e-3) / 1e9 / peak, "launches": 3}
@@ -522,17 +601,8 @@ def run_ours(args):
                 torch.cuda.synchronize()
                 sess4 = st.session(reuse_idx=out["reuse_idx"], reuse_cnt=out["reuse_cnt"])
                 r4, w4, items4 = algorithmic_bytes(ck, out["reuse_idx"].cpu().numpy(), out["reuse_cnt"].cpu().numpy())
-                ts4 = []
-                for i in range(13):
-                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                    a.record(stream)
-                    ctx.restore(geom, pool, [sess4], stream)
-                    b.record(stream)
-                    b.synchronize()
-                    if i >= 3:
-                        ts4.append(a.elapsed_time(b))
+                r_ms = median_ms(lambda: ctx.restore(geom, pool, [sess4], stream), stream, 10)
                 assert ctx.query_status() == 0
-                r_ms = statistics.median(ts4)
                 select_scale["restore_of_its_reuse_set"] = {
                     "ms": r_ms, "block_layers": int(items4), "restored_kv_gbps_bf16_equiv": w4 / (r_ms * 1e-3) / 1e9,
                     "real_gbps": (r4 + w4) / (r_ms * 1e-3) / 1e9, "frac_of_hbm_peak": (r4 + w4) / (r_ms * 1e-3) / 1e9 / peak}
@@ -543,50 +613,17 @@ def run_ours(args):
 
     # ---- the two host-resident workloads: 7B-shaped / 4 KV heads (one session), 70B-shaped stress (8 sessions)
     host_cfg3 = stress = None
+    ceiling = None
     if not args.no_host_configs:
         try:
             ceiling = pinned_copy_ceiling(dev)
-
             ctx_direct = pk.Context(device=local_rank, flags=pk.FLAG_HOST_DIRECT)
 
             def host_leg(cks, label, reps=5, both=False):
-                out_ = host_leg_on(ctx, cks, label, reps)
+                out_ = host_leg_on(ctx, cks, label, ceiling, dev, stream, reps)
                 if both:     # the same through the zero-copy variant: the kernel pulls the records over the link itself
-                    d_ = host_leg_on(ctx_direct, cks, label, reps)
+                    d_ = host_leg_on(ctx_direct, cks, label, ceiling, dev, stream, reps)
                     out_["zero_copy"] = {k_: d_[k_] for k_ in ("ms", "payload_gbps", "frac_of_link", "bytes_copied", "copies")}
-                return out_
-
-            def host_leg_on(ctx, cks, label, reps=5):
-                sts = [StagedCheckpoint(c, dev, payload_on_host=True) for c in cks]
-                for s_ in sts:
-                    ctx.select_repair(s_.select_args(), stream)
-                torch.cuda.synchronize()
-                hk, hv, hpool = device_pool(cks[0], dev)
-                hgeom = sts[0].geom()
-                hss = [s_.host_session() for s_ in sts]
-                useful = written = items_h = 0
-                for c, s_ in zip(cks, sts):
-                    r_, w_, i_ = algorithmic_bytes(c, s_.reuse_idx.cpu().numpy(), s_.reuse_cnt.cpu().numpy())
-                    useful, written, items_h = useful + r_, written + w_, items_h + i_
-                ts_, stats_ = [], None
-                for i in range(2 + reps):
-                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                    torch.cuda.synchronize()
-                    a.record(stream)
-                    rc_, stats_ = ctx.restore_from_host(hgeom, hpool, hss, stream)
-                    b.record(stream)
-                    b.synchronize()
-                    if i >= 2:
-                        ts_.append(a.elapsed_time(b))
-                assert ctx.query_status() == 0 and stats_.bytes_useful == useful
-                t_ms = statistics.median(ts_)
-                out_ = {"workload": label, "ms": t_ms, "restored_kv_gbps_bf16_equiv": written / (t_ms * 1e-3) / 1e9,
-                        "payload_gbps": useful / (t_ms * 1e-3) / 1e9, "link_ceiling_gbps": ceiling,
-                        "frac_of_link": useful / (t_ms * 1e-3) / 1e9 / ceiling, "bytes_useful": int(useful),
-                        "bytes_copied": int(stats_.bytes_copied), "copies": int(stats_.n_copies),
-                        "block_layers": int(items_h), "block_layers_per_s": items_h / (t_ms * 1e-3)}
-                del sts, hk, hv, hss
-                torch.cuda.empty_cache()
                 return out_
 
             try:
@@ -601,35 +638,35 @@ def run_ours(args):
             SLy = args.stress_layers
             waves = []
             for w_ in range(args.stress_waves):          # each wave: SLy of the 80 layers, payload regenerated outside the timed region
-                sess = [pin.config_stress_session(i, device=dev, n_layers=SLy, pin_payload=True, seed=1005 + 17 * i + 1000 * w_)
-                        for i in range(8)]
-                pin.shared_free_list(1005, 8 * 4096, sess)
-                waves.append(host_leg(sess, "", reps=3, both=(w_ == 0)))
-                if w_ + 1 < args.stress_waves:
-                    del sess
+                wave_sess = pin.stress_wave(w_, device=dev, layers=SLy)
+                waves.append(host_leg(wave_sess, "", reps=3, both=(w_ == 0)))
+                del wave_sess
             stress = dict(waves[0])
             stress["workload"] = (f"70b-shaped stress: 8 sessions x 64k-token suffix, H=8 D=128, int4 share 10-60 %, one shared pool "
                                   f"of 32768 pages, pinned host payload; {SLy} of 80 layers resident per wave, {len(waves)} wave(s) "
                                   f"timed (fit rule: the 80-layer pool is 172 GB and its payload 103 GB of pinned memory)")
-            if len(waves) > 1:
-                tot_ms = sum(w["ms"] for w in waves)
-                tot_useful = sum(w["bytes_useful"] for w in waves)
-                stress.update(ms=tot_ms, bytes_useful=tot_useful, layers_covered=SLy * len(waves),
-                              payload_gbps=tot_useful / (tot_ms * 1e-3) / 1e9,
-                              frac_of_link=tot_useful / (tot_ms * 1e-3) / 1e9 / waves[0]["link_ceiling_gbps"],
-                              block_layers=sum(w["block_layers"] for w in waves),
-                              restored_kv_gbps_bf16_equiv=sum(w["restored_kv_gbps_bf16_equiv"] * w["ms"] for w in waves) / tot_ms)
-            del sess
+            tot_ms = sum(w["ms"] for w in waves)
+            tot_useful = sum(w["bytes_useful"] for w in waves)
+            stress.update(ms=tot_ms, bytes_useful=tot_useful, layers_covered=SLy * len(waves), waves=len(waves),
+                          wave_ms=[round(w["ms"], 2) for w in waves],
+                          bytes_copied=sum(w["bytes_copied"] for w in waves), bytes_wasted=sum(w["bytes_wasted"] for w in waves),
+                          copies=sum(w["copies"] for w in waves),
+                          payload_gbps=tot_useful / (tot_ms * 1e-3) / 1e9,
+                          frac_of_link=tot_useful / (tot_ms * 1e-3) / 1e9 / ceiling,
+                          block_layers=sum(w["block_layers"] for w in waves),
+                          block_layers_per_s=sum(w["block_layers"] for w in waves) / (tot_ms * 1e-3),
+                          restored_kv_gbps_bf16_equiv=sum(w["restored_kv_gbps_bf16_equiv"] * w["ms"] for w in waves) / tot_ms)
         except Exception as exc:                          # an optional leg must not cost the bench line
             if world > 1:
                 raise
-            host_cfg3 = leg_failed(exc)
+            host_cfg3 = host_cfg3 or leg_failed(exc)
+            stress = stress or leg_failed(exc)
 
     # ---- the paper's restore microbenchmark shape (Section V-E): an ~8k-token checkpoint of a 64-layer, 8-KV-head,
     #      head_dim-128 model (geometry from the public Qwen3-32B model card, not from the paper), 32-token blocks,
     #      one fp16 scale per 128 channels, restored whole from pinned host memory in each transport format
     paper_shape = None
-    if not args.no_host_configs:
+    if not args.no_host_configs and ceiling is not None:
         try:
             gm = pin.Geometry(64, 8, 128, 128, pin.ROPE_HALF, 1.0e6, 32, 32, 128)
             rows = {}
@@ -638,7 +675,7 @@ def run_ours(args):
                 cm = pin.make_checkpoint(name="paper-microbench", seed=2024, geom=gm, n=8031, delta=-512, tag_probs=probs,
                                          n_outlier=6, outlier_scale=10.0, n_pages=256, dirty_tokens=0, top_k=0,
                                          device=dev, pin_payload=True)
-                r_ = host_leg([cm], label, reps=5)
+                r_ = host_leg_on(ctx, [cm], label, ceiling, dev, stream, reps=5)
                 rows[label] = {"payload_mib": r_["bytes_useful"] / 2 ** 20, "fetch_and_restore_ms": r_["ms"],
                                "payload_gbps": r_["payload_gbps"], "frac_of_link": r_["frac_of_link"], "copies": r_["copies"]}
                 del cm
@@ -672,19 +709,47 @@ def run_ours(args):
             cpu_baseline = leg_failed(exc)
 
     if rank == 0:
+        def get(d, *path):
+            for p_ in path:
+                if not isinstance(d, dict) or p_ not in d:
+                    return None
+                d = d[p_]
+            return d
+        # one compact row per BASELINE configuration; kept as the LAST key so that it is what a truncated record shows
+        configs = {
+            "1_tiny": "parity only (latency-sized)",
+            "2_llama8b_device": {"ms": r3(ms_per_step), "gbps_bf16eq": r3(value), "frac_hbm": r3(roofline["frac"]),
+                                 "select_us": r3(select_us), "restore_kernel_ms": r3(restore_avg_ms)},
+            "3_7b_host": {"ms": r3(get(host_cfg3, "ms")), "gbps_bf16eq": r3(get(host_cfg3, "restored_kv_gbps_bf16_equiv")),
+                          "frac_link": r3(get(host_cfg3, "frac_of_link")),
+                          "zero_copy_frac_link": r3(get(host_cfg3, "zero_copy", "frac_of_link"))},
+            "4_select_scale": {"select_us": r3(get(select_scale, "select_us")), "frac_hbm": r3(get(select_scale, "frac_of_hbm_peak")),
+                               "token_form_us": r3(get(select_scale, "token_form_us_from_attention")),
+                               "token_form_frac_hbm": r3(get(select_scale, "token_form_attn_frac_of_hbm_peak")),
+                               "restore_ms": r3(get(select_scale, "restore_of_its_reuse_set", "ms")),
+                               "restore_gbps_bf16eq": r3(get(select_scale, "restore_of_its_reuse_set", "restored_kv_gbps_bf16_equiv")),
+                               "restore_frac_hbm": r3(get(select_scale, "restore_of_its_reuse_set", "frac_of_hbm_peak"))},
+            "5_stress": {"ms": r3(get(stress, "ms")), "gbps_bf16eq": r3(get(stress, "restored_kv_gbps_bf16_equiv")),
+                         "frac_link": r3(get(stress, "frac_of_link")), "layers_covered": get(stress, "layers_covered"),
+                         "payload_gb": r3((get(stress, "bytes_useful") or 0) / 1e9)},
+            "e2e_llama8b_host": {"ms": r3(get(e2e, "ms_per_step")), "gbps_bf16eq": r3(get(e2e, "value")),
+                                 "frac_link": r3(get(host_link, "frac"))},
+            "writer": {"ms": r3(get(writer, "ms")), "frac_hbm": r3(get(writer, "frac_of_hbm_peak")),
+                       "to_host_frac_link": r3(get(writer, "to_host", "frac_of_link"))},
+        }
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": WORKLOAD if args.layers == 32 else WORKLOAD + f" [PROFILING SLICE: {args.layers} layers]",
-                       "delta": ck.delta, "l2": "working set 3.0 GB per step >> 126 MB L2, no flush",
-                       "parallelism": f"independent replicas x{world}" if world > 1 else "1 gpu"},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": 2 * args.steps,
-            "roofline": roofline, "cpu_baseline": cpu_baseline,
+            "config": workload_config(ck.delta, world, args.layers),
+            "clocks": clocks, "e2e": e2e, "gpu_launches": 2 * K * n_blocks,
+            "gpu_launches_note": f"{n_blocks} timed block(s) x {K} steps x (select_kernel + restore_pipe_kernel)",
+            "roofline": roofline, "cpu_baseline": cpu_baseline, "timing": timing,
             "select_us": select_us, "restore_ms": restore_avg_ms, "cuda_graph_ms_per_step": graph_ms,
             "block_layers_per_s": world * items / (ms_per_step * 1e-3),
             "real_gbps": world * (read_b + written_b) / (ms_per_step * 1e-3) / 1e9,
-            "host_link": host_link, "select_at_scale": select_scale, "host_7b": host_cfg3, "stress": stress, "writer": writer, "paper_microbench_shape": paper_shape,
+            "host_link": host_link, "select_at_scale": select_scale, "host_7b": host_cfg3, "stress": stress,
+            "writer": writer, "paper_microbench_shape": paper_shape, "configs": configs,
         }
         print(json.dumps(line), flush=True)
     ctx.close()
@@ -693,20 +758,144 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------------------ sweeps
+def run_sweep(args):
+    """Restore and writer fractions by tag and by geometry, restore time by suffix length, and the merge-gap sweep of
+    the host path, each on a workload of at most about 2 GB (half of the benchmark's 32 layers).  One JSON line."""
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda:0")
+    from paper_2609_26219_b200 import binding as pk
+    from paper_2609_26219_b200 import build as pkbuild
+    from patchkv_inputs.staging import StagedCheckpoint, device_pool
+    pkbuild.build()
+    ctx = pk.Context(device=0)
+    stream = torch.cuda.current_stream()
+    peak, peak_kind = measured_hbm_peak()
+    LH = 16
+    G = pin.Geometry
+
+    def restore_row(ck, reps=20):
+        st = StagedCheckpoint(ck, dev)
+        k, v, pool = device_pool(ck, dev)
+        geom = st.geom()
+        sa = st.select_args()
+        ctx.select_repair(sa, stream)
+        torch.cuda.synchronize()
+        sess = st.session()
+        r, w, items = algorithmic_bytes(ck, st.reuse_idx.cpu().numpy(), st.reuse_cnt.cpu().numpy())
+        ms = median_ms(lambda: ctx.restore(geom, pool, [sess], stream), stream, reps, warm=5)
+        sel_us = 1e3 * median_ms(lambda: ctx.select_repair(sa, stream), stream, reps, warm=3)
+        assert ctx.query_status() == 0
+        del st, k, v, pool
+        torch.cuda.empty_cache()
+        return {"us": r3(1e3 * ms), "gbps": r3((r + w) / ms / 1e6), "frac_hbm": r3((r + w) / ms / 1e6 / peak),
+                "block_layers": items, "select_us": r3(sel_us)}
+
+    def writer_row(ck, reps=20):
+        g = ck.geom
+        st = StagedCheckpoint(ck, dev)
+        k, v, pool = device_pool(ck, dev)
+        k.view(torch.bfloat16).normal_()
+        v.view(torch.bfloat16).normal_()
+        geom = st.geom()
+        L, NB = g.n_layers, ck.n_blocks
+        off = torch.zeros((L, NB), dtype=torch.int64, device=dev)
+        lb = torch.zeros(L, dtype=torch.int64, device=dev)
+        ctx.plan_checkpoint(geom, ck.n_suffix_tokens, st.tags, off, lb)
+        torch.cuda.synchronize()
+        sizes = [int(x) for x in lb.cpu()]
+        starts = [sum(-(-s // 256) * 256 for s in sizes[:i]) for i in range(L)]
+        out = torch.empty(starts[-1] + sizes[-1] + 256, dtype=torch.uint8, device=dev)
+        ptrs = torch.tensor([out.data_ptr() + o for o in starts], dtype=torch.int64, device=dev)
+        ws = pk.make_session(n_suffix_tokens=ck.n_suffix_tokens, delta=0, dst_shift=ck.dst_shift, block_table=st.block_table,
+                             tags=st.tags, blk_off=off, layer_payload=ptrs, layer_bytes=lb, reuse_idx=None, reuse_cnt=None)
+        ms = median_ms(lambda: ctx.quantize_gather(geom, pool, ws, stream), stream, reps, warm=5)
+        assert ctx.query_status() == 0
+        rd = 2 * L * NB * g.block_tokens * g.n_kv_heads * g.head_dim * 2
+        wr = sum(sizes)
+        del st, k, v, pool, out
+        torch.cuda.empty_cache()
+        return {"us": r3(1e3 * ms), "gbps": r3((rd + wr) / ms / 1e6), "frac_hbm": r3((rd + wr) / ms / 1e6 / peak)}
+
+    def mk(geom, n, seed, probs=pin.MIX, delta=300, shift=0):
+        nb = -(-n // geom.block_tokens)
+        pages = -(-(nb * geom.block_tokens + shift) // geom.page_tokens) + 64
+        return pin.make_checkpoint(name="sweep", seed=seed, geom=geom, n=n, delta=delta, dst_shift=shift, tag_probs=probs,
+                                   n_outlier=6, outlier_scale=10.0, n_pages=pages, dirty_tokens=int(0.088 * n),
+                                   top_k=max(1, nb // 16), device=dev)
+
+    out = {"peak_gbps": peak, "peak_kind": peak_kind, "layers": LH,
+           "note": "half-size workloads (16 layers, <= 2 GB resident); fractions of the measured HBM copy bandwidth"}
+    base = G(LH, 8, 128, 128, pin.ROPE_HALF, 5e5, 16, 16, 32)
+    by_tag = {}
+    for name, probs in (("mix_30_50_20", pin.MIX), ("bf16", (1, 0, 0, 0)), ("k8v8", (0, 1, 0, 0)), ("k8v4", (0, 0, 1, 0)),
+                        ("k4v4", (0, 0, 0, 1))):
+        row = {}
+        for delta in (429, 0):
+            row[f"restore_delta{delta}"] = restore_row(mk(base, 16384, 1002, probs, delta))
+        row["writer"] = writer_row(mk(base, 16384, 1002, probs))
+        by_tag[name] = row
+    out["by_tag"] = by_tag
+    geoms = {
+        "H16_D128_B16": (G(LH, 16, 128, 128, pin.ROPE_HALF, 1e4, 16, 16, 32), 8192),
+        "H8_D128_B16": (base, 16384),
+        "H8_D128_B32_P32_G128": (G(LH, 8, 128, 128, pin.ROPE_HALF, 1e6, 32, 32, 128), 16384),
+        "H8_D128_interleaved": (G(LH, 8, 128, 128, pin.ROPE_INTERLEAVED, 5e5, 16, 16, 32), 16384),
+        "H8_D128_P32_shift5": (G(LH, 8, 128, 128, pin.ROPE_HALF, 5e5, 16, 32, 32), 16384),
+        "H4_D128_B16": (G(LH, 4, 128, 128, pin.ROPE_HALF, 1e6, 16, 16, 32), 32768),
+        "H8_D64_B16": (G(LH, 8, 64, 64, pin.ROPE_HALF, 1e4, 16, 16, 32), 32768),
+        "H2_D128_B16": (G(LH, 2, 128, 128, pin.ROPE_HALF, 1e6, 16, 16, 32), 65536),
+        "H2_D128_B32": (G(LH, 2, 128, 128, pin.ROPE_HALF, 1e6, 32, 32, 32), 65536),
+        "H4_D64_B16": (G(LH, 4, 64, 64, pin.ROPE_HALF, 1e4, 16, 16, 32), 65536),
+    }
+    by_geom = {}
+    for name, (gm, n) in geoms.items():
+        shift = 5 if "shift5" in name else 0
+        by_geom[name] = {"restore": restore_row(mk(gm, n, 7, shift=shift)), "writer": writer_row(mk(gm, n, 7, shift=shift))}
+    out["by_geometry"] = by_geom
+    out["by_suffix_tokens"] = {str(n): restore_row(mk(G(32, 8, 128, 128, pin.ROPE_HALF, 5e5, 16, 16, 32), n, 1002), reps=30)
+                               for n in (256, 1024, 2048, 4096, 8192, 16384)}
+    # merge-gap sweep of the staged host path on the 16-layer 8B-shaped payload, and the zero-copy mode
+    ceiling = pinned_copy_ceiling(dev)
+    ck = mk(base, 16384, 1002)
+    ck.payload = ck.payload.cpu().pin_memory()
+    gaps = {}
+    for gap in (0, 32 << 10, 64 << 10, 128 << 10, 256 << 10, 1 << 20):
+        c = pk.Context(device=0, merge_gap_bytes=gap)
+        r = host_leg_on(c, [ck], "", ceiling, dev, stream, reps=5)
+        gaps[str(gap)] = {"ms": r3(r["ms"]), "frac_link": r3(r["frac_of_link"]), "copies": r["copies"],
+                          "wasted_frac": r3(r["bytes_wasted"] / r["bytes_useful"])}
+        c.close()
+    c = pk.Context(device=0, flags=pk.FLAG_HOST_DIRECT)
+    r = host_leg_on(c, [ck], "", ceiling, dev, stream, reps=5)
+    c.close()
+    r0 = host_leg_on(ctx, [ck], "", ceiling, dev, stream, reps=5)
+    out["host_path"] = {"link_ceiling_gbps": r3(ceiling), "by_merge_gap_bytes": gaps,
+                        "zero_copy": {"ms": r3(r["ms"]), "frac_link": r3(r["frac_of_link"])},
+                        "default": {"ms": r3(r0["ms"]), "frac_link": r3(r0["frac_of_link"]), "copies": r0["copies"],
+                                    "wasted_frac": r3(r0["bytes_wasted"] / r0["bytes_useful"])}}
+    print(json.dumps({"sweep": out}), flush=True)
+    ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--sweep", action="store_true",
+                    help="print the per-tag / per-geometry / suffix-length / merge-gap sweeps instead of the benchmark line")
+    ap.add_argument("--single-block", action="store_true", help="profiling only: time one block of --steps steps")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-scale-select", action="store_true")
     ap.add_argument("--no-host-configs", action="store_true")
     ap.add_argument("--no-writer", action="store_true")
     ap.add_argument("--no-graph", action="store_true")
-    ap.add_argument("--stress-layers", type=int, default=10)
-    ap.add_argument("--stress-waves", type=int, default=1, help="8 waves of 10 layers cover the full 80-layer stress config")
+    ap.add_argument("--stress-layers", type=int, default=pin.STRESS_WAVE_LAYERS)
+    ap.add_argument("--stress-waves", type=int, default=pin.STRESS_LAYERS // pin.STRESS_WAVE_LAYERS,
+                    help="8 waves of 10 layers cover the full 80-layer stress config (the default)")
     ap.add_argument("--scale-layers", type=int, default=32, help="layers of the selection-at-scale leg (profiling: fewer)")
     ap.add_argument("--layers", type=int, default=32,
                     help="profiling only: fewer layers of the same workload (the bench line is quoted on 32)")
@@ -717,6 +906,8 @@ def main():
         args.no_host_configs = args.no_writer = args.no_scale_select = args.no_graph = True
     if args.impl == "reference":
         run_reference(args)
+    elif args.sweep:
+        run_sweep(args)
     else:
         run_ours(args)
 

@@ -240,6 +240,11 @@ PATCHKV_API int patchkv_last_error(patchkv_ctx* ctx, char* buf, size_t n);
  *   H_l        = the min(top_k, #candidates) non-dirty blocks of largest mass; ties go to the lower index.
  *   R_l = dirty u H_l and F_l = the rest, both ascending; unused list entries are set to -1.
  * Asynchronous on `stream`; all outputs are caller-allocated DEVICE arrays. */
+/* Workspace: when the masses are computed here and no mass_out is given, or layer_mode is LAYERS_SHARED, the call
+ * (and patchkv_select_repair_tokens always) uses ONE workspace owned by the context.  Selection calls on one
+ * context must therefore be ordered on the GPU with respect to each other (same stream, or events between
+ * streams); two that overlap race on it.  The workspace grows on demand, which synchronises the device and
+ * reallocates: the first call, and any call with a larger problem, must not be made inside a stream capture. */
 PATCHKV_API int patchkv_select_repair(patchkv_ctx* ctx, const patchkv_select_args* args, void* stream);
 
 /* The selection in the form the paper prints it (Section IV-C, Eqs. 10-12): the importance score is per TOKEN,
@@ -278,9 +283,14 @@ PATCHKV_API int patchkv_select_repair_tokens(patchkv_ctx* ctx, const patchkv_sel
 PATCHKV_API int patchkv_select_repair_static(const patchkv_select_args* args, void* stream, int32_t* device_status);
 
 /* Section IV-D fused restore (dequantise, Eq. 3 RoPE correction of K, page placement) of the reuse sets of
- * up to PATCHKV_MAX_SESSIONS sessions whose payloads are in device memory.  One 4-byte counter reset and one kernel
- * launch, asynchronous on `stream`, no host synchronisation, no allocation; the pair can be captured in a CUDA graph.
- * Launches from one context may overlap on different streams (each takes its own work counter from a ring of 256). */
+ * up to PATCHKV_MAX_SESSIONS sessions whose payloads are in device memory.  One kernel launch, asynchronous on
+ * `stream`, no host synchronisation, no allocation; it can be captured in a CUDA graph.  The kernel is launched with
+ * programmatic stream serialisation, so its set-up overlaps the tail of the kernel in front of it in the stream; it
+ * touches no memory before that kernel has completed.
+ * Launches from one context may overlap on the GPU when they are on different streams: the kernel's work counters
+ * live in a slot that belongs to the stream (at most 191 different streams per context over its life), and a launch
+ * recorded into a graph gets a slot of its own (at most 320 captured launches per context); beyond either limit the
+ * call returns PATCHKV_E_UNSUPPORTED.  The kernel leaves its slot zeroed, so no reset is enqueued. */
 PATCHKV_API int patchkv_restore(patchkv_ctx* ctx, const patchkv_geom* geom, const patchkv_pool* pool,
                                 const patchkv_session* sessions, int n_sessions, void* stream);
 
@@ -361,6 +371,17 @@ PATCHKV_API int patchkv_query_status(patchkv_ctx* ctx, int* device_status);
  * second), so that a caller can check that the limit expires, that patchkv_query_status then reports
  * PATCHKV_E_TIMEOUT, and that the context keeps working afterwards.  Asynchronous on `stream`. */
 PATCHKV_API int patchkv_selftest_bounded_wait(patchkv_ctx* ctx, uint32_t max_polls, void* stream);
+
+/* Diagnostic (the paper has no counterpart).  Arms the NEXT launch of a bulk-copy pipeline kernel on this context
+ * (patchkv_restore, one launch of patchkv_restore_from_host, or patchkv_quantize_gather) to run with a wait limit of
+ * `max_polls` polls (1 .. 2^20) and to have the first consumer group of every CTA withhold the `empty` arrival of
+ * its unit number `after_units` (0-based), so that the warp that feeds the ring runs out of patience while copies it
+ * issued earlier are still landing or have landed.  That launch then takes the path a real timeout would take:
+ * the CTA's abort flag is raised, every role leaves its loop, the feeding warp waits (bounded) for its copies in
+ * flight so that none of them can write the shared memory of a CTA that has gone, and PATCHKV_E_TIMEOUT is latched.
+ * Blocks the launch did not get to are left untouched; no page outside the reuse set is written.  The launch after
+ * it runs normally.  Nothing here faults or spins without a limit. */
+PATCHKV_API int patchkv_selftest_stall_next_launch(patchkv_ctx* ctx, int32_t after_units, uint32_t max_polls);
 
 /* Bytes of one block record for a tag under a geometry; 0 for an unknown tag. */
 PATCHKV_API uint64_t patchkv_record_bytes(int tag, int block_tokens, int n_kv_heads, int head_dim, int group);

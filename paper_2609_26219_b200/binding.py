@@ -105,6 +105,8 @@ def lib():
         l.patchkv_plan_precision.restype = C.c_int
         l.patchkv_query_status.argtypes = [C.c_void_p, C.POINTER(C.c_int)]
         l.patchkv_selftest_bounded_wait.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p]
+        l.patchkv_selftest_stall_next_launch.argtypes = [C.c_void_p, C.c_int32, C.c_uint32]
+        l.patchkv_selftest_stall_next_launch.restype = C.c_int
         l.patchkv_record_bytes.argtypes = [C.c_int] * 5
         l.patchkv_record_bytes.restype = C.c_uint64
         for f in (l.patchkv_create, l.patchkv_destroy, l.patchkv_last_error, l.patchkv_select_repair,
@@ -232,6 +234,11 @@ class Context:
     def selftest_bounded_wait(self, max_polls: int, stream=None, check: bool = True) -> int:
         """Runs the kernels' bounded barrier wait on a barrier that nothing completes; query_status() then reports E_TIMEOUT."""
         return self._check(lib().patchkv_selftest_bounded_wait(self._h, max_polls, _stream_handle(stream)), check)
+
+    def selftest_stall_next_launch(self, after_units: int, max_polls: int, check: bool = True) -> int:
+        """Arms the next pipeline launch on this context to stall one consumer group after `after_units` units with a
+        wait limit of `max_polls` polls; that launch ends early and latches E_TIMEOUT."""
+        return self._check(lib().patchkv_selftest_stall_next_launch(self._h, after_units, max_polls), check)
 
     def query_status(self) -> int:
         v = C.c_int(0)

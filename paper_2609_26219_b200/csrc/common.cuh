@@ -8,6 +8,7 @@
 
 #include <mutex>
 #include <string>
+#include <utility>
 #include <vector>
 
 #include "patchkv.h"
@@ -124,6 +125,36 @@ __device__ __forceinline__ uint16_t lds16(uint32_t a) {
     return v;
 }
 
+// Exclusive prefix sum of v over a CTA of kScanThreads threads; *total receives the CTA sum.  `warp_sums` is 33 ints
+// of shared memory.  Every thread of the CTA has to call it (it contains CTA-wide barriers).
+constexpr int kScanThreads = 1024;
+__device__ __forceinline__ int cta_exclusive_scan(int v, int* warp_sums, int* total) {
+    const unsigned lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    int inc = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int o = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+        if (lane >= (unsigned)d) inc += o;
+    }
+    __syncthreads();                                 // warp_sums free to overwrite
+    if (lane == 31) warp_sums[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        const int w = warp_sums[lane];               // kScanThreads / 32 = 32 warps: one per lane
+        int winc = w;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int o = __shfl_up_sync(0xFFFFFFFFu, winc, d);
+            if (lane >= (unsigned)d) winc += o;
+        }
+        warp_sums[lane] = winc - w;                  // exclusive offset of each warp
+        if (lane == 31) warp_sums[32] = winc;
+    }
+    __syncthreads();
+    *total = warp_sums[32];
+    return warp_sums[warp] + inc - v;
+}
+
 // One session as the restore kernel sees it (all pointers device memory).
 struct SessionDev {
     const int32_t* block_table;
@@ -148,7 +179,11 @@ struct RestoreParams {
     // work: items are (session, layer in [layer_begin, layer_end), position r in the reuse list)
     int32_t n_sessions, layer_begin, layer_end, total_items;
     int32_t* status;        // device status word
-    int32_t* sched;         // work counter of this launch (zeroed on the stream right before it)
+    int32_t* sched;         // this launch's slot of work counters: [0] blocks handed out, [1] CTAs that have left
+                            // (the last CTA to leave zeroes both, so the slot starts the next launch at zero)
+    uint32_t wait_limit;    // polls before a barrier wait gives up (kWaitLimit unless a self-test shortened it)
+    int32_t stall_after;    // self-test only: consumer group 0 of every CTA withholds the `empty` arrival of its
+                            // unit number stall_after (-1: never)
     // bulk-copy pipeline: tokens per staged unit, bytes of one stage's code / scale / offset areas, ring depth
     int32_t unit_tokens, stage_code_bytes, stage_scale_bytes, stage_bytes, n_stages;
     int32_t whole_record;   // 1: a unit is a whole block record (K and V sections together, one bulk copy)
@@ -175,12 +210,21 @@ struct patchkv_ctx {
     int staging_slots = 4;
     int flags = 0;
     int max_smem_optin = 0;
+    int smem_per_sm = 0;
     uint64_t merge_gap = 64 * 1024;
     cudaStream_t copy_stream = nullptr, decode_stream = nullptr;
     cudaEvent_t ev_begin = nullptr, ev_done = nullptr;
     int32_t* d_status = nullptr;
-    int32_t* d_sched = nullptr;     // ring of work counters, one per restore launch in flight
-    unsigned sched_seq = 0;
+    // Work-counter slots of the restore pipeline (two words each, zero between launches: the kernel resets its
+    // own slot).  A slot is private to whatever serialises the launches that use it: slot 0 belongs to the internal
+    // decode stream, every caller stream gets a slot of its own on first use, and a launch recorded into a CUDA
+    // graph gets a slot that nothing else ever uses.
+    int32_t* d_sched = nullptr;
+    std::vector<std::pair<uint64_t, uint64_t>> sched_streams;   // (stream handle, host thread for per-thread streams)
+    int sched_captured = 0;         // slots handed to captured launches so far
+    // self-test: the next pipeline launch runs with this wait limit and stalls one consumer group (see patchkv.h)
+    uint32_t selftest_wait_limit = 0;
+    int32_t selftest_stall_after = -1;
     // select workspace (block masses when the caller gives no mass_out; summed mass for LAYERS_SHARED)
     unsigned long long* d_mass_ws = nullptr;
     size_t mass_ws_elems = 0;
@@ -196,7 +240,9 @@ struct patchkv_ctx {
 
 namespace patchkv {
 
-constexpr int kSchedSlots = 256;
+constexpr int kSchedStreamSlots = 192;      // slot 0: internal decode stream; 1 .. 191: caller streams
+constexpr int kSchedCaptureSlots = 320;     // launches recorded into CUDA graphs over the life of a context
+constexpr int kSchedSlots = kSchedStreamSlots + kSchedCaptureSlots;
 
 struct DeviceGuard {
     int prev = -1;

@@ -18,13 +18,15 @@ extern "C" int patchkv_create(patchkv_ctx** out, const patchkv_config* cfg) {
     ctx->merge_gap = cfg->merge_gap_bytes == UINT64_MAX ? 128 * 1024 : cfg->merge_gap_bytes;
     bool ok = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, cfg->device) == cudaSuccess;
     ok = ok && cudaDeviceGetAttribute(&ctx->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, cfg->device) == cudaSuccess;
+    ok = ok && cudaDeviceGetAttribute(&ctx->smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, cfg->device) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&ctx->decode_stream, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&ctx->ev_begin, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&ctx->ev_done, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->d_status, sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMemset(ctx->d_status, 0, sizeof(int32_t)) == cudaSuccess;
-    ok = ok && cudaMalloc(&ctx->d_sched, kSchedSlots * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc(&ctx->d_sched, 2 * kSchedSlots * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMemset(ctx->d_sched, 0, 2 * kSchedSlots * sizeof(int32_t)) == cudaSuccess;
     if (!ok) {
         patchkv_destroy(ctx);
         return PATCHKV_E_CUDA;
@@ -104,6 +106,16 @@ extern "C" int patchkv_selftest_bounded_wait(patchkv_ctx* ctx, uint32_t max_poll
     if (!guard.ok) return fail(ctx, PATCHKV_E_CUDA, "cudaSetDevice failed");
     patchkv::bounded_wait_selftest_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>(max_polls, ctx->d_status);
     PKV_CUDA(ctx, cudaGetLastError());
+    return PATCHKV_OK;
+}
+
+extern "C" int patchkv_selftest_stall_next_launch(patchkv_ctx* ctx, int32_t after_units, uint32_t max_polls) {
+    if (!ctx) return PATCHKV_E_INVALID;
+    std::lock_guard<std::mutex> lock(ctx->mu);
+    if (after_units < 0 || max_polls == 0 || max_polls > (1u << 20))
+        return fail(ctx, PATCHKV_E_INVALID, "selftest: after_units >= 0, max_polls 1 .. 2^20");
+    ctx->selftest_stall_after = after_units;
+    ctx->selftest_wait_limit = max_polls;
     return PATCHKV_OK;
 }
 

@@ -124,6 +124,24 @@ extern "C" int patchkv_restore_from_host(patchkv_ctx* ctx, const patchkv_geom* g
     PKV_CUDA(ctx, cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_begin, 0));
     PKV_CUDA(ctx, cudaStreamWaitEvent(ctx->decode_stream, ctx->ev_begin, 0));
 
+    // From here on work is enqueued on the internal streams.  Whatever happens below, the call leaves through
+    // `join`, which makes the caller's stream wait for both internal streams and marks the context's arenas and ring
+    // as in use, so that an error half-way never lets a later call (or the caller's stream) overtake queued work.
+    auto join = [&](int code) -> int {
+        cudaError_t e = cudaEventRecord(ctx->ev_begin, ctx->copy_stream);       // ev_begin has served its purpose above
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->decode_stream, ctx->ev_begin, 0);
+        if (e == cudaSuccess) e = cudaEventRecord(ctx->ev_done, ctx->decode_stream);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, ctx->ev_done, 0);
+        if (e == cudaSuccess) ctx->host_call_pending = true;
+        else {                                                                   // cannot order it: drain it here
+            cudaGetLastError();
+            cudaStreamSynchronize(ctx->copy_stream);
+            cudaStreamSynchronize(ctx->decode_stream);
+            if (code == PATCHKV_OK) code = fail(ctx, PATCHKV_E_CUDA, std::string("restore_from_host: ") + cudaGetErrorString(e));
+        }
+        return code;
+    };
+    auto enqueue = [&]() -> int {
     // ---- stage metadata: one pinned image, one copy; unit u (session-major, then layer) uses slot u % n_slots
     size_t cur = 0;
     auto put = [&](const void* src, size_t bytes) -> size_t {
@@ -191,9 +209,6 @@ extern "C" int patchkv_restore_from_host(patchkv_ctx* ctx, const patchkv_geom* g
         q.total_items = (int32_t)items;
         rc = launch_restore(ctx, &q, ctx->decode_stream);
         if (rc != PATCHKV_OK) return rc;
-        PKV_CUDA(ctx, cudaEventRecord(ctx->ev_done, ctx->decode_stream));
-        PKV_CUDA(ctx, cudaStreamWaitEvent(stream, ctx->ev_done, 0));
-        ctx->host_call_pending = true;
         if (stats) *stats = st;
         return PATCHKV_OK;
     }
@@ -248,10 +263,9 @@ extern "C" int patchkv_restore_from_host(patchkv_ctx* ctx, const patchkv_geom* g
         }
     }
 
-    // ---- the caller's stream continues only after copy and decode have drained
-    PKV_CUDA(ctx, cudaEventRecord(ctx->ev_done, ctx->decode_stream));
-    PKV_CUDA(ctx, cudaStreamWaitEvent(stream, ctx->ev_done, 0));
-    ctx->host_call_pending = true;
     if (stats) *stats = st;
     return PATCHKV_OK;
+    };
+    // ---- the caller's stream continues only after copy and decode have drained
+    return join(enqueue());
 }

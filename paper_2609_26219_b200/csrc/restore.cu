@@ -4,6 +4,10 @@
 #include <cuda_fp16.h>
 #include <math.h>
 
+#include <algorithm>
+#include <functional>
+#include <thread>
+
 #include "common.cuh"
 
 namespace patchkv {
@@ -402,6 +406,10 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
     const int off_vec = off_scales + p.stage_scale_bytes;
     const int off_meta = (off_vec + 8 * p.unit_tokens + 15) & ~15;
     volatile int* abortp = &abort_flag;
+    // Launched with programmatic stream serialisation: everything above overlaps the tail of the kernel before this
+    // one in the stream (usually the selection that writes the reuse lists); nothing below may run before that
+    // kernel has completed and its writes are visible.  Without the launch attribute this is a no-op.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     if (threadIdx.x >= 32 && threadIdx.x < kPipeProducers) {
         // ================================================================ resolver warp
@@ -483,7 +491,7 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
                 }
             }
             // hand the round over once the issuing warp has finished with this buffer (bounded, warp-uniform)
-            if (!__all_sync(0xFFFFFFFFu, mbar_wait(&rempty_bar[rb], rphase ^ 1, abortp))) break;
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait(&rempty_bar[rb], rphase ^ 1, abortp, p.wait_limit))) break;
             descs[rb][lane] = d;
             if (lane == 0) round_blocks[rb] = first >= p.total_items ? -1 : round;
             __syncwarp();
@@ -506,7 +514,7 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
         bool alive = true;
 #pragma unroll 1
         while (alive) {
-            if (!__all_sync(0xFFFFFFFFu, mbar_wait(&rfull_bar[ib], iphase, abortp))) { alive = false; break; }
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait(&rfull_bar[ib], iphase, abortp, p.wait_limit))) { alive = false; break; }
             if (round_blocks[ib] < 0) break;
 #pragma unroll 1
             for (int di = 0; di < 32 && alive; di++) {
@@ -524,7 +532,7 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
                 const bool shifted = p.s[si].delta != 0;
                 if (p.whole_record) {
                     // one unit: the record as it lies in the payload, and the destination row of every token
-                    if (!__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], phase ^ 1, abortp))) { alive = false; break; }
+                    if (!__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], phase ^ 1, abortp, p.wait_limit))) { alive = false; break; }
                     uint8_t* sp = ring + (size_t)stage * p.stage_bytes;
                     long long* voff = reinterpret_cast<long long*>(sp + off_vec);
                     for (int i = lane; i < valid; i += 32) {
@@ -557,7 +565,7 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
                     for (int t0 = 0; t0 < valid; t0 += p.unit_tokens) {
                         const int nt = min(p.unit_tokens, valid - t0);
                         // the verdict is made warp-uniform: the lanes meet again at __syncwarp below
-                        if (!__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], phase ^ 1, abortp))) { alive = false; break; }
+                        if (!__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], phase ^ 1, abortp, p.wait_limit))) { alive = false; break; }
                         uint8_t* sp = ring + (size_t)stage * p.stage_bytes;
                         long long* voff = reinterpret_cast<long long*>(sp + off_vec);
                         for (int i = lane; i < nt; i += 32) {                // one destination row per token
@@ -591,7 +599,7 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
         }
         // tell every consumer group that the work list is exhausted: one empty unit each, in the groups' turn order
         for (int g = 0; g < (kPipeConsumers / 32) / p.group_warps && alive; g++) {
-            if (__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], phase ^ 1, abortp))) {
+            if (__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], phase ^ 1, abortp, p.wait_limit))) {
                 if (lane == 0) {
                     StageMeta m; m.nvec = -1; m.fmt = 0; m.flags = 0; m.session = 0;
                     *reinterpret_cast<StageMeta*>(ring + (size_t)stage * p.stage_bytes + off_meta) = m;
@@ -607,7 +615,7 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
             const uint32_t issued = q < (uint32_t)S ? q : (uint32_t)S;
             for (uint32_t k = 0; k < issued; k++) {
                 const uint32_t qq = q - 1 - k;
-                for (uint32_t i = 0; i < kWaitLimit; i++) {
+                for (uint32_t i = 0; i < p.wait_limit; i++) {
                     if (mbar_try_wait(&full_bar[qq % S], (qq / S) & 1)) break;
                     __nanosleep(100);
                 }
@@ -627,8 +635,9 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
         int cur_session = -1;
         int stage = grp;                                 // n_groups <= S
         uint32_t phase = 0;
+        int units_done = 0;
         while (true) {
-            if (!__all_sync(0xFFFFFFFFu, mbar_wait(&full_bar[stage], phase, abortp))) break;
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait(&full_bar[stage], phase, abortp, p.wait_limit))) break;
             uint8_t* sp = ring + (size_t)stage * p.stage_bytes;
             const uint4 mw = lds128(smem_u32(sp) + off_meta);
             StageMeta m;
@@ -661,11 +670,24 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
                 }
             }
             __syncwarp();
-            if ((c & 31) == 0) mbar_arrive(&empty_bar[stage]);
+            // (self-test: group 0 keeps one arrival to itself, so that the issuing warp's wait for this stage runs out)
+            if ((c & 31) == 0 && !(grp == 0 && units_done == p.stall_after)) mbar_arrive(&empty_bar[stage]);
+            units_done++;
             stage += n_groups;
             if (stage >= S) { stage -= S; phase ^= 1; }
         }
         if (c == 0 && *abortp) atomicCAS(p.status, 0, (int)PATCHKV_E_TIMEOUT);
+    }
+    // The last CTA to leave hands the slot of work counters back at zero, so the next launch that uses the slot (the
+    // next one on the same stream, or the next replay of the same graph node) needs no reset of its own.
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        if (atomicAdd(p.sched + 1, 1) == (int)gridDim.x - 1) {
+            p.sched[0] = 0;
+            p.sched[1] = 0;
+            __threadfence();
+        }
     }
 }
 
@@ -720,6 +742,17 @@ int fill_geometry(patchkv_ctx* ctx, const patchkv_geom* g, const patchkv_pool* p
 
 // Sizes the shared-memory ring for a geometry.  Returns false when the bulk-copy pipeline does not apply:
 // per-token code / scale runs that are not multiples of 16 bytes, or a token row too large for one stage.
+static long long pipe_static_smem(bool inter) {
+    static long long cached[2] = {-1, -1};
+    if (cached[inter] < 0) {
+        cudaFuncAttributes fa;
+        cudaError_t e = inter ? cudaFuncGetAttributes(&fa, restore_pipe_kernel<true>) : cudaFuncGetAttributes(&fa, restore_pipe_kernel<false>);
+        if (e != cudaSuccess) { cudaGetLastError(); return 6 * 1024; }
+        cached[inter] = (long long)fa.sharedSizeBytes;
+    }
+    return cached[inter];
+}
+
 static bool plan_pipeline(const patchkv_ctx* ctx, RestoreParams* p) {
     if (ctx->flags & PATCHKV_FLAG_DIRECT_LOADS) return false;
     const long long hd = (long long)p->H * p->D;
@@ -737,7 +770,9 @@ static bool plan_pipeline(const patchkv_ctx* ctx, RestoreParams* p) {
     p->stage_scale_bytes = (int32_t)(p->whole_record ? 0 : ut * (hd / p->G) * 2);
     const long long raw = (long long)p->stage_code_bytes + p->stage_scale_bytes + 8 * ut + 32;
     p->stage_bytes = (int32_t)((raw + 127) / 128 * 128);
-    long long budget = ((long long)ctx->max_smem_optin - 2048) / 2;   // two CTAs per SM
+    // two CTAs per SM: each may use half of what an SM offers, less its static shared memory (descriptor buffers,
+    // barriers) and the 1 KiB the system reserves per CTA
+    long long budget = (long long)ctx->smem_per_sm / 2 - pipe_static_smem(p->rope_style == PATCHKV_ROPE_INTERLEAVED) - 1024;
     if (budget > 112 * 1024) budget = 112 * 1024;
     long long stages = budget / p->stage_bytes;
     if (stages > kMaxStages) stages = kMaxStages;
@@ -764,22 +799,67 @@ static bool plan_pipeline(const patchkv_ctx* ctx, RestoreParams* p) {
     return true;
 }
 
+// The slot of work counters a pipeline launch on `stream` uses.  Launches that share a slot must never overlap on the
+// GPU, so a slot belongs to whatever serialises them: the internal decode stream (slot 0), one caller stream each
+// (slots 1 ...), or one captured launch (a graph node can be replayed from any stream, next to anything).
+static int sched_slot(patchkv_ctx* ctx, cudaStream_t stream, bool capturing, int* slot) {
+    if (stream == ctx->decode_stream && !capturing) { *slot = 0; return PATCHKV_OK; }
+    if (capturing) {
+        if (ctx->sched_captured >= kSchedCaptureSlots)
+            return fail(ctx, PATCHKV_E_UNSUPPORTED, "restore: too many launches captured into CUDA graphs by this context");
+        *slot = kSchedStreamSlots + ctx->sched_captured++;
+        return PATCHKV_OK;
+    }
+    // cudaStreamPerThread is one handle for a different stream in every host thread
+    const uint64_t handle = reinterpret_cast<uintptr_t>(stream);
+    const uint64_t owner = stream == cudaStreamPerThread ? (uint64_t)std::hash<std::thread::id>()(std::this_thread::get_id()) : 0;
+    for (size_t i = 0; i < ctx->sched_streams.size(); i++)
+        if (ctx->sched_streams[i].first == handle && ctx->sched_streams[i].second == owner) { *slot = 1 + (int)i; return PATCHKV_OK; }
+    if ((int)ctx->sched_streams.size() >= kSchedStreamSlots - 1)
+        return fail(ctx, PATCHKV_E_UNSUPPORTED, "restore: this context has been used from too many different streams");
+    ctx->sched_streams.emplace_back(handle, owner);
+    *slot = (int)ctx->sched_streams.size();
+    return PATCHKV_OK;
+}
+
+template <bool INTER>
+static int launch_pipe(patchkv_ctx* ctx, RestoreParams* p, int grid, int smem, cudaStream_t stream, bool pdl) {
+    PKV_CUDA(ctx, cudaFuncSetAttribute(restore_pipe_kernel<INTER>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(kPipeThreads); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = pdl ? 1 : 0;
+    PKV_CUDA(ctx, cudaLaunchKernelEx(&cfg, restore_pipe_kernel<INTER>, *p));
+    return PATCHKV_OK;
+}
+
 int launch_restore(patchkv_ctx* ctx, RestoreParams* p, cudaStream_t stream) {
     if (p->total_items <= 0) return PATCHKV_OK;
     const bool inter = p->rope_style == PATCHKV_ROPE_INTERLEAVED;
     if (plan_pipeline(ctx, p)) {
         const int smem = p->n_stages * p->stage_bytes;
-        if (inter) PKV_CUDA(ctx, cudaFuncSetAttribute(restore_pipe_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        else PKV_CUDA(ctx, cudaFuncSetAttribute(restore_pipe_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         int grid = ctx->sm_count * 2;
         if (grid > p->total_items) grid = p->total_items;
-        // each launch gets its own work counter from a small ring, zeroed in stream order just before it
-        p->sched = ctx->d_sched + (ctx->sched_seq++ % kSchedSlots);
-        PKV_CUDA(ctx, cudaMemsetAsync(p->sched, 0, sizeof(int32_t), stream));
-        if (inter) restore_pipe_kernel<true><<<grid, kPipeThreads, smem, stream>>>(*p);
-        else restore_pipe_kernel<false><<<grid, kPipeThreads, smem, stream>>>(*p);
-        PKV_CUDA(ctx, cudaGetLastError());
-        return PATCHKV_OK;
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        PKV_CUDA(ctx, cudaStreamIsCapturing(stream, &cap));
+        const bool capturing = cap != cudaStreamCaptureStatusNone;
+        int slot = 0;
+        int rc = sched_slot(ctx, stream, capturing, &slot);
+        if (rc != PATCHKV_OK) return rc;
+        p->sched = ctx->d_sched + 2 * slot;
+        p->wait_limit = kWaitLimit;
+        p->stall_after = -1;
+        if (ctx->selftest_stall_after >= 0) {            // armed by patchkv_selftest_stall_next_launch: this launch only
+            p->wait_limit = ctx->selftest_wait_limit;
+            p->stall_after = ctx->selftest_stall_after;
+            ctx->selftest_stall_after = -1;
+        }
+        // The kernel's prologue (barrier set-up, thread map, rotation table) may run under the tail of the kernel in
+        // front of it in the stream; it waits for that kernel before it touches memory.
+        return inter ? launch_pipe<true>(ctx, p, grid, smem, stream, true) : launch_pipe<false>(ctx, p, grid, smem, stream, true);
     }
     int grid = ctx->sm_count * kCtasPerSm;
     if (grid > p->total_items) grid = p->total_items;

@@ -320,35 +320,7 @@ struct TopkParams {
     int32_t* reuse_idx;  int32_t* reuse_cnt;
 };
 
-constexpr int kSelThreads = 1024;
-
-// Exclusive prefix sum of v over the CTA; *total receives the CTA sum.  `warp_sums` is 33 ints of shared memory.
-__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int* total) {
-    const unsigned lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-    int inc = v;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        const int o = __shfl_up_sync(0xFFFFFFFFu, inc, d);
-        if (lane >= (unsigned)d) inc += o;
-    }
-    __syncthreads();                                 // warp_sums free to overwrite
-    if (lane == 31) warp_sums[warp] = inc;
-    __syncthreads();
-    if (warp == 0) {
-        int w = lane < (kSelThreads >> 5) ? warp_sums[lane] : 0;
-        int winc = w;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const int o = __shfl_up_sync(0xFFFFFFFFu, winc, d);
-            if (lane >= (unsigned)d) winc += o;
-        }
-        warp_sums[lane] = winc - w;                  // exclusive offset of each warp
-        if (lane == 31) warp_sums[32] = winc;
-    }
-    __syncthreads();
-    *total = warp_sums[32];
-    return warp_sums[warp] + inc - v;
-}
+constexpr int kSelThreads = kScanThreads;
 
 // Norm of Eq. 10 as the share of the row total: one CTA per row, exact u64 total, quotient in double, one rounding
 // to fp32.  Reported only; the ranking uses the exact masses.
@@ -489,12 +461,12 @@ select_kernel(const TopkParams p) {
         else if (!take_none) {
             const int eq = in && x == T;
             int tot_eq;
-            const int rank = block_exclusive_scan(eq, warp_sums, &tot_eq) + run_eq;
+            const int rank = cta_exclusive_scan(eq, warp_sums, &tot_eq) + run_eq;
             run_eq += tot_eq;
             sel = in && (x > T || (eq && rank < krem));
         }
         int tot_sel;
-        const int before = block_exclusive_scan(sel ? 1 : 0, warp_sums, &tot_sel) + run_sel;
+        const int before = cta_exclusive_scan(sel ? 1 : 0, warp_sums, &tot_sel) + run_sel;
         run_sel += tot_sel;
         if (in) {
             const int j = n_dirty + c;
@@ -532,7 +504,7 @@ block_round_kernel(const uint8_t* token_mask, int n, int B, int NB, uint8_t* mas
             for (int i = j * B; i < e; i++) hit |= tm[i];
         }
         int tot;
-        const int before = block_exclusive_scan(hit, warp_sums, &tot) + run;
+        const int before = cta_exclusive_scan(hit, warp_sums, &tot) + run;
         run += tot;
         if (j < NB) {
             bm[j] = (uint8_t)hit;

@@ -9,36 +9,8 @@
 
 namespace patchkv {
 
-constexpr int kPlanThreads = 1024;
+constexpr int kPlanThreads = kScanThreads;
 constexpr int kGatherThreads = 256;
-
-// Exclusive prefix sum of v over a 1024-thread CTA; *total receives the CTA sum.
-__device__ __forceinline__ int plan_exclusive_scan(int v, int* warp_sums, int* total) {
-    const unsigned lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-    int inc = v;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        const int o = __shfl_up_sync(0xFFFFFFFFu, inc, d);
-        if (lane >= (unsigned)d) inc += o;
-    }
-    __syncthreads();
-    if (lane == 31) warp_sums[warp] = inc;
-    __syncthreads();
-    if (warp == 0) {
-        const int w = warp_sums[lane];
-        int winc = w;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const int o = __shfl_up_sync(0xFFFFFFFFu, winc, d);
-            if (lane >= (unsigned)d) winc += o;
-        }
-        warp_sums[lane] = winc - w;
-        if (lane == 31) warp_sums[32] = winc;
-    }
-    __syncthreads();
-    *total = warp_sums[32];
-    return warp_sums[warp] + inc - v;
-}
 
 // One CTA per layer: offsets of the runs [bf16][int8][int4][k4v4], ascending block index inside a run.
 __global__ void __launch_bounds__(kPlanThreads)
@@ -56,7 +28,7 @@ plan_checkpoint_kernel(const uint8_t* tags, int NB, unsigned long long elems, in
             const int j = j0 + threadIdx.x;
             const int mine = j < NB && tg[j] == tag;
             int tot;
-            const int rank = plan_exclusive_scan(mine, warp_sums, &tot) + run;
+            const int rank = cta_exclusive_scan(mine, warp_sums, &tot) + run;
             run += tot;
             if (mine) off[j] = base + (unsigned long long)rank * rec;
         }
@@ -362,6 +334,9 @@ constexpr int kWPipeMaxPages = 4;                          // logical pages one 
 
 struct WPipeCfg {
     int32_t unit_tokens, stage_bytes, n_stages, heads_contiguous, total_items;
+    uint32_t wait_limit;                                    // polls before a barrier wait gives up
+    int32_t stall_after;                                    // self-test only: consumer warp 0 withholds the `empty`
+                                                            // arrival of its unit number stall_after (-1: never)
     // bytes of a block's / a token's codes and scales per format, and of a record per tag
     uint32_t blk_codes[3], blk_scales[3], tok_codes[3], tok_scales[3], rec_bytes[4];
 };
@@ -486,7 +461,7 @@ quantize_gather_pipe_kernel(const __grid_constant__ GatherParams p, const __grid
                 for (int t0 = 0; t0 < p.B; t0 += cfg.unit_tokens) {
                     const int rows_total = min(cfg.unit_tokens, p.B - t0);
                     const int rows_valid = max(0, min(rows_total, valid - t0));
-                    if (!__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], phase ^ 1, abortp))) { alive = false; break; }
+                    if (!__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], phase ^ 1, abortp, cfg.wait_limit))) { alive = false; break; }
                     uint8_t* sp = ring + (size_t)stage * cfg.stage_bytes;
                     if (lane == 0) {
                         WStageMeta m;
@@ -529,7 +504,7 @@ quantize_gather_pipe_kernel(const __grid_constant__ GatherParams p, const __grid
             cur = nxt;
         }
         if (alive) {                                        // tell the consumers that the list is exhausted
-            if (__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], phase ^ 1, abortp))) {
+            if (__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], phase ^ 1, abortp, cfg.wait_limit))) {
                 if (lane == 0) {
                     WStageMeta m;
                     m.codes = 0; m.scales = 0; m.fmt = 0; m.rows_total = -1; m.rows_valid = 0; m.pad = 0;
@@ -544,7 +519,7 @@ quantize_gather_pipe_kernel(const __grid_constant__ GatherParams p, const __grid
             const uint32_t issued = q < (uint32_t)S ? q : (uint32_t)S;
             for (uint32_t k = 0; k < issued; k++) {
                 const uint32_t qq = q - 1 - k;
-                for (uint32_t i = 0; i < kWaitLimit; i++) {
+                for (uint32_t i = 0; i < cfg.wait_limit; i++) {
                     if (mbar_try_wait(&full_bar[qq % S], (qq / S) & 1)) break;
                     __nanosleep(100);
                 }
@@ -560,8 +535,9 @@ quantize_gather_pipe_kernel(const __grid_constant__ GatherParams p, const __grid
         const int rot = NC > 1 ? (c / (8 / NC)) & (NC - 1) : 0;
         int stage = 0;
         uint32_t phase = 0;
+        int units_done = 0;
         while (true) {
-            if (!__all_sync(0xFFFFFFFFu, mbar_wait(&full_bar[stage], phase, abortp))) break;
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait(&full_bar[stage], phase, abortp, cfg.wait_limit))) break;
             uint8_t* sp = ring + (size_t)stage * cfg.stage_bytes;
             const uint32_t src = smem_u32(sp);
             const uint4 m0 = lds128(src + off_meta), m1 = lds128(src + off_meta + 16);
@@ -589,7 +565,9 @@ quantize_gather_pipe_kernel(const __grid_constant__ GatherParams p, const __grid
             // the stage was rewritten with ordinary stores above; order them before the bulk copy that refills it
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
-            if ((c & 31) == 0) mbar_arrive(&empty_bar[stage]);
+            // (self-test: warp 0 keeps one arrival to itself, so that the producer's wait for this stage runs out)
+            if ((c & 31) == 0 && !(c == 0 && units_done == cfg.stall_after)) mbar_arrive(&empty_bar[stage]);
+            units_done++;
             if (++stage == S) { stage = 0; phase ^= 1; }
         }
         if (c == 0 && *abortp) atomicCAS(p.status, 0, (int)PATCHKV_E_TIMEOUT);
@@ -677,6 +655,12 @@ static int launch_gather(patchkv_ctx* ctx, const patchkv_geom* g, const patchkv_
             WPipeCfg cfg;
             cfg.unit_tokens = ut; cfg.stage_bytes = (int)stage_bytes; cfg.n_stages = n_stages; cfg.heads_contiguous = hc;
             cfg.total_items = p.nb * layers;
+            cfg.wait_limit = kWaitLimit; cfg.stall_after = -1;
+            if (ctx->selftest_stall_after >= 0) {          // armed by patchkv_selftest_stall_next_launch: this launch only
+                cfg.wait_limit = ctx->selftest_wait_limit;
+                cfg.stall_after = ctx->selftest_stall_after;
+                ctx->selftest_stall_after = -1;
+            }
             const uint64_t elems = (uint64_t)g->block_tokens * g->n_kv_heads * g->head_dim, hd = (uint64_t)g->n_kv_heads * g->head_dim;
             for (int f = 0; f < 3; f++) {
                 cfg.blk_codes[f] = (uint32_t)code_bytes(f, elems); cfg.blk_scales[f] = (uint32_t)scale_bytes(f, elems, g->group);
@@ -773,6 +757,23 @@ extern "C" int patchkv_checkpoint_to_host(patchkv_ctx* ctx, const patchkv_geom* 
     PKV_CUDA(ctx, cudaEventRecord(ctx->ev_begin, stream));
     PKV_CUDA(ctx, cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_begin, 0));
     PKV_CUDA(ctx, cudaStreamWaitEvent(ctx->decode_stream, ctx->ev_begin, 0));
+    // From here on work is enqueued on the internal streams; every exit goes through `join`, which makes the caller's
+    // stream wait for both of them and marks the ring as in use, also when a later step fails.
+    auto join = [&](int code) -> int {
+        cudaError_t e = cudaEventRecord(ctx->ev_begin, ctx->decode_stream);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_begin, 0);
+        if (e == cudaSuccess) e = cudaEventRecord(ctx->ev_done, ctx->copy_stream);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, ctx->ev_done, 0);
+        if (e == cudaSuccess) ctx->host_call_pending = true;
+        else {
+            cudaGetLastError();
+            cudaStreamSynchronize(ctx->decode_stream);
+            cudaStreamSynchronize(ctx->copy_stream);
+            if (code == PATCHKV_OK) code = fail(ctx, PATCHKV_E_CUDA, std::string("checkpoint_to_host: ") + cudaGetErrorString(e));
+        }
+        return code;
+    };
+    auto enqueue = [&]() -> int {
     PKV_CUDA(ctx, cudaMemcpyAsync(d_ptrs, h_ptrs, (size_t)L * 8, cudaMemcpyHostToDevice, ctx->decode_stream));
     p.layer_payload = d_ptrs;
     // 3. encode layer l on the decode stream, copy it out on the copy stream; events order slot reuse
@@ -788,10 +789,9 @@ extern "C" int patchkv_checkpoint_to_host(patchkv_ctx* ctx, const patchkv_geom* 
             PKV_CUDA(ctx, cudaMemcpyAsync(host_layer_payload[l], slot.base, h_bytes[l], cudaMemcpyDeviceToHost, ctx->copy_stream));
         PKV_CUDA(ctx, cudaEventRecord(slot.freed, ctx->copy_stream));
     }
-    PKV_CUDA(ctx, cudaEventRecord(ctx->ev_done, ctx->copy_stream));
-    PKV_CUDA(ctx, cudaStreamWaitEvent(stream, ctx->ev_done, 0));
-    ctx->host_call_pending = true;
     return PATCHKV_OK;
+    };
+    return join(enqueue());
 }
 
 // ---------------------------------------------------------------- precision planner (Eqs. 13-14)

@@ -232,7 +232,7 @@ def make_checkpoint(*, name: str, seed: int, geom: Geometry, n: int, delta: int,
                     dirty_tokens: int, top_k: int, layer_mode: int = LAYERS_INDEPENDENT,
                     scores: str = "mass", n_q_heads: int = 0, n_queries: int = 0,
                     device="cpu", payload_device=None, pin_payload: bool = False,
-                    keep_kv: bool = False) -> SuffixCheckpoint:
+                    keep_kv: bool = False, kv_seed: Optional[int] = None) -> SuffixCheckpoint:
     """Build one seeded session.
 
     table: "permutation" (first entries of a seeded permutation of all pages), "identity",
@@ -240,7 +240,8 @@ def make_checkpoint(*, name: str, seed: int, geom: Geometry, n: int, delta: int,
     for the 2x-oversized-pool configuration).
     scores: "mass" (Zipf block masses), "softmax_attn" or "zipf_attn" (fp16 attention).
     The payload is encoded on `device` and moved to `payload_device` (default: same), optionally
-    into pinned host memory.
+    into pinned host memory.  kv_seed, if given, seeds the K/V values on their own (everything else - tags,
+    block table, scores - still follows `seed`).
     """
     g = geom
     gen = torch.Generator(device=device)
@@ -268,8 +269,12 @@ def make_checkpoint(*, name: str, seed: int, geom: Geometry, n: int, delta: int,
     payload.zero_()
     blk_off = torch.empty((L, nb), dtype=torch.int64, device=device)
     raw = []
+    gen_kv = gen
+    if kv_seed is not None:
+        gen_kv = torch.Generator(device=device)
+        gen_kv.manual_seed(kv_seed)
     for l in range(L):
-        k, v = _kv_layer(gen, g, n, n_outlier, outlier_scale, device)
+        k, v = _kv_layer(gen_kv, g, n, n_outlier, outlier_scale, device)
         pl, off = encode_layer(k, v, tags[l], g)
         assert pl.numel() == sizes[l]
         payload[layer_off[l]:layer_off[l] + sizes[l]].copy_(pl)
@@ -371,6 +376,25 @@ def config_stress_session(i: int, device="cpu", n_layers: int = 80, n: int = 655
               n_outlier=6, outlier_scale=10.0, n_pages=n_pages, dirty_tokens=5760, top_k=254, device=device)
     kw.update(over)
     return make_checkpoint(**kw)
+
+
+STRESS_LAYERS = 80
+STRESS_WAVE_LAYERS = 10
+
+
+def stress_wave(w: int, device="cpu", layers: int = STRESS_WAVE_LAYERS, n: int = 65536, pin_payload: bool = True,
+                n_sessions: int = 8, **over) -> List[SuffixCheckpoint]:
+    """Layers [w * layers, (w + 1) * layers) of the 70B-shaped stress workload: the 8 sessions with their own
+    delta and tag mix, pages drawn from one shared shuffled free list.  The whole workload (80 layers, 172 GB of
+    pool, 103 GB of payload) does not fit next to itself, so it is produced and restored one wave of layers at a
+    time.  Tags, delta, masses and pages of a session are the same in every wave (they come from the session's
+    seed); only the K/V values are re-seeded per wave."""
+    nb = -(-n // 16)
+    sess = [config_stress_session(i, device=device, n_layers=layers, n=n, n_pages=nb, pin_payload=pin_payload,
+                                  kv_seed=1005 + 17 * i + 1000 * w, **over)
+            for i in range(n_sessions)]
+    shared_free_list(1005, n_sessions * nb, sess)
+    return sess
 
 
 def shared_free_list(seed: int, n_pages: int, sessions: List[SuffixCheckpoint]) -> None:

@@ -1,7 +1,8 @@
-"""Marshalling of a synthetic SuffixCheckpoint (patchkv_inputs) into the library's argument structs.
+"""Marshalling of a synthetic SuffixCheckpoint into the CUDA library's argument structs.
 
-Used by the GPU tests, the smoke check and the benchmark.  Holds no arithmetic of the method: it moves
-tensors to the device (or to pinned host memory), allocates the output arrays and fills the POD structs.
+Test and benchmark plumbing (used by the GPU tests, the smoke check and bench.py; the CPU checker's tests never
+import it).  Holds no arithmetic of the method: it moves tensors to the device (or to pinned host memory),
+allocates the output arrays and fills the POD structs of paper_2609_26219_b200.binding.
 """
 from __future__ import annotations
 
@@ -10,8 +11,7 @@ from typing import Optional
 import torch
 
 import patchkv_inputs as pin
-
-from . import binding as pk
+from paper_2609_26219_b200 import binding as pk
 
 
 class StagedCheckpoint:

@@ -439,3 +439,42 @@ def test_a_bounded_wait_runs_out_and_the_context_keeps_working(ctx):
     assert ctx.query_status() == 0                       # the latch clears on read
     assert ctx.selftest_bounded_wait(0, check=False) == -1
     run_select_and_restore(ctx, pin.config_tiny(n_pages=256))
+
+
+def test_restore_pipeline_leaves_cleanly_when_a_wait_runs_out():
+    """The path a timeout takes inside the restore pipeline, end to end: one consumer group of every CTA withholds
+    an `empty` arrival (a self-test switch armed for one launch), so the warp that feeds the ring gives up after a
+    short limit with earlier copies already landed.  The launch must return, latch E_TIMEOUT, write nothing outside
+    the reuse set and nothing wrong inside it, and the next launch on the same context must be bit-exact."""
+    import time
+    c = new_context()
+    try:
+        ck = pin.config_llama8b(device=DEV, n_layers=2, delta=77)
+        st = staged(ck)
+        _, sel = oracle_select(ck)
+        c.select_repair(st.select_args())
+        k, v, pool = gpu_pool(ck)
+        geom, sess = st.geom(), st.session()
+        torch.cuda.synchronize()
+        rc, k_ref, v_ref, _ = oracle_restore(ck, sel["reuse_idx"], sel["reuse_cnt"])
+        assert rc == oracle.OK
+        t0 = time.time()
+        c.selftest_stall_next_launch(2, 4096)
+        c.restore(geom, pool, [sess])
+        torch.cuda.synchronize()
+        assert time.time() - t0 < 20.0
+        assert c.query_status() == -5
+        # every halfword is either what the full restore writes there or still the sentinel; some blocks are missing
+        for got, ref in ((np_u16(k), k_ref), (np_u16(v), v_ref)):
+            got = got.reshape(ref.shape)
+            assert np.all((got == ref) | (got == pin.SENTINEL))
+            assert (got != ref).any() and (got[ref != pin.SENTINEL] != pin.SENTINEL).any()
+        # the switch was for one launch: the same context restores everything, bit for bit
+        c.restore(geom, pool, [sess])
+        torch.cuda.synchronize()
+        assert c.query_status() == 0
+        check_pools(k, v, k_ref, v_ref, ck.geom)
+        assert c.selftest_stall_next_launch(-1, 10, check=False) == -1
+        assert c.selftest_stall_next_launch(0, 0, check=False) == -1
+    finally:
+        c.close()

@@ -292,3 +292,33 @@ def test_checkpoint_to_host_streams_the_same_bytes(slots):
         assert c.checkpoint_to_host(geom, pool, sess, ptrs, small, sizes, check=False) == pk.E_INVALID
     finally:
         c.close()
+
+
+def test_writer_pipeline_leaves_cleanly_when_a_wait_runs_out():
+    """The writer's twin of the restore pipeline's timeout path: consumer warp 0 of every CTA withholds one `empty`
+    arrival, the producer warp gives up, waits for its copies in flight and leaves; E_TIMEOUT is latched, every
+    payload byte is either the checker's or untouched, and the next launch on the context writes the whole payload."""
+    import time
+    c = new_context()
+    try:
+        g = pin.Geometry(2, 8, 128, 128, pin.ROPE_HALF, 5e5, 16, 16, 32)
+        ck = _ck(geom=g, n=16384, n_pages=1100, tag_probs=(0.3, 0.5, 0.2, 0.0))
+        kp, vp = pool_from_raw(ck)
+        rc, rc2, off_o, lb_o, bufs_o = run_writer(ck, kp, vp)
+        assert rc == oracle.OK and rc2 == oracle.OK
+        t0 = time.time()
+        c.selftest_stall_next_launch(2, 4096)
+        off, sizes, bufs = gpu_writer(c, ck, kp, vp)
+        assert time.time() - t0 < 30.0
+        assert c.query_status() == -5
+        missing = 0
+        for a, b in zip(bufs, bufs_o):
+            assert np.all((a == b) | (a == 0xEE))
+            missing += int((a != b).sum())
+        assert missing > 0
+        off, sizes, bufs = gpu_writer(c, ck, kp, vp)
+        assert c.query_status() == 0
+        for a, b in zip(bufs, bufs_o):
+            assert np.array_equal(a, b)
+    finally:
+        c.close()

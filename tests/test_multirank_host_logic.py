@@ -52,3 +52,33 @@ def test_single_rank_is_the_identity():
     import bench
     assert bench.max_over_ranks(3.5, 1, torch.device("cpu")) == 3.5
     assert abs(bench.aggregate_value(2.0e9, 4.0, 1) - 0.5e3) < 1e-9
+
+
+def test_both_arms_print_the_same_config_object():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.workload_config(429, 1) == bench.workload_config(429, 1)
+    assert bench.workload_config(429, 1)["workload"] == bench.WORKLOAD
+    assert "PROFILING SLICE" in bench.workload_config(429, 1, layers=4)["workload"]
+
+
+def test_traffic_figure_comes_from_the_committed_capture():
+    sys.path.insert(0, ROOT)
+    import bench
+    kv = dict(x.split(" = ") for x in open(bench.TRAFFIC_FILE).read().splitlines() if " = " in x and not x.startswith("#"))
+    n = int(kv["block_layers"])
+    got, src = bench.captured_traffic(n, int(kv["algorithmic_bytes_written"]))
+    # on the captured slice itself the figure is the capture's own read + write bytes
+    assert abs(got - (int(kv["dram_bytes_read_per_launch"]) + int(kv["dram_bytes_write_per_launch"]))) <= 1
+    assert kv["capture"] in src
+
+
+def test_clock_samples_are_binned_by_block():
+    sys.path.insert(0, ROOT)
+    import bench
+    s = bench.ClockSampler(0)
+    s.proc = None
+    s.lines = [(100.0, "0, 1965, 1965, 400.0, 0x0, Not Active, Not Active, Not Active, Not Active"),
+               (100.5, "0, 1800, 1965, 900.0, 0x4, Not Active, Not Active, Not Active, Active")]
+    rows = s.rows(99.9, 100.6)
+    assert [r[1] for r in rows] == [1965.0, 1800.0] and rows[1][3] == ["sw_power_cap"]

@@ -18,7 +18,7 @@ DEV = "cuda:0"
 
 def _both(ctx, ck):
     from paper_2609_26219_b200 import binding as pk
-    from paper_2609_26219_b200.harness import StagedCheckpoint
+    from patchkv_inputs.staging import StagedCheckpoint
     ref = StagedCheckpoint(ck, DEV)
     new = StagedCheckpoint(ck, DEV)
     ctx.select_repair(ref.select_args())
@@ -52,7 +52,7 @@ def test_static_scratch_variant_matches_the_context_variant_twice_in_a_row():
 
 def test_static_scratch_variant_refuses_what_does_not_fit_and_reports_bad_input():
     from paper_2609_26219_b200 import build, binding as pk
-    from paper_2609_26219_b200.harness import StagedCheckpoint
+    from patchkv_inputs.staging import StagedCheckpoint
     build.build()
     torch.cuda.set_device(0)
     ck = pin.config_tiny()

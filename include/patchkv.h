@@ -374,8 +374,8 @@ PATCHKV_API int patchkv_selftest_bounded_wait(patchkv_ctx* ctx, uint32_t max_pol
 
 /* Diagnostic (the paper has no counterpart).  Arms the NEXT launch of a bulk-copy pipeline kernel on this context
  * (patchkv_restore, one launch of patchkv_restore_from_host, or patchkv_quantize_gather) to run with a wait limit of
- * `max_polls` polls (1 .. 2^20) and to have the first consumer group of every CTA withhold the `empty` arrival of
- * its unit number `after_units` (0-based), so that the warp that feeds the ring runs out of patience while copies it
+ * `max_polls` polls (1 .. 2^20) and to have the consumer warps of every CTA withhold the `empty` arrivals of
+ * their unit number `after_units` (0-based), so that the warp that feeds the ring runs out of patience while copies it
  * issued earlier are still landing or have landed.  That launch then takes the path a real timeout would take:
  * the CTA's abort flag is raised, every role leaves its loop, the feeding warp waits (bounded) for its copies in
  * flight so that none of them can write the shared memory of a CTA that has gone, and PATCHKV_E_TIMEOUT is latched.

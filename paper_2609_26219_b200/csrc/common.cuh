@@ -184,12 +184,14 @@ struct RestoreParams {
     uint32_t wait_limit;    // polls before a barrier wait gives up (kWaitLimit unless a self-test shortened it)
     int32_t stall_after;    // self-test only: consumer group 0 of every CTA withholds the `empty` arrival of its
                             // unit number stall_after (-1: never)
-    // bulk-copy pipeline: tokens per staged unit, bytes of one stage's code / scale / offset areas, ring depth
-    int32_t unit_tokens, stage_code_bytes, stage_scale_bytes, stage_bytes, n_stages;
-    int32_t whole_record;   // 1: a unit is a whole block record (K and V sections together, one bulk copy)
+    // bulk-copy pipeline: bytes of a stage and of its data area, ring depth, tokens per unit of a section slice, and
+    // per tag how many whole records one unit may carry (0: the record is staged a section slice at a time)
+    int32_t unit_tokens, stage_data_bytes, stage_bytes, n_stages;
+    int32_t unit_records[4];
+    int32_t B_shift, P_shift;       // log2 of B / P when a power of two, else -1
     int32_t round_cap, round_div;   // a round of self-scheduled blocks: min(round_cap, left / (round_div * CTAs)), at least 1
-    int32_t group_warps;    // consumer warps that share one unit (8, 4, 2 or 1): small units go to small groups
     uint32_t blk_codes[3], blk_scales[3], tok_codes[3], tok_scales[3];   // bytes per block / per token, by format
+    uint32_t rec_bytes[4];  // bytes of a block record, by tag
     SessionDev s[PATCHKV_MAX_SESSIONS];
     // cos / sin of delta * theta_i per session, fp32, built on the host in double
     float cs[PATCHKV_MAX_SESSIONS][2][PATCHKV_MAX_ROTARY_DIM / 2];

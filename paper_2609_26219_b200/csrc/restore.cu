@@ -311,18 +311,33 @@ restore_kernel(const __grid_constant__ RestoreParams p) {
 
 // ---------------------------------------------------------------- bulk-copy pipeline
 // A resolver warp takes rounds of blocks from the global work counter and resolves the directory entry and the
-// destination pages of each block one round ahead; an issuing warp stages each resolved block's K and V sections
-// (in units of a few tokens; small records whole, K and V in one unit) into a shared-memory ring with bulk
-// asynchronous copies that complete on an mbarrier.
+// destination pages of each block one round ahead; an issuing warp stages the resolved blocks into a shared-memory
+// ring with bulk asynchronous copies that complete on an mbarrier.  What one copy (one "unit") carries depends on the
+// size of the block's record: a record that fits a stage travels whole, K and V sections together, and records of the
+// same tag that lie next to each other in the payload (same-tag runs are contiguous in the checkpoint) share a unit and
+// a copy; a record larger than a stage is staged one K or V section at a time, a few tokens per unit.
 // Eight consumer warps dequantise / rotate from shared memory and write the bf16 rows to the pool with 128-bit
-// stores; when a unit holds few vectors they split into groups that take units in turn.  Directory latency and HBM
-// read latency are hidden by the ring instead of by occupancy.  Every wait is bounded.
+// stores.  Directory latency and HBM read latency are hidden by the ring instead of by occupancy.  Every wait is
+// bounded.
 constexpr int kPipeConsumers = 256;
 constexpr int kPipeProducers = 64;                          // warp 0 feeds the ring, warp 1 resolves the next round of blocks
 constexpr int kPipeThreads = kPipeConsumers + kPipeProducers;
 constexpr int kMaxStages = 8;
+constexpr int kMaxUnitTokens = 128;                         // tokens one unit may carry (rows of its token table)
+constexpr int kMaxUnitRecords = 8;                          // records one unit may carry
 
-struct StageMeta { int32_t nvec, fmt, flags, session; };   // nvec < 0: no more work; flags bit0 = K section, bit1 = rotate
+// Header of a staged unit (32 bytes at the end of the stage).  Section bases are byte offsets from the start of the stage
+// for the first record of the unit; a token's table row adds the offset of its own record.
+struct StageMeta {
+    int32_t nvec;                   // (token, head) vectors in the unit; < 0: no more work
+    int32_t fmt;                    // K format | V format << 4
+    int32_t flags;                  // bit0: unit holds K rows, bit1: rotate K, bit2: unit holds V rows
+    int32_t session;
+    uint32_t k_codes, k_scales, v_codes, v_scales;
+};
+// One row of a unit's token table: where the token's rows go in the pool (element offset without the head term), the byte
+// offset of its record inside the unit, and its index inside that record (or inside the staged slice of a section).
+struct TokenRow { long long dst; uint32_t rec_off; uint32_t tok; };
 constexpr int kMaxItemPages = 8;                            // destination pages one block may touch in this kernel
 struct ItemDesc {                                           // one resolved, validated block (valid == 0: nothing to do)
     const uint8_t* rec;
@@ -349,20 +364,23 @@ __device__ __forceinline__ Chunk lds_chunk(uint32_t codes, uint32_t scales, int 
     return c;
 }
 
+// One section (K or V) of a staged unit: `codes` / `scales` are the shared-memory addresses of the section in the unit's
+// first record, `tok_tab` the unit's token table.
 template <int FMT, bool INTER>
 __device__ __forceinline__ void consume_unit(const RestoreParams& p, uint32_t codes, uint32_t scales,
-                                             uint32_t tok_off, int nvec, uint16_t* dst_base,
+                                             uint32_t tok_tab, int nvec, uint16_t* dst_base,
                                              const ThreadMap& tm, int gpv, const float* tc, const float* ts, bool rotate) {
     const bool hasB = tm.cB >= 0;
     const bool rotA = rotate && tm.rotA, rotB = rotate && tm.rotB;
     int t = tm.t0, h = tm.h0;                              // (token, head) of `vec`, advanced without divisions
 #pragma unroll 1
     for (int vec = tm.ty; vec < nvec; vec += tm.TY) {
-        const Chunk ca = lds_chunk<FMT>(codes, scales, vec, p.D, gpv, tm.cA, tm.gA);
+        const uint4 row = lds128(tok_tab + 16u * (uint32_t)t);
+        const int rv = (int)row.w * p.H + h;               // vector index inside the token's record
+        const Chunk ca = lds_chunk<FMT>(codes + row.z, scales + row.z, rv, p.D, gpv, tm.cA, tm.gA);
         Chunk cb = ca;
-        if (hasB) cb = lds_chunk<FMT>(codes, scales, vec, p.D, gpv, tm.cB, tm.gB);
-        const uint2 vo = lds64(tok_off + 8u * (uint32_t)t);
-        uint16_t* d = dst_base + (long long)(((unsigned long long)vo.y << 32) | vo.x) + (long long)h * p.stride_head;
+        if (hasB) cb = lds_chunk<FMT>(codes + row.z, scales + row.z, rv, p.D, gpv, tm.cB, tm.gB);
+        uint16_t* d = dst_base + (long long)(((unsigned long long)row.y << 32) | row.x) + (long long)h * p.stride_head;
         t += tm.dt; h += tm.dh;
         if (h >= p.H) { h -= p.H; t++; }
         uint4 oa = ca.w, ob = cb.w;
@@ -396,15 +414,14 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
 
     const int S = p.n_stages;
     if (threadIdx.x == 0) {
-        for (int s = 0; s < S; s++) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], p.group_warps); }
+        for (int s = 0; s < S; s++) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], kPipeConsumers / 32); }
         for (int b = 0; b < 2; b++) { mbar_init(&rfull_bar[b], 1); mbar_init(&rempty_bar[b], 1); }
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    const int off_scales = p.stage_code_bytes;
-    const int off_vec = off_scales + p.stage_scale_bytes;
-    const int off_meta = (off_vec + 8 * p.unit_tokens + 15) & ~15;
+    const int off_tab = p.stage_data_bytes;              // stage layout: [data][token table][header]
+    const int off_meta = p.stage_bytes - 32;
     volatile int* abortp = &abort_flag;
     // Launched with programmatic stream serialisation: everything above overlaps the tail of the kernel before this
     // one in the stream (usually the selection that writes the reuse lists); nothing below may run before that
@@ -503,8 +520,9 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
     } else if (threadIdx.x < 32) {
         // ================================================================ issuing warp
         // Feeds the shared-memory ring from the resolved rounds without touching global memory itself: per unit it
-        // waits for a free stage, writes the per-token destination offsets and the unit header, and starts the two
-        // bulk copies.
+        // waits for a free stage, writes the unit's token table and header, and starts the bulk copy (two for a section
+        // of a quantised format: codes and scales).  Lane i keeps block i of the round; a unit of whole records is built
+        // by chaining blocks of the round whose records follow one another in the payload.
         const int lane = threadIdx.x;
         uint32_t q = 0;                                  // units issued
         int stage = 0;                                   // q % S, and the parity of q / S, kept without divisions
@@ -516,47 +534,87 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
         while (alive) {
             if (!__all_sync(0xFFFFFFFFu, mbar_wait(&rfull_bar[ib], iphase, abortp, p.wait_limit))) { alive = false; break; }
             if (round_blocks[ib] < 0) break;
+            const ItemDesc* rd = descs[ib];
+            // this lane's block of the round
+            const unsigned long long my_rec = reinterpret_cast<unsigned long long>(rd[lane].rec);
+            const int my_valid = rd[lane].valid, my_tag = rd[lane].tag, my_l = rd[lane].l, my_si = rd[lane].si;
+            uint32_t todo = __ballot_sync(0xFFFFFFFFu, my_valid != 0);
 #pragma unroll 1
-            for (int di = 0; di < 32 && alive; di++) {
-                const ItemDesc& d = descs[ib][di];
-                const int valid = d.valid;
-                if (valid == 0) continue;
-                const int tag = d.tag, l = d.l, si = d.si;
+            while (todo && alive) {
+                const int di = __ffs(todo) - 1;
+                todo &= todo - 1;
+                const ItemDesc& d = rd[di];
+                const int valid = d.valid, tag = d.tag, l = d.l, si = d.si;
                 const int kf = k_format(tag), vf = v_format(tag);
+                const bool shifted = p.s[si].delta != 0;
+                const int cap_records = p.unit_records[tag];
+                if (cap_records > 0) {
+                    // ---- whole records: this block and up to cap_records - 1 blocks of the round that follow it in the
+                    //      payload (same tag, same layer and session).  Only the last member may be a partial block.
+                    const uint32_t rbytes = p.rec_bytes[tag];
+                    int members = 1, tokens = valid;
+                    int my_member = lane == 0 ? di : -1;     // lane c remembers member c of the unit
+                    unsigned long long want = reinterpret_cast<unsigned long long>(d.rec) + rbytes;
+                    bool open = valid == p.B;
+#pragma unroll 1
+                    while (open && members < cap_records) {
+                        const uint32_t hit = __ballot_sync(0xFFFFFFFFu, ((todo >> lane) & 1u) && my_rec == want && my_tag == tag &&
+                                                                          my_l == l && my_si == si);
+                        if (!hit) break;
+                        const int nx = __ffs(hit) - 1;
+                        todo &= ~(1u << nx);
+                        if (lane == members) my_member = nx;
+                        const int nv = __shfl_sync(0xFFFFFFFFu, my_valid, nx);
+                        members++;
+                        tokens += nv;
+                        want += rbytes;
+                        open = nv == p.B;
+                    }
+                    if (!__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], phase ^ 1, abortp, p.wait_limit))) { alive = false; break; }
+                    uint8_t* sp = ring + (size_t)stage * p.stage_bytes;
+                    TokenRow* tab = reinterpret_cast<TokenRow*>(sp + off_tab);
+                    for (int i0 = 0; i0 < tokens; i0 += 32) {
+                        const int i = i0 + lane;
+                        const int m = p.B_shift >= 0 ? i >> p.B_shift : i / p.B;      // member the token belongs to
+                        const int src = __shfl_sync(0xFFFFFFFFu, my_member, min(m, members - 1));
+                        if (i < tokens) {
+                            const ItemDesc& dm = rd[src];
+                            const int tr = i - m * p.B;
+                            const int us = dm.slot0 + tr;
+                            const int pi = p.P_shift >= 0 ? us >> p.P_shift : us / p.P;
+                            TokenRow row;
+                            row.dst = (long long)l * p.stride_layer + (long long)dm.pages[pi] * p.stride_page +
+                                      (long long)(us - pi * p.P) * p.stride_token;
+                            row.rec_off = (uint32_t)m * rbytes;
+                            row.tok = (uint32_t)tr;
+                            tab[i] = row;
+                        }
+                    }
+                    if (lane == 0) {
+                        StageMeta m;
+                        m.nvec = tokens * p.H; m.fmt = kf | (vf << 4); m.session = si;
+                        m.flags = 1 | 4 | (shifted ? 2 : 0);
+                        m.k_codes = 0; m.k_scales = p.blk_codes[kf];
+                        m.v_codes = m.k_scales + p.blk_scales[kf]; m.v_scales = m.v_codes + p.blk_codes[vf];
+                        *reinterpret_cast<StageMeta*>(sp + off_meta) = m;
+                    }
+                    __syncwarp();
+                    if (lane == 0) {
+                        const uint32_t bytes = (uint32_t)members * rbytes;
+                        mbar_arrive_expect_tx(&full_bar[stage], bytes);
+                        bulk_g2s(sp, d.rec, bytes, &full_bar[stage]);
+                    }
+                    q++;
+                    if (++stage == S) { stage = 0; phase ^= 1; }
+                    continue;
+                }
+                // ---- a record larger than a stage: one section at a time, unit_tokens tokens per unit
                 const uint8_t* sec_codes[2];
                 const uint8_t* sec_scales[2];
                 sec_codes[0] = d.rec;
                 sec_scales[0] = sec_codes[0] + p.blk_codes[kf];
                 sec_codes[1] = sec_scales[0] + p.blk_scales[kf];
                 sec_scales[1] = sec_codes[1] + p.blk_codes[vf];
-                const bool shifted = p.s[si].delta != 0;
-                if (p.whole_record) {
-                    // one unit: the record as it lies in the payload, and the destination row of every token
-                    if (!__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], phase ^ 1, abortp, p.wait_limit))) { alive = false; break; }
-                    uint8_t* sp = ring + (size_t)stage * p.stage_bytes;
-                    long long* voff = reinterpret_cast<long long*>(sp + off_vec);
-                    for (int i = lane; i < valid; i += 32) {
-                        const int us = d.slot0 + i;
-                        const int pi = us / p.P;
-                        voff[i] = (long long)l * p.stride_layer + (long long)d.pages[pi] * p.stride_page +
-                                  (long long)(us - pi * p.P) * p.stride_token;
-                    }
-                    if (lane == 0) {
-                        StageMeta m;
-                        m.nvec = valid * p.H; m.fmt = kf | (vf << 4); m.session = si;
-                        m.flags = 4 | (shifted ? 2 : 0);
-                        *reinterpret_cast<StageMeta*>(sp + off_meta) = m;
-                    }
-                    __syncwarp();
-                    if (lane == 0) {
-                        const uint32_t rb_ = p.blk_codes[kf] + p.blk_scales[kf] + p.blk_codes[vf] + p.blk_scales[vf];
-                        mbar_arrive_expect_tx(&full_bar[stage], rb_);
-                        bulk_g2s(sp, d.rec, rb_, &full_bar[stage]);
-                    }
-                    q++;
-                    if (++stage == S) { stage = 0; phase ^= 1; }
-                    continue;
-                }
 #pragma unroll 1
                 for (int sec = 0; sec < 2 && alive; sec++) {
                     const int fmt = sec ? vf : kf;
@@ -567,25 +625,30 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
                         // the verdict is made warp-uniform: the lanes meet again at __syncwarp below
                         if (!__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], phase ^ 1, abortp, p.wait_limit))) { alive = false; break; }
                         uint8_t* sp = ring + (size_t)stage * p.stage_bytes;
-                        long long* voff = reinterpret_cast<long long*>(sp + off_vec);
+                        TokenRow* tab = reinterpret_cast<TokenRow*>(sp + off_tab);
                         for (int i = lane; i < nt; i += 32) {                // one destination row per token
                             const int us = d.slot0 + t0 + i;               // slot counted from the first page
-                            const int pi = us / p.P;
-                            voff[i] = (long long)l * p.stride_layer + (long long)d.pages[pi] * p.stride_page +
+                            const int pi = p.P_shift >= 0 ? us >> p.P_shift : us / p.P;
+                            TokenRow row;
+                            row.dst = (long long)l * p.stride_layer + (long long)d.pages[pi] * p.stride_page +
                                       (long long)(us - pi * p.P) * p.stride_token;
+                            row.rec_off = 0;
+                            row.tok = (uint32_t)i;
+                            tab[i] = row;
                         }
+                        const uint32_t cb = nt * ctok, sb = nt * stok;
                         if (lane == 0) {
                             StageMeta m;
-                            m.nvec = nt * p.H; m.fmt = fmt; m.session = si;
-                            m.flags = (sec == 0 ? 1 : 0) | ((sec == 0 && shifted) ? 2 : 0);
+                            m.nvec = nt * p.H; m.fmt = fmt | (fmt << 4); m.session = si;
+                            m.flags = sec == 0 ? (1 | (shifted ? 2 : 0)) : 4;
+                            m.k_codes = 0; m.k_scales = cb; m.v_codes = 0; m.v_scales = cb;
                             *reinterpret_cast<StageMeta*>(sp + off_meta) = m;
                         }
                         __syncwarp();
                         if (lane == 0) {
-                            const uint32_t cb = nt * ctok, sb = nt * stok;
                             mbar_arrive_expect_tx(&full_bar[stage], cb + sb);
                             bulk_g2s(sp, sec_codes[sec] + (size_t)t0 * ctok, cb, &full_bar[stage]);
-                            if (sb) bulk_g2s(sp + off_scales, sec_scales[sec] + (size_t)t0 * stok, sb, &full_bar[stage]);
+                            if (sb) bulk_g2s(sp + cb, sec_scales[sec] + (size_t)t0 * stok, sb, &full_bar[stage]);
                         }
                         q++;
                         if (++stage == S) { stage = 0; phase ^= 1; }
@@ -597,11 +660,13 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
             ib ^= 1;
             if (ib == 0) iphase ^= 1;
         }
-        // tell every consumer group that the work list is exhausted: one empty unit each, in the groups' turn order
-        for (int g = 0; g < (kPipeConsumers / 32) / p.group_warps && alive; g++) {
+        // tell the consumers that the work list is exhausted: one empty unit
+        if (alive) {
             if (__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], phase ^ 1, abortp, p.wait_limit))) {
                 if (lane == 0) {
-                    StageMeta m; m.nvec = -1; m.fmt = 0; m.flags = 0; m.session = 0;
+                    StageMeta m;
+                    memset(&m, 0, sizeof(m));
+                    m.nvec = -1;
                     *reinterpret_cast<StageMeta*>(ring + (size_t)stage * p.stage_bytes + off_meta) = m;
                     mbar_arrive(&full_bar[stage]);
                 }
@@ -624,57 +689,47 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
         }
     } else {
         // ================================================================ consumer warps
-        // group g of the consumer warps takes units g, g + n_groups, ... (units are numbered in issue order)
+        // All eight warps work on one unit at a time, in issue order.  (Every waiter has to see every phase of a stage's
+        // barriers - a parity wait cannot tell a phase from the one two before it - so the warps are never split into
+        // groups that would each visit only some uses of a stage.)
         const int c = threadIdx.x - kPipeProducers;
-        const int group_threads = p.group_warps * 32, n_groups = kPipeConsumers / group_threads;
-        const int grp = c / group_threads;
         bool lane_active;
-        const ThreadMap tm = make_thread_map<INTER>(p, group_threads, c - grp * group_threads, &lane_active);
+        const ThreadMap tm = make_thread_map<INTER>(p, kPipeConsumers, c, &lane_active);
         const int gpv = p.D / p.G;
         float tc[8], ts[8];
         int cur_session = -1;
-        int stage = grp;                                 // n_groups <= S
+        int stage = 0;
         uint32_t phase = 0;
         int units_done = 0;
         while (true) {
             if (!__all_sync(0xFFFFFFFFu, mbar_wait(&full_bar[stage], phase, abortp, p.wait_limit))) break;
             uint8_t* sp = ring + (size_t)stage * p.stage_bytes;
-            const uint4 mw = lds128(smem_u32(sp) + off_meta);
-            StageMeta m;
-            m.nvec = (int)mw.x; m.fmt = (int)mw.y; m.flags = (int)mw.z; m.session = (int)mw.w;
-            if (m.nvec < 0) break;
-            if (m.session != cur_session) { cur_session = m.session; load_rotation<INTER>(p, cur_session, tm, tc, ts); }
+            const uint32_t base = smem_u32(sp);
+            const uint4 mw = lds128(base + off_meta), mo = lds128(base + off_meta + 16);
+            const int nvec = (int)mw.x, fmts = (int)mw.y, flags = (int)mw.z, session = (int)mw.w;
+            if (nvec < 0) break;
+            if (session != cur_session) { cur_session = session; load_rotation<INTER>(p, cur_session, tm, tc, ts); }
             if (lane_active) {
-                const uint32_t base = smem_u32(sp);
-                const uint32_t voff = base + off_vec;
-                const bool whole = (m.flags & 4) != 0;
-                const int kf = m.fmt & 15, vf = m.fmt >> 4;          // whole-record units carry both formats
+                const uint32_t tab = base + off_tab;
 #pragma unroll 1
-                for (int sec = 0; sec < (whole ? 2 : 1); sec++) {
-                    int fmt = m.fmt;
-                    uint32_t codes = base, scales = base + off_scales;
-                    uint16_t* dst = (m.flags & 1) ? p.k_base : p.v_base;
-                    bool rotate = (m.flags & 2) != 0;
-                    if (whole) {                                     // sections in record order: K codes, K scales, V codes, V scales
-                        fmt = sec ? vf : kf;
-                        codes = sec ? base + p.blk_codes[kf] + p.blk_scales[kf] : base;
-                        scales = codes + p.blk_codes[fmt];
-                        dst = sec ? p.v_base : p.k_base;
-                        rotate = rotate && sec == 0;
-                    }
+                for (int sec = 0; sec < 2; sec++) {
+                    if (!(flags & (sec ? 4 : 1))) continue;
+                    const int fmt = sec ? fmts >> 4 : fmts & 15;
+                    const uint32_t codes = base + (sec ? mo.z : mo.x), scales = base + (sec ? mo.w : mo.y);
+                    uint16_t* dst = sec ? p.v_base : p.k_base;
+                    const bool rotate = sec == 0 && (flags & 2) != 0;
                     switch (fmt) {
-                        case FMT_BF16: consume_unit<FMT_BF16, INTER>(p, codes, scales, voff, m.nvec, dst, tm, gpv, tc, ts, rotate); break;
-                        case FMT_INT8: consume_unit<FMT_INT8, INTER>(p, codes, scales, voff, m.nvec, dst, tm, gpv, tc, ts, rotate); break;
-                        default:       consume_unit<FMT_INT4, INTER>(p, codes, scales, voff, m.nvec, dst, tm, gpv, tc, ts, rotate); break;
+                        case FMT_BF16: consume_unit<FMT_BF16, INTER>(p, codes, scales, tab, nvec, dst, tm, gpv, tc, ts, rotate); break;
+                        case FMT_INT8: consume_unit<FMT_INT8, INTER>(p, codes, scales, tab, nvec, dst, tm, gpv, tc, ts, rotate); break;
+                        default:       consume_unit<FMT_INT4, INTER>(p, codes, scales, tab, nvec, dst, tm, gpv, tc, ts, rotate); break;
                     }
                 }
             }
             __syncwarp();
-            // (self-test: group 0 keeps one arrival to itself, so that the issuing warp's wait for this stage runs out)
-            if ((c & 31) == 0 && !(grp == 0 && units_done == p.stall_after)) mbar_arrive(&empty_bar[stage]);
+            // (self-test: the arrivals of one unit are withheld, so that the issuing warp's wait for this stage runs out)
+            if ((c & 31) == 0 && units_done != p.stall_after) mbar_arrive(&empty_bar[stage]);
             units_done++;
-            stage += n_groups;
-            if (stage >= S) { stage -= S; phase ^= 1; }
+            if (++stage == S) { stage = 0; phase ^= 1; }
         }
         if (c == 0 && *abortp) atomicCAS(p.status, 0, (int)PATCHKV_E_TIMEOUT);
     }
@@ -740,8 +795,7 @@ int fill_geometry(patchkv_ctx* ctx, const patchkv_geom* g, const patchkv_pool* p
     return PATCHKV_OK;
 }
 
-// Sizes the shared-memory ring for a geometry.  Returns false when the bulk-copy pipeline does not apply:
-// per-token code / scale runs that are not multiples of 16 bytes, or a token row too large for one stage.
+// Static shared memory of the pipeline kernel (descriptor buffers, barriers), asked of the runtime once.
 static long long pipe_static_smem(bool inter) {
     static long long cached[2] = {-1, -1};
     if (cached[inter] < 0) {
@@ -753,49 +807,73 @@ static long long pipe_static_smem(bool inter) {
     return cached[inter];
 }
 
+// Sizes the shared-memory ring for a geometry and decides, per tag, what a unit carries.  Returns false when the
+// bulk-copy pipeline does not apply: per-token code / scale runs that are not multiples of 16 bytes, or a token row
+// too large for one stage.
 static bool plan_pipeline(const patchkv_ctx* ctx, RestoreParams* p) {
     if (ctx->flags & PATCHKV_FLAG_DIRECT_LOADS) return false;
     const long long hd = (long long)p->H * p->D;
     if (hd % 32 != 0 || (hd / p->G) % 8 != 0) return false;
-    long long ut = 16384 / hd;                       // at most 32 KiB of bf16 codes per stage
-    if (ut > p->B) ut = p->B;
-    if (ut > 256 / p->H) ut = 256 / p->H;            // at most 256 (token, head) vectors per stage
-    if (ut < 1) return false;
     if ((p->B + p->P - 2) / p->P + 1 > kMaxItemPages) return false;   // pages one block can straddle
-    // Small records (both bf16 sections of a block within 36 KiB) travel whole: one unit and one bulk copy per block
-    // instead of one per section, which halves the issuing warp's work where it is the limit.
-    p->whole_record = (ut == p->B && 4ll * p->B * hd <= 36 * 1024) ? 1 : 0;
-    p->unit_tokens = (int32_t)ut;
-    p->stage_code_bytes = (int32_t)(p->whole_record ? 4 * ut * hd : ut * hd * 2);      // whole: the largest (bf16) record
-    p->stage_scale_bytes = (int32_t)(p->whole_record ? 0 : ut * (hd / p->G) * 2);
-    const long long raw = (long long)p->stage_code_bytes + p->stage_scale_bytes + 8 * ut + 32;
-    p->stage_bytes = (int32_t)((raw + 127) / 128 * 128);
     // two CTAs per SM: each may use half of what an SM offers, less its static shared memory (descriptor buffers,
     // barriers) and the 1 KiB the system reserves per CTA
     long long budget = (long long)ctx->smem_per_sm / 2 - pipe_static_smem(p->rope_style == PATCHKV_ROPE_INTERLEAVED) - 1024;
     if (budget > 112 * 1024) budget = 112 * 1024;
-    long long stages = budget / p->stage_bytes;
-    if (stages > kMaxStages) stages = kMaxStages;
-    if (stages < 2) return false;
-    p->n_stages = (int32_t)stages;
-    // Consumer groups: a unit of few vectors is not worth the fixed work of all eight consumer warps (barrier wait,
-    // unit header, format switch), so the warps split into groups that take units in turn, sized so that a thread
-    // gets about four (vector, channel-lane) tasks per unit; never more groups than stages.
-    const long long tasks = (p->whole_record ? 2 : 1) * ut * p->H * ((p->D + 15) / 16);
-    int gw = kPipeConsumers / 32;
-    while (gw > 1 && (long long)gw * 32 / 2 * 4 >= tasks && (kPipeConsumers / 32) / (gw / 2) <= stages) gw /= 2;
-    p->group_warps = gw;
-    // Self-scheduled rounds: the resolver's chain of dependent lookups (about 7 us under load) has to stay shorter
-    // than the time the CTA spends issuing the previous round, so small records are claimed in larger rounds
-    // (about 256 KiB of bf16 per round), and shrink later (measured on records of 16 to 128 KiB).
-    const long long rec_bf16 = 4ll * p->B * hd;
-    p->round_cap = (int32_t)std::max<long long>(4, std::min<long long>(16, (256 * 1024) / rec_bf16));
-    p->round_div = (int32_t)std::max<long long>(2, std::min<long long>(8, rec_bf16 / 8192));
+    if (budget > ctx->max_smem_optin) budget = ctx->max_smem_optin;
+    // Three stages of about 36 KiB each (measured: fewer, larger units beat more, smaller ones as long as three fit).
+    long long stage_total = budget / 3 / 128 * 128;
+    if (stage_total > 40 * 1024) stage_total = 40 * 1024;
     const uint64_t elems = (uint64_t)p->B * hd;
     for (int f = 0; f < 3; f++) {                     // section sizes per format: no divisions in the issuing warp
         p->blk_codes[f] = (uint32_t)code_bytes(f, elems); p->blk_scales[f] = (uint32_t)scale_bytes(f, elems, p->G);
         p->tok_codes[f] = (uint32_t)code_bytes(f, hd); p->tok_scales[f] = (uint32_t)scale_bytes(f, hd, p->G);
     }
+    for (int t = 0; t < 4; t++) p->rec_bytes[t] = (uint32_t)record_bytes(t, elems, p->G);
+    // A record that fits the data area of a stage travels whole, and as many records of a same-tag run as fit (at most
+    // kMaxUnitRecords, at most kMaxUnitTokens tokens) share a unit; a larger record is staged a section slice at a time.
+    // The token table grows with the tokens a unit may carry, so the two sizes are settled together.
+    long long rows = std::min<long long>(p->B, kMaxUnitTokens), cap = 0, ut = 0;
+    for (int pass = 0; pass < 3; pass++) {
+        cap = (stage_total - 32 - 16 * rows) / 16 * 16;
+        if (cap < 2 * hd) return false;               // not even one token of a bf16 section
+        ut = std::min<long long>(std::min<long long>(p->B, cap / (2 * hd)), std::max<long long>(1, 256 / p->H));
+        ut = std::min<long long>(ut, kMaxUnitTokens);
+        long long want = ut;
+        for (int t = 0; t < 4; t++) {
+            long long m = 0;
+            if (p->B <= kMaxUnitTokens && (long long)p->rec_bytes[t] <= cap)
+                m = std::min<long long>(std::min<long long>(kMaxUnitRecords, cap / p->rec_bytes[t]), kMaxUnitTokens / p->B);
+            p->unit_records[t] = (int32_t)m;
+            want = std::max(want, m * p->B);
+        }
+        if (want == rows) break;
+        rows = want;
+    }
+    cap = (stage_total - 32 - 16 * rows) / 16 * 16;
+    for (int t = 0; t < 4; t++)
+        while (p->unit_records[t] > 0 && ((long long)p->unit_records[t] * p->rec_bytes[t] > cap || (long long)p->unit_records[t] * p->B > rows))
+            p->unit_records[t]--;
+    if (ut < 1 || 2 * ut * hd > cap || ut > rows) return false;
+    p->unit_tokens = (int32_t)ut;
+    p->stage_data_bytes = (int32_t)cap;
+    p->stage_bytes = (int32_t)((cap + 16 * rows + 32 + 127) / 128 * 128);
+    long long stages = budget / p->stage_bytes;
+    if (stages > kMaxStages) stages = kMaxStages;
+    if (stages < 2) return false;
+    p->n_stages = (int32_t)stages;
+    p->B_shift = (p->B & (p->B - 1)) == 0 ? 31 - __builtin_clz((unsigned)p->B) : -1;
+    p->P_shift = (p->P & (p->P - 1)) == 0 ? 31 - __builtin_clz((unsigned)p->P) : -1;
+    // Self-scheduled rounds.  The resolver's chain of dependent lookups (about 5 us under load) has to stay shorter than
+    // the time the CTA spends issuing the previous round, so a round carries about 100 KiB of traffic (a block moves
+    // about 1.6 x its bf16 size) - measured best at 2 blocks for 64-KiB records, 4 for 32- and 16-KiB records; larger
+    // rounds only cost balance, a deeper ring of resolved rounds was slower at every size (it commits work too early).
+    // Rounds shrink towards the end of the list: a fraction 1 / round_div of what is left per CTA.
+    const long long rec_bf16 = 4ll * p->B * hd;
+    const long long traffic = rec_bf16 * 13 / 8;
+    long long rcap = (105 * 1024 + traffic - 1) / traffic;
+    rcap = std::max<long long>(rcap, rec_bf16 >= 64 * 1024 ? 2 : 4);
+    p->round_cap = (int32_t)std::min<long long>(rcap, 32);
+    p->round_div = (int32_t)std::max<long long>(2, std::min<long long>(8, rec_bf16 / 8192));
     return true;
 }
 

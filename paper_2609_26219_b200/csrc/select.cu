@@ -351,6 +351,9 @@ select_kernel(const TopkParams p) {
     __shared__ int s_krem;
     __shared__ unsigned int s_or[2];
 
+    // The kernel that follows in the stream (the restore, launched with programmatic stream serialisation) may be
+    // brought onto the SMs now; it still waits for this grid to finish before it reads the lists written here.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int l = blockIdx.x;
     const unsigned long long* key = p.mass + (p.shared ? 0 : (long long)l * p.NB);
     const int NB = p.NB, n_dirty = min(p.n_dirty, NB);
@@ -490,6 +493,7 @@ __global__ void __launch_bounds__(kSelThreads)
 block_round_kernel(const uint8_t* token_mask, int n, int B, int NB, uint8_t* mask, int32_t* repair_idx,
                    int32_t* repair_cnt, int32_t* reuse_idx, int32_t* reuse_cnt) {
     __shared__ int warp_sums[33];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");      // see select_kernel
     const int l = blockIdx.x;
     const uint8_t* tm = token_mask + (long long)l * n;
     uint8_t* bm = mask + (long long)l * NB;

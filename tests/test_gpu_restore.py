@@ -478,3 +478,26 @@ def test_restore_pipeline_leaves_cleanly_when_a_wait_runs_out():
         assert c.selftest_stall_next_launch(0, 0, check=False) == -1
     finally:
         c.close()
+
+
+SMALL_RECORD_GEOMETRIES = {
+    "H2_D128_B16": dict(geom=pin.Geometry(4, 2, 128, 128, pin.ROPE_HALF, 1e6, 16, 16, 32), n=16380),
+    "H1_D128_B16": dict(geom=pin.Geometry(4, 1, 128, 128, pin.ROPE_HALF, 5e5, 16, 16, 32), n=32768),
+    "H4_D64_B8_P16": dict(geom=pin.Geometry(4, 4, 64, 64, pin.ROPE_INTERLEAVED, 1e4, 8, 16, 32), n=16383, dst_shift=3),
+    "H2_D64_B32_P16": dict(geom=pin.Geometry(3, 2, 64, 32, pin.ROPE_HALF, 1e4, 32, 16, 16), n=40000, dst_shift=5),
+    "H4_D128_B16": dict(geom=pin.Geometry(3, 4, 128, 128, pin.ROPE_HALF, 1e6, 16, 16, 32), n=32768),
+}
+
+
+@pytest.mark.parametrize("name", sorted(SMALL_RECORD_GEOMETRIES))
+def test_small_records_share_units(ctx, name):
+    """Records far smaller than a stage of the pipeline travel several to a unit (neighbours of a same-tag run, one
+    bulk copy, one token table); enough blocks per CTA that rounds hold several blocks, all four tags, a partial last
+    block, pages that do not line up with blocks.  Compared in full with the oracle."""
+    kw = dict(SMALL_RECORD_GEOMETRIES[name])
+    g, n, shift = kw["geom"], kw["n"], kw.get("dst_shift", 0)
+    ck = pin.make_checkpoint(name=name, seed=11, geom=g, n=n, delta=-777, dst_shift=shift, tag_probs=(0.3, 0.3, 0.2, 0.2),
+                             n_outlier=3, outlier_scale=8.0, n_pages=-(-(n + shift) // g.page_tokens) + 37,
+                             dirty_tokens=n // 20, top_k=max(1, n // g.block_tokens // 40), device=DEV)
+    run_select_and_restore(ctx, ck)
+    run_select_and_restore(ctx, ck, host=True)

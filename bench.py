@@ -330,7 +330,8 @@ def host_leg_on(ctx, cks, label, ceiling, dev, stream, reps=5):
             "payload_gbps": useful / (t_ms * 1e-3) / 1e9, "link_ceiling_gbps": ceiling,
             "frac_of_link": useful / (t_ms * 1e-3) / 1e9 / ceiling, "bytes_useful": int(useful),
             "bytes_copied": int(stats_.bytes_copied), "bytes_wasted": int(stats_.bytes_copied - useful),
-            "copies": int(stats_.n_copies), "block_layers": int(items_h), "block_layers_per_s": items_h / (t_ms * 1e-3)}
+            "bytes_direct": int(stats_.bytes_direct), "copies": int(stats_.n_copies), "block_layers": int(items_h),
+            "block_layers_per_s": items_h / (t_ms * 1e-3)}
     del sts, hk, hv, hss
     torch.cuda.empty_cache()
     return out_
@@ -628,12 +629,14 @@ def run_ours(args):
         try:
             ceiling = pinned_copy_ceiling(dev)
             ctx_direct = pk.Context(device=local_rank, flags=pk.FLAG_HOST_DIRECT)
+            ctx_staged = pk.Context(device=local_rank, flags=pk.FLAG_HOST_STAGED)
 
             def host_leg(cks, label, reps=5, both=False):
                 out_ = host_leg_on(ctx, cks, label, ceiling, dev, stream, reps)
-                if both:     # the same through the zero-copy variant: the kernel pulls the records over the link itself
-                    d_ = host_leg_on(ctx_direct, cks, label, ceiling, dev, stream, reps)
-                    out_["zero_copy"] = {k_: d_[k_] for k_ in ("ms", "payload_gbps", "frac_of_link", "bytes_copied", "copies")}
+                if both:     # the same with staging copies only, and with none (the kernel pulls every record itself)
+                    for name_, c_ in (("staged_only", ctx_staged), ("zero_copy", ctx_direct)):
+                        d_ = host_leg_on(c_, cks, label, ceiling, dev, stream, reps)
+                        out_[name_] = {k_: d_[k_] for k_ in ("ms", "payload_gbps", "frac_of_link", "bytes_copied", "bytes_wasted", "copies")}
                 return out_
 
             try:
@@ -732,6 +735,7 @@ def run_ours(args):
                                  "select_us": r3(select_us), "restore_kernel_ms": r3(restore_avg_ms)},
             "3_7b_host": {"ms": r3(get(host_cfg3, "ms")), "gbps_bf16eq": r3(get(host_cfg3, "restored_kv_gbps_bf16_equiv")),
                           "frac_link": r3(get(host_cfg3, "frac_of_link")),
+                          "staged_only_frac_link": r3(get(host_cfg3, "staged_only", "frac_of_link")),
                           "zero_copy_frac_link": r3(get(host_cfg3, "zero_copy", "frac_of_link"))},
             "4_select_scale": {"select_us": r3(get(select_scale, "select_us")), "frac_hbm": r3(get(select_scale, "frac_of_hbm_peak")),
                                "token_form_us": r3(get(select_scale, "token_form_us_from_attention")),
@@ -871,7 +875,7 @@ def run_sweep(args):
     ck.payload = ck.payload.cpu().pin_memory()
     gaps = {}
     for gap in (0, 32 << 10, 64 << 10, 128 << 10, 256 << 10, 1 << 20):
-        c = pk.Context(device=0, merge_gap_bytes=gap)
+        c = pk.Context(device=0, merge_gap_bytes=gap, flags=pk.FLAG_HOST_STAGED)
         r = host_leg_on(c, [ck], "", ceiling, dev, stream, reps=5)
         gaps[str(gap)] = {"ms": r3(r["ms"]), "frac_link": r3(r["frac_of_link"]), "copies": r["copies"],
                           "wasted_frac": r3(r["bytes_wasted"] / r["bytes_useful"])}
@@ -880,10 +884,11 @@ def run_sweep(args):
     r = host_leg_on(c, [ck], "", ceiling, dev, stream, reps=5)
     c.close()
     r0 = host_leg_on(ctx, [ck], "", ceiling, dev, stream, reps=5)
-    out["host_path"] = {"link_ceiling_gbps": r3(ceiling), "by_merge_gap_bytes": gaps,
+    out["host_path"] = {"link_ceiling_gbps": r3(ceiling), "staged_only_by_merge_gap_bytes": gaps,
                         "zero_copy": {"ms": r3(r["ms"]), "frac_link": r3(r["frac_of_link"])},
-                        "default": {"ms": r3(r0["ms"]), "frac_link": r3(r0["frac_of_link"]), "copies": r0["copies"],
-                                    "wasted_frac": r3(r0["bytes_wasted"] / r0["bytes_useful"])}}
+                        "default_hybrid": {"ms": r3(r0["ms"]), "frac_link": r3(r0["frac_of_link"]), "copies": r0["copies"],
+                                           "direct_frac": r3(r0["bytes_direct"] / r0["bytes_useful"]),
+                                           "wasted_frac": r3(r0["bytes_wasted"] / r0["bytes_useful"])}}
     print(json.dumps({"sweep": out}), flush=True)
     ctx.close()
 

@@ -92,8 +92,10 @@ enum { PATCHKV_SCORE_ATTN_F16 = 0 /* stored attention */, PATCHKV_SCORE_BLOCK_MA
 
 enum {
     PATCHKV_FLAG_DIRECT_LOADS = 1, /* restore with the plain-load kernel even where the bulk-copy pipeline applies */
-    PATCHKV_FLAG_HOST_DIRECT = 2   /* restore_from_host: no staging copies; the restore kernel reads the pinned payload
+    PATCHKV_FLAG_HOST_DIRECT = 2,  /* restore_from_host: no staging copies; the restore kernel reads the pinned payload
                                       through its device alias, so exactly the reused records cross the link */
+    PATCHKV_FLAG_HOST_STAGED = 4   /* restore_from_host: staging copies only (ranges closer than merge_gap_bytes merged);
+                                      without either flag long runs are staged and short ones read directly, at once */
 };
 
 enum {
@@ -108,8 +110,9 @@ typedef struct {
     int32_t device;            /* CUDA device ordinal */
     int32_t staging_slots;     /* restore_from_host: depth of the device staging ring (0 = 4) */
     int32_t flags;             /* PATCHKV_FLAG_* */
-    uint64_t merge_gap_bytes;  /* restore_from_host: two reused records closer than this are fetched by one copy
-                                  (the bytes between them are transferred and ignored); UINT64_MAX = default 128 KiB */
+    uint64_t merge_gap_bytes;  /* restore_from_host with PATCHKV_FLAG_HOST_STAGED: two reused records closer than this
+                                  are fetched by one copy (the bytes between them are transferred and ignored);
+                                  UINT64_MAX = default 128 KiB */
 } patchkv_config;
 
 /* Model / cache geometry shared by all sessions of a call. */
@@ -222,6 +225,7 @@ typedef struct {
     uint64_t bytes_copied;       /* bytes that crossed the link */
     uint64_t bytes_useful;       /* bytes of reused records among them */
     uint64_t n_block_layers;     /* reused (layer, block) records */
+    uint64_t bytes_direct;       /* of bytes_copied: read over the link by the kernel itself (no staging copy) */
 } patchkv_restore_stats;
 
 /* Create / destroy a context bound to one device.  Creation allocates two streams, a few events and the
@@ -288,20 +292,26 @@ PATCHKV_API int patchkv_select_repair_static(const patchkv_select_args* args, vo
  * programmatic stream serialisation, so its set-up overlaps the tail of the kernel in front of it in the stream; it
  * touches no memory before that kernel has completed.
  * Launches from one context may overlap on the GPU when they are on different streams: the kernel's work counters
- * live in a slot that belongs to the stream (at most 191 different streams per context over its life), and a launch
+ * live in a slot that belongs to the stream (at most 190 different streams per context over its life), and a launch
  * recorded into a graph gets a slot of its own (at most 320 captured launches per context); beyond either limit the
  * call returns PATCHKV_E_UNSUPPORTED.  The kernel leaves its slot zeroed, so no reset is enqueued. */
 PATCHKV_API int patchkv_restore(patchkv_ctx* ctx, const patchkv_geom* geom, const patchkv_pool* pool,
                                 const patchkv_session* sessions, int n_sessions, void* stream);
 
 /* The same restore with the payloads in PINNED host memory (the CPU-resident checkpoint of Section II-C /
- * Section V-A): only the records of F are fetched, by asynchronous copies on an internal copy stream into a
- * ring of device staging slots (one layer of one session per slot), each decoded by the restore kernel on
- * an internal decode stream as soon as it has landed, so that transfer and decode overlap.  The internal
- * streams start after the work already on `stream` and `stream` waits for them before anything enqueued
- * later, so pages are complete for whatever follows on `stream`.  The call returns once everything is
- * enqueued; host arrays are consumed before it returns, the pinned payload must stay valid until the
- * stream work completes.  `stats` is optional. */
+ * Section V-A).  Only the records of F cross the link, layer by layer, by two routes at once: the long runs of records
+ * that lie back to back in a layer payload (same-tag runs are contiguous in the checkpoint) are fetched by the copy
+ * engine, one asynchronous copy per run on an internal copy stream into a ring of device staging slots (one layer of
+ * one session per slot), and decoded by the restore kernel on an internal decode stream as soon as the layer has
+ * landed; the layer's short runs are read over the link by a small side launch of the same kernel, whose bulk copies
+ * address the pinned payload through its device alias, while the engine works.  Nothing but reused records is
+ * transferred, and transfer and decode overlap.  PATCHKV_FLAG_HOST_STAGED (copy engine only, neighbouring ranges
+ * merged across gaps of up to merge_gap_bytes) and PATCHKV_FLAG_HOST_DIRECT (no staging at all: one launch reads every
+ * record itself) select the two routes on their own; a payload without a device alias is always staged.
+ * The internal streams start after the work already on `stream` and `stream` waits for them before anything enqueued
+ * later, so pages are complete for whatever follows on `stream`, also when the call returns an error half-way.
+ * The call returns once everything is enqueued; host arrays are consumed before it returns, the pinned payload must
+ * stay valid until the stream work completes.  `stats` is optional. */
 PATCHKV_API int patchkv_restore_from_host(patchkv_ctx* ctx, const patchkv_geom* geom, const patchkv_pool* pool,
                                           const patchkv_session_host* sessions, int n_sessions, void* stream,
                                           patchkv_restore_stats* stats);

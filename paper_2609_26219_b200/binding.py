@@ -25,6 +25,7 @@ SCORE_ATTN_F16, SCORE_BLOCK_MASS, SCORE_TOKEN_MASS = 0, 1, 2
 MAX_SESSIONS = 8
 FLAG_DIRECT_LOADS = 1
 FLAG_HOST_DIRECT = 2
+FLAG_HOST_STAGED = 4
 
 
 class Config(C.Structure):
@@ -69,7 +70,7 @@ class SelectArgs(C.Structure):
 
 class RestoreStats(C.Structure):
     _fields_ = [("struct_size", C.c_uint32), ("n_copies", C.c_uint32), ("bytes_copied", C.c_uint64),
-                ("bytes_useful", C.c_uint64), ("n_block_layers", C.c_uint64)]
+                ("bytes_useful", C.c_uint64), ("n_block_layers", C.c_uint64), ("bytes_direct", C.c_uint64)]
 
 
 _lib = None

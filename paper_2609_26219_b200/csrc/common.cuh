@@ -165,6 +165,7 @@ struct SessionDev {
     const int32_t* reuse_idx;
     const int32_t* reuse_cnt;
     int32_t n, nb, delta, dst_shift, n_table;
+    int32_t list_nb;        // row stride of reuse_idx, and work items per layer (nb unless the host path split the list)
     int32_t item_begin;     // first work item of this session in the launch's item numbering
 };
 
@@ -178,6 +179,7 @@ struct RestoreParams {
     int32_t n_pages;
     // work: items are (session, layer in [layer_begin, layer_end), position r in the reuse list)
     int32_t n_sessions, layer_begin, layer_end, total_items;
+    int32_t grid_cap;       // > 0: launch at most this many CTAs (the host path's side launch that reads over the link)
     int32_t* status;        // device status word
     int32_t* sched;         // this launch's slot of work counters: [0] blocks handed out, [1] CTAs that have left
                             // (the last CTA to leave zeroes both, so the slot starts the next launch at zero)
@@ -214,8 +216,12 @@ struct patchkv_ctx {
     int max_smem_optin = 0;
     int smem_per_sm = 0;
     uint64_t merge_gap = 64 * 1024;
-    cudaStream_t copy_stream = nullptr, decode_stream = nullptr;
-    cudaEvent_t ev_begin = nullptr, ev_done = nullptr;
+    int direct_percent = 48;                // hybrid host path: share of a layer's bytes that its side launch reads directly ...
+    uint64_t pause_fill_bytes = 100 * 1024; // ... plus this much per copy left to the engine (half of what the side launch
+                                            // reads during the engine's pause between two copies, ~4 us at ~50 GB/s)
+    int direct_ctas = 4;                    // hybrid host path: CTAs of a side launch
+    cudaStream_t copy_stream = nullptr, decode_stream = nullptr, direct_stream = nullptr;
+    cudaEvent_t ev_begin = nullptr, ev_done = nullptr, ev_direct = nullptr;
     int32_t* d_status = nullptr;
     // Work-counter slots of the restore pipeline (two words each, zero between launches: the kernel resets its
     // own slot).  A slot is private to whatever serialises the launches that use it: slot 0 belongs to the internal
@@ -234,6 +240,7 @@ struct patchkv_ctx {
     std::vector<patchkv::Staging> slots;
     uint8_t* d_meta = nullptr;
     uint8_t* h_meta = nullptr;      // pinned mirror
+    uint8_t* h_meta_alias = nullptr;    // its device alias (the host path's kernels read their reuse lists there)
     size_t meta_bytes = 0;
     bool host_call_pending = false;
     std::string last_error;
@@ -242,7 +249,7 @@ struct patchkv_ctx {
 
 namespace patchkv {
 
-constexpr int kSchedStreamSlots = 192;      // slot 0: internal decode stream; 1 .. 191: caller streams
+constexpr int kSchedStreamSlots = 192;      // slots 0, 1: the internal decode and direct streams; 2 .. 191: caller streams
 constexpr int kSchedCaptureSlots = 320;     // launches recorded into CUDA graphs over the life of a context
 constexpr int kSchedSlots = kSchedStreamSlots + kSchedCaptureSlots;
 

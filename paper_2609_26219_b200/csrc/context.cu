@@ -21,6 +21,8 @@ extern "C" int patchkv_create(patchkv_ctx** out, const patchkv_config* cfg) {
     ok = ok && cudaDeviceGetAttribute(&ctx->smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, cfg->device) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&ctx->decode_stream, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&ctx->direct_stream, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&ctx->ev_direct, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&ctx->ev_begin, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&ctx->ev_done, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->d_status, sizeof(int32_t)) == cudaSuccess;
@@ -54,6 +56,8 @@ extern "C" int patchkv_destroy(patchkv_ctx* ctx) {
         if (ctx->ev_done) cudaEventDestroy(ctx->ev_done);
         if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
         if (ctx->decode_stream) cudaStreamDestroy(ctx->decode_stream);
+        if (ctx->direct_stream) cudaStreamDestroy(ctx->direct_stream);
+        if (ctx->ev_direct) cudaEventDestroy(ctx->ev_direct);
     }
     delete ctx;
     return PATCHKV_OK;

@@ -255,14 +255,14 @@ restore_kernel(const __grid_constant__ RestoreParams p) {
         for (int k = 1; k < p.n_sessions; k++) if (item >= p.s[k].item_begin) si = k;
         const SessionDev& S = p.s[si];
         const int local = item - S.item_begin;
-        const int l = p.layer_begin + local / S.nb;
-        const int r = local - (l - p.layer_begin) * S.nb;
+        const int l = p.layer_begin + local / S.list_nb;
+        const int r = local - (l - p.layer_begin) * S.list_nb;
         if (r >= __ldg(S.reuse_cnt + l)) continue;                     // uniform over the CTA
 
         if (si != cur_session) { cur_session = si; load_rotation<INTER>(p, si, tm, tc, ts); }
 
         // ---- directory entry of the block; every thread reads the same words (broadcast)
-        const int j = __ldg(S.reuse_idx + (size_t)l * S.nb + r);
+        const int j = __ldg(S.reuse_idx + (size_t)l * S.list_nb + r);
         bool bad = j < 0 || j >= S.nb;
         int tag = 0;
         unsigned long long off = 0, rec = 0, lbytes = 0;
@@ -475,11 +475,11 @@ restore_pipe_kernel(const __grid_constant__ RestoreParams p) {
                 for (int k = 1; k < p.n_sessions; k++) if (item >= p.s[k].item_begin) si = k;
                 const SessionDev& Sd = p.s[si];
                 const int local = (int)item - Sd.item_begin;
-                const int l = p.layer_begin + local / Sd.nb;
-                const int r = local - (l - p.layer_begin) * Sd.nb;
-                // r < nb, so the list entry can be read before the list length is known
+                const int l = p.layer_begin + local / Sd.list_nb;
+                const int r = local - (l - p.layer_begin) * Sd.list_nb;
+                // r < list_nb, so the list entry can be read before the list length is known
                 const int cnt = __ldg(Sd.reuse_cnt + l);
-                const int j = __ldg(Sd.reuse_idx + (size_t)l * Sd.nb + r);
+                const int j = __ldg(Sd.reuse_idx + (size_t)l * Sd.list_nb + r);
                 if (r < cnt) {
                     bool bad = j < 0 || j >= Sd.nb;
                     if (!bad) {
@@ -878,10 +878,11 @@ static bool plan_pipeline(const patchkv_ctx* ctx, RestoreParams* p) {
 }
 
 // The slot of work counters a pipeline launch on `stream` uses.  Launches that share a slot must never overlap on the
-// GPU, so a slot belongs to whatever serialises them: the internal decode stream (slot 0), one caller stream each
-// (slots 1 ...), or one captured launch (a graph node can be replayed from any stream, next to anything).
+// GPU, so a slot belongs to whatever serialises them: the two internal streams (slots 0 and 1), one caller stream each
+// (slots 2 ...), or one captured launch (a graph node can be replayed from any stream, next to anything).
 static int sched_slot(patchkv_ctx* ctx, cudaStream_t stream, bool capturing, int* slot) {
     if (stream == ctx->decode_stream && !capturing) { *slot = 0; return PATCHKV_OK; }
+    if (stream == ctx->direct_stream && !capturing) { *slot = 1; return PATCHKV_OK; }
     if (capturing) {
         if (ctx->sched_captured >= kSchedCaptureSlots)
             return fail(ctx, PATCHKV_E_UNSUPPORTED, "restore: too many launches captured into CUDA graphs by this context");
@@ -892,11 +893,11 @@ static int sched_slot(patchkv_ctx* ctx, cudaStream_t stream, bool capturing, int
     const uint64_t handle = reinterpret_cast<uintptr_t>(stream);
     const uint64_t owner = stream == cudaStreamPerThread ? (uint64_t)std::hash<std::thread::id>()(std::this_thread::get_id()) : 0;
     for (size_t i = 0; i < ctx->sched_streams.size(); i++)
-        if (ctx->sched_streams[i].first == handle && ctx->sched_streams[i].second == owner) { *slot = 1 + (int)i; return PATCHKV_OK; }
-    if ((int)ctx->sched_streams.size() >= kSchedStreamSlots - 1)
+        if (ctx->sched_streams[i].first == handle && ctx->sched_streams[i].second == owner) { *slot = 2 + (int)i; return PATCHKV_OK; }
+    if ((int)ctx->sched_streams.size() >= kSchedStreamSlots - 2)
         return fail(ctx, PATCHKV_E_UNSUPPORTED, "restore: this context has been used from too many different streams");
     ctx->sched_streams.emplace_back(handle, owner);
-    *slot = (int)ctx->sched_streams.size();
+    *slot = 1 + (int)ctx->sched_streams.size();
     return PATCHKV_OK;
 }
 
@@ -921,6 +922,7 @@ int launch_restore(patchkv_ctx* ctx, RestoreParams* p, cudaStream_t stream) {
         const int smem = p->n_stages * p->stage_bytes;
         int grid = ctx->sm_count * 2;
         if (grid > p->total_items) grid = p->total_items;
+        if (p->grid_cap > 0 && grid > p->grid_cap) grid = p->grid_cap;
         cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
         PKV_CUDA(ctx, cudaStreamIsCapturing(stream, &cap));
         const bool capturing = cap != cudaStreamCaptureStatusNone;
@@ -960,7 +962,7 @@ extern "C" int patchkv_restore(patchkv_ctx* ctx, const patchkv_geom* geom, const
     static thread_local RestoreParams p;
     int rc = fill_geometry(ctx, geom, pool, &p);
     if (rc != PATCHKV_OK) return rc;
-    p.n_sessions = n_sessions; p.layer_begin = 0; p.layer_end = geom->n_layers;
+    p.n_sessions = n_sessions; p.layer_begin = 0; p.layer_end = geom->n_layers; p.grid_cap = 0;
     long long items = 0;
     for (int i = 0; i < n_sessions; i++) {
         const patchkv_session& s = sessions[i];
@@ -976,7 +978,7 @@ extern "C" int patchkv_restore(patchkv_ctx* ctx, const patchkv_geom* geom, const
         d.layer_payload = s.layer_payload;
         d.layer_bytes = reinterpret_cast<const unsigned long long*>(s.layer_bytes);
         d.reuse_idx = s.reuse_idx; d.reuse_cnt = s.reuse_cnt;
-        d.n = s.n_suffix_tokens; d.nb = nb; d.delta = s.delta; d.dst_shift = s.dst_shift; d.n_table = s.n_table;
+        d.n = s.n_suffix_tokens; d.nb = nb; d.list_nb = nb; d.delta = s.delta; d.dst_shift = s.dst_shift; d.n_table = s.n_table;
         d.item_begin = (int32_t)items;
         items += (long long)nb * geom->n_layers;
         if (items > 0x7fff0000LL) return fail(ctx, PATCHKV_E_UNSUPPORTED, "restore: more than 2^31 work items");

@@ -125,6 +125,25 @@ __device__ __forceinline__ uint16_t lds16(uint32_t a) {
     return v;
 }
 
+// Programmatic dependent launch (sm_90+).  A kernel launched with launch_pdl may be brought onto the SMs while the kernel
+// in front of it in the stream is still running; it calls pdl_wait() before it touches global memory, which returns
+// once that kernel has completed and its writes are visible.  pdl_trigger() tells the runtime that the kernel behind
+// this one may be brought on.  Both are no-ops for kernels launched the ordinary way.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args&&... args) {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
 // Exclusive prefix sum of v over a CTA of kScanThreads threads; *total receives the CTA sum.  `warp_sums` is 33 ints
 // of shared memory.  Every thread of the CTA has to call it (it contains CTA-wide barriers).
 constexpr int kScanThreads = 1024;

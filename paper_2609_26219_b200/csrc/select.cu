@@ -32,6 +32,8 @@ struct MassParams {
     int Hq, Q, n, B, NB;
     int rows_per_cta;
     unsigned long long* mass;   // [L][NB], zeroed before the launch
+    long long mass_stride;      // elements between the rows of two layers (0: every layer adds into one row, which is
+                                // the layer-summed mass of LAYERS_SHARED; exact, so the order of the adds is immaterial)
     int32_t* status;
 };
 
@@ -92,6 +94,8 @@ constexpr int kMassBatch = 8;      // rows whose loads are issued before any of 
 // grid = (octet tiles, row groups, layers).
 __global__ void __launch_bounds__(256)
 block_mass_octet_kernel(const MassParams p) {
+    pdl_wait();
+    pdl_trigger();
     const int oct = blockIdx.x * blockDim.x + threadIdx.x;
     const int col = oct * 8;
     const int l = blockIdx.z;
@@ -155,16 +159,18 @@ block_mass_octet_kernel(const MassParams p) {
             const unsigned long long o = __shfl_down_sync(0xFFFFFFFFu, acc, d);
             if ((lane & (2 * d - 1)) == 0) acc += o;     // only segment-aligned lanes keep a full sum
         }
-        if (in_range && (lane & (opb - 1)) == 0 && acc) atomicAdd(p.mass + (long long)l * p.NB + col / p.B, acc);
+        if (in_range && (lane & (opb - 1)) == 0 && acc) atomicAdd(p.mass + (long long)l * p.mass_stride + col / p.B, acc);
     } else if (in_range && acc) {
-        atomicAdd(p.mass + (long long)l * p.NB + col / p.B, acc);
+        atomicAdd(p.mass + (long long)l * p.mass_stride + col / p.B, acc);
     }
 }
 
 // Token granularity (the score of Eq. 10 per token): one thread owns eight consecutive tokens and keeps one exact sum
 // per token over the rows of its CTA.  Same loads and the same exact-fp32 fast path as the block kernel.
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 4)
 token_mass_octet_kernel(const MassParams p) {
+    pdl_wait();
+    pdl_trigger();
     const int oct = blockIdx.x * blockDim.x + threadIdx.x;
     const int col = oct * 8;
     const int l = blockIdx.z;
@@ -180,7 +186,7 @@ token_mass_octet_kernel(const MassParams p) {
                 acc += units_any(__ldg(p.attn + (long long)l * p.stride_layer + (long long)h * p.stride_head +
                                        (long long)q * p.stride_query + col + i), &bad);
             }
-            if (acc) atomicAdd(p.mass + (long long)l * p.NB + col + i, acc);
+            if (acc) atomicAdd(p.mass + (long long)l * p.mass_stride + col + i, acc);
         }
         if (bad) atomicCAS(p.status, 0, (int)PATCHKV_E_BADINPUT);
         return;
@@ -277,13 +283,15 @@ token_mass_octet_kernel(const MassParams p) {
 #pragma unroll
     for (int k = 0; k < 8; k++) {
         const unsigned long long v = acc[k] + __float2uint_rz(facc[k] * 16777216.0f);
-        if (v) atomicAdd(p.mass + (long long)l * p.NB + col + k, v);
+        if (v) atomicAdd(p.mass + (long long)l * p.mass_stride + col + k, v);
     }
 }
 
 // Any B, any strides, any alignment: one thread per key position.
 __global__ void __launch_bounds__(256)
 block_mass_generic_kernel(const MassParams p) {
+    pdl_wait();
+    pdl_trigger();
     const int col = blockIdx.x * blockDim.x + threadIdx.x;
     const int l = blockIdx.z;
     const int R = p.Hq * p.Q;
@@ -299,14 +307,24 @@ block_mass_generic_kernel(const MassParams p) {
         acc += units_any(x, &bad);
     }
     if (bad) atomicCAS(p.status, 0, (int)PATCHKV_E_BADINPUT);
-    if (acc) atomicAdd(p.mass + (long long)l * p.NB + col / p.B, acc);
+    if (acc) atomicAdd(p.mass + (long long)l * p.mass_stride + col / p.B, acc);
 }
 
 __global__ void sum_layers_kernel(const unsigned long long* mass, int L, int NB, unsigned long long* out) {
+    pdl_wait();
+    pdl_trigger();
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= NB) return;
     unsigned long long s = 0;
-    for (int l = 0; l < L; l++) s += mass[(long long)l * NB + j];
+    int l = 0;
+    for (; l + 8 <= L; l += 8) {                         // eight loads in flight, then the adds
+        unsigned long long v[8];
+#pragma unroll
+        for (int u = 0; u < 8; u++) v[u] = mass[(long long)(l + u) * NB + j];
+#pragma unroll
+        for (int u = 0; u < 8; u++) s += v[u];
+    }
+    for (; l < L; l++) s += mass[(long long)l * NB + j];
     out[j] = s;
 }
 
@@ -314,6 +332,7 @@ __global__ void sum_layers_kernel(const unsigned long long* mass, int L, int NB,
 struct TopkParams {
     const unsigned long long* mass;     // [L][NB], or [NB] when shared
     int shared;                         // 1: every layer ranks on mass[0..NB)
+    int spill_keys;                     // candidates the kernel may keep in its dynamic shared memory
     int NB, n_dirty, top_k;
     uint8_t* mask;
     int32_t* repair_idx; int32_t* repair_cnt;
@@ -326,6 +345,8 @@ constexpr int kSelThreads = kScanThreads;
 // to fp32.  Reported only; the ranking uses the exact masses.
 __global__ void __launch_bounds__(256)
 normalise_kernel(const unsigned long long* mass, int NB, float* score) {
+    pdl_wait();
+    pdl_trigger();
     __shared__ unsigned long long part[8];
     const unsigned long long* m = mass + (long long)blockIdx.x * NB;
     unsigned long long t = 0;
@@ -348,12 +369,14 @@ select_kernel(const TopkParams p) {
     __shared__ unsigned int hist[256];
     __shared__ int warp_sums[33];
     __shared__ unsigned long long s_prefix;
-    __shared__ int s_krem;
+    __shared__ int s_krem, s_eq;
     __shared__ unsigned int s_or[2];
 
     // The kernel that follows in the stream (the restore, launched with programmatic stream serialisation) may be
     // brought onto the SMs now; it still waits for this grid to finish before it reads the lists written here.
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    pdl_wait();
+    pdl_trigger();
+    extern __shared__ unsigned long long spill[];        // candidates beyond the register-cached ones (p.spill_keys of them)
     const int l = blockIdx.x;
     const unsigned long long* key = p.mass + (p.shared ? 0 : (long long)l * p.NB);
     const int NB = p.NB, n_dirty = min(p.n_dirty, NB);
@@ -363,16 +386,22 @@ select_kernel(const TopkParams p) {
     const int iters = (ncand + kSelThreads - 1) / kSelThreads;
     const unsigned lane = threadIdx.x & 31u;
 
-    // candidate c = threadIdx.x + i * kSelThreads is block n_dirty + c; the first kKeysPerThread rounds live in registers
+    // candidate c = threadIdx.x + i * kSelThreads is block n_dirty + c; the first kKeysPerThread rounds live in registers,
+    // the next p.spill_keys candidates in shared memory, anything beyond that is re-read from global memory
     unsigned long long kreg[kKeysPerThread];
 #pragma unroll
     for (int i = 0; i < kKeysPerThread; i++) {
         const int c = threadIdx.x + i * kSelThreads;
         kreg[i] = c < ncand ? key[n_dirty + c] : 0ull;
     }
+    const int reg_keys = kKeysPerThread * kSelThreads;
+    for (int c = reg_keys + threadIdx.x; c < ncand && c - reg_keys < p.spill_keys; c += kSelThreads) spill[c - reg_keys] = key[n_dirty + c];
+    auto later_key = [&](int c) -> unsigned long long {      // a candidate of a later round (a thread reads back its own writes only)
+        return c - reg_keys < p.spill_keys ? spill[c - reg_keys] : key[n_dirty + c];
+    };
 
     unsigned long long T = 0;
-    int krem = 0;
+    int krem = 0, n_eq = 0;                      // keys equal to T: krem of them are taken, n_eq exist
     if (!take_all && !take_none) {
         // highest byte that is non-zero in any candidate: the passes above it would all pick digit 0
         unsigned long long orv = 0;
@@ -380,9 +409,9 @@ select_kernel(const TopkParams p) {
         for (int i = 0; i < kKeysPerThread; i++) orv |= kreg[i];
         for (int i = kKeysPerThread; i < iters; i++) {
             const int c = threadIdx.x + i * kSelThreads;
-            if (c < ncand) orv |= key[n_dirty + c];
+            if (c < ncand) orv |= later_key(c);
         }
-        if (threadIdx.x == 0) { s_or[0] = 0; s_or[1] = 0; s_prefix = 0; s_krem = k; }
+        if (threadIdx.x == 0) { s_or[0] = 0; s_or[1] = 0; s_prefix = 0; s_krem = k; s_eq = ncand; }
         __syncthreads();
         const unsigned lo = __reduce_or_sync(0xFFFFFFFFu, (unsigned)orv);
         const unsigned hi = __reduce_or_sync(0xFFFFFFFFu, (unsigned)(orv >> 32));
@@ -398,20 +427,28 @@ select_kernel(const TopkParams p) {
             __syncthreads();
             const unsigned long long prefix = s_prefix;
             const int need = s_krem;
+            // In the high bytes most keys share one digit (a long tail of small masses), and thousands of atomics on one
+            // counter serialise; a warp whose live lanes all hold the same digit adds its count with one atomic.
+            auto count_digit = [&](bool live, unsigned long long x) {
+                const unsigned digit = (unsigned)(x >> (8 * b)) & 255u;
+                const unsigned act = __ballot_sync(0xFFFFFFFFu, live);
+                if (live) {
+                    int same;
+                    __match_all_sync(act, digit, &same);
+                    if (!same) atomicAdd(&hist[digit], 1u);
+                    else if (lane == (unsigned)(__ffs(act) - 1)) atomicAdd(&hist[digit], (unsigned)__popc(act));
+                }
+            };
 #pragma unroll
             for (int i = 0; i < kKeysPerThread; i++) {
                 const int c = threadIdx.x + i * kSelThreads;
                 const unsigned long long x = kreg[i];
-                if (c < ncand && (b == 7 || ((x ^ prefix) >> (8 * (b + 1))) == 0))
-                    atomicAdd(&hist[(unsigned)(x >> (8 * b)) & 255u], 1u);
+                count_digit(c < ncand && (b == 7 || ((x ^ prefix) >> (8 * (b + 1))) == 0), x);
             }
             for (int i = kKeysPerThread; i < iters; i++) {
                 const int c = threadIdx.x + i * kSelThreads;
-                if (c < ncand) {
-                    const unsigned long long x = key[n_dirty + c];
-                    if (b == 7 || ((x ^ prefix) >> (8 * (b + 1))) == 0)
-                        atomicAdd(&hist[(unsigned)(x >> (8 * b)) & 255u], 1u);
-                }
+                const unsigned long long x = c < ncand ? later_key(c) : 0ull;
+                count_digit(c < ncand && (b == 7 || ((x ^ prefix) >> (8 * (b + 1))) == 0), x);
             }
             __syncthreads();
             if (threadIdx.x < 32) {
@@ -433,6 +470,7 @@ select_kernel(const TopkParams p) {
                         if (cum < need && need <= cum + cnt[t]) {
                             s_prefix = prefix | ((unsigned long long)(255 - 8 * (int)lane - t) << (8 * b));
                             s_krem = need - cum;
+                            s_eq = cnt[t];               // after the last pass: how many keys equal the k-th largest
                         }
                         cum += cnt[t];
                     }
@@ -442,7 +480,10 @@ select_kernel(const TopkParams p) {
         }
         T = s_prefix;
         krem = s_krem;                           // keys equal to T to take, lowest block index first
+        n_eq = s_eq;
     }
+    // Ranking among equal keys (a prefix count in index order) is needed only when some of them stay out.
+    const bool ties_matter = !take_all && !take_none && n_eq > krem;
 
     // ---- emit mask and ascending lists: the dirty window first, then the candidates in index order
     uint8_t* mask = p.mask + (long long)l * NB;
@@ -458,19 +499,25 @@ select_kernel(const TopkParams p) {
         if (i < kKeysPerThread) {
 #pragma unroll
             for (int t = 0; t < kKeysPerThread; t++) if (t == i) x = kreg[t];
-        } else if (in) x = key[n_dirty + c];
+        } else if (in) x = later_key(c);
         bool sel = false;
         if (take_all) sel = in;
         else if (!take_none) {
-            const int eq = in && x == T;
-            int tot_eq;
-            const int rank = cta_exclusive_scan(eq, warp_sums, &tot_eq) + run_eq;
-            run_eq += tot_eq;
-            sel = in && (x > T || (eq && rank < krem));
+            sel = in && x >= T;
+            if (ties_matter) {
+                const int eq = in && x == T;
+                int tot_eq;
+                const int rank = cta_exclusive_scan(eq, warp_sums, &tot_eq) + run_eq;
+                run_eq += tot_eq;
+                sel = in && (x > T || (eq && rank < krem));
+            }
         }
-        int tot_sel;
-        const int before = cta_exclusive_scan(sel ? 1 : 0, warp_sums, &tot_sel) + run_sel;
-        run_sel += tot_sel;
+        int before = 0;
+        if (lists) {                                     // the mask alone needs no compaction
+            int tot_sel;
+            before = cta_exclusive_scan(sel ? 1 : 0, warp_sums, &tot_sel) + run_sel;
+            run_sel += tot_sel;
+        }
         if (in) {
             const int j = n_dirty + c;
             mask[j] = sel ? 1 : 0;
@@ -490,12 +537,13 @@ select_kernel(const TopkParams p) {
 // BlockRound of Eq. 12: a block is repaired when any of its tokens is in D u H.  One CTA per layer turns the token
 // mask into the block mask and the ascending repair / reuse lists.
 __global__ void __launch_bounds__(kSelThreads)
-block_round_kernel(const uint8_t* token_mask, int n, int B, int NB, uint8_t* mask, int32_t* repair_idx,
+block_round_kernel(const uint8_t* token_mask, long long mask_stride, int n, int B, int NB, uint8_t* mask, int32_t* repair_idx,
                    int32_t* repair_cnt, int32_t* reuse_idx, int32_t* reuse_cnt) {
     __shared__ int warp_sums[33];
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");      // see select_kernel
+    pdl_wait();
+    pdl_trigger();                                        // see select_kernel
     const int l = blockIdx.x;
-    const uint8_t* tm = token_mask + (long long)l * n;
+    const uint8_t* tm = token_mask + (long long)l * mask_stride;      // stride 0: one request-level token set for every layer
     uint8_t* bm = mask + (long long)l * NB;
     int32_t* ridx = repair_idx + (long long)l * NB;
     int32_t* fidx = reuse_idx + (long long)l * NB;
@@ -505,7 +553,14 @@ block_round_kernel(const uint8_t* token_mask, int n, int B, int NB, uint8_t* mas
         int hit = 0;
         if (j < NB) {
             const int e = min(n, (j + 1) * B);
-            for (int i = j * B; i < e; i++) hit |= tm[i];
+            if ((B & 15) == 0 && e == (j + 1) * B && ((reinterpret_cast<uintptr_t>(tm) + (size_t)j * B) & 15u) == 0) {
+                for (int i = j * B; i < e; i += 16) {
+                    const uint4 w = *reinterpret_cast<const uint4*>(tm + i);
+                    hit |= (w.x | w.y | w.z | w.w) != 0;
+                }
+            } else {
+                for (int i = j * B; i < e; i++) hit |= tm[i];
+            }
         }
         int tot;
         const int before = cta_exclusive_scan(hit, warp_sums, &tot) + run;
@@ -520,6 +575,20 @@ block_round_kernel(const uint8_t* token_mask, int n, int B, int NB, uint8_t* mas
     for (int i = n_r + threadIdx.x; i < NB; i += kSelThreads) ridx[i] = -1;
     for (int i = n_f + threadIdx.x; i < NB; i += kSelThreads) fidx[i] = -1;
     if (threadIdx.x == 0) { repair_cnt[l] = n_r; reuse_cnt[l] = n_f; }
+}
+
+// Shared memory for the candidates that select_kernel cannot keep in registers (it would otherwise re-read them from
+// global memory in every radix pass).
+static int select_spill(patchkv_ctx* ctx, int ncand, int* keys, int* bytes) {
+    long long want = (long long)ncand - (long long)kKeysPerThread * kSelThreads;
+    const long long cap = ((long long)ctx->max_smem_optin - 4096) / 8;
+    if (want < 0) want = 0;
+    if (want > cap) want = cap;
+    *keys = (int)want;
+    *bytes = (int)want * 8;
+    if (*bytes > 48 * 1024)
+        PKV_CUDA(ctx, cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, *bytes));
+    return PATCHKV_OK;
 }
 
 static int ensure_mass_ws(patchkv_ctx* ctx, size_t elems) {
@@ -576,7 +645,9 @@ extern "C" int patchkv_select_repair(patchkv_ctx* ctx, const patchkv_select_args
 
     const bool shared = a->layer_mode == PATCHKV_LAYERS_SHARED && L > 1;
     const bool from_attn = a->kind == PATCHKV_SCORE_ATTN_F16;
-    size_t ws_need = (from_attn && !a->mass_out ? (size_t)L * NB : 0) + (shared ? (size_t)NB : 0);
+    // (request-level ranking with nobody asking for the per-layer masses: every layer adds straight into the summed row)
+    const bool sum_direct = shared && from_attn && !a->mass_out;
+    size_t ws_need = (from_attn && !a->mass_out && !sum_direct ? (size_t)L * NB : 0) + (shared ? (size_t)NB : 0);
     if (ws_need) { int rc = ensure_mass_ws(ctx, ws_need); if (rc != PATCHKV_OK) return rc; }
     unsigned long long* ws = ctx->d_mass_ws;
 
@@ -585,16 +656,16 @@ extern "C" int patchkv_select_repair(patchkv_ctx* ctx, const patchkv_select_args
         if (a->n_q_heads < 0 || a->n_queries < 0 || (NB > 0 && a->n_q_heads > 0 && a->n_queries > 0 && !a->attn))
             return fail(ctx, PATCHKV_E_INVALID, "select: attention shape / pointer");
         unsigned long long* m = a->mass_out ? reinterpret_cast<unsigned long long*>(a->mass_out) : ws;
-        if (!a->mass_out) ws += (size_t)L * NB;
+        if (!a->mass_out && !sum_direct) ws += (size_t)L * NB;
         const long long rows = (long long)a->n_q_heads * a->n_queries;
-        if (NB > 0) PKV_CUDA(ctx, cudaMemsetAsync(m, 0, (size_t)L * NB * sizeof(unsigned long long), stream));
+        if (NB > 0) PKV_CUDA(ctx, cudaMemsetAsync(m, 0, (size_t)(sum_direct ? 1 : L) * NB * sizeof(unsigned long long), stream));
         if (NB > 0 && rows > 0) {
             if (rows > 0x7fffffffLL) return fail(ctx, PATCHKV_E_UNSUPPORTED, "select: Hq * Q too large");
             MassParams mp;
             mp.attn = static_cast<const uint16_t*>(a->attn);
             mp.stride_layer = a->attn_stride_layer; mp.stride_head = a->attn_stride_head; mp.stride_query = a->attn_stride_query;
             mp.Hq = a->n_q_heads; mp.Q = a->n_queries; mp.n = n; mp.B = B; mp.NB = NB;
-            mp.mass = m; mp.status = ctx->d_status;
+            mp.mass = m; mp.mass_stride = sum_direct ? 0 : NB; mp.status = ctx->d_status;
             const bool octet = (B % 8 == 0) && ((reinterpret_cast<uintptr_t>(a->attn) & 15u) == 0) &&
                                ((a->attn_stride_layer | a->attn_stride_head | a->attn_stride_query) & 7) == 0;
             const int cols = octet ? (n + 7) / 8 : n;
@@ -611,9 +682,7 @@ extern "C" int patchkv_select_repair(patchkv_ctx* ctx, const patchkv_select_args
             if (groups > 65535 || L > 65535) return fail(ctx, PATCHKV_E_UNSUPPORTED, "select: grid too large");
             mp.rows_per_cta = (int)rpc;
             dim3 grid(tiles, (unsigned)groups, L);
-            if (octet) block_mass_octet_kernel<<<grid, 256, 0, stream>>>(mp);
-            else block_mass_generic_kernel<<<grid, 256, 0, stream>>>(mp);
-            PKV_CUDA(ctx, cudaGetLastError());
+            PKV_CUDA(ctx, launch_pdl(octet ? block_mass_octet_kernel : block_mass_generic_kernel, grid, dim3(256), 0, stream, mp));
         }
         mass = m;
     } else if (NB > 0 && !mass) {
@@ -623,16 +692,18 @@ extern "C" int patchkv_select_repair(patchkv_ctx* ctx, const patchkv_select_args
     TopkParams tp;
     tp.mass = mass; tp.shared = 0;
     if (shared && NB > 0) {
-        sum_layers_kernel<<<(NB + 255) / 256, 256, 0, stream>>>(mass, L, NB, ws);
-        PKV_CUDA(ctx, cudaGetLastError());
+        if (!sum_direct) PKV_CUDA(ctx, launch_pdl(sum_layers_kernel, dim3((NB + 255) / 256), dim3(256), 0, stream, mass, L, NB, ws));
         tp.mass = ws; tp.shared = 1;
     }
     tp.NB = NB; tp.n_dirty = n_dirty; tp.top_k = a->top_k;
     tp.mask = a->repair_mask; tp.repair_idx = a->repair_idx; tp.repair_cnt = a->repair_cnt;
     tp.reuse_idx = a->reuse_idx; tp.reuse_cnt = a->reuse_cnt;
-    if (a->score_out && NB > 0) normalise_kernel<<<tp.shared ? 1 : L, 256, 0, stream>>>(tp.mass, NB, a->score_out);
-    select_kernel<<<L, kSelThreads, 0, stream>>>(tp);
-    PKV_CUDA(ctx, cudaGetLastError());
+    if (a->score_out && NB > 0)
+        PKV_CUDA(ctx, launch_pdl(normalise_kernel, dim3(tp.shared ? 1 : L), dim3(256), 0, stream, tp.mass, NB, a->score_out));
+    int spill_bytes = 0;
+    int rc2 = select_spill(ctx, NB - n_dirty, &tp.spill_keys, &spill_bytes);
+    if (rc2 != PATCHKV_OK) return rc2;
+    PKV_CUDA(ctx, launch_pdl(select_kernel, dim3(L), dim3(kSelThreads), (size_t)spill_bytes, stream, tp));
     PKV_CUDA(ctx, mirror_to_host(a, L, NB, stream));
     return PATCHKV_OK;
 }
@@ -661,7 +732,9 @@ extern "C" int patchkv_select_repair_tokens(patchkv_ctx* ctx, const patchkv_sele
     const bool shared = a->layer_mode == PATCHKV_LAYERS_SHARED && L > 1;
     const bool from_attn = a->kind == PATCHKV_SCORE_ATTN_F16;
     // workspace: [token mass L*n (if computed here and not handed out)] [summed mass n (shared)] [token mask L*n bytes]
-    const size_t mass_elems = from_attn && !a->mass_out ? (size_t)L * n : 0;
+    // (request-level ranking with nobody asking for the per-layer masses: every layer adds straight into the summed row)
+    const bool sum_direct = shared && from_attn && !a->mass_out;
+    const size_t mass_elems = from_attn && !a->mass_out && !sum_direct ? (size_t)L * n : 0;
     const size_t sum_elems = shared ? (size_t)n : 0;
     const size_t mask_words = ((size_t)L * n + 7) / 8;
     int rc = ensure_mass_ws(ctx, mass_elems + sum_elems + mask_words + 1);
@@ -674,16 +747,16 @@ extern "C" int patchkv_select_repair_tokens(patchkv_ctx* ctx, const patchkv_sele
     if (from_attn) {
         if (a->n_q_heads < 0 || a->n_queries < 0 || (n > 0 && a->n_q_heads > 0 && a->n_queries > 0 && !a->attn))
             return fail(ctx, PATCHKV_E_INVALID, "select: attention shape / pointer");
-        unsigned long long* m = a->mass_out ? reinterpret_cast<unsigned long long*>(a->mass_out) : ws;
+        unsigned long long* m = a->mass_out ? reinterpret_cast<unsigned long long*>(a->mass_out) : (sum_direct ? ws_sum : ws);
         const long long rows = (long long)a->n_q_heads * a->n_queries;
         if (rows > 0x7fffffffLL) return fail(ctx, PATCHKV_E_UNSUPPORTED, "select: Hq * Q too large");
-        if (n > 0) PKV_CUDA(ctx, cudaMemsetAsync(m, 0, (size_t)L * n * sizeof(unsigned long long), stream));
+        if (n > 0) PKV_CUDA(ctx, cudaMemsetAsync(m, 0, (size_t)(sum_direct ? 1 : L) * n * sizeof(unsigned long long), stream));
         if (n > 0 && rows > 0) {
             MassParams mp;                         // token granularity: a block of one token
             mp.attn = static_cast<const uint16_t*>(a->attn);
             mp.stride_layer = a->attn_stride_layer; mp.stride_head = a->attn_stride_head; mp.stride_query = a->attn_stride_query;
             mp.Hq = a->n_q_heads; mp.Q = a->n_queries; mp.n = n; mp.B = 1; mp.NB = n;
-            mp.mass = m; mp.status = ctx->d_status;
+            mp.mass = m; mp.mass_stride = sum_direct ? 0 : n; mp.status = ctx->d_status;
             const bool octet = ((reinterpret_cast<uintptr_t>(a->attn) & 15u) == 0) &&
                                ((a->attn_stride_layer | a->attn_stride_head | a->attn_stride_query) & 7) == 0;
             const int cols = octet ? (n + 7) / 8 : n;
@@ -710,9 +783,8 @@ extern "C" int patchkv_select_repair_tokens(patchkv_ctx* ctx, const patchkv_sele
             long long groups = (rows + rpc - 1) / rpc;
             if (groups > 65535) return fail(ctx, PATCHKV_E_UNSUPPORTED, "select: grid too large");
             mp.rows_per_cta = (int)rpc;
-            if (octet) token_mass_octet_kernel<<<dim3(tiles, (unsigned)groups, L), 256, 0, stream>>>(mp);
-            else block_mass_generic_kernel<<<dim3(tiles, (unsigned)groups, L), 256, 0, stream>>>(mp);
-            PKV_CUDA(ctx, cudaGetLastError());
+            PKV_CUDA(ctx, launch_pdl(octet ? token_mass_octet_kernel : block_mass_generic_kernel,
+                                     dim3(tiles, (unsigned)groups, L), dim3(256), 0, stream, mp));
         }
         mass = m;
     } else if (n > 0 && !mass) {
@@ -722,18 +794,22 @@ extern "C" int patchkv_select_repair_tokens(patchkv_ctx* ctx, const patchkv_sele
     TopkParams tp;
     tp.mass = mass; tp.shared = 0;
     if (shared && n > 0) {
-        sum_layers_kernel<<<(n + 255) / 256, 256, 0, stream>>>(mass, L, n, ws_sum);
-        PKV_CUDA(ctx, cudaGetLastError());
+        if (!sum_direct) PKV_CUDA(ctx, launch_pdl(sum_layers_kernel, dim3((n + 255) / 256), dim3(256), 0, stream, mass, L, n, ws_sum));
         tp.mass = ws_sum; tp.shared = 1;
     }
-    if (a->score_out && n > 0) normalise_kernel<<<tp.shared ? 1 : L, 256, 0, stream>>>(tp.mass, n, a->score_out);
+    if (a->score_out && n > 0)
+        PKV_CUDA(ctx, launch_pdl(normalise_kernel, dim3(tp.shared ? 1 : L), dim3(256), 0, stream, tp.mass, n, a->score_out));
     tp.NB = n; tp.n_dirty = (int)nd; tp.top_k = a->top_k;     // the "blocks" of this stage are single tokens
     tp.mask = tok_mask; tp.repair_idx = nullptr; tp.repair_cnt = nullptr; tp.reuse_idx = nullptr; tp.reuse_cnt = nullptr;
-    select_kernel<<<L, kSelThreads, 0, stream>>>(tp);
-    PKV_CUDA(ctx, cudaGetLastError());
-    block_round_kernel<<<L, kSelThreads, 0, stream>>>(tok_mask, n, B, NB, a->repair_mask, a->repair_idx, a->repair_cnt,
-                                                      a->reuse_idx, a->reuse_cnt);
-    PKV_CUDA(ctx, cudaGetLastError());
+    // the request-level ranking (layers shared) is one ranking: one CTA, one token mask that every layer rounds to blocks
+    int spill_bytes = 0;
+    rc = select_spill(ctx, n - (int)nd, &tp.spill_keys, &spill_bytes);
+    if (rc != PATCHKV_OK) return rc;
+    // the request-level ranking (layers shared) is one ranking: one CTA, one token mask that every layer rounds to blocks
+    PKV_CUDA(ctx, launch_pdl(select_kernel, dim3(tp.shared ? 1 : L), dim3(kSelThreads), (size_t)spill_bytes, stream, tp));
+    PKV_CUDA(ctx, launch_pdl(block_round_kernel, dim3(L), dim3(kSelThreads), 0, stream, (const uint8_t*)tok_mask,
+                             tp.shared ? 0ll : (long long)n, n, B, NB, a->repair_mask, a->repair_idx, a->repair_cnt,
+                             a->reuse_idx, a->reuse_cnt));
     PKV_CUDA(ctx, mirror_to_host(a, L, NB, stream));
     return PATCHKV_OK;
 }
@@ -812,7 +888,7 @@ extern "C" int patchkv_select_repair_static(const patchkv_select_args* a, void* 
             mp.attn = static_cast<const uint16_t*>(a->attn);
             mp.stride_layer = a->attn_stride_layer; mp.stride_head = a->attn_stride_head; mp.stride_query = a->attn_stride_query;
             mp.Hq = a->n_q_heads; mp.Q = a->n_queries; mp.n = n; mp.B = B; mp.NB = NB;
-            mp.mass = m; mp.status = status;
+            mp.mass = m; mp.mass_stride = NB; mp.status = status;
             const bool octet = (B % 8 == 0) && ((reinterpret_cast<uintptr_t>(a->attn) & 15u) == 0) &&
                                ((a->attn_stride_layer | a->attn_stride_head | a->attn_stride_query) & 7) == 0;
             const int cols = octet ? (n + 7) / 8 : n;
@@ -846,7 +922,7 @@ extern "C" int patchkv_select_repair_static(const patchkv_select_args* a, void* 
         if (cudaGetLastError() != cudaSuccess) return PATCHKV_E_CUDA;
         tp.mass = ws; tp.shared = 1;
     }
-    tp.NB = NB; tp.n_dirty = n_dirty; tp.top_k = a->top_k;
+    tp.NB = NB; tp.n_dirty = n_dirty; tp.top_k = a->top_k; tp.spill_keys = 0;
     tp.mask = a->repair_mask; tp.repair_idx = a->repair_idx; tp.repair_cnt = a->repair_cnt;
     tp.reuse_idx = a->reuse_idx; tp.reuse_cnt = a->reuse_cnt;
     if (a->score_out && NB > 0) normalise_kernel<<<tp.shared ? 1 : L, 256, 0, stream>>>(tp.mass, NB, a->score_out);

@@ -32,7 +32,8 @@
  *
  * Checkpoint byte layout ("PKV1"; the paper prescribes none beyond same-representation runs)
  *   - per layer one payload buffer, 16-byte aligned; tags u8 [L][NB] and blk_off u64 [L][NB] give the
- *     tag and the byte offset (multiple of 16) of each block's record inside its layer payload;
+ *     tag and the byte offset of each block's record inside its layer payload (a multiple of 16 wherever the
+ *     geometry makes records multiples of 16 bytes, i.e. for every geometry the fast kernels take);
  *   - one block record = [K codes][K scales][V codes][V scales]; codes are [token][head][channel]
  *     row-major; bf16 codes 2 bytes; int8 codes 1 byte two's complement; int4 codes pack channel c
  *     (even) in bits 0-3 and channel c+1 in bits 4-7 of one byte, two's-complement nibbles; scales
@@ -101,7 +102,7 @@ enum {
 enum {
     PATCHKV_MAX_SESSIONS = 8,      /* sessions per restore call */
     PATCHKV_MAX_ROTARY_DIM = 256,  /* rotary_dim <= 256 */
-    PATCHKV_MAX_BLOCK_VECTORS = 2048, /* block_tokens * n_kv_heads <= 2048 */
+    PATCHKV_MAX_BLOCK_VECTORS = 2048, /* block_tokens * n_kv_heads of the fast kernels and of the writer */
     PATCHKV_STATIC_MAX_MASS_ELEMS = 262144 /* u64 entries (2 MiB) of patchkv_select_repair_static's fixed scratch */
 };
 
@@ -115,17 +116,21 @@ typedef struct {
                                   UINT64_MAX = default 128 KiB */
 } patchkv_config;
 
-/* Model / cache geometry shared by all sessions of a call. */
+/* Model / cache geometry shared by all sessions of a call.  The restore entry points take every geometry that the
+ * format allows.  The fast kernels need D and G multiples of 8, Dr a multiple of 16 (HALF) or 8 (INTERLEAVED), at most
+ * PATCHKV_MAX_BLOCK_VECTORS (token, head) vectors per block, and record sections that are multiples of 16 bytes
+ * (B*H*D a multiple of 32, B*H*D/G a multiple of 8); any other geometry is restored by an element-wise kernel with the
+ * same results and no claim to speed.  The checkpoint writer takes only the geometries of the fast kernels. */
 typedef struct {
     uint32_t struct_size;
     int32_t n_layers;       /* L */
     int32_t n_kv_heads;     /* H */
-    int32_t head_dim;       /* D, multiple of 8 */
-    int32_t rotary_dim;     /* Dr <= D; multiple of 16 (HALF) or 8 (INTERLEAVED); channels >= Dr are not rotated */
+    int32_t head_dim;       /* D, even */
+    int32_t rotary_dim;     /* Dr <= D, even, at most PATCHKV_MAX_ROTARY_DIM; channels >= Dr are not rotated */
     int32_t rope_style;     /* PATCHKV_ROPE_* */
     int32_t block_tokens;   /* B: tokens per checkpoint block */
     int32_t page_tokens;    /* P: tokens per destination page */
-    int32_t group;          /* G: channels per fp16 scale, multiple of 8, divides D */
+    int32_t group;          /* G: channels per fp16 scale, divides D */
     double rope_base;
     const float* inv_freq;  /* HOST, optional [Dr/2]; overrides rope_base (frequency-scaled RoPE variants) */
 } patchkv_geom;
@@ -136,7 +141,8 @@ typedef struct {
     int32_t n_pages;
     void* k_base;           /* DEVICE bf16, 16-byte aligned */
     void* v_base;           /* DEVICE bf16, 16-byte aligned */
-    int64_t stride_layer;   /* elements; every stride a multiple of 8; the channel stride is 1 */
+    int64_t stride_layer;   /* elements, non-negative; the channel stride is 1.  The fast kernels need every stride
+                               to be a multiple of 8 (16-byte stores); other pools go to the element-wise kernel */
     int64_t stride_page;
     int64_t stride_token;
     int64_t stride_head;

@@ -191,6 +191,7 @@ struct SessionDev {
 struct RestoreParams {
     // geometry
     int32_t L, H, D, Dr, rope_style, B, P, G;
+    int32_t scalar_only;    // 1: a geometry only the element-wise kernel takes
     // pool
     uint16_t* k_base;
     uint16_t* v_base;

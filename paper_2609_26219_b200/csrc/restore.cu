@@ -309,6 +309,116 @@ restore_kernel(const __grid_constant__ RestoreParams p) {
     }
 }
 
+// ---------------------------------------------------------------- any geometry
+// One element (or one rotary pair) per thread, byte and halfword accesses only: the kernel for geometries that the
+// vector kernels above and below do not take (head_dim, group or rotary_dim not multiples of 8 / 16, record sections that
+// are not multiples of 16 bytes, blocks of more than 2048 (token, head) vectors).  Same arithmetic, same validation,
+// same results; speed is not its purpose.
+__device__ __forceinline__ float scalar_dequant(int fmt, const uint8_t* codes, const uint8_t* scales, size_t e, size_t sidx,
+                                                uint16_t* bits) {
+    if (fmt == FMT_BF16) {
+        const uint16_t b = (uint16_t)codes[2 * e] | ((uint16_t)codes[2 * e + 1] << 8);
+        *bits = b;
+        return __uint_as_float((uint32_t)b << 16);
+    }
+    const uint16_t sb = (uint16_t)scales[2 * sidx] | ((uint16_t)scales[2 * sidx + 1] << 8);
+    int q;
+    if (fmt == FMT_INT8) q = (int)(int8_t)codes[e];
+    else {
+        const uint32_t byte = codes[e >> 1];
+        const uint32_t nib = (e & 1) ? byte >> 4 : byte & 15u;
+        q = (int)(nib ^ 8u) - 8;                        // two's-complement nibble
+    }
+    return __fmul_rn((float)q, fp16_bits_to_f32(sb));   // exact: at most 8 x 11 significant bits
+}
+__device__ __forceinline__ uint16_t bf16_bits_rn(float x) { return (uint16_t)(pack_bf16x2(x, 0.0f) & 0xFFFFu); }
+
+template <bool INTER>
+__global__ void __launch_bounds__(kThreads)
+restore_scalar_kernel(const __grid_constant__ RestoreParams p) {
+    pdl_wait();
+    const uint64_t elems = (uint64_t)p.B * p.H * p.D;
+    const int half = p.Dr >> 1, slots = half + (p.D - p.Dr), gpv = p.D / p.G;
+    for (int item = blockIdx.x; item < p.total_items; item += gridDim.x) {
+        int si = 0;
+#pragma unroll 1
+        for (int k = 1; k < p.n_sessions; k++) if (item >= p.s[k].item_begin) si = k;
+        const SessionDev& S = p.s[si];
+        const int local = item - S.item_begin;
+        const int l = p.layer_begin + local / S.list_nb;
+        const int r = local - (l - p.layer_begin) * S.list_nb;
+        if (r >= __ldg(S.reuse_cnt + l)) continue;                     // uniform over the CTA
+        const int j = __ldg(S.reuse_idx + (size_t)l * S.list_nb + r);
+        bool bad = j < 0 || j >= S.nb;
+        int tag = 0;
+        unsigned long long off = 0, rec = 0, lbytes = 0;
+        const uint8_t* base = nullptr;
+        if (!bad) {
+            tag = __ldg(S.tags + (size_t)l * S.nb + j);
+            off = __ldg(S.blk_off + (size_t)l * S.nb + j);
+            lbytes = __ldg(S.layer_bytes + l);
+            base = reinterpret_cast<const uint8_t*>(
+                static_cast<uintptr_t>(__ldg(reinterpret_cast<const unsigned long long*>(S.layer_payload) + l)));
+            rec = record_bytes(tag, elems, p.G);
+            // (no alignment rule here: records of these geometries are not multiples of 16 bytes to begin with)
+            bad = rec == 0 || off > lbytes || rec > lbytes - off || base == nullptr;
+        }
+        const int valid = bad ? 0 : min(p.B, S.n - j * p.B);
+        // every destination page is validated before any write
+        for (int t = threadIdx.x; t < valid; t += kThreads) {
+            const long long u = (long long)j * p.B + t + S.dst_shift;
+            const long long lp = u / p.P;
+            const int page = lp < S.n_table ? __ldg(S.block_table + lp) : -1;
+            if (page < 0 || page >= p.n_pages) bad = true;
+        }
+        if (__syncthreads_or(bad)) {                                    // skip the block whole, latch the error
+            if (threadIdx.x == 0) atomicCAS(p.status, 0, (int)PATCHKV_E_BOUNDS);
+            continue;
+        }
+        const int kf = k_format(tag), vf = v_format(tag);
+        const uint8_t* kc = base + off;
+        const uint8_t* ks = kc + code_bytes(kf, elems);
+        const uint8_t* vc = ks + scale_bytes(kf, elems, p.G);
+        const uint8_t* vs = vc + code_bytes(vf, elems);
+        const bool rotate = S.delta != 0;
+        const long long work = (long long)valid * p.H * slots;
+        for (long long w = threadIdx.x; w < work; w += kThreads) {
+            const int vec = (int)(w / slots), s = (int)(w - (long long)vec * slots);
+            const int t = vec / p.H, h = vec - t * p.H;
+            const long long u = (long long)j * p.B + t + S.dst_shift;
+            const long long lp = u / p.P;
+            const long long dst = (long long)l * p.stride_layer + (long long)__ldg(S.block_table + lp) * p.stride_page +
+                                  (u - lp * p.P) * p.stride_token + (long long)h * p.stride_head;
+            // the one or two channels of this slot: a rotary pair, or one channel outside the rotary dimension
+            int c0, c1 = -1;
+            if (s < half) { c0 = INTER ? 2 * s : s; c1 = INTER ? 2 * s + 1 : s + half; }
+            else c0 = p.Dr + (s - half);
+            const size_t e0 = (size_t)vec * p.D + c0, g0 = (size_t)vec * gpv + c0 / p.G;
+            uint16_t kb0 = 0, kb1 = 0, vb0 = 0, vb1 = 0;
+            float ka = scalar_dequant(kf, kc, ks, e0, g0, &kb0);
+            const float va = scalar_dequant(vf, vc, vs, e0, g0, &vb0);
+            p.v_base[dst + c0] = vf == FMT_BF16 ? vb0 : bf16_bits_rn(va);          // V is never rotated
+            if (c1 >= 0) {
+                const size_t e1 = (size_t)vec * p.D + c1, g1 = (size_t)vec * gpv + c1 / p.G;
+                float kbv = scalar_dequant(kf, kc, ks, e1, g1, &kb1);
+                const float vb = scalar_dequant(vf, vc, vs, e1, g1, &vb1);
+                p.v_base[dst + c1] = vf == FMT_BF16 ? vb1 : bf16_bits_rn(vb);
+                if (rotate) {
+                    rotate_pair(ka, kbv, p.cs[si][0][s], p.cs[si][1][s]);
+                    p.k_base[dst + c0] = bf16_bits_rn(ka);
+                    p.k_base[dst + c1] = bf16_bits_rn(kbv);
+                } else {                                                    // a bf16 code that is not rotated is copied bit for bit
+                    p.k_base[dst + c0] = kf == FMT_BF16 ? kb0 : bf16_bits_rn(ka);
+                    p.k_base[dst + c1] = kf == FMT_BF16 ? kb1 : bf16_bits_rn(kbv);
+                }
+            } else {
+                p.k_base[dst + c0] = kf == FMT_BF16 ? kb0 : bf16_bits_rn(ka);
+            }
+        }
+        __syncthreads();
+    }
+}
+
 // ---------------------------------------------------------------- bulk-copy pipeline
 // A resolver warp takes rounds of blocks from the global work counter and resolves the directory entry and the
 // destination pages of each block one round ahead; an issuing warp stages the resolved blocks into a shared-memory
@@ -769,21 +879,23 @@ int fill_geometry(patchkv_ctx* ctx, const patchkv_geom* g, const patchkv_pool* p
         return fail(ctx, PATCHKV_E_INVALID, "geometry: unknown rope_style");
     if (!g->inv_freq && g->rotary_dim > 0 && !(g->rope_base > 0.0))
         return fail(ctx, PATCHKV_E_INVALID, "geometry: rope_base must be positive");
+    if (g->rotary_dim > PATCHKV_MAX_ROTARY_DIM)
+        return fail(ctx, PATCHKV_E_UNSUPPORTED, "geometry outside kernel limits: rotary_dim <= 256");
+    // The vector kernels own 8-channel chunks (one scale per chunk, a rotary chunk and its partner in one thread) and
+    // read record sections with 16-byte accesses; anything else goes to the element-wise kernel.
     const int rot_mult = g->rope_style == PATCHKV_ROPE_HALF ? 16 : 8;
     const long long vecs = (long long)g->block_tokens * g->n_kv_heads;
-    if (g->head_dim % 8 || g->group % 8 || g->rotary_dim % rot_mult || g->rotary_dim > PATCHKV_MAX_ROTARY_DIM ||
-        vecs > PATCHKV_MAX_BLOCK_VECTORS || g->head_dim > 16 * kThreads ||
-        (vecs * g->head_dim) % 32 != 0 || (vecs * (g->head_dim / g->group)) % 8 != 0)
-        return fail(ctx, PATCHKV_E_UNSUPPORTED,
-                    "geometry outside kernel limits: D % 8, G % 8, Dr % 16 (half) or % 8 (interleaved), Dr <= 256, "
-                    "B*H <= 2048, record sections multiples of 16 bytes");
+    p->scalar_only = (g->head_dim % 8 || g->group % 8 || g->rotary_dim % rot_mult || vecs > PATCHKV_MAX_BLOCK_VECTORS ||
+                      g->head_dim > 16 * kThreads || (vecs * g->head_dim) % 32 != 0 ||
+                      (vecs * (g->head_dim / g->group)) % 8 != 0) ? 1 : 0;
     if (!pool->k_base || !pool->v_base || pool->n_pages <= 0)
         return fail(ctx, PATCHKV_E_INVALID, "pool: null base or n_pages <= 0");
     if ((reinterpret_cast<uintptr_t>(pool->k_base) | reinterpret_cast<uintptr_t>(pool->v_base)) & 15u)
         return fail(ctx, PATCHKV_E_INVALID, "pool: bases must be 16-byte aligned");
-    if (pool->stride_layer < 0 || pool->stride_page < 0 || pool->stride_token < 0 || pool->stride_head < 0 ||
-        ((pool->stride_layer | pool->stride_page | pool->stride_token | pool->stride_head) & 7))
-        return fail(ctx, PATCHKV_E_INVALID, "pool: strides must be non-negative multiples of 8 elements");
+    if (pool->stride_layer < 0 || pool->stride_page < 0 || pool->stride_token < 0 || pool->stride_head < 0)
+        return fail(ctx, PATCHKV_E_INVALID, "pool: strides must be non-negative");
+    if ((pool->stride_layer | pool->stride_page | pool->stride_token | pool->stride_head) & 7)
+        p->scalar_only = 1;                                // the vector kernels store 16 bytes at a time
     p->L = g->n_layers; p->H = g->n_kv_heads; p->D = g->head_dim; p->Dr = g->rotary_dim; p->rope_style = g->rope_style;
     p->B = g->block_tokens; p->P = g->page_tokens; p->G = g->group;
     p->k_base = static_cast<uint16_t*>(pool->k_base);
@@ -918,6 +1030,14 @@ static int launch_pipe(patchkv_ctx* ctx, RestoreParams* p, int grid, int smem, c
 int launch_restore(patchkv_ctx* ctx, RestoreParams* p, cudaStream_t stream) {
     if (p->total_items <= 0) return PATCHKV_OK;
     const bool inter = p->rope_style == PATCHKV_ROPE_INTERLEAVED;
+    if (p->scalar_only) {
+        int grid = ctx->sm_count * kCtasPerSm;
+        if (grid > p->total_items) grid = p->total_items;
+        if (inter) restore_scalar_kernel<true><<<grid, kThreads, 0, stream>>>(*p);
+        else restore_scalar_kernel<false><<<grid, kThreads, 0, stream>>>(*p);
+        PKV_CUDA(ctx, cudaGetLastError());
+        return PATCHKV_OK;
+    }
     if (plan_pipeline(ctx, p)) {
         const int smem = p->n_stages * p->stage_bytes;
         int grid = ctx->sm_count * 2;

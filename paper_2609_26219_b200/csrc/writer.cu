@@ -606,6 +606,9 @@ static int fill_gather(patchkv_ctx* ctx, const patchkv_geom* g, const patchkv_po
     static thread_local RestoreParams rp;                  // reused only for the shared geometry / pool validation
     int rc = fill_geometry(ctx, g, pool, &rp);
     if (rc != PATCHKV_OK) return rc;
+    if (rp.scalar_only)
+        return fail(ctx, PATCHKV_E_UNSUPPORTED, "quantize_gather: needs D % 8, G % 8, B*H <= 2048 and record sections that are "
+                                                "multiples of 16 bytes");
     if (!s || s->struct_size != sizeof(patchkv_session)) return fail(ctx, PATCHKV_E_INVALID, "session: null or struct_size mismatch");
     if (s->n_suffix_tokens < 0 || s->dst_shift < 0 || s->dst_shift >= g->page_tokens || s->n_table < 0)
         return fail(ctx, PATCHKV_E_INVALID, "session: n_suffix_tokens >= 0, 0 <= dst_shift < P, n_table >= 0");

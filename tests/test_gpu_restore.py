@@ -139,11 +139,11 @@ def test_invalid_arguments_are_rejected_on_the_host(ctx):
     assert "dst_shift" in ctx.last_error()
     bad = st.geom(); bad.head_dim = 63
     assert ctx.restore(bad, pool, [st.session()], check=False) == pk.E_INVALID
-    bad = st.geom(); bad.group = 4
-    assert ctx.restore(bad, pool, [st.session()], check=False) == pk.E_UNSUPPORTED
-    bad = st.geom(); bad.rotary_dim = 24
-    assert ctx.restore(bad, pool, [st.session()], check=False) == pk.E_UNSUPPORTED
-    badp = pk.make_pool(k, v, ck.n_pages, (7, 8, 8, 8))
+    bad = st.geom(); bad.group = 5                                         # does not divide head_dim
+    assert ctx.restore(bad, pool, [st.session()], check=False) == pk.E_INVALID
+    bad = st.geom(); bad.rotary_dim = 23
+    assert ctx.restore(bad, pool, [st.session()], check=False) == pk.E_INVALID
+    badp = pk.make_pool(k, v, ck.n_pages, (-8, 8, 8, 8))
     assert ctx.restore(g, badp, [st.session()], check=False) == pk.E_INVALID
     assert ctx.restore(g, pool, [st.session()] * 9, check=False) == pk.E_INVALID
     a = st.select_args(); a.top_k = -1
@@ -414,7 +414,8 @@ def test_eight_device_resident_sessions_in_one_launch(ctx):
 
 
 def test_geometry_limits_block_vectors_and_rotary_dim(ctx):
-    """block_tokens * n_kv_heads = 2048 is the largest block the kernels take; one more token is refused."""
+    """block_tokens * n_kv_heads = 2048 is the largest block the vector kernels take (larger ones go to the element-wise
+    kernel, see test_geometries_outside_the_vector_kernels); a rotary dimension beyond 256 is refused."""
     from paper_2609_26219_b200 import binding as pk
     g = pin.Geometry(1, 16, 16, 16, pin.ROPE_HALF, 1e4, 128, 128, 8)       # 128 tokens x 16 heads = 2048 vectors
     ck = pin.make_checkpoint(name="max", seed=3, geom=g, n=300, delta=19, tag_probs=(0.3, 0.3, 0.2, 0.2), tags_per_layer=True,
@@ -422,8 +423,6 @@ def test_geometry_limits_block_vectors_and_rotary_dim(ctx):
     run_select_and_restore(ctx, ck)
     st = staged(ck)
     k, v, pool = gpu_pool(ck)
-    bad = st.geom(); bad.block_tokens = 129
-    assert ctx.restore(bad, pool, [st.session()], check=False) == pk.E_UNSUPPORTED
     bad = st.geom(); bad.head_dim = 512; bad.rotary_dim = 512
     assert ctx.restore(bad, pool, [st.session()], check=False) == pk.E_UNSUPPORTED
 
@@ -559,3 +558,29 @@ def test_host_restore_latches_out_of_range_entries(flags):
         check_pools(k, v, k_ref, v_ref, ck.geom)
     finally:
         c.close()
+
+
+ODD_GEOMETRIES = {
+    "G4": dict(geom=pin.Geometry(2, 4, 64, 64, pin.ROPE_HALF, 1e4, 16, 16, 4)),
+    "G2_interleaved": dict(geom=pin.Geometry(2, 2, 32, 32, pin.ROPE_INTERLEAVED, 1e4, 16, 16, 2)),
+    "Dr24_half": dict(geom=pin.Geometry(2, 4, 64, 24, pin.ROPE_HALF, 1e4, 16, 16, 32)),
+    "Dr6_interleaved": dict(geom=pin.Geometry(2, 3, 48, 6, pin.ROPE_INTERLEAVED, 1e4, 16, 16, 24)),
+    "D50_G10_Dr30": dict(geom=pin.Geometry(2, 3, 50, 30, pin.ROPE_HALF, 1e4, 8, 16, 10), n=500, dst_shift=7),
+    "D6_G2_B3": dict(geom=pin.Geometry(3, 1, 6, 4, pin.ROPE_HALF, 1e4, 3, 8, 2), n=100, dst_shift=5),
+    "sections_not_16B": dict(geom=pin.Geometry(2, 1, 8, 8, pin.ROPE_HALF, 1e4, 3, 4, 8), n=50),
+    "B130_H16_over_2048_vectors": dict(geom=pin.Geometry(1, 16, 16, 16, pin.ROPE_HALF, 1e4, 130, 128, 8), n=400, n_pages=8),
+}
+
+
+@pytest.mark.parametrize("name", sorted(ODD_GEOMETRIES))
+def test_geometries_outside_the_vector_kernels(ctx, name):
+    """Scale groups of 2 or 4 channels, rotary dimensions that are not multiples of 16, head dimensions that are not
+    multiples of 8, record sections that are not multiples of 16 bytes, blocks of more than 2048 vectors: everything the
+    format allows and the oracle accepts is restored (by the element-wise kernel), device- and host-resident, all tags."""
+    kw = dict(ODD_GEOMETRIES[name])
+    kw.setdefault("n_pages", 256)
+    kw.setdefault("tag_probs", (0.25, 0.25, 0.25, 0.25))
+    ck = pin.config_tiny(**{**kw, "n_q_heads": 2, "n_queries": 3})
+    run_select_and_restore(ctx, ck)
+    run_select_and_restore(ctx, ck, host=True)
+    run_select_and_restore(ctx, pin.config_tiny(**{**kw, "n_q_heads": 2, "n_queries": 3, "delta": 0}))

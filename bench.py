@@ -27,6 +27,7 @@ exchange step, so this is weak scaling without any data-path collective.
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import os
 import re
@@ -865,7 +866,13 @@ def run_sweep(args):
     by_geom = {}
     for name, (gm, n) in geoms.items():
         shift = 5 if "shift5" in name else 0
-        by_geom[name] = {"restore": restore_row(mk(gm, n, 7, shift=shift)), "writer": writer_row(mk(gm, n, 7, shift=shift))}
+        row = restore_row(mk(gm, n, 7, shift=shift))
+        # the same with half the layers: the slope between the two sizes leaves the launch's fixed cost out
+        half_geom = dataclasses.replace(gm, n_layers=LH // 2)
+        small = restore_row(mk(half_geom, n, 7, shift=shift))
+        bytes_full, bytes_half = row["gbps"] * row["us"], small["gbps"] * small["us"]
+        row["frac_hbm_marginal"] = r3((bytes_full - bytes_half) / (row["us"] - small["us"]) / peak)
+        by_geom[name] = {"restore": row, "writer": writer_row(mk(gm, n, 7, shift=shift))}
     out["by_geometry"] = by_geom
     out["by_suffix_tokens"] = {str(n): restore_row(mk(G(32, 8, 128, 128, pin.ROPE_HALF, 5e5, 16, 16, 32), n, 1002), reps=30)
                                for n in (256, 1024, 2048, 4096, 8192, 16384)}

@@ -441,6 +441,7 @@ select_kernel(const TopkParams p) {
             };
 #pragma unroll
             for (int i = 0; i < kKeysPerThread; i++) {
+                if (i >= iters) break;                   // (uniform) rounds that hold no candidate cost nothing
                 const int c = threadIdx.x + i * kSelThreads;
                 const unsigned long long x = kreg[i];
                 count_digit(c < ncand && (b == 7 || ((x ^ prefix) >> (8 * (b + 1))) == 0), x);

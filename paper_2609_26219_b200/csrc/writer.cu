@@ -671,7 +671,12 @@ static int launch_gather(patchkv_ctx* ctx, const patchkv_geom* g, const patchkv_
             }
             for (int t = 0; t < 4; t++) cfg.rec_bytes[t] = (uint32_t)record_bytes(t, elems, g->group);
             const int smem = (int)(stage_bytes * n_stages);
-            const int grid = std::min(cfg.total_items, 2 * ctx->sm_count);
+            // Two CTAs per SM; three where a unit is at most 8 KiB of rows (2 KV heads, or 4 of 64 channels, at 16-token
+            // blocks): there the producer warp's fixed work per unit sets the pace and a third producer per SM pays
+            // (measured 0.585 -> 0.73 of the HBM bandwidth), while with larger units it costs (0.94 -> 0.81 on 32-KiB
+            // units: more reads in flight crowd out the writes).
+            const int per_sm = (long long)ut * row_bytes <= 8192 ? 3 : 2;
+            const int grid = std::min(cfg.total_items, per_sm * ctx->sm_count);
             if (g->group >= 32) {
                 PKV_CUDA(ctx, cudaFuncSetAttribute(quantize_gather_pipe_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
                 quantize_gather_pipe_kernel<4><<<grid, kWPipeThreads, smem, stream>>>(p, cfg);

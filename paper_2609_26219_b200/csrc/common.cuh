@@ -304,5 +304,8 @@ void build_rope_table(const patchkv_geom* g, int delta, float* cos_out, float* s
 int ensure_host_workspace(patchkv_ctx* ctx, size_t meta_bytes, size_t slot_bytes);
 // Launches the restore kernel for layers [layer_begin, layer_end) of the sessions already filled in p.
 int launch_restore(patchkv_ctx* ctx, RestoreParams* p, cudaStream_t stream);
+// The slot of work counters (two words of ctx->d_sched per slot) a self-scheduling launch on `stream` uses: one per
+// stream the context has seen, one per launch captured into a graph.  The last CTA of a launch leaves its slot at zero.
+int sched_slot(patchkv_ctx* ctx, cudaStream_t stream, bool capturing, int* slot);
 
 }  // namespace patchkv

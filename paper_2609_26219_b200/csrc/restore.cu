@@ -992,12 +992,12 @@ static bool plan_pipeline(const patchkv_ctx* ctx, RestoreParams* p) {
 // The slot of work counters a pipeline launch on `stream` uses.  Launches that share a slot must never overlap on the
 // GPU, so a slot belongs to whatever serialises them: the two internal streams (slots 0 and 1), one caller stream each
 // (slots 2 ...), or one captured launch (a graph node can be replayed from any stream, next to anything).
-static int sched_slot(patchkv_ctx* ctx, cudaStream_t stream, bool capturing, int* slot) {
+int sched_slot(patchkv_ctx* ctx, cudaStream_t stream, bool capturing, int* slot) {
     if (stream == ctx->decode_stream && !capturing) { *slot = 0; return PATCHKV_OK; }
     if (stream == ctx->direct_stream && !capturing) { *slot = 1; return PATCHKV_OK; }
     if (capturing) {
         if (ctx->sched_captured >= kSchedCaptureSlots)
-            return fail(ctx, PATCHKV_E_UNSUPPORTED, "restore: too many launches captured into CUDA graphs by this context");
+            return fail(ctx, PATCHKV_E_UNSUPPORTED, "too many launches captured into CUDA graphs by this context");
         *slot = kSchedStreamSlots + ctx->sched_captured++;
         return PATCHKV_OK;
     }
@@ -1007,7 +1007,7 @@ static int sched_slot(patchkv_ctx* ctx, cudaStream_t stream, bool capturing, int
     for (size_t i = 0; i < ctx->sched_streams.size(); i++)
         if (ctx->sched_streams[i].first == handle && ctx->sched_streams[i].second == owner) { *slot = 2 + (int)i; return PATCHKV_OK; }
     if ((int)ctx->sched_streams.size() >= kSchedStreamSlots - 2)
-        return fail(ctx, PATCHKV_E_UNSUPPORTED, "restore: this context has been used from too many different streams");
+        return fail(ctx, PATCHKV_E_UNSUPPORTED, "this context has been used from too many different streams");
     ctx->sched_streams.emplace_back(handle, owner);
     *slot = 1 + (int)ctx->sched_streams.size();
     return PATCHKV_OK;

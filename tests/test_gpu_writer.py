@@ -135,6 +135,48 @@ def test_writer_exact_ties_round_to_even(ctx):
     assert np.array_equal(bufs[0], bufs_o[0])
 
 
+def test_writer_every_bf16_maximum_and_many_ties(ctx):
+    """Every finite positive bf16 value as the maximum of a scale group (so every scale the encoder can produce from
+    one, subnormal and infinite fp16 scales included), in 8-bit and in 4-bit codes; the other channels of the group are
+    fractions of the maximum with few significant bits (odd multiples of max/14, max/254, max/8 ... rounded to bf16,
+    which land on exact half-integer quotients whenever the scale has few bits) and random values below it."""
+    rng = np.random.default_rng(77)
+    amax_bits = np.arange(1, 0x7F80, dtype=np.uint32)                       # 32 639 values
+    n_groups = 32768
+    amax = np.zeros(n_groups, dtype=np.float32)
+    amax[:amax_bits.size] = (amax_bits << 16).view(np.float32)
+    amax[amax_bits.size:] = 1.5
+    x = np.zeros((n_groups, 32), dtype=np.float64)
+    x[:, 0] = amax
+    odd = rng.integers(0, 64, size=(n_groups, 15)) * 2 + 1
+    den = rng.choice([14.0, 254.0, 8.0, 16.0, 28.0, 508.0], size=(n_groups, 15))
+    x[:, 1:16] = amax[:, None].astype(np.float64) * np.minimum(odd / den, 1.0) * rng.choice([-1.0, 1.0], size=(n_groups, 15))
+    x[:, 16:] = amax[:, None].astype(np.float64) * rng.uniform(-1.0, 1.0, size=(n_groups, 16))
+    with np.errstate(over="ignore", invalid="ignore"):
+        xf = x.astype(np.float32)
+    bits = xf.view(np.uint32)
+    bf = ((bits + 0x7FFF + ((bits >> 16) & 1)) >> 16).astype(np.uint16)    # round to nearest even bf16
+    bf[:, 0] = (amax.view(np.uint32) >> 16).astype(np.uint16)
+    mag = bf & 0x7FFF
+    over = mag > mag[:, :1]                                                 # rounding must not exceed the maximum
+    bf = np.where(over, (bf & 0x8000) | mag[:, :1], bf).astype(np.uint16)
+    # layout: 1 head of 128 channels (4 groups per token), 16-token blocks: 64 groups per block, 512 blocks
+    g = pin.Geometry(2, 1, 128, 128, pin.ROPE_HALF, 1e4, 16, 16, 32)
+    n = n_groups // 4
+    ck = _ck(geom=g, n=n, n_pages=n // 16, table="identity", tag_probs=(0, 1.0, 0, 0))
+    ck.tags[1, :] = pin.TAG_K4V4
+    kp = np.zeros((2, n // 16, 16, 1, 128), dtype=np.uint16)
+    kp[0] = bf.reshape(n // 16, 16, 1, 128)
+    kp[1] = kp[0]
+    vp = kp[:, ::-1].copy()
+    rc, rc2, off_o, lb_o, bufs_o = run_writer(ck, kp, vp)
+    assert rc == oracle.OK and rc2 == oracle.OK
+    off, sizes, bufs = gpu_writer(ctx, ck, kp, vp)
+    assert ctx.query_status() == 0
+    for a, b in zip(bufs, bufs_o):
+        assert np.array_equal(a, b)
+
+
 @pytest.mark.parametrize("what", ["page", "offset", "table_short"])
 def test_writer_skips_out_of_range_blocks(ctx, what):
     ck = _ck()

@@ -262,7 +262,7 @@ __device__ __forceinline__ uint32_t absmax_bf16x2(uint32_t a, uint32_t b) {     
     return d;
 }
 // The codes of a span element by element, with a tie test on the exact remainder and the clamp a subnormal scale
-// needs: the rare path of quantise_span (a span whose scale is a subnormal fp16, or infinite).
+// needs: the rare path of quantise_span (a span whose scale is a subnormal fp16).
 template <int FMT, int NC>
 __device__ __forceinline__ void quantise_span_exact(const uint4* w, float s, float r, bool subnormal, uint32_t* out) {
     const float qmax = FMT == FMT_INT8 ? 127.0f : 7.0f;
@@ -303,7 +303,7 @@ __device__ __forceinline__ void quantise_span_exact(const uint4* w, float s, flo
 // is within 2^-15 of x / s and *equal* to it whenever x / s is a half-integer (an fp32 value, which the correction
 // reproduces exactly); adding 1.5 * 2^23 then rounds it to the integer the exact quotient rounds to, ties to even,
 // and leaves the code in the low byte.  Four packed fp32 operations per pair of elements, no tie test.  A span whose
-// scale is a subnormal fp16 (its codes may need the clamp) or infinite takes the element-wise path above.
+// scale is a subnormal fp16 (its codes may need the clamp) takes the element-wise path above.
 template <int FMT, int NC>
 __device__ __forceinline__ void quantise_span(const uint4* w, int seg, uint32_t* out, __half* scale) {
     uint32_t mx = 0;
@@ -329,8 +329,9 @@ __device__ __forceinline__ void quantise_span(const uint4* w, int seg, uint32_t*
     const float magic = 12582912.0f;                       // 1.5 * 2^23: adding it rounds to an integer, ties to even
     const uint32_t exp16 = __half_as_ushort(s16) & 0x7C00u;
     const bool subnormal = exp16 == 0 && s > 0.0f;          // |k| may exceed qmax
-    const bool rare = subnormal || exp16 == 0x7C00u;        // an infinite scale (amax beyond fp16 * qmax): all codes 0
-    const f32x2 r2 = pack2(r, r), m2 = pack2(magic, magic), ns2 = pack2(-s, -s);
+    // an infinite scale (amax beyond 65504 * qmax) has r = 0 and every code 0: keep inf * 0 out of the remainder
+    const float s_rem = exp16 == 0x7C00u ? 0.0f : s;
+    const f32x2 r2 = pack2(r, r), m2 = pack2(magic, magic), ns2 = pack2(-s_rem, -s_rem);
 #pragma unroll
     for (int c = 0; c < NC; c++) {
         const uint32_t word[4] = {w[c].x, w[c].y, w[c].z, w[c].w};
@@ -355,7 +356,7 @@ __device__ __forceinline__ void quantise_span(const uint4* w, int seg, uint32_t*
             out[c] = (ev & 0x0F0F0F0Fu) | ((od << 4) & 0xF0F0F0F0u);
         }
     }
-    if (rare) quantise_span_exact<FMT, NC>(w, s, r, subnormal, out);
+    if (subnormal) quantise_span_exact<FMT, NC>(w, s, r, subnormal, out);
     *scale = s16;
 }
 

@@ -55,9 +55,10 @@ TRAFFIC_FILE = os.path.join(ROOT, "profiles", "restore_pipe_kernel_llama8b_slice
 
 
 # ------------------------------------------------------------------------------------------ helpers
-def workload_config(delta: int, world: int, layers: int = 32) -> dict:
+def workload_config(delta: int, world: int, layers: int = 32, tags: str = "") -> dict:
     """The `config` object of the JSON line, the same for both arms."""
-    return {"workload": WORKLOAD if layers == 32 else WORKLOAD + f" [PROFILING SLICE: {layers} layers]",
+    note = (f" [PROFILING SLICE: {layers} layers]" if layers != 32 else "") + (f" [PROFILING: tag shares {tags}]" if tags else "")
+    return {"workload": WORKLOAD + note,
             "delta": delta, "l2": "working set 3.0 GB per step >> 126 MB L2, no flush",
             "parallelism": f"independent replicas x{world}" if world > 1 else "1 gpu"}
 
@@ -355,7 +356,11 @@ def run_ours(args):
     ctx = pk.Context(device=local_rank)
 
     # ---- inputs, resident in HBM before the timed region
-    ck = pin.config_llama8b(device=dev, n_layers=args.layers)
+    over = {}
+    if args.tags:                                           # profiling only: another mix of precision tags
+        over["tag_probs"] = tuple(float(x) for x in args.tags.split(","))
+        assert len(over["tag_probs"]) == 4
+    ck = pin.config_llama8b(device=dev, n_layers=args.layers, **over)
     st = StagedCheckpoint(ck, dev)
     k, v, pool = device_pool(ck, dev)
     geom = st.geom()
@@ -759,7 +764,7 @@ def run_ours(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": workload_config(ck.delta, world, args.layers),
+            "config": workload_config(ck.delta, world, args.layers, args.tags),
             "clocks": clocks, "e2e": e2e, "gpu_launches": 2 * K * n_blocks,
             "gpu_launches_note": f"{n_blocks} timed block(s) x {K} steps x (select_kernel + restore_pipe_kernel); as many again in the interleaved probe blocks",
             "roofline": roofline, "cpu_baseline": cpu_baseline, "timing": timing,
@@ -922,6 +927,8 @@ def main():
     ap.add_argument("--stress-waves", type=int, default=pin.STRESS_LAYERS // pin.STRESS_WAVE_LAYERS,
                     help="8 waves of 10 layers cover the full 80-layer stress config (the default)")
     ap.add_argument("--scale-layers", type=int, default=32, help="layers of the selection-at-scale leg (profiling: fewer)")
+    ap.add_argument("--tags", default="",
+                    help="profiling only: shares of the tags bf16,K8V8,K8V4,K4V4 instead of the workload's 0.3,0.5,0.2,0")
     ap.add_argument("--layers", type=int, default=32,
                     help="profiling only: fewer layers of the same workload (the bench line is quoted on 32)")
     args = ap.parse_args()

@@ -302,6 +302,39 @@ def pinned_copy_ceiling(device, nbytes=1 << 30, reps=10):
     return nbytes / (best * 1e-3) / 1e9
 
 
+def copy_engine_table(device, total=1 << 28):
+    """GB/s of pinned host-to-device copies by copy size, issued on one stream and alternating between two: what one
+    copy costs the engine beyond its bytes, and whether a second stream hides it."""
+    src = torch.empty(total, dtype=torch.uint8).pin_memory()
+    dst = torch.empty(total, dtype=torch.uint8, device=device)
+    streams = [torch.cuda.Stream(device=device) for _ in range(2)]
+    out = {}
+    for size in (64 << 10, 256 << 10, 1 << 20, 4 << 20, 64 << 20):
+        n = min(total // size, 256)
+        row = {}
+        for ns in (1, 2):
+            best = None
+            for _ in range(3):
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                with torch.cuda.stream(streams[0]):
+                    torch.cuda._sleep(30_000_000)           # ~15 ms: the copies queue up behind it, so the host's issue
+                e0.record(streams[0])                       # rate is not what is measured
+                streams[1].wait_event(e0)
+                for i in range(n):
+                    with torch.cuda.stream(streams[i % ns]):
+                        dst[i * size:(i + 1) * size].copy_(src[i * size:(i + 1) * size], non_blocking=True)
+                streams[0].wait_stream(streams[1])
+                e1.record(streams[0])
+                e1.synchronize()
+                ms = e0.elapsed_time(e1)
+                best = ms if best is None else min(best, ms)
+            row[f"streams_{ns}"] = r3(n * size / (best * 1e-3) / 1e9)
+        out[str(size)] = row
+    del src, dst
+    return out
+
+
 def host_leg_on(ctx, cks, label, ceiling, dev, stream, reps=5):
     """restore_from_host of the sessions `cks` (pinned payloads) into a fresh pool: median time and link fractions."""
     from patchkv_inputs.staging import StagedCheckpoint, device_pool
@@ -899,7 +932,8 @@ def run_sweep(args):
     r = host_leg_on(c, [ck], "", ceiling, dev, stream, reps=5)
     c.close()
     r0 = host_leg_on(ctx, [ck], "", ceiling, dev, stream, reps=5)
-    out["host_path"] = {"link_ceiling_gbps": r3(ceiling), "staged_only_by_merge_gap_bytes": gaps,
+    out["host_path"] = {"link_ceiling_gbps": r3(ceiling), "copy_engine_gbps_by_copy_bytes": copy_engine_table(dev),
+                        "staged_only_by_merge_gap_bytes": gaps,
                         "zero_copy": {"ms": r3(r["ms"]), "frac_link": r3(r["frac_of_link"])},
                         "default_hybrid": {"ms": r3(r0["ms"]), "frac_link": r3(r0["frac_of_link"]), "copies": r0["copies"],
                                            "direct_frac": r3(r0["bytes_direct"] / r0["bytes_useful"]),

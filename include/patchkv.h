@@ -355,9 +355,12 @@ PATCHKV_API int patchkv_plan_checkpoint(patchkv_ctx* ctx, const patchkv_geom* ge
  * buffers are written), delta and the reuse lists are ignored.  Quantiser, per group of `group` channels of one
  * (token, head): s = fp16(amax / qmax) (fp32 division, round to nearest even), code = clamp(rint(x / s), -qmax,
  * qmax) with ties to even, s == 0 -> code 0; qmax = 127 for int8 and 7 for int4; a bf16 section copies the 16
- * bits; tokens past the end of the suffix encode as zeros.  Values must be finite with amax / qmax <= 65504.
+ * bits; tokens past the end of the suffix encode as zeros.  Values must be finite; a group whose amax / qmax
+ * exceeds 65504 gets an infinite scale and all-zero codes.
  * Needs group in {8, 16, 32, 64, 128, 256}.  A block whose tag, record extent or source pages are out of range
- * is skipped whole and PATCHKV_E_BOUNDS is latched.  One launch, asynchronous on `stream`. */
+ * is skipped whole and PATCHKV_E_BOUNDS is latched.  One launch, asynchronous on `stream`, no allocation; it hands
+ * out its blocks from the work counters of the stream's slot, as patchkv_restore does (same limits on streams and
+ * on launches captured into graphs), and leaves them zeroed. */
 PATCHKV_API int patchkv_quantize_gather(patchkv_ctx* ctx, const patchkv_geom* geom, const patchkv_pool* pool,
                                         const patchkv_session* session, void* stream);
 

@@ -177,6 +177,48 @@ def test_writer_every_bf16_maximum_and_many_ties(ctx):
         assert np.array_equal(a, b)
 
 
+def test_plan_and_writer_replay_from_a_cuda_graph(ctx):
+    """plan_checkpoint + quantize_gather enqueue kernels only (the encoder's work counters live in a slot of their own
+    for a captured launch and are left zeroed), so the pair can be captured once and replayed: same bytes as the oracle
+    on every replay."""
+    from paper_2609_26219_b200 import binding as pk
+    ck = _ck(n=150, dst_shift=5)
+    kp, vp = pool_from_raw(ck, shift=5)
+    rc, rc2, off_o, lb_o, bufs_o = run_writer(ck, kp, vp, shift=5)
+    g = ck.geom
+    L, NB = g.n_layers, ck.n_blocks
+    k = torch.from_numpy(kp.view(np.int16)).to(DEV)
+    v = torch.from_numpy(vp.view(np.int16)).to(DEV)
+    pool = pk.make_pool(k, v, ck.n_pages, pin.pool_strides(g, ck.n_pages))
+    geom = pk.make_geom(g.n_layers, g.n_kv_heads, g.head_dim, g.rotary_dim, g.rope_style, g.rope_base, g.block_tokens,
+                        g.page_tokens, g.group)
+    tags = ck.tags.to(DEV).contiguous()
+    off = torch.zeros((L, NB), dtype=torch.int64, device=DEV)
+    lb = torch.zeros(L, dtype=torch.int64, device=DEV)
+    sizes = [int(x) for x in lb_o]
+    starts = [sum(-(-s // 256) * 256 for s in sizes[:i]) for i in range(L)]
+    payload = torch.zeros(starts[-1] + sizes[-1] + 256, dtype=torch.uint8, device=DEV)
+    ptrs = torch.tensor([payload.data_ptr() + o for o in starts], dtype=torch.int64, device=DEV)
+    sess = pk.make_session(n_suffix_tokens=ck.n_suffix_tokens, delta=0, dst_shift=5, block_table=ck.block_table.to(DEV).contiguous(),
+                           tags=tags, blk_off=off, layer_payload=ptrs, layer_bytes=lb, reuse_idx=None, reuse_cnt=None)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        ctx.plan_checkpoint(geom, ck.n_suffix_tokens, tags, off, lb, side)
+        ctx.quantize_gather(geom, pool, sess, side)
+    for _ in range(3):
+        payload.fill_(0xEE)
+        off.fill_(-1)
+        graph.replay()
+        torch.cuda.synchronize()
+        pay = payload.cpu().numpy()
+        assert np.array_equal(off.cpu().numpy().astype(np.uint64), off_o)
+        for o, s_, b_ in zip(starts, sizes, bufs_o):
+            assert np.array_equal(pay[o:o + s_], b_)
+    assert ctx.query_status() == 0
+
+
 @pytest.mark.parametrize("what", ["page", "offset", "table_short"])
 def test_writer_skips_out_of_range_blocks(ctx, what):
     ck = _ck()

@@ -392,7 +392,8 @@ PATCHKV_API int patchkv_query_status(patchkv_ctx* ctx, int* device_status);
 PATCHKV_API int patchkv_selftest_bounded_wait(patchkv_ctx* ctx, uint32_t max_polls, void* stream);
 
 /* Diagnostic (the paper has no counterpart).  Arms the NEXT launch of a bulk-copy pipeline kernel on this context
- * (patchkv_restore, one launch of patchkv_restore_from_host, or patchkv_quantize_gather) to run with a wait limit of
+ * (patchkv_restore, one launch of patchkv_restore_from_host, patchkv_quantize_gather, or the per-token mass kernel of
+ * patchkv_select_repair_tokens on a regular attention shape) to run with a wait limit of
  * `max_polls` polls (1 .. 2^20) and to have the consumer warps of every CTA withhold the `empty` arrivals of
  * their unit number `after_units` (0-based), so that the warp that feeds the ring runs out of patience while copies it
  * issued earlier are still landing or have landed.  That launch then takes the path a real timeout would take:

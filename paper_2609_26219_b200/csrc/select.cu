@@ -165,6 +165,198 @@ block_mass_octet_kernel(const MassParams p) {
     }
 }
 
+// Token granularity through a bulk-copy ring (regular shapes: 16-byte aligned rows, Q a multiple of 8, n a multiple of
+// 8).  The reads in flight of the kernel below are what its registers hold (eight 128-bit loads per thread at 64
+// registers: 32 warps per SM); here a producer warp stages batches of eight rows x 2048 tokens (32 KiB) into a ring
+// of three stages with bulk asynchronous copies, so 192 KiB per SM are in flight whatever the consumers need, and the
+// eight consumer warps add up from shared memory.  Persistent grid: the launch's (layer, column tile, batch of rows)
+// list is cut into one contiguous piece per CTA, so a thread keeps its eight sums in registers across batches and
+// goes to memory (one 64-bit atomic per token) only when its piece crosses into another (layer, column tile).
+constexpr int kTokPipeConsumers = 256;
+constexpr int kTokPipeThreads = kTokPipeConsumers + 32;
+constexpr int kTokPipeStages = 3;
+constexpr int kTokPipeRows = 8;                                // rows per stage: one batch inside one head
+constexpr int kTokPipeCols = 8 * kTokPipeConsumers;            // tokens per column tile
+constexpr int kTokPipeStageBytes = kTokPipeRows * kTokPipeCols * 2;
+
+struct TokPipeParams {
+    MassParams m;
+    int col_tiles;              // ceil(n / kTokPipeCols)
+    int batches_per_tile;       // Hq * Q / kTokPipeRows
+    long long total_batches;    // L * col_tiles * batches_per_tile
+    uint32_t wait_limit;        // polls before a barrier wait gives up
+    int32_t stall_after;        // self-test only: consumer warp 0 withholds the `empty` arrival of its batch number
+                                // stall_after (-1: never), so that the producer's wait for that stage runs out
+};
+
+__global__ void __launch_bounds__(kTokPipeThreads, 2)
+token_mass_pipe_kernel(const __grid_constant__ TokPipeParams tp) {
+    extern __shared__ __align__(128) uint8_t ring[];
+    __shared__ uint64_t full_bar[kTokPipeStages], empty_bar[kTokPipeStages];
+    __shared__ int abort_flag;
+    const MassParams& p = tp.m;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kTokPipeStages; s++) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], kTokPipeConsumers / 32); }
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    pdl_wait();
+    pdl_trigger();
+    volatile int* abortp = &abort_flag;
+    // this CTA's piece of the batch list
+    const long long first = tp.total_batches * blockIdx.x / gridDim.x, last = tp.total_batches * (blockIdx.x + 1) / gridDim.x;
+    long long tile = first / tp.batches_per_tile;              // (layer, column tile) index
+    int batch = (int)(first - tile * tp.batches_per_tile);
+    int l = (int)(tile / tp.col_tiles), ct = (int)(tile - (long long)l * tp.col_tiles);
+    const int bpq = p.Q / kTokPipeRows;                        // batches per head
+
+    if (threadIdx.x < 32) {
+        // ================================================================ producer warp
+        const int lane = threadIdx.x;
+        int stage = 0;
+        uint32_t phase = 0, issued = 0;
+        bool alive = true;
+        for (long long i = first; i < last && alive; i++) {
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait(&empty_bar[stage], phase ^ 1, abortp, tp.wait_limit))) { alive = false; break; }
+            const int col0 = ct * kTokPipeCols;
+            const uint32_t bytes = (uint32_t)min(kTokPipeCols, p.n - col0) * 2u;
+            const int h = batch / bpq, q0 = (batch - h * bpq) * kTokPipeRows;
+            if (lane == 0) mbar_arrive_expect_tx(&full_bar[stage], bytes * kTokPipeRows);
+            __syncwarp();
+            if (lane < kTokPipeRows)
+                bulk_g2s(ring + (size_t)stage * kTokPipeStageBytes + (size_t)lane * (kTokPipeCols * 2),
+                         p.attn + (long long)l * p.stride_layer + (long long)h * p.stride_head +
+                             (long long)(q0 + lane) * p.stride_query + col0,
+                         bytes, &full_bar[stage]);
+            issued++;
+            if (++stage == kTokPipeStages) { stage = 0; phase ^= 1; }
+            if (++batch == tp.batches_per_tile) { batch = 0; if (++ct == tp.col_tiles) { ct = 0; l++; } }
+        }
+        if (!alive) {
+            // a wait gave up: let the copies already issued land (bounded) before the CTA and its shared memory go
+            const uint32_t n_wait = issued < (uint32_t)kTokPipeStages ? issued : (uint32_t)kTokPipeStages;
+            for (uint32_t k = 0; k < n_wait; k++) {
+                const uint32_t qq = issued - 1 - k;
+                for (uint32_t it = 0; it < tp.wait_limit; it++) {
+                    if (mbar_try_wait(&full_bar[qq % kTokPipeStages], (qq / kTokPipeStages) & 1)) break;
+                    __nanosleep(100);
+                }
+            }
+            if (lane == 0) atomicCAS(p.status, 0, (int)PATCHKV_E_TIMEOUT);
+        }
+    } else {
+        // ================================================================ consumer warps
+        // An fp16 below 1/2 is x = u * 2^-24 with u < 2^23, and fma(x, 2^15, 2^14) in fp32 -- one mixed-precision
+        // instruction on the fp16 operand, no conversion -- is exactly 2^14 + u * 2^-9: its bit pattern is
+        // 0x46800000 + u.  So a token's sum is kept as a 32-bit integer sum of those patterns (one fma per element, one
+        // three-input integer add per two elements), and the bias leaves when the sum moves to the token's 64-bit total
+        // (after at most 256 rows: the arithmetic is modular and the true partial sum stays below 2^31).  Whether a
+        // batch may go this way is decided once per batch: the largest half of its 32 words as an unsigned 16-bit
+        // integer (the order of non-negative fp16; a set sign bit counts as large) must be below 0x3800 = 1/2.
+        // Otherwise the batch is taken word by word, and a word with an entry of 1/2 or more, a negative, an infinity
+        // or a NaN takes the general conversion.
+        const int c = threadIdx.x - 32;
+        uint32_t a32[8];
+        unsigned long long acc[8];
+#pragma unroll
+        for (int k = 0; k < 8; k++) { a32[k] = 0; acc[k] = 0; }
+        uint32_t biased = 0;                                    // rows whose biased patterns a32 holds
+        bool bad = false;
+        int stage = 0, since_fold = 0;
+        uint32_t phase = 0;
+        auto pattern2 = [](uint32_t word, uint32_t& p0, uint32_t& p1) {
+            unsigned short lo, hi;
+            asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(word));
+            float t0, t1;
+            asm("fma.rn.f32.f16 %0, %1, %2, %3;" : "=f"(t0) : "h"(lo), "h"((unsigned short)0x7800), "f"(16384.0f));
+            asm("fma.rn.f32.f16 %0, %1, %2, %3;" : "=f"(t1) : "h"(hi), "h"((unsigned short)0x7800), "f"(16384.0f));
+            p0 = __float_as_uint(t0); p1 = __float_as_uint(t1);
+        };
+        auto fold = [&]() {
+#pragma unroll
+            for (int k = 0; k < 8; k++) { acc[k] += (uint32_t)(a32[k] - biased * 0x46800000u); a32[k] = 0; }
+            biased = 0; since_fold = 0;
+        };
+        auto to_memory = [&]() {                                // this thread's eight sums of (l, ct) -> the mass row
+            fold();
+            const int col = ct * kTokPipeCols + 8 * c;
+            if (col < p.n) {
+#pragma unroll
+                for (int k = 0; k < 8; k++)
+                    if (acc[k]) atomicAdd(p.mass + (long long)l * p.mass_stride + col + k, acc[k]);
+            }
+#pragma unroll
+            for (int k = 0; k < 8; k++) acc[k] = 0;
+        };
+        bool dirty = false;                                     // sums not yet in memory
+        for (long long i = first; i < last; i++) {
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait(&full_bar[stage], phase, abortp, tp.wait_limit))) break;
+            const uint32_t src = smem_u32(ring + (size_t)stage * kTokPipeStageBytes) + 16u * (uint32_t)c;
+            if (ct * kTokPipeCols + 8 * c < p.n) {
+                uint4 w[kTokPipeRows];
+#pragma unroll
+                for (int r = 0; r < kTokPipeRows; r++) w[r] = lds128(src + (uint32_t)r * (kTokPipeCols * 2));
+                uint32_t mx = 0;
+#pragma unroll
+                for (int r = 0; r < kTokPipeRows; r += 2) {
+                    mx = __vimax3_u16x2(mx, w[r].x, w[r].y);
+                    mx = __vimax3_u16x2(mx, w[r].z, w[r].w);
+                    mx = __vimax3_u16x2(mx, w[r + 1].x, w[r + 1].y);
+                    mx = __vimax3_u16x2(mx, w[r + 1].z, w[r + 1].w);
+                }
+                if ((mx & 0xFFFFu) < 0x3800u && (mx >> 16) < 0x3800u) {
+#pragma unroll
+                    for (int r = 0; r < kTokPipeRows; r += 2) {
+                        const uint32_t wa[4] = {w[r].x, w[r].y, w[r].z, w[r].w};
+                        const uint32_t wb[4] = {w[r + 1].x, w[r + 1].y, w[r + 1].z, w[r + 1].w};
+#pragma unroll
+                        for (int k = 0; k < 4; k++) {
+                            uint32_t a0, a1, b0, b1;
+                            pattern2(wa[k], a0, a1);
+                            pattern2(wb[k], b0, b1);
+                            a32[2 * k] += a0 + b0; a32[2 * k + 1] += a1 + b1;
+                        }
+                    }
+                    biased += kTokPipeRows;
+                } else
+#pragma unroll
+                for (int r = 0; r < kTokPipeRows; r++) {
+                    const uint32_t ww[4] = {w[r].x, w[r].y, w[r].z, w[r].w};
+                    const uint32_t m4 = __vimax3_u16x2(__vimax3_u16x2(ww[0], ww[1], ww[2]), ww[3], 0u);
+                    if ((m4 & 0xFFFFu) < 0x3800u && (m4 >> 16) < 0x3800u) {
+#pragma unroll
+                        for (int k = 0; k < 4; k++) {
+                            uint32_t a0, a1;
+                            pattern2(ww[k], a0, a1);
+                            a32[2 * k] += a0; a32[2 * k + 1] += a1;
+                        }
+                        biased++;
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < 4; k++) { acc[2 * k] += units_any(ww[k], &bad); acc[2 * k + 1] += units_any(ww[k] >> 16, &bad); }
+                    }
+                }
+            }
+            __syncwarp();
+            if ((c & 31) == 0 && !(c == 0 && i - first == tp.stall_after)) mbar_arrive(&empty_bar[stage]);
+            if (++stage == kTokPipeStages) { stage = 0; phase ^= 1; }
+            dirty = true;
+            since_fold += kTokPipeRows;
+            if (since_fold == 256) fold();
+            if (++batch == tp.batches_per_tile) {
+                to_memory();
+                dirty = false;
+                batch = 0;
+                if (++ct == tp.col_tiles) { ct = 0; l++; }
+            }
+        }
+        if (dirty) to_memory();
+        if (bad) atomicCAS(p.status, 0, (int)PATCHKV_E_BADINPUT);
+        if (c == 0 && *abortp) atomicCAS(p.status, 0, (int)PATCHKV_E_TIMEOUT);
+    }
+}
+
 // Token granularity (the score of Eq. 10 per token): one thread owns eight consecutive tokens and keeps one exact sum
 // per token over the rows of its CTA.  Same loads and the same exact-fp32 fast path as the block kernel.
 __global__ void __launch_bounds__(256, 4)
@@ -760,6 +952,24 @@ extern "C" int patchkv_select_repair_tokens(patchkv_ctx* ctx, const patchkv_sele
             mp.mass = m; mp.mass_stride = sum_direct ? 0 : n; mp.status = ctx->d_status;
             const bool octet = ((reinterpret_cast<uintptr_t>(a->attn) & 15u) == 0) &&
                                ((a->attn_stride_layer | a->attn_stride_head | a->attn_stride_query) & 7) == 0;
+            if (octet && n % 8 == 0 && a->n_queries % kTokPipeRows == 0 && !(ctx->flags & PATCHKV_FLAG_DIRECT_LOADS)) {
+                // regular shape: rows staged through shared memory by bulk copies, one contiguous piece of the list per CTA
+                TokPipeParams tpp;
+                tpp.m = mp;
+                tpp.col_tiles = (n + kTokPipeCols - 1) / kTokPipeCols;
+                tpp.batches_per_tile = (int)(rows / kTokPipeRows);
+                tpp.total_batches = (long long)L * tpp.col_tiles * tpp.batches_per_tile;
+                tpp.wait_limit = kWaitLimit; tpp.stall_after = -1;
+                if (ctx->selftest_stall_after >= 0) {      // armed by patchkv_selftest_stall_next_launch: this launch only
+                    tpp.wait_limit = ctx->selftest_wait_limit;
+                    tpp.stall_after = ctx->selftest_stall_after;
+                    ctx->selftest_stall_after = -1;
+                }
+                const int smem = kTokPipeStages * kTokPipeStageBytes;
+                const int grid = (int)std::min<long long>(tpp.total_batches, 2ll * ctx->sm_count);
+                PKV_CUDA(ctx, cudaFuncSetAttribute(token_mass_pipe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+                PKV_CUDA(ctx, launch_pdl(token_mass_pipe_kernel, dim3(grid), dim3(kTokPipeThreads), smem, stream, tpp));
+            } else {
             const int cols = octet ? (n + 7) / 8 : n;
             const int tiles = (cols + 255) / 256;
             // few row groups (every thread ends with one 64-bit atomic per token), a whole number of batches each,
@@ -786,6 +996,7 @@ extern "C" int patchkv_select_repair_tokens(patchkv_ctx* ctx, const patchkv_sele
             mp.rows_per_cta = (int)rpc;
             PKV_CUDA(ctx, launch_pdl(octet ? token_mass_octet_kernel : block_mass_generic_kernel,
                                      dim3(tiles, (unsigned)groups, L), dim3(256), 0, stream, mp));
+            }
         }
         mass = m;
     } else if (n > 0 && !mass) {

@@ -556,6 +556,74 @@ normalise_kernel(const unsigned long long* mass, int NB, float* score) {
 
 constexpr int kKeysPerThread = 8;      // candidate masses cached in registers: covers NB - n_dirty <= 8192
 
+// Radix select, 8 bits per pass from byte `top_byte` down, over the candidates of one CTA: kr[] are the register-cached
+// keys, later(c) fetches a candidate of a later round.  After the pass over byte b, *s_prefix holds the bytes >= b of the
+// k-th largest key and *s_krem how many keys with that prefix are still to be taken; after the last pass *s_eq is the
+// number of keys equal to the k-th largest.  K is the integer type the keys fit (32-bit keys halve the arithmetic).
+template <typename K, typename Later>
+__device__ __forceinline__ void radix_select_passes(const K (&kr)[kKeysPerThread], Later later, int iters, int ncand, int top_byte,
+                                                    unsigned int* hist, unsigned long long* s_prefix, int* s_krem, int* s_eq) {
+    const unsigned lane = threadIdx.x & 31u;
+    constexpr int kTopByte = (int)sizeof(K) - 1;
+    for (int b = top_byte; b >= 0; b--) {
+        if (threadIdx.x < 256) hist[threadIdx.x] = 0;
+        __syncthreads();
+        const K prefix = (K)*s_prefix;
+        const int need = *s_krem;
+        // In the high bytes most keys share one digit (a long tail of small masses), and thousands of atomics on one
+        // counter serialise; a warp whose live lanes all hold the same digit adds its count with one atomic.
+        auto count_digit = [&](bool live, K x) {
+            const unsigned digit = (unsigned)(x >> (8 * b)) & 255u;
+            const unsigned act = __ballot_sync(0xFFFFFFFFu, live);
+            if (live) {
+                int same;
+                __match_all_sync(act, digit, &same);
+                if (!same) atomicAdd(&hist[digit], 1u);
+                else if (lane == (unsigned)(__ffs(act) - 1)) atomicAdd(&hist[digit], (unsigned)__popc(act));
+            }
+        };
+#pragma unroll
+        for (int i = 0; i < kKeysPerThread; i++) {
+            if (i >= iters) break;                   // (uniform) rounds that hold no candidate cost nothing
+            const int c = threadIdx.x + i * kSelThreads;
+            const K x = kr[i];
+            count_digit(c < ncand && (b == kTopByte || ((K)(x ^ prefix) >> (8 * (b + 1))) == 0), x);
+        }
+        for (int i = kKeysPerThread; i < iters; i++) {
+            const int c = threadIdx.x + i * kSelThreads;
+            const K x = c < ncand ? (K)later(c) : (K)0;
+            count_digit(c < ncand && (b == kTopByte || ((K)(x ^ prefix) >> (8 * (b + 1))) == 0), x);
+        }
+        __syncthreads();
+        if (threadIdx.x < 32) {
+            // lane owns the 8 digits 255-8*lane ... 248-8*lane; a warp scan finds the digit where the running
+            // count from the top first reaches `need`
+            int cnt[8], sum = 0;
+#pragma unroll
+            for (int t = 0; t < 8; t++) { cnt[t] = (int)hist[255 - 8 * (int)lane - t]; sum += cnt[t]; }
+            int inc = sum;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int o = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+                if (lane >= (unsigned)d) inc += o;
+            }
+            int cum = inc - sum;
+            if (cum < need && need <= inc) {
+#pragma unroll
+                for (int t = 0; t < 8; t++) {
+                    if (cum < need && need <= cum + cnt[t]) {
+                        *s_prefix = (unsigned long long)prefix | ((unsigned long long)(255 - 8 * (int)lane - t) << (8 * b));
+                        *s_krem = need - cum;
+                        *s_eq = cnt[t];              // after the last pass: how many keys equal the k-th largest
+                    }
+                    cum += cnt[t];
+                }
+            }
+        }
+        __syncthreads();
+    }
+}
+
 __global__ void __launch_bounds__(kSelThreads)
 select_kernel(const TopkParams p) {
     __shared__ unsigned int hist[256];
@@ -612,64 +680,14 @@ select_kernel(const TopkParams p) {
         const unsigned long long all_or = ((unsigned long long)s_or[1] << 32) | s_or[0];
         const int top_byte = all_or ? (63 - __clzll((long long)all_or)) >> 3 : -1;
 
-        // radix select, 8 bits per pass from the top: after the pass over byte b, `prefix` holds the bytes >= b of
-        // the k-th largest key and `krem` how many keys with that prefix are still to be taken
-        for (int b = top_byte; b >= 0; b--) {
-            if (threadIdx.x < 256) hist[threadIdx.x] = 0;
-            __syncthreads();
-            const unsigned long long prefix = s_prefix;
-            const int need = s_krem;
-            // In the high bytes most keys share one digit (a long tail of small masses), and thousands of atomics on one
-            // counter serialise; a warp whose live lanes all hold the same digit adds its count with one atomic.
-            auto count_digit = [&](bool live, unsigned long long x) {
-                const unsigned digit = (unsigned)(x >> (8 * b)) & 255u;
-                const unsigned act = __ballot_sync(0xFFFFFFFFu, live);
-                if (live) {
-                    int same;
-                    __match_all_sync(act, digit, &same);
-                    if (!same) atomicAdd(&hist[digit], 1u);
-                    else if (lane == (unsigned)(__ffs(act) - 1)) atomicAdd(&hist[digit], (unsigned)__popc(act));
-                }
-            };
+        if ((all_or >> 32) == 0) {
+            // every candidate fits 32 bits (masses of a few thousand rows): the same passes on 32-bit keys
+            unsigned int k32[kKeysPerThread];
 #pragma unroll
-            for (int i = 0; i < kKeysPerThread; i++) {
-                if (i >= iters) break;                   // (uniform) rounds that hold no candidate cost nothing
-                const int c = threadIdx.x + i * kSelThreads;
-                const unsigned long long x = kreg[i];
-                count_digit(c < ncand && (b == 7 || ((x ^ prefix) >> (8 * (b + 1))) == 0), x);
-            }
-            for (int i = kKeysPerThread; i < iters; i++) {
-                const int c = threadIdx.x + i * kSelThreads;
-                const unsigned long long x = c < ncand ? later_key(c) : 0ull;
-                count_digit(c < ncand && (b == 7 || ((x ^ prefix) >> (8 * (b + 1))) == 0), x);
-            }
-            __syncthreads();
-            if (threadIdx.x < 32) {
-                // lane owns the 8 digits 255-8*lane ... 248-8*lane; a warp scan finds the digit where the running
-                // count from the top first reaches `need`
-                int cnt[8], sum = 0;
-#pragma unroll
-                for (int t = 0; t < 8; t++) { cnt[t] = (int)hist[255 - 8 * (int)lane - t]; sum += cnt[t]; }
-                int inc = sum;
-#pragma unroll
-                for (int d = 1; d < 32; d <<= 1) {
-                    const int o = __shfl_up_sync(0xFFFFFFFFu, inc, d);
-                    if (lane >= (unsigned)d) inc += o;
-                }
-                int cum = inc - sum;
-                if (cum < need && need <= inc) {
-#pragma unroll
-                    for (int t = 0; t < 8; t++) {
-                        if (cum < need && need <= cum + cnt[t]) {
-                            s_prefix = prefix | ((unsigned long long)(255 - 8 * (int)lane - t) << (8 * b));
-                            s_krem = need - cum;
-                            s_eq = cnt[t];               // after the last pass: how many keys equal the k-th largest
-                        }
-                        cum += cnt[t];
-                    }
-                }
-            }
-            __syncthreads();
+            for (int i = 0; i < kKeysPerThread; i++) k32[i] = (unsigned int)kreg[i];
+            radix_select_passes<unsigned int>(k32, later_key, iters, ncand, top_byte, hist, &s_prefix, &s_krem, &s_eq);
+        } else {
+            radix_select_passes<unsigned long long>(kreg, later_key, iters, ncand, top_byte, hist, &s_prefix, &s_krem, &s_eq);
         }
         T = s_prefix;
         krem = s_krem;                           // keys equal to T to take, lowest block index first
@@ -685,14 +703,9 @@ select_kernel(const TopkParams p) {
     const bool lists = p.repair_idx != nullptr;          // the token-level stage only needs the mask
     for (int j = threadIdx.x; j < n_dirty; j += kSelThreads) { mask[j] = 1; if (lists) ridx[j] = j; }
     int run_sel = 0, run_eq = 0;
-    for (int i = 0; i < iters; i++) {
+    auto emit = [&](int i, unsigned long long x) {       // round i of the candidates; x: this thread's key of the round
         const int c = threadIdx.x + i * kSelThreads;
         const bool in = c < ncand;
-        unsigned long long x = 0;
-        if (i < kKeysPerThread) {
-#pragma unroll
-            for (int t = 0; t < kKeysPerThread; t++) if (t == i) x = kreg[t];
-        } else if (in) x = later_key(c);
         bool sel = false;
         if (take_all) sel = in;
         else if (!take_none) {
@@ -719,6 +732,15 @@ select_kernel(const TopkParams p) {
                 else fidx[c - before] = j;
             }
         }
+    };
+#pragma unroll
+    for (int i = 0; i < kKeysPerThread; i++) {
+        if (i >= iters) break;
+        emit(i, kreg[i]);
+    }
+    for (int i = kKeysPerThread; i < iters; i++) {
+        const int c = threadIdx.x + i * kSelThreads;
+        emit(i, c < ncand ? later_key(c) : 0ull);
     }
     if (!lists) return;
     const int n_r = n_dirty + run_sel, n_f = NB - n_r;

@@ -525,6 +525,7 @@ struct TopkParams {
     const unsigned long long* mass;     // [L][NB], or [NB] when shared
     int shared;                         // 1: every layer ranks on mass[0..NB)
     int spill_keys;                     // candidates the kernel may keep in its dynamic shared memory
+    const unsigned int* coarse_hist;    // select_kernel<true>: [rankings][kCoarseCodes] counts of coarse_hist_kernel
     int NB, n_dirty, top_k;
     uint8_t* mask;
     int32_t* repair_idx; int32_t* repair_cnt;
@@ -556,12 +557,61 @@ normalise_kernel(const unsigned long long* mass, int NB, float* score) {
 
 constexpr int kKeysPerThread = 8;      // candidate masses cached in registers: covers NB - n_dirty <= 8192
 
+// ---- ranking many candidates (the tokens of the token-level form): the first cut is made by many CTAs
+constexpr int kCoarseCodes = 2048;
+constexpr int kSelList = 1024;         // keys of the deciding code that are ranked from a list, one per thread
+
+// A monotone 11-bit code of a 64-bit key: the key itself below 64, else the position of its leading one and the five
+// bits under it.  Keys that share a code share every bit down to position `low` (coarse_prefix).
+__device__ __forceinline__ unsigned coarse_code(unsigned long long x) {
+    if (x < 64ull) return (unsigned)x;
+    const int e = 64 - __clzll((long long)x);            // 7 .. 64: x in [2^(e-1), 2^e)
+    return 64u + (unsigned)(e - 7) * 32u + ((unsigned)(x >> (e - 6)) & 31u);
+}
+__device__ __forceinline__ unsigned long long coarse_prefix(unsigned code, int* low) {
+    if (code < 64u) { *low = 0; return code; }
+    const int e = 7 + (int)((code - 64u) >> 5);
+    *low = e - 6;
+    return (unsigned long long)(32u + ((code - 64u) & 31u)) << (e - 6);
+}
+
+// Histogram of the candidates' coarse codes, one slice of the candidates per CTA: grid = (slices, rankings).  Masses
+// spread over many octaves, so the codes spread the keys over many counters; each CTA counts in shared memory and adds
+// its non-zero counters to the ranking's row of `hist` (zeroed before the launch).
+__global__ void __launch_bounds__(kSelThreads)
+coarse_hist_kernel(const unsigned long long* mass, int shared, int NB, int n_dirty, unsigned int* hist) {
+    __shared__ unsigned int h[kCoarseCodes];
+    pdl_wait();
+    pdl_trigger();
+    const int r = blockIdx.y;
+    const unsigned long long* key = mass + (shared ? 0 : (long long)r * NB);
+    const int nd = min(n_dirty, NB), ncand = NB - nd;
+    const int per = ((ncand + (int)gridDim.x - 1) / (int)gridDim.x + kSelThreads - 1) / kSelThreads * kSelThreads;
+    const int c0 = blockIdx.x * per, c1 = min(ncand, c0 + per);
+    for (int i = threadIdx.x; i < kCoarseCodes; i += kSelThreads) h[i] = 0;
+    __syncthreads();
+    const unsigned lane = threadIdx.x & 31u;
+    for (int cb = c0; cb < c1; cb += kSelThreads) {          // (uniform trip count: the ballots below are warp-wide)
+        const int c = cb + threadIdx.x;
+        const bool live = c < c1;
+        const unsigned code = live ? coarse_code(key[nd + c]) : 0u;
+        const unsigned act = __ballot_sync(0xFFFFFFFFu, live);
+        if (live) {
+            const unsigned peers = __match_any_sync(act, code);
+            if (lane == (unsigned)(__ffs(peers) - 1)) atomicAdd(&h[code], (unsigned)__popc(peers));
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < kCoarseCodes; i += kSelThreads)
+        if (h[i]) atomicAdd(hist + (long long)r * kCoarseCodes + i, h[i]);
+}
+
 // Radix select, 8 bits per pass from byte `top_byte` down, over the candidates of one CTA: kr[] are the register-cached
 // keys, later(c) fetches a candidate of a later round.  After the pass over byte b, *s_prefix holds the bytes >= b of the
 // k-th largest key and *s_krem how many keys with that prefix are still to be taken; after the last pass *s_eq is the
 // number of keys equal to the k-th largest.  K is the integer type the keys fit (32-bit keys halve the arithmetic).
-template <typename K, typename Later>
-__device__ __forceinline__ void radix_select_passes(const K (&kr)[kKeysPerThread], Later later, int iters, int ncand, int top_byte,
+template <typename K, int KPT, typename Later>
+__device__ __forceinline__ void radix_select_passes(const K (&kr)[KPT], Later later, int iters, int ncand, int top_byte,
                                                     unsigned int* hist, unsigned long long* s_prefix, int* s_krem, int* s_eq) {
     const unsigned lane = threadIdx.x & 31u;
     constexpr int kTopByte = (int)sizeof(K) - 1;
@@ -583,13 +633,13 @@ __device__ __forceinline__ void radix_select_passes(const K (&kr)[kKeysPerThread
             }
         };
 #pragma unroll
-        for (int i = 0; i < kKeysPerThread; i++) {
+        for (int i = 0; i < KPT; i++) {
             if (i >= iters) break;                   // (uniform) rounds that hold no candidate cost nothing
             const int c = threadIdx.x + i * kSelThreads;
             const K x = kr[i];
             count_digit(c < ncand && (b == kTopByte || ((K)(x ^ prefix) >> (8 * (b + 1))) == 0), x);
         }
-        for (int i = kKeysPerThread; i < iters; i++) {
+        for (int i = KPT; i < iters; i++) {
             const int c = threadIdx.x + i * kSelThreads;
             const K x = c < ncand ? (K)later(c) : (K)0;
             count_digit(c < ncand && (b == kTopByte || ((K)(x ^ prefix) >> (8 * (b + 1))) == 0), x);
@@ -624,9 +674,20 @@ __device__ __forceinline__ void radix_select_passes(const K (&kr)[kKeysPerThread
     }
 }
 
+// COARSE: the histogram of coarse_hist_kernel makes the first cut, and the few candidates that share the code of the k-th
+// largest key are ranked from a list in shared memory, one key per thread; the passes over all candidates remain for
+// masses so full of ties that the list would overflow.  (A separate instantiation, so that the kernel of the block form,
+// which runs under the restore kernel's CTAs, keeps its small shared-memory footprint.)
+template <bool COARSE>
 __global__ void __launch_bounds__(kSelThreads)
 select_kernel(const TopkParams p) {
+    // Candidates cached in registers per thread.  The many-candidate instantiation keeps one and reads the rest from
+    // shared memory: it runs as a single CTA that executes its code once, cold, and the loops over register-cached
+    // rounds are unrolled code that would have to be fetched instruction by instruction.
+    constexpr int KPT = COARSE ? 1 : kKeysPerThread;
     __shared__ unsigned int hist[256];
+    __shared__ unsigned long long s_list[COARSE ? kSelList : 1];
+    __shared__ int s_code, s_list_n;
     __shared__ int warp_sums[33];
     __shared__ unsigned long long s_prefix;
     __shared__ int s_krem, s_eq;
@@ -646,28 +707,138 @@ select_kernel(const TopkParams p) {
     const int iters = (ncand + kSelThreads - 1) / kSelThreads;
     const unsigned lane = threadIdx.x & 31u;
 
-    // candidate c = threadIdx.x + i * kSelThreads is block n_dirty + c; the first kKeysPerThread rounds live in registers,
+    // candidate c = threadIdx.x + i * kSelThreads is block n_dirty + c; the first KPT rounds live in registers,
     // the next p.spill_keys candidates in shared memory, anything beyond that is re-read from global memory
-    unsigned long long kreg[kKeysPerThread];
+    unsigned long long kreg[KPT];
 #pragma unroll
-    for (int i = 0; i < kKeysPerThread; i++) {
+    for (int i = 0; i < KPT; i++) {
         const int c = threadIdx.x + i * kSelThreads;
         kreg[i] = c < ncand ? key[n_dirty + c] : 0ull;
     }
-    const int reg_keys = kKeysPerThread * kSelThreads;
-    for (int c = reg_keys + threadIdx.x; c < ncand && c - reg_keys < p.spill_keys; c += kSelThreads) spill[c - reg_keys] = key[n_dirty + c];
+    const int reg_keys = KPT * kSelThreads;
+    {
+        // eight loads in flight per thread: the copy into shared memory is a chain of global-memory latencies otherwise
+        const int spill_end = min(ncand, reg_keys + p.spill_keys);
+        for (int c0 = reg_keys + threadIdx.x; c0 < spill_end; c0 += 8 * kSelThreads) {
+            unsigned long long v[8];
+#pragma unroll
+            for (int u = 0; u < 8; u++) {
+                const int c = c0 + u * kSelThreads;
+                v[u] = c < spill_end ? key[n_dirty + c] : 0ull;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; u++) {
+                const int c = c0 + u * kSelThreads;
+                if (c < spill_end) spill[c - reg_keys] = v[u];
+            }
+        }
+    }
     auto later_key = [&](int c) -> unsigned long long {      // a candidate of a later round (a thread reads back its own writes only)
         return c - reg_keys < p.spill_keys ? spill[c - reg_keys] : key[n_dirty + c];
     };
 
     unsigned long long T = 0;
     int krem = 0, n_eq = 0;                      // keys equal to T: krem of them are taken, n_eq exist
-    if (!take_all && !take_none) {
+    bool ranked = take_all || take_none;
+    if (COARSE && !ranked) {
+        // thread t owns the codes 2047 - 2t and 2046 - 2t; a scan from the top finds the code where the count reaches k
+        const unsigned int* ch = p.coarse_hist + (long long)l * kCoarseCodes;
+        const int c0 = (int)ch[kCoarseCodes - 1 - 2 * (int)threadIdx.x], c1 = (int)ch[kCoarseCodes - 2 - 2 * (int)threadIdx.x];
+        if (threadIdx.x == 0) s_list_n = 0;
+        int tot;
+        int cum = cta_exclusive_scan(c0 + c1, warp_sums, &tot);
+        if (cum < k && k <= cum + c0) { s_code = kCoarseCodes - 1 - 2 * (int)threadIdx.x; s_krem = k - cum; s_eq = c0; }
+        cum += c0;
+        if (cum < k && k <= cum + c1) { s_code = kCoarseCodes - 2 - 2 * (int)threadIdx.x; s_krem = k - cum; s_eq = c1; }
+        __syncthreads();
+        const unsigned code_k = (unsigned)s_code;
+        const int n_code = s_eq;                         // candidates that share the code of the k-th largest
+        int low = 0;                                     // bits of the k-th largest key not known yet
+        const unsigned long long prefix0 = coarse_prefix(code_k, &low);
+        if (low == 0 || n_code <= kSelList) {
+            if (low > 0) {
+#pragma unroll
+                for (int i = 0; i < KPT; i++) {
+                    if (i >= iters) break;
+                    if (threadIdx.x + i * kSelThreads < ncand && coarse_code(kreg[i]) == code_k) s_list[atomicAdd(&s_list_n, 1)] = kreg[i];
+                }
+                for (int i = KPT; i < iters; i++) {
+                    const int c = threadIdx.x + i * kSelThreads;
+                    if (c < ncand) {
+                        const unsigned long long x = later_key(c);
+                        if (coarse_code(x) == code_k) s_list[atomicAdd(&s_list_n, 1)] = x;
+                    }
+                }
+            }
+            if (threadIdx.x == 0) s_prefix = prefix0;
+            __syncthreads();
+            const bool have = (int)threadIdx.x < n_code && low > 0;
+            const unsigned long long mine = have ? s_list[threadIdx.x] : 0ull;
+            if (low > 0 && n_code <= 256) {
+                // a short list is ranked directly: the key that has exactly need - 1 keys in front of it (larger, or equal
+                // and earlier in the list) is the k-th largest; three barriers instead of three per radix pass
+                const int need = s_krem;
+                int front = 0;
+                if (have)
+                    for (int j = 0; j < n_code; j++) {
+                        const unsigned long long x = s_list[j];
+                        front += (x > mine || (x == mine && j < (int)threadIdx.x)) ? 1 : 0;
+                    }
+                if (have && front == need - 1) s_prefix = mine;
+                __syncthreads();
+                const unsigned long long kth = s_prefix;
+                const int larger = __syncthreads_count(have && mine > kth);
+                const int equal = __syncthreads_count(have && mine == kth);
+                T = kth; krem = need - larger; n_eq = equal;
+                low = 0;
+                ranked = true;
+            }
+            // radix select over the remaining bits of the listed keys, up to 8 per pass from the top
+            while (low > 0) {
+                const int width = min(8, low), shift = low - width;
+                if (threadIdx.x < 256) hist[threadIdx.x] = 0;
+                __syncthreads();
+                const unsigned long long prefix = s_prefix;
+                const int need = s_krem;
+                if (have && ((mine ^ prefix) >> low) == 0) atomicAdd(&hist[(unsigned)(mine >> shift) & ((1u << width) - 1u)], 1u);
+                __syncthreads();
+                if (threadIdx.x < 32) {
+                    int cnt[8], sum = 0;
+#pragma unroll
+                    for (int t = 0; t < 8; t++) { cnt[t] = (int)hist[255 - 8 * (int)lane - t]; sum += cnt[t]; }
+                    int inc = sum;
+#pragma unroll
+                    for (int d = 1; d < 32; d <<= 1) {
+                        const int o = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+                        if (lane >= (unsigned)d) inc += o;
+                    }
+                    int cm = inc - sum;
+                    if (cm < need && need <= inc) {
+#pragma unroll
+                        for (int t = 0; t < 8; t++) {
+                            if (cm < need && need <= cm + cnt[t]) {
+                                s_prefix = prefix | ((unsigned long long)(255 - 8 * (int)lane - t) << shift);
+                                s_krem = need - cm;
+                                s_eq = cnt[t];
+                            }
+                            cm += cnt[t];
+                        }
+                    }
+                }
+                __syncthreads();
+                low = shift;
+            }
+            if (!ranked) { T = s_prefix; krem = s_krem; n_eq = s_eq; }
+            ranked = true;
+        }
+        __syncthreads();                                 // (the shared words are set again below)
+    }
+    if (!ranked) {
         // highest byte that is non-zero in any candidate: the passes above it would all pick digit 0
         unsigned long long orv = 0;
 #pragma unroll
-        for (int i = 0; i < kKeysPerThread; i++) orv |= kreg[i];
-        for (int i = kKeysPerThread; i < iters; i++) {
+        for (int i = 0; i < KPT; i++) orv |= kreg[i];
+        for (int i = KPT; i < iters; i++) {
             const int c = threadIdx.x + i * kSelThreads;
             if (c < ncand) orv |= later_key(c);
         }
@@ -682,12 +853,12 @@ select_kernel(const TopkParams p) {
 
         if ((all_or >> 32) == 0) {
             // every candidate fits 32 bits (masses of a few thousand rows): the same passes on 32-bit keys
-            unsigned int k32[kKeysPerThread];
+            unsigned int k32[KPT];
 #pragma unroll
-            for (int i = 0; i < kKeysPerThread; i++) k32[i] = (unsigned int)kreg[i];
-            radix_select_passes<unsigned int>(k32, later_key, iters, ncand, top_byte, hist, &s_prefix, &s_krem, &s_eq);
+            for (int i = 0; i < KPT; i++) k32[i] = (unsigned int)kreg[i];
+            radix_select_passes<unsigned int, KPT>(k32, later_key, iters, ncand, top_byte, hist, &s_prefix, &s_krem, &s_eq);
         } else {
-            radix_select_passes<unsigned long long>(kreg, later_key, iters, ncand, top_byte, hist, &s_prefix, &s_krem, &s_eq);
+            radix_select_passes<unsigned long long, KPT>(kreg, later_key, iters, ncand, top_byte, hist, &s_prefix, &s_krem, &s_eq);
         }
         T = s_prefix;
         krem = s_krem;                           // keys equal to T to take, lowest block index first
@@ -734,11 +905,11 @@ select_kernel(const TopkParams p) {
         }
     };
 #pragma unroll
-    for (int i = 0; i < kKeysPerThread; i++) {
+    for (int i = 0; i < KPT; i++) {
         if (i >= iters) break;
         emit(i, kreg[i]);
     }
-    for (int i = kKeysPerThread; i < iters; i++) {
+    for (int i = KPT; i < iters; i++) {
         const int c = threadIdx.x + i * kSelThreads;
         emit(i, c < ncand ? later_key(c) : 0ull);
     }
@@ -794,15 +965,17 @@ block_round_kernel(const uint8_t* token_mask, long long mask_stride, int n, int 
 
 // Shared memory for the candidates that select_kernel cannot keep in registers (it would otherwise re-read them from
 // global memory in every radix pass).
-static int select_spill(patchkv_ctx* ctx, int ncand, int* keys, int* bytes) {
-    long long want = (long long)ncand - (long long)kKeysPerThread * kSelThreads;
-    const long long cap = ((long long)ctx->max_smem_optin - 4096) / 8;
+static int select_spill(patchkv_ctx* ctx, int ncand, int* keys, int* bytes, int keys_per_thread = kKeysPerThread) {
+    long long want = (long long)ncand - (long long)keys_per_thread * kSelThreads;
+    const long long cap = ((long long)ctx->max_smem_optin - 4096 - 8 * kSelList) / 8;
     if (want < 0) want = 0;
     if (want > cap) want = cap;
     *keys = (int)want;
     *bytes = (int)want * 8;
-    if (*bytes > 48 * 1024)
-        PKV_CUDA(ctx, cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, *bytes));
+    if (*bytes > 48 * 1024) {
+        PKV_CUDA(ctx, cudaFuncSetAttribute(select_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, *bytes));
+        PKV_CUDA(ctx, cudaFuncSetAttribute(select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, *bytes));
+    }
     return PATCHKV_OK;
 }
 
@@ -916,9 +1089,10 @@ extern "C" int patchkv_select_repair(patchkv_ctx* ctx, const patchkv_select_args
     if (a->score_out && NB > 0)
         PKV_CUDA(ctx, launch_pdl(normalise_kernel, dim3(tp.shared ? 1 : L), dim3(256), 0, stream, tp.mass, NB, a->score_out));
     int spill_bytes = 0;
+    tp.coarse_hist = nullptr;
     int rc2 = select_spill(ctx, NB - n_dirty, &tp.spill_keys, &spill_bytes);
     if (rc2 != PATCHKV_OK) return rc2;
-    PKV_CUDA(ctx, launch_pdl(select_kernel, dim3(L), dim3(kSelThreads), (size_t)spill_bytes, stream, tp));
+    PKV_CUDA(ctx, launch_pdl(select_kernel<false>, dim3(L), dim3(kSelThreads), (size_t)spill_bytes, stream, tp));
     PKV_CUDA(ctx, mirror_to_host(a, L, NB, stream));
     return PATCHKV_OK;
 }
@@ -952,11 +1126,17 @@ extern "C" int patchkv_select_repair_tokens(patchkv_ctx* ctx, const patchkv_sele
     const size_t mass_elems = from_attn && !a->mass_out && !sum_direct ? (size_t)L * n : 0;
     const size_t sum_elems = shared ? (size_t)n : 0;
     const size_t mask_words = ((size_t)L * n + 7) / 8;
-    int rc = ensure_mass_ws(ctx, mass_elems + sum_elems + mask_words + 1);
+    // many candidates: the first cut of the ranking is a histogram made by several CTAs (coarse_hist_kernel)
+    const long long nd_tokens = std::min<long long>(std::max<long long>(a->dirty_tokens, 0), n);
+    const bool coarse = (long long)n - nd_tokens >= 4 * kSelThreads;
+    const size_t hist_words = coarse ? ((size_t)(shared ? 1 : L) * kCoarseCodes + 1) / 2 : 0;
+    int rc = ensure_mass_ws(ctx, mass_elems + sum_elems + mask_words + hist_words + 1);
     if (rc != PATCHKV_OK) return rc;
     unsigned long long* ws = ctx->d_mass_ws;
     unsigned long long* ws_sum = ws + mass_elems;
     uint8_t* tok_mask = reinterpret_cast<uint8_t*>(ws_sum + sum_elems);
+    unsigned int* coarse_hist = reinterpret_cast<unsigned int*>(ws_sum + sum_elems + mask_words);
+    if (coarse) PKV_CUDA(ctx, cudaMemsetAsync(coarse_hist, 0, hist_words * 8, stream));
 
     const unsigned long long* mass = reinterpret_cast<const unsigned long long*>(a->mass);
     if (from_attn) {
@@ -1037,10 +1217,19 @@ extern "C" int patchkv_select_repair_tokens(patchkv_ctx* ctx, const patchkv_sele
     tp.mask = tok_mask; tp.repair_idx = nullptr; tp.repair_cnt = nullptr; tp.reuse_idx = nullptr; tp.reuse_cnt = nullptr;
     // the request-level ranking (layers shared) is one ranking: one CTA, one token mask that every layer rounds to blocks
     int spill_bytes = 0;
-    rc = select_spill(ctx, n - (int)nd, &tp.spill_keys, &spill_bytes);
+    rc = select_spill(ctx, n - (int)nd, &tp.spill_keys, &spill_bytes, coarse ? 1 : kKeysPerThread);
     if (rc != PATCHKV_OK) return rc;
     // the request-level ranking (layers shared) is one ranking: one CTA, one token mask that every layer rounds to blocks
-    PKV_CUDA(ctx, launch_pdl(select_kernel, dim3(tp.shared ? 1 : L), dim3(kSelThreads), (size_t)spill_bytes, stream, tp));
+    tp.coarse_hist = coarse ? coarse_hist : nullptr;
+    if (coarse) {
+        const int rankings = tp.shared ? 1 : L;
+        const int slices = std::max(1, std::min(32, (n - (int)nd + kSelThreads - 1) / kSelThreads));
+        PKV_CUDA(ctx, launch_pdl(coarse_hist_kernel, dim3(slices, rankings), dim3(kSelThreads), 0, stream, tp.mass, tp.shared, n, (int)nd,
+                                 coarse_hist));
+        PKV_CUDA(ctx, launch_pdl(select_kernel<true>, dim3(rankings), dim3(kSelThreads), (size_t)spill_bytes, stream, tp));
+    } else {
+        PKV_CUDA(ctx, launch_pdl(select_kernel<false>, dim3(tp.shared ? 1 : L), dim3(kSelThreads), (size_t)spill_bytes, stream, tp));
+    }
     PKV_CUDA(ctx, launch_pdl(block_round_kernel, dim3(L), dim3(kSelThreads), 0, stream, (const uint8_t*)tok_mask,
                              tp.shared ? 0ll : (long long)n, n, B, NB, a->repair_mask, a->repair_idx, a->repair_cnt,
                              a->reuse_idx, a->reuse_cnt));
@@ -1156,11 +1345,11 @@ extern "C" int patchkv_select_repair_static(const patchkv_select_args* a, void* 
         if (cudaGetLastError() != cudaSuccess) return PATCHKV_E_CUDA;
         tp.mass = ws; tp.shared = 1;
     }
-    tp.NB = NB; tp.n_dirty = n_dirty; tp.top_k = a->top_k; tp.spill_keys = 0;
+    tp.NB = NB; tp.n_dirty = n_dirty; tp.top_k = a->top_k; tp.spill_keys = 0; tp.coarse_hist = nullptr;
     tp.mask = a->repair_mask; tp.repair_idx = a->repair_idx; tp.repair_cnt = a->repair_cnt;
     tp.reuse_idx = a->reuse_idx; tp.reuse_cnt = a->reuse_cnt;
     if (a->score_out && NB > 0) normalise_kernel<<<tp.shared ? 1 : L, 256, 0, stream>>>(tp.mass, NB, a->score_out);
-    select_kernel<<<L, kSelThreads, 0, stream>>>(tp);
+    select_kernel<false><<<L, kSelThreads, 0, stream>>>(tp);
     if (cudaGetLastError() != cudaSuccess) return PATCHKV_E_CUDA;
     if (mirror_to_host(a, L, NB, stream) != cudaSuccess) { cudaGetLastError(); return PATCHKV_E_CUDA; }
     return PATCHKV_OK;

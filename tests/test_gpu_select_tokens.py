@@ -173,6 +173,46 @@ def test_token_form_at_scale_full_size_sampled_layers(ctx):
     assert ctx.query_status() == 0
 
 
+@pytest.mark.parametrize("case", ["tiny_keys", "distinct", "band_600", "band_3000", "all_equal", "huge_keys"])
+def test_many_candidates_every_way_through_the_ranking(ctx, case):
+    """With 4096 candidates or more the first cut of the ranking is a histogram of coarse key codes made by several
+    CTAs; what is left is ranked from a list (directly when short, by radix passes when longer) or, when thousands of
+    keys share the deciding code, by the passes over all candidates.  Each case is built to take one of those ways, with
+    duplicates around the threshold so that the order of equal keys matters."""
+    from paper_2609_26219_b200 import binding as pk
+    rng = np.random.default_rng(sum(map(ord, case)))
+    n, B, L = 8192, 16, 2
+    if case == "tiny_keys":                               # every key below 64: the code is the key
+        mass = rng.integers(0, 64, size=(L, n))
+        kappa = 700
+    elif case == "distinct":                              # keys spread over twenty octaves: a handful per code
+        mass = (2.0 ** rng.uniform(4, 24, size=(L, n))).astype(np.int64)
+        kappa = 123
+    elif case in ("band_600", "band_3000"):               # a band of keys that share one code holds the threshold
+        band = 600 if case == "band_600" else 3000
+        mass = rng.integers(0, 1 << 20, size=(L, n))
+        pos = rng.permutation(n)[:band]
+        mass[:, pos] = (1 << 30) + (rng.integers(0, 40, size=(L, band)) << 12)
+        kappa = band // 2
+    elif case == "all_equal":
+        mass = np.full((L, n), 12345, dtype=np.int64)
+        kappa = 1000
+    else:                                                 # keys with the top bit of 64 set (one layer: no sum to overflow)
+        L = 1
+        mass = rng.integers(0, 1 << 62, size=(L, n)).astype(np.uint64)
+        mass[:, ::3] |= np.uint64(1 << 63)
+        kappa = 2000
+    mass = np.ascontiguousarray(mass.astype(np.uint64))
+    for mode in (0, 1):
+        sel = oracle.select_tokens(mass, B, 100, kappa, mode)
+        out = _outputs(L, n // B)
+        a = pk.select_args(kind=pk.SCORE_TOKEN_MASS, n_layers=L, n_suffix_tokens=n, block_tokens=B, dirty_tokens=100,
+                           top_k=kappa, layer_mode=mode, mass=torch.from_numpy(mass.view(np.int64)).to(DEV), **out)
+        ctx.select_repair_tokens(a)
+        _check(out, sel)
+    assert ctx.query_status() == 0
+
+
 def test_token_form_and_block_form_differ_on_the_constructed_case(ctx):
     from paper_2609_26219_b200 import binding as pk
     n, B = 128, 16

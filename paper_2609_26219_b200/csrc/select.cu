@@ -1120,7 +1120,8 @@ extern "C" int patchkv_select_repair_tokens(patchkv_ctx* ctx, const patchkv_sele
 
     const bool shared = a->layer_mode == PATCHKV_LAYERS_SHARED && L > 1;
     const bool from_attn = a->kind == PATCHKV_SCORE_ATTN_F16;
-    // workspace: [token mass L*n (if computed here and not handed out)] [summed mass n (shared)] [token mask L*n bytes]
+    // workspace: [token mass L*n (if computed here and not handed out)] [summed mass n (shared)] [code histogram] [token
+    // mask L*n bytes]; what has to start at zero (masses computed here, the histogram) is contiguous: one memset
     // (request-level ranking with nobody asking for the per-layer masses: every layer adds straight into the summed row)
     const bool sum_direct = shared && from_attn && !a->mass_out;
     const size_t mass_elems = from_attn && !a->mass_out && !sum_direct ? (size_t)L * n : 0;
@@ -1134,9 +1135,11 @@ extern "C" int patchkv_select_repair_tokens(patchkv_ctx* ctx, const patchkv_sele
     if (rc != PATCHKV_OK) return rc;
     unsigned long long* ws = ctx->d_mass_ws;
     unsigned long long* ws_sum = ws + mass_elems;
-    uint8_t* tok_mask = reinterpret_cast<uint8_t*>(ws_sum + sum_elems);
-    unsigned int* coarse_hist = reinterpret_cast<unsigned int*>(ws_sum + sum_elems + mask_words);
-    if (coarse) PKV_CUDA(ctx, cudaMemsetAsync(coarse_hist, 0, hist_words * 8, stream));
+    unsigned int* coarse_hist = reinterpret_cast<unsigned int*>(ws_sum + sum_elems);
+    uint8_t* tok_mask = reinterpret_cast<uint8_t*>(ws_sum + sum_elems + hist_words);
+    const bool mass_in_ws = from_attn && !a->mass_out && n > 0;       // the masses are computed into the workspace
+    if (mass_in_ws) PKV_CUDA(ctx, cudaMemsetAsync(ws, 0, (mass_elems + sum_elems + hist_words) * 8, stream));
+    else if (coarse) PKV_CUDA(ctx, cudaMemsetAsync(coarse_hist, 0, hist_words * 8, stream));
 
     const unsigned long long* mass = reinterpret_cast<const unsigned long long*>(a->mass);
     if (from_attn) {
@@ -1145,7 +1148,7 @@ extern "C" int patchkv_select_repair_tokens(patchkv_ctx* ctx, const patchkv_sele
         unsigned long long* m = a->mass_out ? reinterpret_cast<unsigned long long*>(a->mass_out) : (sum_direct ? ws_sum : ws);
         const long long rows = (long long)a->n_q_heads * a->n_queries;
         if (rows > 0x7fffffffLL) return fail(ctx, PATCHKV_E_UNSUPPORTED, "select: Hq * Q too large");
-        if (n > 0) PKV_CUDA(ctx, cudaMemsetAsync(m, 0, (size_t)(sum_direct ? 1 : L) * n * sizeof(unsigned long long), stream));
+        if (n > 0 && !mass_in_ws) PKV_CUDA(ctx, cudaMemsetAsync(m, 0, (size_t)L * n * sizeof(unsigned long long), stream));
         if (n > 0 && rows > 0) {
             MassParams mp;                         // token granularity: a block of one token
             mp.attn = static_cast<const uint16_t*>(a->attn);

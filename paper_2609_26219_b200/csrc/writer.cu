@@ -819,7 +819,7 @@ static int fill_gather(patchkv_ctx* ctx, const patchkv_geom* g, const patchkv_po
     if (nb == 0) return PATCHKV_OK;
     if (!s->block_table || !s->tags || !s->blk_off || !s->layer_bytes)
         return fail(ctx, PATCHKV_E_INVALID, "session: null pointer");
-    if ((long long)nb * g->n_layers > 0x7fffffffLL) return fail(ctx, PATCHKV_E_UNSUPPORTED, "quantize_gather: too many blocks");
+    if ((long long)nb * g->n_layers > 0x7fff0000LL) return fail(ctx, PATCHKV_E_UNSUPPORTED, "quantize_gather: too many blocks");
     p->L = g->n_layers; p->H = g->n_kv_heads; p->D = g->head_dim; p->B = g->block_tokens; p->P = g->page_tokens; p->G = G;
     p->k_base = static_cast<const uint16_t*>(pool->k_base);
     p->v_base = static_cast<const uint16_t*>(pool->v_base);

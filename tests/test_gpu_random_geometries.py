@@ -149,3 +149,41 @@ def test_selection_random_configuration(sctx, seed):
     sctx.select_repair_tokens(a)
     check(out, oracle.select_tokens(tmass, B, d_hat, kappa, mode))
     assert sctx.query_status() == 0
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_token_selection_random_many_candidates(sctx, seed):
+    """Token form with 4096 candidates or more (the ranking whose first cut is a code histogram by several CTAs): suffix
+    lengths, block sizes, dirty windows and budgets at random, scores full of ties, spread over many octaves, or both."""
+    from gpu_common import DEV
+    from paper_2609_26219_b200 import binding as pk
+    rng = np.random.default_rng(9000 + seed)
+    L = int(rng.integers(1, 4))
+    n = int(rng.integers(4200, 30000))
+    B = int(rng.choice([1, 8, 16, 20, 32, 64]))
+    NB = -(-n // B)
+    d_hat = int(rng.integers(0, 100))
+    mode = int(rng.integers(0, 2))
+    kind = seed % 3
+    if kind == 0:                                           # a handful of distinct values
+        tmass = rng.integers(0, 6, size=(L, n)).astype(np.uint64) << np.uint64(int(rng.integers(0, 40)))
+    elif kind == 1:                                         # twenty octaves, nearly all distinct
+        tmass = (2.0 ** rng.uniform(0, 40, size=(L, n))).astype(np.uint64)
+    else:                                                   # a crowd of near-equal scores with duplicates under a few large ones
+        tmass = ((1 << 28) + (rng.integers(0, 300, size=(L, n)) << 8)).astype(np.uint64)
+        tmass[:, rng.permutation(n)[:50]] <<= np.uint64(5)
+    kappa = int(rng.choice([1, 17, n // 64, n // 7, n]))
+    sel = oracle.select_tokens(np.ascontiguousarray(tmass), B, d_hat, kappa, mode)
+    out = dict(repair_mask=torch.full((L, NB), 9, dtype=torch.uint8, device=DEV),
+               repair_idx=torch.full((L, NB), -7, dtype=torch.int32, device=DEV),
+               repair_cnt=torch.full((L,), -7, dtype=torch.int32, device=DEV),
+               reuse_idx=torch.full((L, NB), -7, dtype=torch.int32, device=DEV),
+               reuse_cnt=torch.full((L,), -7, dtype=torch.int32, device=DEV))
+    a = pk.select_args(kind=pk.SCORE_TOKEN_MASS, n_layers=L, n_suffix_tokens=n, block_tokens=B, dirty_tokens=d_hat,
+                       top_k=kappa, layer_mode=mode, mass=torch.from_numpy(tmass.view(np.int64)).to(DEV), **out)
+    sctx.select_repair_tokens(a)
+    torch.cuda.synchronize()
+    for name, key in (("repair_mask", "mask"), ("repair_idx", "repair_idx"), ("reuse_idx", "reuse_idx"),
+                      ("repair_cnt", "repair_cnt"), ("reuse_cnt", "reuse_cnt")):
+        assert np.array_equal(out[name].cpu().numpy(), sel[key]), name
+    assert sctx.query_status() == 0

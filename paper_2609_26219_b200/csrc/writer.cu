@@ -179,12 +179,6 @@ __device__ __forceinline__ void encode_chunk(const uint4& w, uint8_t* codes, uin
     if (((threadIdx.x & 31) & (seg - 1)) == 0) *reinterpret_cast<__half*>(scales + 2 * scale_index) = s16;
 }
 
-__device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b) {
-    uint32_t d;
-    asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
-    return d;
-}
-
 // One CTA per (layer, block).
 __global__ void __launch_bounds__(kGatherThreads)
 quantize_gather_kernel(const GatherParams p) {

@@ -401,9 +401,10 @@ __device__ __forceinline__ void encode_pass(uint32_t region, int u0, int units, 
 }
 
 // ---------------------------------------------------------------- persistent bulk-copy pipeline
-// The block encoder as a persistent kernel: one producer warp walks this CTA's share of the (layer, block) list
-// (block i of the launch goes to CTA i mod grid), looks up and validates the directory entries and source pages a
-// round of 32 blocks ahead, and stages the blocks' K and V rows into a shared-memory ring with bulk asynchronous
+// The block encoder as a persistent kernel: one producer warp takes rounds of consecutive (layer, block) entries (the
+// first dealt out statically, the rest claimed from the launch's work counter in shrinking rounds), looks up and
+// validates the directory entries and source pages a round of up to 32 blocks ahead, one block per lane, and stages
+// the blocks' K and V rows into a shared-memory ring with bulk asynchronous
 // copies that complete on an mbarrier; the consumer warps quantise from shared memory and write the record with
 // warp-contiguous stores.  A stage (a unit) carries up to kWMaxSub pieces -- a piece is a run of tokens of one section
 // of one block -- so that geometries with small rows still move about 32 KiB per barrier round trip, and the

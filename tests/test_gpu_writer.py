@@ -199,7 +199,8 @@ def test_plan_and_writer_replay_from_a_cuda_graph(ctx):
     starts = [sum(-(-s // 256) * 256 for s in sizes[:i]) for i in range(L)]
     payload = torch.zeros(starts[-1] + sizes[-1] + 256, dtype=torch.uint8, device=DEV)
     ptrs = torch.tensor([payload.data_ptr() + o for o in starts], dtype=torch.int64, device=DEV)
-    sess = pk.make_session(n_suffix_tokens=ck.n_suffix_tokens, delta=0, dst_shift=5, block_table=ck.block_table.to(DEV).contiguous(),
+    table = ck.block_table.to(DEV).contiguous()           # (the session holds raw pointers: keep the tensors alive)
+    sess = pk.make_session(n_suffix_tokens=ck.n_suffix_tokens, delta=0, dst_shift=5, block_table=table,
                            tags=tags, blk_off=off, layer_payload=ptrs, layer_bytes=lb, reuse_idx=None, reuse_cnt=None)
     side = torch.cuda.Stream()
     side.wait_stream(torch.cuda.current_stream())
@@ -215,6 +216,48 @@ def test_plan_and_writer_replay_from_a_cuda_graph(ctx):
         pay = payload.cpu().numpy()
         assert np.array_equal(off.cpu().numpy().astype(np.uint64), off_o)
         for o, s_, b_ in zip(starts, sizes, bufs_o):
+            assert np.array_equal(pay[o:o + s_], b_)
+    assert ctx.query_status() == 0
+
+
+def test_two_writers_on_two_streams_of_one_context(ctx):
+    """Two checkpoints encoded at the same time on two streams of one context (each stream has its own work counters):
+    both match the oracle, over several rounds without a synchronisation in between."""
+    from paper_2609_26219_b200 import binding as pk
+    jobs = []
+    for seed, n in ((31, 640), (32, 1000)):
+        g = pin.Geometry(3, 4, 64, 64, pin.ROPE_HALF, 1e4, 16, 16, 32)
+        ck = _ck(geom=g, n=n, n_pages=n // 16 + 8, seed=seed)
+        kp, vp = pool_from_raw(ck)
+        rc, rc2, off_o, lb_o, bufs_o = run_writer(ck, kp, vp)
+        L, NB = g.n_layers, ck.n_blocks
+        k = torch.from_numpy(kp.view(np.int16)).to(DEV)
+        v = torch.from_numpy(vp.view(np.int16)).to(DEV)
+        pool = pk.make_pool(k, v, ck.n_pages, pin.pool_strides(g, ck.n_pages))
+        geom = pk.make_geom(g.n_layers, g.n_kv_heads, g.head_dim, g.rotary_dim, g.rope_style, g.rope_base, g.block_tokens,
+                            g.page_tokens, g.group)
+        tags = ck.tags.to(DEV).contiguous()
+        off = torch.from_numpy(off_o.astype(np.int64)).to(DEV)
+        lb = torch.from_numpy(np.asarray(lb_o).astype(np.int64)).to(DEV)
+        sizes = [int(x) for x in lb_o]
+        starts = [sum(-(-s // 256) * 256 for s in sizes[:i]) for i in range(L)]
+        payload = torch.zeros(starts[-1] + sizes[-1] + 256, dtype=torch.uint8, device=DEV)
+        ptrs = torch.tensor([payload.data_ptr() + o for o in starts], dtype=torch.int64, device=DEV)
+        table = ck.block_table.to(DEV).contiguous()
+        sess = pk.make_session(n_suffix_tokens=ck.n_suffix_tokens, delta=0, dst_shift=0, block_table=table,
+                               tags=tags, blk_off=off, layer_payload=ptrs, layer_bytes=lb, reuse_idx=None, reuse_cnt=None)
+        jobs.append(dict(geom=geom, pool=pool, sess=sess, payload=payload, starts=starts, sizes=sizes, want=bufs_o,
+                         stream=torch.cuda.Stream(), keep=(k, v, tags, off, lb, ptrs, table)))   # the session holds raw pointers
+    torch.cuda.synchronize()
+    for _ in range(6):
+        for j in jobs:
+            with torch.cuda.stream(j["stream"]):
+                j["payload"].fill_(0xEE)
+            ctx.quantize_gather(j["geom"], j["pool"], j["sess"], j["stream"])
+    torch.cuda.synchronize()
+    for j in jobs:
+        pay = j["payload"].cpu().numpy()
+        for o, s_, b_ in zip(j["starts"], j["sizes"], j["want"]):
             assert np.array_equal(pay[o:o + s_], b_)
     assert ctx.query_status() == 0
 

@@ -851,7 +851,29 @@ select_kernel(const TopkParams p) {
         const unsigned long long all_or = ((unsigned long long)s_or[1] << 32) | s_or[0];
         const int top_byte = all_or ? (63 - __clzll((long long)all_or)) >> 3 : -1;
 
-        if ((all_or >> 32) == 0) {
+        if (!COARSE && iters == 1) {
+            // One candidate per thread (the block form: at most 1024 blocks per layer): the k-th largest key by bisection
+            // on its bits from the top, one counting barrier per bit.  As soon as exactly k keys lie at or above the
+            // trial value the selection is decided and the remaining bits do not matter (masses spread over many
+            // octaves: a dozen steps); masses full of ties go through every bit and end with the exact key and the
+            // number of its equals.
+            const bool cand = (int)threadIdx.x < ncand;
+            const unsigned long long x = kreg[0];
+            unsigned long long t = 0;
+            bool exact_k = false;
+            for (int bit = all_or ? 63 - __clzll((long long)all_or) : -1; bit >= 0; bit--) {
+                const unsigned long long trial = t | (1ull << bit);
+                const int c = __syncthreads_count(cand && x >= trial);
+                if (c >= k) { t = trial; if (c == k) { exact_k = true; break; } }
+            }
+            T = t;
+            if (exact_k) { krem = 0; n_eq = 0; }         // x >= T takes exactly k keys: no equals to rank
+            else {
+                const int larger = __syncthreads_count(cand && x > t);
+                n_eq = __syncthreads_count(cand && x == t);
+                krem = k - larger;
+            }
+        } else if ((all_or >> 32) == 0) {
             // every candidate fits 32 bits (masses of a few thousand rows): the same passes on 32-bit keys
             unsigned int k32[KPT];
 #pragma unroll
@@ -860,9 +882,11 @@ select_kernel(const TopkParams p) {
         } else {
             radix_select_passes<unsigned long long, KPT>(kreg, later_key, iters, ncand, top_byte, hist, &s_prefix, &s_krem, &s_eq);
         }
-        T = s_prefix;
-        krem = s_krem;                           // keys equal to T to take, lowest block index first
-        n_eq = s_eq;
+        if (COARSE || iters != 1) {
+            T = s_prefix;
+            krem = s_krem;                       // keys equal to T to take, lowest block index first
+            n_eq = s_eq;
+        }
     }
     // Ranking among equal keys (a prefix count in index order) is needed only when some of them stay out.
     const bool ties_matter = !take_all && !take_none && n_eq > krem;
